@@ -1,0 +1,5 @@
+"""fp64 CPU oracle for the CLP decode-step attention (test infrastructure, not part of the product).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
+"""
+from .plt_oracle import build, decode_attn, decode_attn_rows, threads, set_threads  # noqa: F401
