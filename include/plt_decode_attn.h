@@ -1,0 +1,162 @@
+/*
+ * plt_decode_attn.h - C ABI of the Cross-Loop-Parallel (CLP) decode-step
+ * attention of the Parallel Loop Transformer, for NVIDIA B200 (sm_100a).
+ *
+ * One call computes, for a batch of B sequences, the attention of ONE layer at
+ * ONE decode step for all L loops at once (the paper's displaced micro-batch,
+ * Algorithm 1 line 5 and the "Inference" paragraph of Sec. 2.2.1): loop l
+ * (1-indexed) serves token i-l+1, so its query may see the first
+ * cut(b,l) = max(0, N_b - delta_l) entries of the single shared first-loop KV
+ * cache (delta_l = l-1 unless overridden).  Every loop attends that one cache
+ * ("KV-cache sharing from the first loop", Sec. 2.2.2, Algorithm 3 line 2),
+ * which the kernels read from HBM once per sequence, not once per loop.
+ * Loops 2..L additionally attend their private window of the most recent
+ * <= w entries (Algorithm 3 line 3) and the two normalised results are mixed
+ * with a per-head sigmoid gate (Algorithm 3 lines 4-5, Eq. 2):
+ *
+ *   y_global = softmax(sm_scale * q K_share[0:cut]^T) V_share[0:cut]
+ *   y_local  = softmax(sm_scale * q K_win[0:wl]^T)    V_win[0:wl]
+ *   g        = sigmoid(gate_logit)
+ *   O        = g * y_local + (1 - g) * y_global        (loops 2..L)
+ *   O        = y_global                                (loop 1)
+ *
+ * Rows whose loop has no token yet (cut == 0) are written as zeros.  With
+ * cut > 0 and wl == 0, y_local is taken as 0.  Query head h reads KV head
+ * h / (Hq / Hkv).
+ *
+ * All tensor pointers are DEVICE pointers owned by the caller unless a comment
+ * says "host".  No exception crosses this boundary; every function returns a
+ * plt_status.  There is no CPU fallback: without a CUDA device every call that
+ * needs one fails with PLT_ERR_CUDA.
+ */
+#ifndef PLT_DECODE_ATTN_H
+#define PLT_DECODE_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct plt_decode_attn* plt_decode_attn_t; /* opaque; owned by the library */
+
+typedef enum {
+    PLT_OK = 0,
+    PLT_ERR_INVALID_ARG = 1,  /* null pointer, bad size, misaligned base, struct_size mismatch */
+    PLT_ERR_UNSUPPORTED = 2,  /* shape outside what the kernels implement (never a silent fallback) */
+    PLT_ERR_OUT_OF_MEMORY = 3,
+    PLT_ERR_CUDA = 4,         /* a CUDA runtime/driver call failed; see plt_decode_attn_last_error */
+    PLT_ERR_CAPACITY = 5,     /* batch > max_batch, or a table smaller than the configuration needs */
+    PLT_ERR_DEVICE_CHECK = 6  /* plt_decode_attn_check: a kernel clamped a device-resident value or gave up a wait */
+} plt_status;
+
+typedef enum { PLT_F32 = 0, PLT_BF16 = 1 } plt_dtype;
+
+/* Bits of the device status word reported by plt_decode_attn_check. */
+#define PLT_DEV_SEQ_LEN_CLAMPED 1u  /* a seq_lens entry was outside [0, max_seq_len] */
+#define PLT_DEV_PAGE_ID_CLAMPED 2u  /* a page id was outside [0, num_pool_pages) */
+#define PLT_DEV_WAIT_TIMEOUT 4u     /* a bounded wait inside a kernel ran out; the output is not valid */
+#define PLT_DEV_WIN_LEN_CLAMPED 8u  /* a win_lens entry was outside [0, w] */
+
+/*
+ * Fixed at create.  struct_size = sizeof(plt_decode_attn_config) (versioning).
+ * Supported: d in {64, 128}; Hq % Hkv == 0; L * (Hq / Hkv) <= 64 packed query
+ * rows per KV head; L <= 8; paged caches need page_size % 16 == 0.
+ */
+typedef struct {
+    uint32_t struct_size;
+    int32_t dtype;        /* plt_dtype of Q, K, V, Kwin, Vwin and O; gate logits are always fp32 */
+    int32_t max_batch;    /* largest batch any run may pass (<= 4096) */
+    int32_t L;            /* loops computed in parallel (CLP micro-batch size), >= 1 */
+    int32_t Hq, Hkv, d;   /* query heads, KV heads, head dimension */
+    int32_t max_seq_len;  /* capacity of the shared cache per sequence, in tokens */
+    int32_t w;            /* window capacity in tokens (G-SWA, Sec. 2.2.2); may be 0 only if L == 1 */
+    int32_t page_size;    /* 0: contiguous shared cache; > 0: tokens per page */
+    float sm_scale;       /* score scale; <= 0 selects 1/sqrt(d) */
+    int32_t device;       /* CUDA device ordinal */
+    const int32_t* loop_offset; /* host, L entries delta_l >= 0; NULL: delta_l = l-1. Copied at create. */
+    /* Launch tuning, 0 = automatic. Results do not depend on these beyond rounding order. */
+    int32_t heads_per_cta; /* KV heads one thread block streams together (bf16 path; divides Hkv) */
+    int32_t key_slices;    /* 16-key slices per pipeline tile (bf16 path; 1, 2 or 4) */
+    int32_t stages;        /* depth of the shared-memory pipeline (bf16 path) */
+    int32_t ctas_per_sm;   /* persistent thread blocks per SM */
+} plt_decode_attn_config;
+
+/*
+ * Per call.  struct_size = sizeof(plt_decode_attn_args).  Every tensor base
+ * must be 16-byte aligned.  Inputs are read-only; `out` is fully overwritten
+ * for sequences [0, batch).
+ */
+typedef struct {
+    uint32_t struct_size;
+    int32_t batch;                 /* B, 0 <= B <= max_batch */
+    const void* q;                 /* [B, L, Hq, d] contiguous */
+    const void* k_cache;           /* shared first-loop keys: contiguous [B, N, Hkv, d] (strides below) */
+    const void* v_cache;           /*   or page pool [num_pool_pages, page_size, Hkv, d] */
+    int64_t kv_stride_b;           /* elements between sequences (contiguous) or between pages (paged) */
+    int64_t kv_stride_n;           /* elements between tokens */
+    int64_t kv_stride_h;           /* elements between KV heads; the head dimension itself is dense */
+                                   /* all three 0: dense layout as written above. Each a multiple of 8 (bf16) / 4 (fp32). */
+    const int32_t* seq_lens;       /* [B]; N_b counts the current token; values outside [0, max_seq_len] are clamped */
+    const int32_t* page_table;     /* [B, max_pages] page ids (paged only; else NULL) */
+    int32_t max_pages;             /* row length of page_table; >= ceil(max_seq_len / page_size) */
+    int32_t num_pool_pages;        /* pages in the pool */
+    const void* k_win;             /* [B, L-1, w, Hkv, d] contiguous; slots [0, wl) are attended (any order) */
+    const void* v_win;             /*   (both NULL allowed when L == 1) */
+    const int32_t* win_lens;       /* optional [B, L-1]; NULL: wl = min(w, cut(b,l)) */
+    const float* gate_logits;      /* [B, L-1, Hq] pre-sigmoid; +-inf allowed (NULL allowed when L == 1) */
+    void* out;                     /* [B, L, Hq, d], same dtype as q */
+} plt_decode_attn_args;
+
+/*
+ * Validates the configuration, selects the kernel variant and allocates the
+ * handle's workspace on config->device (split partials, plan, status word).
+ * This is the only call that allocates device memory for plt_decode_attn_run.
+ */
+plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_decode_attn_t* out_handle);
+
+/*
+ * Enqueues one decode-step attention (Algorithm 3 lines 2-5 for all L loops of
+ * all B sequences) on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ * Asynchronous: no allocation and no host synchronisation.  Host-visible
+ * arguments are validated first and nothing is launched on error.  Two kernels
+ * are launched: the split-KV main kernel and the merge/gate kernel.
+ * Calls on the same handle must be stream-ordered (they share the workspace).
+ */
+plt_status plt_decode_attn_run(plt_decode_attn_t handle, const plt_decode_attn_args* args, void* cuda_stream);
+
+/*
+ * Same computation with every tensor pointer in `args` pointing to HOST memory
+ * (pinned memory makes the copies asynchronous).  Copies the inputs into
+ * device staging buffers owned by the handle (allocated on the first call,
+ * sized for max_batch), runs, copies `out` back and synchronises the stream.
+ * Shared-cache strides must be 0 (dense); a paged pool must have
+ * num_pool_pages <= max_batch * max_pages.
+ */
+plt_status plt_decode_attn_run_host(plt_decode_attn_t handle, const plt_decode_attn_args* host_args, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the device status word and clears it.
+ * PLT_OK if it was 0; else PLT_ERR_DEVICE_CHECK with *out_bits (optional) = PLT_DEV_* bits. */
+plt_status plt_decode_attn_check(plt_decode_attn_t handle, void* cuda_stream, uint32_t* out_bits);
+
+/* Frees the workspace. NULL is accepted. The caller makes sure no run is in flight. */
+plt_status plt_decode_attn_destroy(plt_decode_attn_t handle);
+
+/* Message for the last non-OK status of this handle (or of the last failed create when handle == NULL).
+ * Owned by the library; valid until the next call on the same handle / thread. */
+const char* plt_decode_attn_last_error(plt_decode_attn_t handle);
+
+/* Device bytes plt_decode_attn_create would allocate for this configuration (no device needed for the arithmetic,
+ * but the SM count of config->device is queried when a device is present; 148 is assumed otherwise). */
+plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config* config, size_t* out_bytes);
+
+/* Number of kernels one plt_decode_attn_run launches, and the variant chosen at create
+ * (heads_per_cta, key_slices, stages, ctas_per_sm, grid size); any pointer may be NULL. */
+plt_status plt_decode_attn_launch_info(plt_decode_attn_t handle, int32_t* kernels_per_run, int32_t* heads_per_cta,
+                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PLT_DECODE_ATTN_H */

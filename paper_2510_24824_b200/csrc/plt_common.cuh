@@ -1,0 +1,221 @@
+// Shared device-side definitions of the CLP decode-attention kernels: the kernel parameter block,
+// the tile plan (how the key tiles of all sequences are laid on one line and cut into equal
+// ranges, one per persistent thread block) and the layout of split partials.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace plt {
+
+constexpr int kMaxLoops = 8;
+constexpr int kMaxRows = 64;     // packed query rows per KV head: L * (Hq / Hkv)
+constexpr int kMaxBatch = 4096;
+
+// Device status bits (mirrors the PLT_DEV_* values of the public header).
+constexpr uint32_t kDevSeqLenClamped = 1u;
+constexpr uint32_t kDevPageIdClamped = 2u;
+constexpr uint32_t kDevWaitTimeout = 4u;
+constexpr uint32_t kDevWinLenClamped = 8u;
+
+// Everything a kernel needs besides its TMA descriptors. Passed by value.
+struct Params {
+    const void* q;             // [B, L, Hq, d]
+    const void* k_cache;       // only the fp32 path dereferences these directly
+    const void* v_cache;
+    const void* k_win;
+    const void* v_win;
+    const int32_t* seq_lens;   // [B]
+    const int32_t* win_lens;   // [B, L-1] or null
+    const int32_t* page_table; // [B, max_pages] or null
+    const float* gate_logits;  // [B, L-1, Hq]
+    void* out;                 // [B, L, Hq, d]
+    float* part_acc;           // [slots][hpc][R][d]  unnormalised sum of p * V
+    float* part_ml;            // [slots][hpc][R][2]  running max (log2 units) and sum of p
+    int32_t* prefix;           // [B + 1] tile prefix written by block 0 of the main kernel
+    uint32_t* status;          // device status word
+    int64_t kv_stride_b, kv_stride_n, kv_stride_h;  // elements
+    int32_t B, L, Hq, Hkv, G, R, d, w;
+    int32_t max_seq_len, page_size, max_pages, num_pool_pages;
+    int32_t hpc;               // KV heads per work item
+    int32_t tile_keys;         // keys per plan tile
+    int32_t num_ctas;          // persistent grid size of the main kernel
+    float scale_log2;          // sm_scale * log2(e)
+    int32_t delta[kMaxLoops];  // per-loop causal offset
+};
+
+// ---- per-sequence plan -------------------------------------------------------------------------
+// Sequence b contributes, per group of `hpc` KV heads, gt tiles of the shared cache followed by the
+// tiles of the windows of loops 2..L. All head groups of a sequence are laid one after the other.
+struct SeqPlan {
+    int32_t n;                 // clamped N_b
+    int32_t cmax;              // largest cutoff over loops = keys of the shared cache that are read
+    int32_t gt;                // tiles of the shared cache
+    int32_t lt;                // tiles of all windows
+    int32_t cut[kMaxLoops];    // keys loop l may see
+    int32_t wl[kMaxLoops];     // wl[l] valid window slots of loop l (index 1..L-1; wl[0] unused)
+};
+
+__device__ __forceinline__ int32_t ceil_div(int32_t a, int32_t b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ void seq_plan(const Params& p, int b, SeqPlan& s, uint32_t& flags) {
+    int32_t n = p.seq_lens[b];
+    if (n < 0 || n > p.max_seq_len) {
+        flags |= kDevSeqLenClamped;
+        n = n < 0 ? 0 : p.max_seq_len;
+    }
+    s.n = n;
+    s.cmax = 0;
+    s.lt = 0;
+#pragma unroll
+    for (int l = 0; l < kMaxLoops; ++l) {
+        s.cut[l] = 0;
+        s.wl[l] = 0;
+        if (l < p.L) {
+            int32_t c = n - p.delta[l];
+            c = c > 0 ? c : 0;
+            s.cut[l] = c;
+            s.cmax = c > s.cmax ? c : s.cmax;
+            if (l >= 1) {
+                int32_t wl = c < p.w ? c : p.w;
+                if (p.win_lens != nullptr && c > 0) {
+                    wl = p.win_lens[b * (p.L - 1) + (l - 1)];
+                    if (wl < 0 || wl > p.w) {
+                        flags |= kDevWinLenClamped;
+                        wl = wl < 0 ? 0 : p.w;
+                    }
+                }
+                s.wl[l] = wl;
+                s.lt += ceil_div(wl, p.tile_keys);
+            }
+        }
+    }
+    s.gt = ceil_div(s.cmax, p.tile_keys);
+}
+
+// Tiles sequence b puts on the line.
+__device__ __forceinline__ int32_t seq_tiles(const Params& p, int b, uint32_t& flags) {
+    SeqPlan s;
+    seq_plan(p, b, s, flags);
+    return (p.Hkv / p.hpc) * (s.gt + s.lt);
+}
+
+// Range of the tile line owned by block c of C: [c*T/C, (c+1)*T/C).
+__device__ __forceinline__ int64_t cta_begin(int64_t T, int c, int C) { return (T * c) / C; }
+
+// The block that owns tile position pos.
+__device__ __forceinline__ int cta_of(int64_t T, int64_t pos, int C) {
+    return (int)(((pos + 1) * C - 1) / T);
+}
+
+// Work item index: (sequence, head group, kind) with kind 0 = shared cache, 1 = windows.
+__device__ __forceinline__ int item_index(const Params& p, int b, int hg, int kind) {
+    return (b * (p.Hkv / p.hpc) + hg) * 2 + kind;
+}
+
+// A piece (the part of an item done by one block) stores its partial in slot item + block.
+__device__ __forceinline__ int64_t slot_of(int item, int cta) { return (int64_t)item + cta; }
+
+// Block-wide exclusive prefix of seq_tiles into sp[0..B] (shared memory). All threads of the block call it.
+__device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint32_t& flags) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    for (int b = tid; b < p.B; b += nt) sp[b + 1] = seq_tiles(p, b, flags);
+    if (tid == 0) sp[0] = 0;
+    __syncthreads();
+    if (tid < 32) {
+        // warp 0: each lane owns a contiguous chunk, then a warp scan of the chunk sums
+        const int per = (p.B + 31) / 32;
+        const int lo = tid * per, hi = min(lo + per, p.B);
+        int32_t sum = 0;
+        for (int b = lo; b < hi; ++b) sum += sp[b + 1];
+        int32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (tid >= o) incl += v;
+        }
+        int32_t run = incl - sum;
+        for (int b = lo; b < hi; ++b) {
+            run += sp[b + 1];
+            sp[b + 1] = run;
+        }
+    }
+    __syncthreads();
+}
+
+// Largest b with sp[b] <= pos (pos < sp[B]).
+__device__ __forceinline__ int find_seq(const int32_t* sp, int B, int64_t pos) {
+    int lo = 0, hi = B;  // invariant: sp[lo] <= pos < sp[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if ((int64_t)sp[mid] <= pos) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// One piece of work: the tiles [t0, t1) of item (b, hg, kind).
+struct Piece {
+    int b, hg, kind;
+    int t0, t1;
+    SeqPlan sp;
+};
+
+// Walks the pieces of the range [pos, hi). Usage: PieceWalk w(p, sp, lo, hi); while (w.next(piece)) {...}
+struct PieceWalk {
+    const Params& p;
+    const int32_t* sp;
+    int64_t pos, hi;
+    int b;
+    __device__ PieceWalk(const Params& p_, const int32_t* sp_, int64_t lo_, int64_t hi_)
+        : p(p_), sp(sp_), pos(lo_), hi(hi_), b(0) {
+        if (pos < hi) b = find_seq(sp, p.B, pos);
+    }
+    __device__ bool next(Piece& pc, uint32_t& flags) {
+        if (pos >= hi) return false;
+        while ((int64_t)sp[b + 1] <= pos) ++b;
+        seq_plan(p, b, pc.sp, flags);
+        const int per = pc.sp.gt + pc.sp.lt;
+        const int o = (int)(pos - sp[b]);
+        pc.b = b;
+        pc.hg = o / per;
+        const int o2 = o - pc.hg * per;
+        int64_t item_end;
+        if (o2 < pc.sp.gt) {
+            pc.kind = 0;
+            pc.t0 = o2;
+            item_end = pos + (pc.sp.gt - o2);
+        } else {
+            pc.kind = 1;
+            pc.t0 = o2 - pc.sp.gt;
+            item_end = pos + (per - o2);
+        }
+        const int64_t end = item_end < hi ? item_end : hi;
+        pc.t1 = pc.t0 + (int)(end - pos);
+        pos = end;
+        return true;
+    }
+};
+
+// Window tile cursor: maps the running tile index of a windows item to (loop, first key in that window).
+struct WinCursor {
+    int l;      // loop index (0-based), 1..L-1
+    int key0;   // first key of the tile inside the window of loop l
+    __device__ void seek(const Params& p, const SeqPlan& s, int t) {
+        l = 1;
+        while (l < p.L - 1) {
+            int nt = ceil_div(s.wl[l], p.tile_keys);
+            if (t < nt) break;
+            t -= nt;
+            ++l;
+        }
+        key0 = t * p.tile_keys;
+    }
+    __device__ void advance(const Params& p, const SeqPlan& s) {
+        key0 += p.tile_keys;
+        while (key0 >= s.wl[l] && l < p.L - 1) {
+            ++l;
+            key0 = 0;
+        }
+    }
+};
+
+}  // namespace plt

@@ -1,0 +1,506 @@
+// C ABI of the CLP decode-step attention: argument validation, variant selection, workspace,
+// TMA descriptors and the two launches (split-KV main kernel, merge/gate kernel) per run.
+#include "../../include/plt_decode_attn.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "plt_host.h"
+
+using namespace plt;
+
+namespace {
+
+thread_local char g_create_error[512] = "";
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapKey {
+    const void* base;
+    int64_t s1, s2, s3;
+    int64_t d1, d2, d3;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && s1 == o.s1 && s2 == o.s2 && s3 == o.s3 && d1 == o.d1 && d2 == o.d2 && d3 == o.d3;
+    }
+};
+
+struct Staging {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct plt_decode_attn {
+    plt_decode_attn_config cfg;
+    int32_t delta[kMaxLoops];
+    int G, R;
+    bool bf16;
+    int sm_count;
+    MainVariant var;      // bf16: full variant; fp32: only grid/smem used
+    int ctas_per_sm;
+    float scale_log2;
+    // workspace
+    float* part_acc = nullptr;
+    float* part_ml = nullptr;
+    int32_t* prefix = nullptr;
+    uint32_t* status = nullptr;
+    size_t ws_bytes = 0;
+    // TMA descriptors, re-encoded only when a base pointer, stride or extent changes
+    EncodeTiledFn encode = nullptr;
+    CUtensorMap maps[4];
+    MapKey keys[4];
+    bool map_valid[4] = {false, false, false, false};
+    // device staging for plt_decode_attn_run_host (grow-only)
+    Staging st[10];
+    char err[512];
+};
+
+namespace {
+
+plt_status fail(plt_decode_attn_t h, plt_status code, const char* fmt, ...) {
+    char* dst = h ? h->err : g_create_error;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(dst, 512, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+plt_status cuda_fail(plt_decode_attn_t h, const char* what, cudaError_t e) {
+    return fail(h, PLT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+int elem_size(bool bf16) { return bf16 ? 2 : 4; }
+
+struct Geometry {
+    int G, R, MT;
+};
+
+plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
+    if (!c) return fail(nullptr, PLT_ERR_INVALID_ARG, "config is NULL");
+    if (c->struct_size != sizeof(plt_decode_attn_config))
+        return fail(nullptr, PLT_ERR_INVALID_ARG, "config.struct_size %u != %zu", c->struct_size,
+                    sizeof(plt_decode_attn_config));
+    if (c->dtype != PLT_F32 && c->dtype != PLT_BF16) return fail(nullptr, PLT_ERR_INVALID_ARG, "unknown dtype %d", c->dtype);
+    if (c->max_batch < 1 || c->L < 1 || c->Hq < 1 || c->Hkv < 1 || c->max_seq_len < 1 || c->w < 0 || c->page_size < 0)
+        return fail(nullptr, PLT_ERR_INVALID_ARG, "non-positive size in config");
+    if (c->max_batch > kMaxBatch) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch %d > %d", c->max_batch, kMaxBatch);
+    if (c->L > kMaxLoops) return fail(nullptr, PLT_ERR_UNSUPPORTED, "L %d > %d", c->L, kMaxLoops);
+    if (c->Hq % c->Hkv != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "Hq %d is not a multiple of Hkv %d", c->Hq, c->Hkv);
+    if (c->d != 64 && c->d != 128) return fail(nullptr, PLT_ERR_UNSUPPORTED, "head dim %d (supported: 64, 128)", c->d);
+    if (c->L > 1 && c->w < 1) return fail(nullptr, PLT_ERR_INVALID_ARG, "w must be >= 1 when L > 1");
+    g->G = c->Hq / c->Hkv;
+    g->R = c->L * g->G;
+    if (g->R > kMaxRows)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "L * Hq/Hkv = %d packed rows > %d", g->R, kMaxRows);
+    g->MT = g->R <= 16 ? 1 : (g->R <= 32 ? 2 : 4);
+    if (c->page_size > 0 && c->page_size % 16 != 0)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "page_size %d is not a multiple of 16", c->page_size);
+    if (c->loop_offset)
+        for (int l = 0; l < c->L; ++l)
+            if (c->loop_offset[l] < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "loop_offset[%d] < 0", l);
+    return PLT_OK;
+}
+
+// Picks (heads per block, key slices, stages, blocks per SM) for the bf16 kernel.
+plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, MainVariant* v, int* want_ctas_per_sm) {
+    v->D = c->d;
+    v->MT = g.MT;
+    int hpc = c->heads_per_cta, kw = c->key_slices;
+    if (hpc == 0) {
+        hpc = 1;
+        const int cap = g.MT >= 4 ? 1 : (g.MT == 2 ? 2 : 4);
+        for (int h = cap; h >= 1; h >>= 1)
+            if (c->Hkv % h == 0) { hpc = h; break; }
+    }
+    if (kw == 0) {
+        kw = 4 / (hpc * g.MT);
+        if (kw < 1) kw = 1;
+        if (kw > 4) kw = 4;
+    }
+    if (c->Hkv % hpc != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "heads_per_cta %d does not divide Hkv %d", hpc, c->Hkv);
+    while (c->page_size > 0 && c->page_size % (16 * kw) != 0 && kw > 1) kw >>= 1;
+    if (!main_bf16_exists(v->D, v->MT, hpc, kw))
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "no bf16 kernel for heads_per_cta=%d key_slices=%d with %d row tiles", hpc,
+                    kw, g.MT);
+    v->HPC = hpc;
+    v->KW = kw;
+    const int ncw = hpc * kw * g.MT;
+    int cps = c->ctas_per_sm > 0 ? c->ctas_per_sm : (ncw <= 4 ? 2 : 1);
+    const size_t budget = (size_t)(cps >= 2 ? 227 * 1024 / cps - 1024 : 227 * 1024);
+    int stages = c->stages;
+    if (stages == 0) {
+        stages = 2;
+        while (stages < 12 && main_bf16_smem(v->D, v->MT, hpc, kw, stages + 1, c->max_batch) <= budget) ++stages;
+        if (stages > 8) stages = 8;
+    }
+    if (stages < 2 || stages > 12) return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [2, 12]", stages);
+    v->stages = stages;
+    v->smem = main_bf16_smem(v->D, v->MT, hpc, kw, stages, c->max_batch);
+    if (v->smem > 227 * 1024)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "variant needs %zu bytes of shared memory (> 227 KB)", v->smem);
+    *want_ctas_per_sm = cps;
+    return PLT_OK;
+}
+
+size_t workspace_bytes_for(const plt_decode_attn_config* c, const Geometry& g, int hpc, int grid, size_t* acc_floats,
+                           size_t* ml_floats) {
+    const size_t slots = (size_t)c->max_batch * (c->Hkv / hpc) * 2 + (size_t)grid;
+    *acc_floats = slots * hpc * g.R * c->d;
+    *ml_floats = slots * hpc * g.R * 2;
+    return (*acc_floats + *ml_floats) * 4 + (size_t)(c->max_batch + 1) * 4 + 256;
+}
+
+plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, int D, int64_t d1, int64_t d2, int64_t d3,
+                      int64_t s1, int64_t s2, int64_t s3, int box_keys, int box_heads) {
+    MapKey key{base, s1, s2, s3, d1, d2, d3};
+    if (h->map_valid[idx] && h->keys[idx] == key) return PLT_OK;
+    cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)d1, (cuuint64_t)d2, (cuuint64_t)d3};
+    cuuint64_t strides[3] = {(cuuint64_t)(s1 * es), (cuuint64_t)(s2 * es), (cuuint64_t)(s3 * es)};
+    cuuint32_t box[4] = {64u, (cuuint32_t)box_keys, (cuuint32_t)box_heads, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    CUresult r = h->encode(&h->maps[idx], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        h->map_valid[idx] = false;
+        return fail(h, PLT_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d for tensor %d", (int)r, idx);
+    }
+    h->keys[idx] = key;
+    h->map_valid[idx] = true;
+    return PLT_OK;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+}  // namespace
+
+#define PLT_API __attribute__((visibility("default")))
+extern "C" {
+
+PLT_API plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config* config, size_t* out_bytes) {
+    Geometry g;
+    plt_status s = check_config(config, &g);
+    if (s != PLT_OK) return s;
+    if (!out_bytes) return fail(nullptr, PLT_ERR_INVALID_ARG, "out_bytes is NULL");
+    int sms = 148;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, config->device) == cudaSuccess) sms = prop.multiProcessorCount;
+    else (void)cudaGetLastError();
+    int hpc = 1, cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
+    if (config->dtype == PLT_BF16) {
+        MainVariant v;
+        s = choose_variant(config, g, &v, &cps);
+        if (s != PLT_OK) return s;
+        hpc = v.HPC;
+    }
+    size_t a, m;
+    *out_bytes = workspace_bytes_for(config, g, hpc, sms * cps, &a, &m);
+    return PLT_OK;
+}
+
+PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_decode_attn_t* out_handle) {
+    if (!out_handle) return fail(nullptr, PLT_ERR_INVALID_ARG, "out_handle is NULL");
+    *out_handle = nullptr;
+    Geometry g;
+    plt_status s = check_config(config, &g);
+    if (s != PLT_OK) return s;
+
+    cudaError_t e = cudaSetDevice(config->device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaSetDevice", e);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, config->device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDeviceProperties", e);
+    if (prop.major != 10)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only",
+                    config->device, prop.major, prop.minor);
+
+    plt_decode_attn* h = new (std::nothrow) plt_decode_attn();
+    if (!h) return fail(nullptr, PLT_ERR_OUT_OF_MEMORY, "host allocation failed");
+    h->cfg = *config;
+    h->cfg.loop_offset = nullptr;
+    for (int l = 0; l < kMaxLoops; ++l) h->delta[l] = config->loop_offset && l < config->L ? config->loop_offset[l] : l;
+    h->G = g.G;
+    h->R = g.R;
+    h->bf16 = config->dtype == PLT_BF16;
+    h->sm_count = prop.multiProcessorCount;
+    const float scale = config->sm_scale > 0.f ? config->sm_scale : 1.0f / sqrtf((float)config->d);
+    h->scale_log2 = scale * 1.4426950408889634f;
+    h->err[0] = 0;
+
+    int blocks = 0;
+    if (h->bf16) {
+        int cps = 0;
+        s = choose_variant(config, g, &h->var, &cps);
+        if (s != PLT_OK) { delete h; return s; }
+        e = main_bf16_prepare(h->var, &blocks);
+        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, "preparing the bf16 main kernel", e); }
+        if (blocks < 1) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM"); }
+        h->ctas_per_sm = blocks < cps ? blocks : cps;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) {
+            delete h;
+            return fail(nullptr, PLT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        }
+        h->encode = (EncodeTiledFn)fn;
+    } else {
+        h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
+        e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
+        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, "preparing the fp32 main kernel", e); }
+        if (blocks < 1) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM"); }
+        const int cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
+        h->ctas_per_sm = blocks < cps ? blocks : cps;
+    }
+    h->var.grid = h->sm_count * h->ctas_per_sm;
+
+    // The tile line must fit 31 bits.
+    const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+    const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
+                         ((double)(config->max_seq_len + tk - 1) / tk + (double)(config->L - 1) * ((config->w + tk - 1) / tk));
+    if (tiles >= 2147483647.0) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan"); }
+
+    size_t acc_floats, ml_floats;
+    h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
+    void* ws = nullptr;
+    e = cudaMalloc(&ws, h->ws_bytes);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete h;
+        return fail(nullptr, PLT_ERR_OUT_OF_MEMORY, "cudaMalloc of %zu workspace bytes failed", h->ws_bytes);
+    }
+    h->part_acc = (float*)ws;
+    h->part_ml = h->part_acc + acc_floats;
+    h->prefix = (int32_t*)(h->part_ml + ml_floats);
+    h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
+    e = cudaMemset(h->status, 0, 4);
+    if (e != cudaSuccess) { cudaFree(ws); delete h; return cuda_fail(nullptr, "cudaMemset", e); }
+    *out_handle = h;
+    return PLT_OK;
+}
+
+PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if (!a) return fail(h, PLT_ERR_INVALID_ARG, "args is NULL");
+    if (a->struct_size != sizeof(plt_decode_attn_args))
+        return fail(h, PLT_ERR_INVALID_ARG, "args.struct_size %u != %zu", a->struct_size, sizeof(plt_decode_attn_args));
+    const plt_decode_attn_config& c = h->cfg;
+    if (a->batch < 0) return fail(h, PLT_ERR_INVALID_ARG, "batch %d < 0", a->batch);
+    if (a->batch > c.max_batch) return fail(h, PLT_ERR_CAPACITY, "batch %d > max_batch %d", a->batch, c.max_batch);
+    if (a->batch == 0) return PLT_OK;
+    if (!a->q || !a->k_cache || !a->v_cache || !a->seq_lens || !a->out)
+        return fail(h, PLT_ERR_INVALID_ARG, "q, k_cache, v_cache, seq_lens and out must not be NULL");
+    if (c.L > 1 && (!a->k_win || !a->v_win || !a->gate_logits))
+        return fail(h, PLT_ERR_INVALID_ARG, "k_win, v_win and gate_logits must not be NULL when L > 1");
+    if (!aligned16(a->q) || !aligned16(a->k_cache) || !aligned16(a->v_cache) || !aligned16(a->out) ||
+        (c.L > 1 && (!aligned16(a->k_win) || !aligned16(a->v_win))))
+        return fail(h, PLT_ERR_INVALID_ARG, "tensor base pointers must be 16-byte aligned");
+    const int es = elem_size(h->bf16);
+    int64_t sb = a->kv_stride_b, sn = a->kv_stride_n, sh = a->kv_stride_h;
+    if (sb == 0 && sn == 0 && sh == 0) {
+        sh = c.d;
+        sn = (int64_t)c.Hkv * c.d;
+        sb = (int64_t)(c.page_size > 0 ? c.page_size : c.max_seq_len) * sn;
+    }
+    const int64_t unit = 16 / es;
+    if (sb <= 0 || sn <= 0 || sh <= 0 || sb % unit || sn % unit || sh % unit)
+        return fail(h, PLT_ERR_INVALID_ARG, "kv strides must be positive multiples of %lld elements", (long long)unit);
+    if (sh < c.d) return fail(h, PLT_ERR_INVALID_ARG, "kv_stride_h %lld < d", (long long)sh);
+    if ((double)sb * es >= 1099511627776.0 || (double)sn * es >= 1099511627776.0)
+        return fail(h, PLT_ERR_UNSUPPORTED, "kv stride of 2^40 bytes or more");
+    if (c.page_size > 0) {
+        if (!a->page_table) return fail(h, PLT_ERR_INVALID_ARG, "page_table is NULL for a paged cache");
+        const int need = (c.max_seq_len + c.page_size - 1) / c.page_size;
+        if (a->max_pages < need) return fail(h, PLT_ERR_CAPACITY, "max_pages %d < %d", a->max_pages, need);
+        if (a->num_pool_pages < 1) return fail(h, PLT_ERR_INVALID_ARG, "num_pool_pages %d < 1", a->num_pool_pages);
+    }
+
+    Params p;
+    memset(&p, 0, sizeof p);
+    p.q = a->q; p.k_cache = a->k_cache; p.v_cache = a->v_cache; p.k_win = a->k_win; p.v_win = a->v_win;
+    p.seq_lens = a->seq_lens; p.win_lens = a->win_lens; p.page_table = a->page_table; p.gate_logits = a->gate_logits;
+    p.out = a->out;
+    p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.status = h->status;
+    p.kv_stride_b = sb; p.kv_stride_n = sn; p.kv_stride_h = sh;
+    p.B = a->batch; p.L = c.L; p.Hq = c.Hq; p.Hkv = c.Hkv; p.G = h->G; p.R = h->R; p.d = c.d; p.w = c.w;
+    p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
+    p.num_pool_pages = a->num_pool_pages;
+    p.hpc = h->var.HPC;
+    p.tile_keys = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+    p.num_ctas = h->var.grid;
+    p.scale_log2 = h->scale_log2;
+    for (int l = 0; l < kMaxLoops; ++l) p.delta[l] = h->delta[l];
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (h->bf16) {
+        const int tk = 16 * h->var.KW;
+        plt_status s;
+        if (c.page_size > 0) {
+            s = encode_map(h, 0, a->k_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, h->var.HPC);
+            if (s == PLT_OK)
+                s = encode_map(h, 1, a->v_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, h->var.HPC);
+        } else {
+            s = encode_map(h, 0, a->k_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, h->var.HPC);
+            if (s == PLT_OK)
+                s = encode_map(h, 1, a->v_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, h->var.HPC);
+        }
+        if (s != PLT_OK) return s;
+        if (c.L > 1) {
+            const int64_t wn = (int64_t)c.Hkv * c.d, wb = (int64_t)c.w * wn;
+            s = encode_map(h, 2, a->k_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tk, h->var.HPC);
+            if (s == PLT_OK)
+                s = encode_map(h, 3, a->v_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tk,
+                               h->var.HPC);
+            if (s != PLT_OK) return s;
+        } else {
+            h->maps[2] = h->maps[0];
+            h->maps[3] = h->maps[1];
+        }
+        e = launch_main_bf16(h->var, h->maps, p, stream);
+    } else {
+        e = launch_main_f32(p, h->var.grid, h->var.smem, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(h, "launching the main kernel", e);
+    e = launch_reduce(p, h->bf16, stream);
+    if (e != cudaSuccess) return cuda_fail(h, "launching the merge kernel", e);
+    return PLT_OK;
+}
+
+static plt_status stage_in(plt_decode_attn_t h, int idx, const void* host, size_t bytes, cudaStream_t stream,
+                           const void** dev) {
+    *dev = nullptr;
+    if (!host || bytes == 0) return PLT_OK;
+    Staging& s = h->st[idx];
+    if (s.bytes < bytes) {
+        if (s.ptr) cudaFree(s.ptr);
+        s.ptr = nullptr;
+        s.bytes = 0;
+        cudaError_t e = cudaMalloc(&s.ptr, bytes);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return fail(h, PLT_ERR_OUT_OF_MEMORY, "cudaMalloc of %zu staging bytes failed", bytes);
+        }
+        s.bytes = bytes;
+    }
+    cudaError_t e = cudaMemcpyAsync(s.ptr, host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaMemcpyAsync (host to device)", e);
+    *dev = s.ptr;
+    return PLT_OK;
+}
+
+PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if (!a) return fail(h, PLT_ERR_INVALID_ARG, "args is NULL");
+    if (a->struct_size != sizeof(plt_decode_attn_args))
+        return fail(h, PLT_ERR_INVALID_ARG, "args.struct_size %u != %zu", a->struct_size, sizeof(plt_decode_attn_args));
+    const plt_decode_attn_config& c = h->cfg;
+    if (a->batch < 0) return fail(h, PLT_ERR_INVALID_ARG, "batch %d < 0", a->batch);
+    if (a->batch > c.max_batch) return fail(h, PLT_ERR_CAPACITY, "batch %d > max_batch %d", a->batch, c.max_batch);
+    if (a->batch == 0) return PLT_OK;
+    if (a->kv_stride_b || a->kv_stride_n || a->kv_stride_h)
+        return fail(h, PLT_ERR_UNSUPPORTED, "run_host takes dense shared caches only (strides must be 0)");
+    if (!a->q || !a->k_cache || !a->v_cache || !a->seq_lens || !a->out)
+        return fail(h, PLT_ERR_INVALID_ARG, "q, k_cache, v_cache, seq_lens and out must not be NULL");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const size_t es = elem_size(h->bf16), B = (size_t)a->batch;
+    const size_t row = (size_t)c.Hkv * c.d * es;
+    size_t kv_bytes;
+    if (c.page_size > 0) {
+        if (a->num_pool_pages < 1 || (size_t)a->num_pool_pages > (size_t)c.max_batch * (size_t)(a->max_pages > 0 ? a->max_pages : 0))
+            return fail(h, PLT_ERR_CAPACITY, "num_pool_pages %d outside [1, max_batch * max_pages]", a->num_pool_pages);
+        kv_bytes = (size_t)a->num_pool_pages * c.page_size * row;
+    } else {
+        kv_bytes = B * c.max_seq_len * row;
+    }
+    const size_t qo_bytes = B * c.L * c.Hq * c.d * es;
+    const size_t win_bytes = c.L > 1 ? B * (c.L - 1) * c.w * row : 0;
+    plt_decode_attn_args d = *a;
+    plt_status s;
+    const void* ptr;
+#define PLT_STAGE(idx, field, bytes)                                                   \
+    s = stage_in(h, idx, a->field, bytes, stream, &ptr);                               \
+    if (s != PLT_OK) return s;                                                         \
+    d.field = (decltype(d.field))ptr;
+    PLT_STAGE(0, q, qo_bytes)
+    PLT_STAGE(1, k_cache, kv_bytes)
+    PLT_STAGE(2, v_cache, kv_bytes)
+    PLT_STAGE(3, seq_lens, B * 4)
+    PLT_STAGE(4, page_table, c.page_size > 0 ? B * (size_t)a->max_pages * 4 : 0)
+    PLT_STAGE(5, k_win, win_bytes)
+    PLT_STAGE(6, v_win, win_bytes)
+    PLT_STAGE(7, win_lens, c.L > 1 ? B * (c.L - 1) * 4 : 0)
+    PLT_STAGE(8, gate_logits, c.L > 1 ? B * (c.L - 1) * c.Hq * 4 : 0)
+#undef PLT_STAGE
+    Staging& so = h->st[9];
+    if (so.bytes < qo_bytes) {
+        if (so.ptr) cudaFree(so.ptr);
+        so.ptr = nullptr;
+        so.bytes = 0;
+        if (cudaMalloc(&so.ptr, qo_bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return fail(h, PLT_ERR_OUT_OF_MEMORY, "cudaMalloc of %zu staging bytes failed", qo_bytes);
+        }
+        so.bytes = qo_bytes;
+    }
+    d.out = so.ptr;
+    s = plt_decode_attn_run(h, &d, cuda_stream);
+    if (s != PLT_OK) return s;
+    cudaError_t e = cudaMemcpyAsync(a->out, so.ptr, qo_bytes, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaMemcpyAsync (device to host)", e);
+    e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaStreamSynchronize", e);
+    return PLT_OK;
+}
+
+PLT_API plt_status plt_decode_attn_check(plt_decode_attn_t h, void* cuda_stream, uint32_t* out_bits) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    uint32_t bits = 0;
+    cudaError_t e = cudaMemcpyAsync(&bits, h->status, 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->status, 0, 4, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(h, "reading the device status word", e);
+    if (out_bits) *out_bits = bits;
+    if (bits == 0) return PLT_OK;
+    return fail(h, PLT_ERR_DEVICE_CHECK, "device status 0x%x:%s%s%s%s", bits,
+                (bits & PLT_DEV_SEQ_LEN_CLAMPED) ? " seq_lens entry out of range (clamped)" : "",
+                (bits & PLT_DEV_PAGE_ID_CLAMPED) ? " page id out of range (clamped)" : "",
+                (bits & PLT_DEV_WAIT_TIMEOUT) ? " a bounded wait ran out (output invalid)" : "",
+                (bits & PLT_DEV_WIN_LEN_CLAMPED) ? " win_lens entry out of range (clamped)" : "");
+}
+
+PLT_API plt_status plt_decode_attn_destroy(plt_decode_attn_t h) {
+    if (!h) return PLT_OK;
+    if (h->part_acc) cudaFree(h->part_acc);
+    for (Staging& s : h->st)
+        if (s.ptr) cudaFree(s.ptr);
+    delete h;
+    return PLT_OK;
+}
+
+PLT_API const char* plt_decode_attn_last_error(plt_decode_attn_t h) { return h ? h->err : g_create_error; }
+
+PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* kernels_per_run, int32_t* heads_per_cta,
+                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if (kernels_per_run) *kernels_per_run = 2;
+    if (heads_per_cta) *heads_per_cta = h->var.HPC;
+    if (key_slices) *key_slices = h->bf16 ? h->var.KW : kF32TileKeys / 16;
+    if (stages) *stages = h->var.stages;
+    if (ctas_per_sm) *ctas_per_sm = h->ctas_per_sm;
+    if (grid) *grid = h->var.grid;
+    return PLT_OK;
+}
+
+}  // extern "C"

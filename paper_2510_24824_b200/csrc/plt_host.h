@@ -1,0 +1,34 @@
+// Host-side interface between the C-ABI layer and the kernel translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "plt_common.cuh"
+
+namespace plt {
+
+// Variant of the bf16 main kernel.
+struct MainVariant {
+    int D, MT, HPC, KW;  // head dim, 16-row tiles, KV heads per block, 16-key slices per tile
+    int stages;          // ring depth
+    int grid;            // persistent blocks
+    size_t smem;         // dynamic shared memory per block
+};
+
+bool main_bf16_exists(int D, int MT, int HPC, int KW);
+size_t main_bf16_smem(int D, int MT, int HPC, int KW, int stages, int max_batch);
+// Sets the shared-memory attribute and reports how many blocks fit one SM.
+cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
+cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, cudaStream_t stream);
+
+// fp32 SIMT main kernel (same plan, tile of kF32TileKeys keys, one KV head per block).
+constexpr int kF32TileKeys = 32;
+constexpr int kF32Threads = 256;
+size_t main_f32_smem(int D, int R, int max_batch);
+cudaError_t main_f32_prepare(int D, int R, int max_batch, int* blocks_per_sm);
+cudaError_t launch_main_f32(const Params& p, int grid, size_t smem, cudaStream_t stream);
+
+cudaError_t launch_reduce(const Params& p, bool bf16, cudaStream_t stream);
+
+}  // namespace plt

@@ -1,0 +1,109 @@
+"""Device plumbing around the C ABI: moves a host problem into torch device tensors and calls the library.
+
+torch is used for device memory and streams only; the attention itself runs in libplt_decode_attn.so.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def _to_torch(a: Optional[np.ndarray], dtype: str, device, pin: bool = False):
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if a.dtype == np.uint16 and dtype == "bf16":
+        t = t.view(torch.bfloat16)
+    if device is None:
+        return t.pin_memory() if pin else t
+    return t.to(device, non_blocking=False)
+
+
+class DeviceProblem:
+    """Tensors of one decode step on a device (or, with device=None, in pinned host memory)."""
+
+    FIELDS = ("q", "k_cache", "v_cache", "seq_lens", "k_win", "v_win", "gate_logits", "page_table", "win_lens")
+
+    def __init__(self, p, device="cuda:0", pin: bool = False):
+        self.problem = p
+        self.device = device
+        for f in self.FIELDS:
+            a = getattr(p, f)
+            is_data = f in ("q", "k_cache", "v_cache", "k_win", "v_win")
+            setattr(self, f, _to_torch(a, p.dtype if is_data else "", device, pin))
+        tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+        if device is None:
+            self.out = torch.empty((p.B, p.L, p.Hq, p.d), dtype=tdt)
+            if pin:
+                self.out = self.out.pin_memory()
+        else:
+            self.out = torch.empty((p.B, p.L, p.Hq, p.d), dtype=tdt, device=device)
+
+    def args(self, out=None) -> B.Args:
+        p = self.problem
+        return B.make_args(
+            p.B, self.q, self.k_cache, self.v_cache, self.seq_lens, self.out if out is None else out,
+            k_win=self.k_win if p.L > 1 else None, v_win=self.v_win if p.L > 1 else None,
+            gate_logits=self.gate_logits if p.L > 1 else None, page_table=self.page_table,
+            max_pages=p.max_pages, num_pool_pages=p.num_pool_pages, win_lens=self.win_lens)
+
+    def h2d_bytes(self) -> int:
+        n = 0
+        for f in self.FIELDS:
+            t = getattr(self, f)
+            if t is not None and not (self.problem.L == 1 and f in ("k_win", "v_win", "gate_logits", "win_lens")):
+                n += t.numel() * t.element_size()
+        return n
+
+    def d2h_bytes(self) -> int:
+        return self.out.numel() * self.out.element_size()
+
+
+class DecodeAttn:
+    """Owns one plt_decode_attn handle sized for a problem (or for explicit limits)."""
+
+    def __init__(self, p, device_index: int = 0, max_batch: Optional[int] = None, **tuning):
+        self.config = B.make_config(
+            p.dtype, max_batch or max(p.B, 1), p.L, p.Hq, p.Hkv, p.d, p.max_seq_len, p.w, page_size=p.page_size,
+            sm_scale=p.sm_scale, device=device_index,
+            loop_offset=None if p.loop_offset is None else [int(x) for x in p.loop_offset], **tuning)
+        self.handle = B.plt_decode_attn_create(self.config)
+        self.info = B.plt_decode_attn_launch_info(self.handle)
+
+    def run(self, dp: DeviceProblem, stream: Optional[int] = None, out=None):
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        B.plt_decode_attn_run(self.handle, dp.args(out), stream)
+        return dp.out if out is None else out
+
+    def run_host(self, hp: DeviceProblem, stream: Optional[int] = None):
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        B.plt_decode_attn_run_host(self.handle, hp.args(), stream)
+        return hp.out
+
+    def check(self, stream: Optional[int] = None) -> int:
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        return B.plt_decode_attn_check(self.handle, stream)
+
+    def close(self):
+        if self.handle is not None:
+            B.plt_decode_attn_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,35 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI, compare with the oracle."""
+import numpy as np
+import torch
+
+from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
+
+# Tolerances of the parity bar: bf16 inputs max-abs 2e-2 and mean-abs 2e-3; fp32 inputs 1e-5 relative.
+BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
+F32_REL = 1e-5
+
+
+def run_gpu(p, check_status=True, **tuning) -> np.ndarray:
+    dp = DeviceProblem(p, "cuda:0")
+    dp.out.fill_(float("nan"))
+    with DecodeAttn(p, **tuning) as op:
+        op.run(dp)
+        bits = op.check()
+    if check_status:
+        assert bits == 0, f"device status 0x{bits:x}"
+    return dp.out.float().cpu().numpy().astype(np.float64)
+
+
+def assert_parity(got: np.ndarray, ref: np.ndarray, dtype: str, what: str = ""):
+    assert got.shape == ref.shape
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - ref)
+    if dtype == "bf16":
+        assert err.max() <= BF16_MAX_ABS, f"{what}: max abs err {err.max():.3e}"
+        assert err.mean() <= BF16_MEAN_ABS, f"{what}: mean abs err {err.mean():.3e}"
+    else:
+        scale = np.abs(ref).max()
+        assert err.max() <= F32_REL * max(scale, 1e-30), f"{what}: max err {err.max():.3e} vs max|ref| {scale:.3e}"
+        bad = err > F32_REL * np.abs(ref) + 1e-6
+        assert not bad.any(), f"{what}: {bad.sum()} elements beyond 1e-5 relative + 1e-6"
+    return float(err.max()), float(err.mean())

@@ -1,0 +1,94 @@
+"""CPU-only checks of the boundary: the library loads, exports what the header declares, and the
+binding's structs match the C layout. No compute call is made here."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parents[1]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2510_24824_b200 import build
+    build.build()
+    from paper_2510_24824_b200 import binding
+    return binding.load_library()
+
+
+def header_functions():
+    text = (ROOT / "include" / "plt_decode_attn.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(plt_decode_attn_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = header_functions()
+    assert "plt_decode_attn_create" in names and "plt_decode_attn_run" in names and "plt_decode_attn_destroy" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in the header but not exported"
+    from paper_2510_24824_b200 import binding
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_struct_layout_matches_c(tmp_path):
+    """Compile a tiny C program against the header and compare sizeof/offsetof with the ctypes structs."""
+    import subprocess
+    from paper_2510_24824_b200 import binding
+    fields_c = [f for f, _ in binding.Config._fields_]
+    fields_a = [f for f, _ in binding.Args._fields_]
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', f'#include "{ROOT}/include/plt_decode_attn.h"', 'int main(void){',
+             'printf("%zu\\n", sizeof(plt_decode_attn_config));']
+    lines += [f'printf("%zu\\n", offsetof(plt_decode_attn_config, {f}));' for f in fields_c]
+    lines += ['printf("%zu\\n", sizeof(plt_decode_attn_args));']
+    lines += [f'printf("%zu\\n", offsetof(plt_decode_attn_args, {f}));' for f in fields_a]
+    lines += ['return 0;}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c11", "-o", str(exe), str(src)], check=True)
+    vals = [int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
+    want = [ctypes.sizeof(binding.Config)] + [getattr(binding.Config, f).offset for f in fields_c]
+    want += [ctypes.sizeof(binding.Args)] + [getattr(binding.Args, f).offset for f in fields_a]
+    assert vals == want
+
+
+def test_host_side_validation_needs_no_gpu(lib):
+    """Argument checks that run before any CUDA call return their codes on a machine without a GPU."""
+    from paper_2510_24824_b200 import binding as B
+    ok = dict(dtype="bf16", max_batch=4, L=2, Hq=8, Hkv=2, d=128, max_seq_len=512, w=64)
+    bad = [
+        (dict(ok, d=96), B.PLT_ERR_UNSUPPORTED),
+        (dict(ok, Hq=7), B.PLT_ERR_INVALID_ARG),
+        (dict(ok, L=9), B.PLT_ERR_UNSUPPORTED),
+        (dict(ok, L=4, Hq=64, Hkv=2), B.PLT_ERR_UNSUPPORTED),  # 128 packed rows
+        (dict(ok, w=0), B.PLT_ERR_INVALID_ARG),
+        (dict(ok, page_size=24), B.PLT_ERR_UNSUPPORTED),
+        (dict(ok, max_batch=0), B.PLT_ERR_INVALID_ARG),
+        (dict(ok, max_batch=5000), B.PLT_ERR_UNSUPPORTED),
+        (dict(ok, loop_offset=[0, -1]), B.PLT_ERR_INVALID_ARG),
+        (dict(ok, heads_per_cta=3), B.PLT_ERR_INVALID_ARG),
+    ]
+    for kw, code in bad:
+        with pytest.raises(B.PltError) as e:
+            B.plt_decode_attn_workspace_bytes(B.make_config(**kw))
+        assert e.value.status == code, (kw, e.value)
+        assert e.value.message
+    cfg = B.make_config(**ok)
+    cfg.struct_size = 8
+    with pytest.raises(B.PltError) as e:
+        B.plt_decode_attn_workspace_bytes(cfg)
+    assert e.value.status == B.PLT_ERR_INVALID_ARG
+    assert B.plt_decode_attn_workspace_bytes(B.make_config(**ok)) > 0
+    B.plt_decode_attn_destroy(None)  # NULL is accepted
+
+
+def test_create_without_a_device_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    from paper_2510_24824_b200 import binding as B
+    with pytest.raises(B.PltError) as e:
+        B.plt_decode_attn_create(B.make_config("bf16", 4, 2, 8, 2, 128, 512, 64))
+    assert e.value.status == B.PLT_ERR_CUDA
