@@ -156,6 +156,11 @@ plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config* config,
 plt_status plt_decode_attn_launch_info(plt_decode_attn_t handle, int32_t* kernels_per_run, int32_t* heads_per_cta,
                                        int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid);
 
+/* Measurement aid: when both are non-NULL (cudaEvent_t created by the caller, with timing enabled), every later
+ * plt_decode_attn_run records ev_main_begin just before and ev_main_end just after the split-KV main kernel on
+ * the run's stream, so that the caller can time that kernel apart from the merge kernel. NULL, NULL switches it off. */
+plt_status plt_decode_attn_set_profile_events(plt_decode_attn_t handle, void* ev_main_begin, void* ev_main_end);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ PLT_DEV_SEQ_LEN_CLAMPED, PLT_DEV_PAGE_ID_CLAMPED, PLT_DEV_WAIT_TIMEOUT, PLT_DEV_
 EXPORTS = (
     "plt_decode_attn_create", "plt_decode_attn_run", "plt_decode_attn_run_host", "plt_decode_attn_check",
     "plt_decode_attn_destroy", "plt_decode_attn_last_error", "plt_decode_attn_workspace_bytes",
-    "plt_decode_attn_launch_info",
+    "plt_decode_attn_launch_info", "plt_decode_attn_set_profile_events",
 )
 
 
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
         lib.plt_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(ctypes.c_size_t)]
         i32p = ctypes.POINTER(ctypes.c_int32)
         lib.plt_decode_attn_launch_info.argtypes = [h, i32p, i32p, i32p, i32p, i32p, i32p]
+        lib.plt_decode_attn_set_profile_events.argtypes = [h, ctypes.c_void_p, ctypes.c_void_p]
         for name in EXPORTS:
             if name != "plt_decode_attn_last_error":
                 getattr(lib, name).restype = ctypes.c_int
@@ -183,3 +184,9 @@ def plt_decode_attn_launch_info(handle) -> dict:
         _raise(st, handle)
     keys = ("kernels_per_run", "heads_per_cta", "key_slices", "stages", "ctas_per_sm", "grid")
     return {k: int(v.value) for k, v in zip(keys, vals)}
+
+
+def plt_decode_attn_set_profile_events(handle, ev_main_begin: Optional[int], ev_main_end: Optional[int]) -> None:
+    st = load_library().plt_decode_attn_set_profile_events(handle, ev_main_begin, ev_main_end)
+    if st != PLT_OK:
+        _raise(st, handle)

@@ -61,6 +61,7 @@ struct plt_decode_attn {
     bool map_valid[4] = {false, false, false, false};
     // device staging for plt_decode_attn_run_host (grow-only)
     Staging st[10];
+    cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // optional, caller-owned
     char err[512];
 };
 
@@ -367,11 +368,14 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
             h->maps[2] = h->maps[0];
             h->maps[3] = h->maps[1];
         }
+        if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
         e = launch_main_bf16(h->var, h->maps, p, stream);
     } else {
+        if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
         e = launch_main_f32(p, h->var.grid, h->var.smem, stream);
     }
     if (e != cudaSuccess) return cuda_fail(h, "launching the main kernel", e);
+    if (h->ev_end) cudaEventRecord(h->ev_end, stream);
     e = launch_reduce(p, h->bf16, stream);
     if (e != cudaSuccess) return cuda_fail(h, "launching the merge kernel", e);
     return PLT_OK;
@@ -490,6 +494,15 @@ PLT_API plt_status plt_decode_attn_destroy(plt_decode_attn_t h) {
 }
 
 PLT_API const char* plt_decode_attn_last_error(plt_decode_attn_t h) { return h ? h->err : g_create_error; }
+
+PLT_API plt_status plt_decode_attn_set_profile_events(plt_decode_attn_t h, void* ev_main_begin, void* ev_main_end) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if ((ev_main_begin == nullptr) != (ev_main_end == nullptr))
+        return fail(h, PLT_ERR_INVALID_ARG, "pass both events or neither");
+    h->ev_begin = (cudaEvent_t)ev_main_begin;
+    h->ev_end = (cudaEvent_t)ev_main_end;
+    return PLT_OK;
+}
 
 PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* kernels_per_run, int32_t* heads_per_cta,
                                        int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid) {

@@ -121,7 +121,11 @@ def test_peaked_softmax_and_large_scores():
     p = make_problem(custom(B=2, L=2, lens=("list", [2000, 300]), peaks=0.02))
     assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", "peaks")
     big = p.with_(sm_scale=4.0)  # scores of magnitude ~50: softmax collapses onto a few keys
-    assert_parity(run_gpu(big), oracle.decode_attn(big), "bf16", "large scores")
+    got, ref = run_gpu(big), oracle.decode_attn(big)
+    # Outputs reach |O| ~ 7 here, where one bf16 output ulp is already 3e-2: bound the error relative to max(1, |O|).
+    assert np.isfinite(got).all()
+    assert (np.abs(got - ref) / np.maximum(1.0, np.abs(ref))).max() <= 2e-2
+    assert np.abs(got - ref).mean() <= 2e-3
 
 
 # ---- layouts ---------------------------------------------------------------------------------------------------
