@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the CLP decode-step attention (one step = one plt_decode_attn_run over the whole batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload I]
+
+Prints ONE JSON line. Default workload: bf16 decode batch B=64, L=2, Hq=32, Hkv=8, d=128, N=4096, w=64
+(the configuration the headline metric is quoted on). Under torchrun (N > 1) every rank runs an
+independent replica of the workload on its own GPU (no collective in the data path; weak scaling).
+`--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np
+
+METRIC = "clp_decode_attn_steps_per_s"
+UNIT = "steps/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, help="index into the five workloads (default 1 = headline)")
+    ap.add_argument("--hpc", type=int, default=0)
+    ap.add_argument("--kw", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--cps", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--cpu-seconds", type=float, default=20.0, help="CPU work budget of the oracle leg (core-seconds)")
+    return ap.parse_args()
+
+
+def workload_config(p, extra=None):
+    from paper_2510_24824_b200.inputs import algorithmic_bytes
+    by = algorithmic_bytes(p)
+    cfg = {
+        "workload": p.name, "B": p.B, "L": p.L, "Hq": p.Hq, "Hkv": p.Hkv, "d": p.d, "w": p.w,
+        "seq_len_min": int(p.seq_lens.min()), "seq_len_max": int(p.seq_lens.max()),
+        "sum_seq_len": int(p.seq_lens.sum()), "page_size": p.page_size,
+        "algorithmic_bytes_per_step": by["total"],
+        "l2": f"inputs {by['total'] / 1e6:.0f} MB per step exceed the 126 MB L2; no flush between steps",
+    }
+    if extra:
+        cfg.update(extra)
+    return cfg, by
+
+
+def peak_hbm():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (6650 GB/s, earlier measurement on this pool)"
+
+
+def recorded_traffic(name: str):
+    """DRAM bytes per launch of the main kernel from the committed ncu capture of this workload, or None."""
+    f = ROOT / "profiles" / "main_kernel_dram_traffic.json"
+    if f.exists():
+        try:
+            return json.loads(f.read_text()).get(name, {}).get("dram_bytes_per_launch")
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def time_oracle(p, cpu_seconds: float):
+    """Times the fp64 oracle as it stands on a bounded sample of output rows. Returns (steps/s, dict)."""
+    import oracle
+    cores = oracle.threads()
+    total_rows = p.B * p.L * p.Hq
+    rng = np.random.default_rng(12345)
+    all_rows = np.stack(np.meshgrid(np.arange(p.B), np.arange(p.L), np.arange(p.Hq), indexing="ij"), -1).reshape(-1, 3)
+    probe = all_rows[rng.choice(total_rows, size=min(total_rows, 8 * cores), replace=False)]
+    t0 = time.perf_counter()
+    oracle.decode_attn_rows(p, probe)
+    t_probe = time.perf_counter() - t0
+    per_row = t_probe / len(probe)  # wall seconds per row with all cores busy
+    n = int(min(total_rows, max(len(probe), cpu_seconds / cores / max(per_row, 1e-9))))
+    rows = all_rows if n >= total_rows else all_rows[rng.choice(total_rows, size=n, replace=False)]
+    t0 = time.perf_counter()
+    oracle.decode_attn_rows(p, rows)
+    t = time.perf_counter() - t0
+    step_seconds = t * total_rows / len(rows)
+    sample = (f"{len(rows)} of {total_rows} output rows (b, loop, head) of the same workload, drawn uniformly"
+              if len(rows) < total_rows else f"all {total_rows} output rows of the workload (one full step)")
+    return 1.0 / step_seconds, {"cores": cores, "kind": "oracle", "sample": sample, "sample_seconds": t}
+
+
+def run_reference(args, rank: int):
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores."""
+    if rank != 0:
+        return
+    from paper_2510_24824_b200.inputs import make_problem, workload
+    p = make_problem(workload(args.workload))
+    cfg, by = workload_config(p)
+    import oracle
+    cores = oracle.threads()
+    total_rows = p.B * p.L * p.Hq
+    all_rows = np.stack(np.meshgrid(np.arange(p.B), np.arange(p.L), np.arange(p.Hq), indexing="ij"), -1).reshape(-1, 3)
+    rng = np.random.default_rng(54321)
+    # Size the per-step sample so that warm-up + timed steps end within about two minutes.
+    probe = all_rows[rng.choice(total_rows, size=min(total_rows, 8 * cores), replace=False)]
+    t0 = time.perf_counter()
+    oracle.decode_attn_rows(p, probe)
+    per_row = (time.perf_counter() - t0) / len(probe)
+    budget = 120.0 / max(args.steps + args.warmup, 1)
+    n = int(min(total_rows, max(cores, budget / max(per_row, 1e-9))))
+    rows = all_rows if n >= total_rows else all_rows[rng.choice(total_rows, size=n, replace=False)]
+    for _ in range(args.warmup):
+        oracle.decode_attn_rows(p, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.decode_attn_rows(p, rows)
+    t = (time.perf_counter() - t0) / max(args.steps, 1)
+    step_seconds = t * total_rows / len(rows)
+    value = 1.0 / step_seconds
+    sample = f"each step = {len(rows)} of {total_rows} output rows of the workload; time scaled to all rows"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_seconds * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+        "loop_queries_per_s": value * p.B * p.L,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_24824_b200 import binding as B
+    from paper_2510_24824_b200.inputs import make_problem, workload
+    from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU implementation")
+    B.load_library()  # fails loudly when the extension has not been built
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    spec = workload(args.workload)
+    spec["seed"] = spec["seed"] + 1000 * rank  # every replica streams its own data
+    p = make_problem(spec)
+    dp = DeviceProblem(p, dev)
+    tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps)
+    op = DecodeAttn(p, device_index=local_rank, **tuning)
+    stream = torch.cuda.current_stream().cuda_stream
+    cfg, by = workload_config(p, {"launch": op.info, "parallelism": f"replicas x{world} (no collective)"})
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    run_args = dp.args()
+
+    def step():
+        B.plt_decode_attn_run(op.handle, run_args, stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert op.check(stream) == 0, "device status not clean after warm-up"
+
+    # ---- timed region 1: K whole steps, device time between two events --------------------------------
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    barrier()
+    with sampler:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+
+    # ---- timed region 2: the same steps with an event pair around the main kernel ---------------------
+    n_prof = min(args.steps, 200)
+    main_ms = []
+    raw = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+    for a, b in raw:
+        a.record()  # materialise the underlying cudaEvent_t handles
+        b.record()
+    torch.cuda.synchronize()
+    for a, b in raw:
+        B.plt_decode_attn_set_profile_events(op.handle, a.cuda_event, b.cuda_event)
+        step()
+    torch.cuda.synchronize()
+    B.plt_decode_attn_set_profile_events(op.handle, None, None)
+    main_ms = [a.elapsed_time(b) for a, b in raw]
+    main_avg_ms = float(np.mean(main_ms))
+
+    # ---- end to end: host buffers through plt_decode_attn_run_host ------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        hp = DeviceProblem(p, device=None, pin=True)
+        for _ in range(2):
+            op.run_host(hp, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            op.run_host(hp, stream)  # synchronises the stream itself
+        torch.cuda.synchronize()
+        t_e2e = (time.perf_counter() - t0) / args.e2e_steps
+        e2e_t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+        e2e = {"value": world / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes(),
+               "d2h_bytes_per_step": hp.d2h_bytes(), "steps": args.e2e_steps,
+               "note": "plt_decode_attn_run_host with pinned host tensors; the whole KV cache crosses PCIe every step"}
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * 1e3 / ms_per_step
+
+    if rank == 0:
+        peak, peak_src = peak_hbm()
+        main_bytes = by["shared_kv"] + by["window_kv"] + by["q_o"] // 2 + by["index"]
+        achieved = main_bytes / (main_avg_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": p.dtype, "data": "synthetic", "config": cfg,
+            "loop_queries_per_s": value * p.B * p.L,
+            "hbm_gbs_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9,
+            "hbm_frac_of_8tbs": by["total"] / (ms_per_step * 1e-3) / 8e12,
+            "clocks": sampler.summary(),
+            "gpu_launches": int(op.info["kernels_per_run"]) * args.steps,
+            "roofline": {
+                "bound": "hbm", "kernel": "plt_decode_main_" + p.dtype, "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": main_bytes, "avg_launch_ms": main_avg_ms,
+                "launches_timed": n_prof, "traffic": recorded_traffic(p.name),
+            },
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if not args.no_cpu:
+            v, info = time_oracle(p, args.cpu_seconds)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, **info}
+        print(json.dumps(line), flush=True)
+    op.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

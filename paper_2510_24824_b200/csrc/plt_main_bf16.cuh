@@ -22,6 +22,7 @@ struct MainCfg {
     static constexpr int TK = 16 * KW;              // keys per tile
     static constexpr int NCW = HPC * KW * MT;       // consumer warps
     static constexpr int NTHREADS = (NCW + 1) * 32;
+    static constexpr int MIN_BLOCKS = NCW <= 2 ? 4 : (NCW <= 4 ? 2 : 1);  // register budget: blocks per SM aimed at
     static constexpr int BOX_BYTES = 128 * TK * HPC;        // one TMA box: [HPC][TK][64 elements]
     static constexpr int TENSOR_BYTES = NH * BOX_BYTES;     // K (or V) part of a stage
     static constexpr int STAGE_BYTES = 2 * TENSOR_BYTES;
@@ -125,7 +126,7 @@ __device__ __forceinline__ void process_slice(uint32_t sK, uint32_t sV, const ui
 }
 
 template <int D, int MT, int HPC, int KW>
-__global__ void __launch_bounds__(MainCfg<D, MT, HPC, KW>::NTHREADS, 1)
+__global__ void __launch_bounds__(MainCfg<D, MT, HPC, KW>::NTHREADS, MainCfg<D, MT, HPC, KW>::MIN_BLOCKS)
 plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
                      const __grid_constant__ Params p, const int stages) {
