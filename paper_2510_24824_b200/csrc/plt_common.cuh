@@ -33,6 +33,9 @@ struct Params {
     float* part_ml;            // [slots][hpc][R][2]  running max (log2 units) and sum of p
     int32_t* prefix;           // [B + 1] tile prefix written by block 0 of the main kernel
     uint32_t* status;          // device status word
+#ifdef PLT_TIMELINE
+    void* timeline;            // [grid][8] u64, instrumentation builds only
+#endif
     int64_t kv_stride_b, kv_stride_n, kv_stride_h;  // elements
     int32_t B, L, Hq, Hkv, G, R, d, w;
     int32_t max_seq_len, page_size, max_pages, num_pool_pages;

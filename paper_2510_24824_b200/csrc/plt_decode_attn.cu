@@ -62,6 +62,9 @@ struct plt_decode_attn {
     // device staging for plt_decode_attn_run_host (grow-only)
     Staging st[10];
     cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // optional, caller-owned
+#ifdef PLT_TIMELINE
+    void* timeline = nullptr;
+#endif
     char err[512];
 };
 
@@ -140,8 +143,12 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
     const size_t budget = (size_t)(cps >= 2 ? 227 * 1024 / cps - 1024 : 227 * 1024);
     int stages = c->stages;
     if (stages == 0) {
-        stages = 2;
-        while (stages < 12 && main_bf16_smem(v->D, v->MT, hpc, kw, stages + 1, c->max_batch) <= budget) ++stages;
+        // About 128 KB of loads in flight per SM measured fastest on B200; more only delays the first data.
+        const size_t stage_bytes = main_bf16_smem(v->D, v->MT, hpc, kw, 3, c->max_batch) -
+                                   main_bf16_smem(v->D, v->MT, hpc, kw, 2, c->max_batch);
+        stages = (int)((128 * 1024) / (stage_bytes * (size_t)cps));
+        if (stages < 2) stages = 2;
+        while (stages > 2 && main_bf16_smem(v->D, v->MT, hpc, kw, stages, c->max_batch) > budget) --stages;
         if (stages > 8) stages = 8;
     }
     if (stages < 2 || stages > 12) return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [2, 12]", stages);
@@ -286,6 +293,10 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
     e = cudaMemset(h->status, 0, 4);
     if (e != cudaSuccess) { cudaFree(ws); delete h; return cuda_fail(nullptr, "cudaMemset", e); }
+#ifdef PLT_TIMELINE
+    cudaMalloc(&h->timeline, (size_t)h->var.grid * 64);
+    cudaMemset(h->timeline, 0, (size_t)h->var.grid * 64);
+#endif
     *out_handle = h;
     return PLT_OK;
 }
@@ -332,6 +343,9 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     p.seq_lens = a->seq_lens; p.win_lens = a->win_lens; p.page_table = a->page_table; p.gate_logits = a->gate_logits;
     p.out = a->out;
     p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.status = h->status;
+#ifdef PLT_TIMELINE
+    p.timeline = h->timeline;
+#endif
     p.kv_stride_b = sb; p.kv_stride_n = sn; p.kv_stride_h = sh;
     p.B = a->batch; p.L = c.L; p.Hq = c.Hq; p.Hkv = c.Hkv; p.G = h->G; p.R = h->R; p.d = c.d; p.w = c.w;
     p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
@@ -517,3 +531,11 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
 }
 
 }  // extern "C"
+
+#ifdef PLT_TIMELINE
+extern "C" PLT_API int plt_debug_timeline(plt_decode_attn_t h, unsigned long long* host, int max_ctas) {
+    int n = h->var.grid < max_ctas ? h->var.grid : max_ctas;
+    cudaMemcpy(host, h->timeline, (size_t)n * 64, cudaMemcpyDeviceToHost);
+    return n;
+}
+#endif

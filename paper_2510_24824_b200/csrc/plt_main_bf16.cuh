@@ -143,6 +143,15 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
     bool ok = true;
+#ifdef PLT_TIMELINE
+    unsigned long long* tl = (unsigned long long*)p.timeline + (size_t)blockIdx.x * 8;
+    if (tid == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        tl[0] = smid;
+        tl[1] = global_timer_ns();
+    }
+#endif
 
     if (tid == 0) {
         s_ctl[0] = 0;
@@ -159,6 +168,10 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
     if (cta == 0)
         for (int b = tid; b <= p.B; b += C::NTHREADS) p.prefix[b] = s_prefix[b];
     const int64_t lo = cta_begin(T, cta, nctas), hi = cta_begin(T, cta + 1, nctas);
+#ifdef PLT_TIMELINE
+    if (tid == 0) { tl[2] = global_timer_ns(); tl[7] = (unsigned long long)(hi - lo); }
+    bool tl_first = true;
+#endif
 
     if (wid == C::NCW) {
         // =========================== producer warp (one lane issues) ==============================
@@ -208,6 +221,9 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         ok = mbar_wait_bounded(&empty_bar[stage], (use - 1) & 1, kWaitLimitNs);
                         if (!ok) flags |= kDevWaitTimeout;
                     }
+#ifdef PLT_TIMELINE
+                    if (tl_first) { tl[3] = global_timer_ns(); tl_first = false; }
+#endif
                     if (ok) {
                         uint8_t* dst = smem + (size_t)stage * C::STAGE_BYTES;
                         mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
@@ -279,6 +295,10 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     ok = mbar_wait_bounded(&full_bar[stage], use & 1, kWaitLimitNs);
                     if (!ok) flags |= kDevWaitTimeout;
                 }
+#ifdef PLT_TIMELINE
+                if (tl_first && tid == 0) { tl[4] = global_timer_ns(); }
+                tl_first = false;
+#endif
                 const uint32_t sK = smem_u32(smem + (size_t)stage * C::STAGE_BYTES);
                 const uint32_t sV = sK + C::TENSOR_BYTES;
                 if (pc.kind == 0) {
@@ -394,9 +414,15 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
         }
     }
+#ifdef PLT_TIMELINE
+    if (tid == 0) tl[5] = global_timer_ns();
+#endif
     if (flags) atomicOr(p.status, flags);
     if (flags & kDevWaitTimeout) s_ctl[0] = 1;
     __syncthreads();
+#ifdef PLT_TIMELINE
+    if (tid == 0) tl[6] = global_timer_ns();
+#endif
     // A wait ran out somewhere: before the block retires, give every copy that was issued a bounded
     // chance to land (in the normal path the consumers have waited for all of them already).
     if (s_ctl[0] != 0 && tid == 0) {

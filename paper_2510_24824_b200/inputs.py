@@ -5,8 +5,9 @@ types.  It contains none of the attention arithmetic and is the one piece of
 code that both the tests' CPU oracle and the CUDA binding are fed from.
 
 Recipe: numpy ``default_rng(seed)``, draw order fixed: ``Q, lens, page permutation,
-(K, V) per sequence, Kwin, Vwin, gate``; the positions of sharp peaks come from a
-second stream ``default_rng([seed, 1])`` (per sequence, then the windows).
+Kwin, Vwin, gate``; the shared cache of sequence ``b`` comes from its own stream
+``default_rng([seed, 2, b])`` (K, then V, then the positions of its sharp peaks), and the
+peak positions of the windows from ``default_rng([seed, 1])``.
 All values are drawn in float32 and, for bf16 problems, rounded to bfloat16
 (round-to-nearest-even) and kept as uint16 bit patterns, so that every consumer
 sees exactly the same stored values.
@@ -14,6 +15,8 @@ sees exactly the same stored values.
 from __future__ import annotations
 
 import math
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field, replace
 from typing import Optional
 
@@ -213,27 +216,30 @@ def make_problem(spec: dict, seed: Optional[int] = None, tail_fill: Optional[flo
         P = int(pages_per_seq.sum()) + int(spec.get("spare_pages", 3))
         perm = rng.permutation(P).astype(np.int32)
         page_table = np.zeros((B, cap // page), dtype=np.int32)
-        k_cache = np.full((P, page, Hkv, d), fill, dtype=st)
-        v_cache = np.full((P, page, Hkv, d), fill, dtype=st)
+        shape = (P, page, Hkv, d)
     else:
-        k_cache = np.full((B, cap, Hkv, d), fill, dtype=st)
-        v_cache = np.full((B, cap, Hkv, d), fill, dtype=st)
-    nxt = 0
-    for b in range(B):
+        shape = (B, cap, Hkv, d)
+    if fill == 0:
+        k_cache, v_cache = np.zeros(shape, dtype=st), np.zeros(shape, dtype=st)
+    else:
+        k_cache, v_cache = np.full(shape, fill, dtype=st), np.full(shape, fill, dtype=st)
+    starts = np.concatenate([[0], np.cumsum(pages_per_seq)]) if page else None
+
+    def fill_sequence(b: int) -> None:
+        # Sequence b draws from its own stream (seed, 2, b), so sequences can be generated concurrently.
         n = int(lens[b])
-        kb = rng.standard_normal((n, Hkv, d), dtype=np.float32)
-        vb = rng.standard_normal((n, Hkv, d), dtype=np.float32)
+        rb = np.random.default_rng([seed, 2, b])
+        kb = rb.standard_normal((n, Hkv, d), dtype=np.float32)
+        vb = rb.standard_normal((n, Hkv, d), dtype=np.float32)
         if peaks:
             # Sharp softmax peaks: a Bernoulli(peaks) set of token positions has its K and V rows (all heads) tripled.
-            hot = rng_peaks.random(n) < peaks
+            hot = rb.random(n) < peaks
             kb[hot] *= 3.0
             vb[hot] *= 3.0
         kb, vb = _store(kb, dtype), _store(vb, dtype)
         if page:
-            npg = int(pages_per_seq[b])
-            ids = perm[nxt:nxt + npg]
-            nxt += npg
-            page_table[b, :npg] = ids
+            ids = perm[int(starts[b]):int(starts[b + 1])]
+            page_table[b, :len(ids)] = ids
             for i, pid in enumerate(ids):
                 lo, hi = i * page, min((i + 1) * page, n)
                 k_cache[pid, : hi - lo] = kb[lo:hi]
@@ -241,6 +247,14 @@ def make_problem(spec: dict, seed: Optional[int] = None, tail_fill: Optional[flo
         else:
             k_cache[b, :n] = kb
             v_cache[b, :n] = vb
+
+    workers = min(B, os.cpu_count() or 1, 16)
+    if workers > 1:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(fill_sequence, range(B)))
+    else:
+        for b in range(B):
+            fill_sequence(b)
 
     k_win_f = rng.standard_normal((B, Lm, w, Hkv, d), dtype=np.float32)
     v_win_f = rng.standard_normal((B, Lm, w, Hkv, d), dtype=np.float32)
