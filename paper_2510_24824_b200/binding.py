@@ -190,3 +190,4 @@ def plt_decode_attn_set_profile_events(handle, ev_main_begin: Optional[int], ev_
     st = load_library().plt_decode_attn_set_profile_events(handle, ev_main_begin, ev_main_end)
     if st != PLT_OK:
         _raise(st, handle)
+

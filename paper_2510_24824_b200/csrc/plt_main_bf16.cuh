@@ -85,9 +85,14 @@ __device__ __forceinline__ void process_slice(uint32_t sK, uint32_t sV, const ui
         const float p01 = fast_exp2(fmaf(s[0][2 * i + 1], scale_log2, -m_use));
         const float p10 = fast_exp2(fmaf(s[1][2 * i], scale_log2, -m_use));
         const float p11 = fast_exp2(fmaf(s[1][2 * i + 1], scale_log2, -m_use));
-        lsum[i] = fmaf(lsum[i], alpha, (p00 + p01) + (p10 + p11));
         pa[i] = pack_bf16x2(p00, p01);       // keys 2tq, 2tq+1
         pa[2 + i] = pack_bf16x2(p10, p11);   // keys 8 + 2tq, 9 + 2tq
+        // The denominator sums the probabilities as rounded to bf16, i.e. exactly the weights the P V
+        // product uses: numerator and denominator then carry the same rounding, which cancels when a few
+        // keys dominate the softmax.
+        const float r00 = __uint_as_float(pa[i] << 16), r01 = __uint_as_float(pa[i] & 0xffff0000u);
+        const float r10 = __uint_as_float(pa[2 + i] << 16), r11 = __uint_as_float(pa[2 + i] & 0xffff0000u);
+        lsum[i] = fmaf(lsum[i], alpha, (r00 + r01) + (r10 + r11));
 #pragma unroll
         for (int nd = 0; nd < D / 8; ++nd) {
             acc[nd][2 * i] *= alpha;

@@ -26,12 +26,15 @@ __device__ __forceinline__ float merge_item(const Params& p, int item, int hl, i
     const int c0 = cta_of(T, s, p.num_ctas), c1 = cta_of(T, e - 1, p.num_ctas);
     float mstar = -INFINITY;
     for (int c = c0; c <= c1; ++c) {
+        // With fewer tiles than blocks some blocks in between own nothing and wrote no partial.
+        if (cta_begin(T, c, p.num_ctas) == cta_begin(T, c + 1, p.num_ctas)) continue;
         const int64_t row = (slot_of(item, c) * p.hpc + hl) * p.R + r;
         mstar = fmaxf(mstar, p.part_ml[row * 2]);
     }
     if (mstar == -INFINITY) return 0.f;  // no visible key anywhere
     float denom = 0.f;
     for (int c = c0; c <= c1; ++c) {
+        if (cta_begin(T, c, p.num_ctas) == cta_begin(T, c + 1, p.num_ctas)) continue;
         const int64_t row = (slot_of(item, c) * p.hpc + hl) * p.R + r;
         const float2 ml = *(const float2*)(p.part_ml + row * 2);
         const float sc = exp2f(ml.x - mstar);  // exp2f(-inf) = 0 for pieces that saw nothing

@@ -8,7 +8,7 @@ import oracle
 from paper_2510_24824_b200.inputs import make_problem, workload
 from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
 
-from gpu_util import BF16_MAX_ABS, BF16_MEAN_ABS
+from gpu_util import BF16_MEAN_ABS, bf16_bound
 
 pytestmark = pytest.mark.gpu
 
@@ -35,7 +35,7 @@ def test_full_size_sampled_rows(index):
     got = dp.out.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     # convexity: every output lies within the range of the values it can mix
-    vmax = float(max(np.abs(dp.v_cache.float()).max().item(), np.abs(dp.v_win.float()).max().item()))
+    vmax = float(max(dp.v_cache.float().abs().max().item(), dp.v_win.float().abs().max().item()))
     assert np.abs(got).max() <= vmax * (1 + 2 ** -7)
     inactive = p.cuts() == 0
     assert np.all(got[inactive] == 0.0)
@@ -51,5 +51,5 @@ def test_full_size_sampled_rows(index):
     ref = oracle.decode_attn_rows(p, rows)
     sel = got[rows[:, 0], rows[:, 1], rows[:, 2]]
     err = np.abs(sel - ref)
-    assert err.max() <= BF16_MAX_ABS, f"{p.name}: max abs err {err.max():.3e}"
+    assert (err / bf16_bound(ref)).max() <= 1.0, f"{p.name}: max abs err {err.max():.3e}"
     assert err.mean() <= BF16_MEAN_ABS, f"{p.name}: mean abs err {err.mean():.3e}"
