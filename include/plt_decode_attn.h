@@ -161,6 +161,35 @@ plt_status plt_decode_attn_launch_info(plt_decode_attn_t handle, int32_t* kernel
  * the run's stream, so that the caller can time that kernel apart from the merge kernel. NULL, NULL switches it off. */
 plt_status plt_decode_attn_set_profile_events(plt_decode_attn_t handle, void* ev_main_begin, void* ev_main_end);
 
+/*
+ * plt_decode_attn_run_no_alloc - the same decode-step attention for callers that cannot allocate device memory.
+ * (An addition of this library; the paper has no counterpart.)
+ *
+ * Who needs it: a serving process that has given every byte of HBM to its KV cache and has no allocator left to
+ * ask, code that must not trigger the device-wide synchronisation a cudaMalloc implies, or a plug-in that is
+ * handed tensors without the right to create device buffers. Such callers skip plt_decode_attn_create: this call
+ * takes the configuration and the per-call arguments together and keeps its scratch (split partials, tile prefix,
+ * status word) in a device array compiled into the library, PLT_NO_ALLOC_SCRATCH_BYTES large, which every
+ * process that loads the library holds on each GPU it touches until the process exits.
+ *
+ * - It never calls cudaMalloc, cudaFree or any allocating routine. `args` is as for plt_decode_attn_run
+ *   (device pointers owned by the caller; `out` fully overwritten); `config` as for plt_decode_attn_create.
+ * - config->device must be the current device of the calling thread.
+ * - A configuration whose scratch (it grows with max_batch * Hkv * L * Hq/Hkv * d; ask
+ *   plt_decode_attn_workspace_bytes) exceeds the array is refused with PLT_ERR_CAPACITY and a message that states
+ *   both sizes. Set max_batch to the batch actually used.
+ * - The first call on a device looks up the array's device address and prepares the kernels; make that first
+ *   call outside any stream capture. Later calls with the same configuration reuse the prepared state.
+ * - All calls on one device share the one array, which keeps what the previous call left. The call clears the
+ *   part that must start at zero (the status word) itself. Two calls whose GPU work overlaps (different streams,
+ *   or different host threads) race on the partials: keep calls on a device stream-ordered and issue them from
+ *   one thread at a time.
+ * - Errors are reported like those of create: plt_decode_attn_last_error(NULL) holds the message.
+ */
+#define PLT_NO_ALLOC_SCRATCH_BYTES (16u << 20)
+plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn_config* config, const plt_decode_attn_args* args,
+                                        void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,8 +21,9 @@ PLT_DEV_SEQ_LEN_CLAMPED, PLT_DEV_PAGE_ID_CLAMPED, PLT_DEV_WAIT_TIMEOUT, PLT_DEV_
 EXPORTS = (
     "plt_decode_attn_create", "plt_decode_attn_run", "plt_decode_attn_run_host", "plt_decode_attn_check",
     "plt_decode_attn_destroy", "plt_decode_attn_last_error", "plt_decode_attn_workspace_bytes",
-    "plt_decode_attn_launch_info", "plt_decode_attn_set_profile_events",
+    "plt_decode_attn_launch_info", "plt_decode_attn_set_profile_events", "plt_decode_attn_run_no_alloc",
 )
+PLT_NO_ALLOC_SCRATCH_BYTES = 16 << 20
 
 
 class PltError(RuntimeError):
@@ -77,6 +78,7 @@ def load_library() -> ctypes.CDLL:
         i32p = ctypes.POINTER(ctypes.c_int32)
         lib.plt_decode_attn_launch_info.argtypes = [h, i32p, i32p, i32p, i32p, i32p, i32p]
         lib.plt_decode_attn_set_profile_events.argtypes = [h, ctypes.c_void_p, ctypes.c_void_p]
+        lib.plt_decode_attn_run_no_alloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Args), ctypes.c_void_p]
         for name in EXPORTS:
             if name != "plt_decode_attn_last_error":
                 getattr(lib, name).restype = ctypes.c_int
@@ -191,3 +193,10 @@ def plt_decode_attn_set_profile_events(handle, ev_main_begin: Optional[int], ev_
     if st != PLT_OK:
         _raise(st, handle)
 
+
+def plt_decode_attn_run_no_alloc(config: Config, args: Args, stream: int = 0) -> None:
+    """The decode-step attention without a handle and without any device allocation (scratch is built into the
+    library). For callers that may not allocate; config.device must be the current device."""
+    st = load_library().plt_decode_attn_run_no_alloc(ctypes.byref(config), ctypes.byref(args), ctypes.c_void_p(stream))
+    if st != PLT_OK:
+        _raise(st, None)

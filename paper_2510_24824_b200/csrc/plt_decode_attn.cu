@@ -539,3 +539,154 @@ extern "C" PLT_API int plt_debug_timeline(plt_decode_attn_t h, unsigned long lon
     return n;
 }
 #endif
+
+// ===================================================================================================
+// Allocation-free entry point.
+//
+// Some callers are not allowed to allocate device memory at the moment they need this attention:
+// code that runs inside a memory-budgeted serving process whose allocator has handed every byte of
+// HBM to the KV cache, code called from a context where cudaMalloc's implicit device synchronisation
+// is unacceptable, or a plug-in that is given tensors but no right to create any. For them the split
+// partials, the tile prefix and the status word live in one file-scope device array of fixed size,
+// which every process that loads this library holds on each GPU it uses until it exits.
+// ===================================================================================================
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = PLT_NO_ALLOC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_no_alloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+
+struct NoAllocDevice {
+    bool ready = false;          // set-up done for this device
+    void* scratch = nullptr;     // DEVICE address of g_no_alloc_scratch on this device
+    int sm_count = 0;
+    EncodeTiledFn encode = nullptr;
+    bool have_handle = false;    // `handle` is prepared for `cfg`
+    plt_decode_attn_config cfg;
+    int32_t offsets[kMaxLoops];
+    plt_decode_attn handle;      // host-side state only; its workspace pointers point into `scratch`
+};
+
+NoAllocDevice g_no_alloc[kNoAllocMaxDevices];
+
+// Once per device, with that device current: take the device address of the scratch array. In host
+// code the array's name is only a stand-in for the symbol; a kernel must be given this address.
+plt_status no_alloc_setup(NoAllocDevice& dv, int device) {
+    if (dv.ready) return PLT_OK;
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_no_alloc_scratch);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetSymbolAddress(scratch)", e);
+    if (ptr == nullptr || ((uintptr_t)ptr & 255u) != 0)
+        return fail(nullptr, PLT_ERR_CUDA, "scratch symbol address %p is null or not 256-byte aligned", ptr);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDeviceProperties", e);
+    if (prop.major != 10)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only", device,
+                    prop.major, prop.minor);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess)
+        return fail(nullptr, PLT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    dv.scratch = ptr;
+    dv.sm_count = prop.multiProcessorCount;
+    dv.encode = (EncodeTiledFn)fn;
+    dv.ready = true;
+    return PLT_OK;
+}
+
+bool same_config(const NoAllocDevice& dv, const plt_decode_attn_config* c) {
+    plt_decode_attn_config a = dv.cfg, b = *c;
+    a.loop_offset = nullptr;
+    b.loop_offset = nullptr;
+    if (memcmp(&a, &b, sizeof a) != 0) return false;
+    for (int l = 0; l < c->L; ++l)
+        if ((c->loop_offset ? c->loop_offset[l] : l) != dv.offsets[l]) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" PLT_API plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn_config* config,
+                                                           const plt_decode_attn_args* args, void* cuda_stream) {
+    Geometry g;
+    plt_status s = check_config(config, &g);
+    if (s != PLT_OK) return s;
+    int current = -1;
+    cudaError_t e = cudaGetDevice(&current);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaGetDevice", e);
+    if (current != config->device)
+        return fail(nullptr, PLT_ERR_INVALID_ARG, "config.device %d is not the current device %d", config->device, current);
+    if (current < 0 || current >= kNoAllocMaxDevices)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "device ordinal %d beyond %d", current, kNoAllocMaxDevices - 1);
+    NoAllocDevice& dv = g_no_alloc[current];
+    s = no_alloc_setup(dv, current);
+    if (s != PLT_OK) return s;
+
+    plt_decode_attn* h = &dv.handle;
+    if (!dv.have_handle || !same_config(dv, config)) {
+        // Prepare the host-side state for this configuration: the same choices create makes, minus cudaMalloc.
+        dv.have_handle = false;
+        h->cfg = *config;
+        h->cfg.loop_offset = nullptr;
+        for (int l = 0; l < kMaxLoops; ++l) h->delta[l] = config->loop_offset && l < config->L ? config->loop_offset[l] : l;
+        h->G = g.G;
+        h->R = g.R;
+        h->bf16 = config->dtype == PLT_BF16;
+        h->sm_count = dv.sm_count;
+        const float scale = config->sm_scale > 0.f ? config->sm_scale : 1.0f / sqrtf((float)config->d);
+        h->scale_log2 = scale * 1.4426950408889634f;
+        h->err[0] = 0;
+        h->encode = dv.encode;
+        for (bool& v : h->map_valid) v = false;
+        int blocks = 0;
+        if (h->bf16) {
+            int cps = 0;
+            s = choose_variant(config, g, &h->var, &cps);
+            if (s != PLT_OK) return s;
+            e = main_bf16_prepare(h->var, &blocks);
+            if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the bf16 main kernel", e);
+            if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
+            h->ctas_per_sm = blocks < cps ? blocks : cps;
+        } else {
+            h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
+            e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
+            if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the fp32 main kernel", e);
+            if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM");
+            const int cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
+            h->ctas_per_sm = blocks < cps ? blocks : cps;
+        }
+        h->var.grid = h->sm_count * h->ctas_per_sm;
+        const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+        const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
+                             ((double)(config->max_seq_len + tk - 1) / tk +
+                              (double)(config->L - 1) * ((config->w + tk - 1) / tk));
+        if (tiles >= 2147483647.0) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan");
+        size_t acc_floats, ml_floats;
+        h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
+        if (h->ws_bytes > kNoAllocScratchBytes)
+            return fail(nullptr, PLT_ERR_CAPACITY,
+                        "this configuration needs %zu bytes of scratch but the built-in array holds %zu: lower max_batch "
+                        "(scratch grows with max_batch * Hkv * L * Hq/Hkv * d) or use plt_decode_attn_create",
+                        h->ws_bytes, kNoAllocScratchBytes);
+        h->part_acc = (float*)dv.scratch;
+        h->part_ml = h->part_acc + acc_floats;
+        h->prefix = (int32_t*)(h->part_ml + ml_floats);
+        h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
+        dv.cfg = *config;
+        for (int l = 0; l < kMaxLoops; ++l) dv.offsets[l] = h->delta[l];
+        dv.have_handle = true;
+    }
+    // The array keeps whatever the previous call left. Partials and the prefix are rewritten before they are
+    // read; only the status word must start at zero.
+    e = cudaMemsetAsync(h->status, 0, 4, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "cudaMemsetAsync(status)", e);
+    s = plt_decode_attn_run(h, args, cuda_stream);
+    if (s != PLT_OK) {
+        snprintf(g_create_error, sizeof g_create_error, "%s", h->err);
+        return s;
+    }
+    return PLT_OK;
+}
