@@ -137,6 +137,30 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def replica_spec(index: int, rank: int) -> dict:
+    """Workload of one replica: every rank streams its own data (seed offset by rank), same shapes."""
+    from paper_2510_24824_b200.inputs import workload
+    spec = workload(index)
+    spec["seed"] = spec["seed"] + 1000 * rank
+    return spec
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Slowest rank's time: all-reduce MAX over the default process group (identity for one rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_steps_per_s(world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas that each did one step per ms_per_step."""
+    return world * 1e3 / ms_per_step
+
+
 def physical_gpu_index(local_index: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -234,9 +258,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    spec = workload(args.workload)
-    spec["seed"] = spec["seed"] + 1000 * rank  # every replica streams its own data
-    p = make_problem(spec)
+    p = make_problem(replica_spec(args.workload, rank))
     dp = DeviceProblem(p, dev)
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps)
     op = DecodeAttn(p, device_index=local_rank, **tuning)
@@ -299,19 +321,14 @@ def main():
             op.run_host(hp, stream)  # synchronises the stream itself
         torch.cuda.synchronize()
         t_e2e = (time.perf_counter() - t0) / args.e2e_steps
-        e2e_t = torch.tensor([t_e2e], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-        e2e = {"value": world / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes(),
+        t_e2e = max_over_ranks(t_e2e, world, dev)
+        e2e = {"value": job_steps_per_s(world, t_e2e * 1e3), "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes(),
                "d2h_bytes_per_step": hp.d2h_bytes(), "steps": args.e2e_steps,
                "note": "plt_decode_attn_run_host with pinned host tensors; the whole KV cache crosses PCIe every step"}
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
-    value = world * 1e3 / ms_per_step
+    value = job_steps_per_s(world, ms_per_step)
 
     if rank == 0:
         peak, peak_src = peak_hbm()
