@@ -102,6 +102,10 @@ __device__ __forceinline__ int32_t seq_tiles(const Params& p, int b, uint32_t& f
     return (p.Hkv / p.hpc) * (s.gt + s.lt);
 }
 
+// Blocks that take part in the plan: never more than there are tiles, so that every taking-part
+// block owns at least one tile and the blocks of one item are consecutive.
+__device__ __forceinline__ int plan_ctas(int64_t T, int launched) { return T < launched ? (int)T : launched; }
+
 // Range of the tile line owned by block c of C: [c*T/C, (c+1)*T/C).
 __device__ __forceinline__ int64_t cta_begin(int64_t T, int c, int C) { return (T * c) / C; }
 

@@ -390,7 +390,8 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     }
     if (e != cudaSuccess) return cuda_fail(h, "launching the main kernel", e);
     if (h->ev_end) cudaEventRecord(h->ev_end, stream);
-    e = launch_reduce(p, h->bf16, stream);
+    // The merge kernel may set up while the main kernel drains, unless an event sits between the two launches.
+    e = launch_reduce(p, h->bf16, /*overlap=*/h->ev_end == nullptr, stream);
     if (e != cudaSuccess) return cuda_fail(h, "launching the merge kernel", e);
     return PLT_OK;
 }

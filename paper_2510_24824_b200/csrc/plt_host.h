@@ -29,6 +29,6 @@ size_t main_f32_smem(int D, int R, int max_batch);
 cudaError_t main_f32_prepare(int D, int R, int max_batch, int* blocks_per_sm);
 cudaError_t launch_main_f32(const Params& p, int grid, size_t smem, cudaStream_t stream);
 
-cudaError_t launch_reduce(const Params& p, bool bf16, cudaStream_t stream);
+cudaError_t launch_reduce(const Params& p, bool bf16, bool overlap, cudaStream_t stream);
 
 }  // namespace plt

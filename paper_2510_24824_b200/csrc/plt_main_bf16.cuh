@@ -167,12 +167,14 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         mbar_fence_init();
     }
+    grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags);  // contains __syncthreads
     const int64_t T = s_prefix[p.B];
-    const int cta = blockIdx.x, nctas = gridDim.x;
+    const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
     if (cta == 0)
         for (int b = tid; b <= p.B; b += C::NTHREADS) p.prefix[b] = s_prefix[b];
-    const int64_t lo = cta_begin(T, cta, nctas), hi = cta_begin(T, cta + 1, nctas);
+    const bool in_plan = cta < nctas;
+    const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
 #ifdef PLT_TIMELINE
     if (tid == 0) { tl[2] = global_timer_ns(); tl[7] = (unsigned long long)(hi - lo); }
     bool tl_first = true;

@@ -5,6 +5,7 @@
 // memory so that every K/V tile is read from global memory once for all loops.
 #include "plt_common.cuh"
 #include "plt_host.h"
+#include "plt_ptx.cuh"
 
 namespace plt {
 
@@ -39,12 +40,15 @@ __global__ void __launch_bounds__(NT) plt_decode_main_f32(const __grid_constant_
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int R = p.R;
     uint32_t flags = 0;
+    grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags);
     const int64_t T = s_prefix[p.B];
     const int cta = blockIdx.x;
     if (cta == 0)
         for (int b = tid; b <= p.B; b += NT) p.prefix[b] = s_prefix[b];
-    const int64_t lo = cta_begin(T, cta, gridDim.x), hi = cta_begin(T, cta + 1, gridDim.x);
+    const int nctas = plan_ctas(T, (int)gridDim.x);
+    const bool in_plan = cta < nctas;
+    const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
 
     const float* kc = (const float*)p.k_cache;
     const float* vc = (const float*)p.v_cache;

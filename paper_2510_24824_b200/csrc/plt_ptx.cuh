@@ -84,6 +84,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// In a kernel launched with programmatic stream serialisation: blocks until the kernel before it in
+// the stream has completed and its writes are visible. A no-op for an ordinary launch.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream, if it was launched with programmatic stream serialisation,
+// start setting up its blocks once every block of this grid has passed this point (or exited).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- math --------------------------------------------------------------------------------------
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;

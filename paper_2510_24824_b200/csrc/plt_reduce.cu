@@ -2,13 +2,24 @@
 // attention (y_global, Algorithm 3 line 2) and of the window attention (y_local, line 3) by their
 // running maxima, normalises each, and applies the sigmoid gate mix of Eq. 2 (lines 4-5):
 //   O = g * y_local + (1 - g) * y_global for loops 2..L,  O = y_global for loop 1.
-// One warp per output row (b, l, h).
+// One block per (sequence, KV-head group, chunk of 8 packed rows); one warp per output row. The
+// first warp works out once per block which blocks of the main kernel hold pieces of the two items.
 #include <cuda_bf16.h>
 
 #include "plt_common.cuh"
 #include "plt_host.h"
+#include "plt_ptx.cuh"
 
 namespace plt {
+
+namespace {
+
+constexpr int kReduceWarps = 8;
+
+struct ReduceCtl {
+    int32_t c0[2], c1[2];        // first and last main-kernel block of the shared-cache item [0] and the windows item [1]
+    int32_t cut[kMaxLoops];
+};
 
 template <int D>
 struct Vec {
@@ -16,72 +27,108 @@ struct Vec {
     float v[N];
 };
 
-// Sum over the pieces [s, e) of one item, rescaled to a common maximum. Returns the denominator.
 template <int D>
-__device__ __forceinline__ float merge_item(const Params& p, int item, int hl, int r, int64_t T, int64_t s, int64_t e,
-                                            int lane, Vec<D>& y) {
+__device__ __forceinline__ void load_vec(const float* src, Vec<D>& x) {
+    if constexpr (Vec<D>::N == 4) {
+        const float4 t = *(const float4*)src;
+        x.v[0] = t.x; x.v[1] = t.y; x.v[2] = t.z; x.v[3] = t.w;
+    } else {
+        const float2 t = *(const float2*)src;
+        x.v[0] = t.x; x.v[1] = t.y;
+    }
+}
+
+// Sum over the pieces held by blocks [c0, c1] of one item, rescaled to a common maximum. Returns the denominator.
+template <int D>
+__device__ __forceinline__ float merge_item(const Params& p, int item, int hl, int r, int c0, int c1, int lane,
+                                            Vec<D>& y) {
 #pragma unroll
     for (int i = 0; i < Vec<D>::N; ++i) y.v[i] = 0.f;
-    if (s >= e) return 0.f;
-    const int c0 = cta_of(T, s, p.num_ctas), c1 = cta_of(T, e - 1, p.num_ctas);
-    float mstar = -INFINITY;
-    for (int c = c0; c <= c1; ++c) {
-        // With fewer tiles than blocks some blocks in between own nothing and wrote no partial.
-        if (cta_begin(T, c, p.num_ctas) == cta_begin(T, c + 1, p.num_ctas)) continue;
-        const int64_t row = (slot_of(item, c) * p.hpc + hl) * p.R + r;
-        mstar = fmaxf(mstar, p.part_ml[row * 2]);
+    if (c0 > c1) return 0.f;
+    const int64_t row0 = (slot_of(item, c0) * p.hpc + hl) * p.R + r;
+    const int64_t step = (int64_t)p.hpc * p.R;  // rows between the slots of consecutive blocks
+    if (c0 == c1) {
+        // The usual case: the whole item was done by one block, nothing to rescale.
+        const float2 ml = *(const float2*)(p.part_ml + row0 * 2);
+        if (ml.x == -INFINITY) return 0.f;
+        load_vec<D>(p.part_acc + row0 * D + lane * Vec<D>::N, y);
+        return ml.y;
     }
+    float mstar = -INFINITY;
+    for (int c = c0; c <= c1; ++c) mstar = fmaxf(mstar, p.part_ml[(row0 + (c - c0) * step) * 2]);
     if (mstar == -INFINITY) return 0.f;  // no visible key anywhere
     float denom = 0.f;
     for (int c = c0; c <= c1; ++c) {
-        if (cta_begin(T, c, p.num_ctas) == cta_begin(T, c + 1, p.num_ctas)) continue;
-        const int64_t row = (slot_of(item, c) * p.hpc + hl) * p.R + r;
+        const int64_t row = row0 + (c - c0) * step;
         const float2 ml = *(const float2*)(p.part_ml + row * 2);
         const float sc = exp2f(ml.x - mstar);  // exp2f(-inf) = 0 for pieces that saw nothing
         denom = fmaf(ml.y, sc, denom);
-        const float* a = p.part_acc + row * D + lane * Vec<D>::N;
+        Vec<D> a;
+        load_vec<D>(p.part_acc + row * D + lane * Vec<D>::N, a);
 #pragma unroll
-        for (int i = 0; i < Vec<D>::N; ++i) y.v[i] = fmaf(a[i], sc, y.v[i]);
+        for (int i = 0; i < Vec<D>::N; ++i) y.v[i] = fmaf(a.v[i], sc, y.v[i]);
     }
     return denom;
 }
 
 template <int D, bool BF16>
-__global__ void __launch_bounds__(128) plt_decode_reduce(const __grid_constant__ Params p) {
-    const int lane = threadIdx.x & 31;
-    const int64_t row_id = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (row_id >= (int64_t)p.B * p.L * p.Hq) return;
-    const int h = (int)(row_id % p.Hq);
-    const int l = (int)((row_id / p.Hq) % p.L);
-    const int b = (int)(row_id / ((int64_t)p.Hq * p.L));
-    const int kvh = h / p.G, g = h - kvh * p.G;
-    const int hg = kvh / p.hpc, hl = kvh - hg * p.hpc;
-    const int r = l * p.G + g;
+__global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __grid_constant__ Params p, const int chunks) {
+    __shared__ ReduceCtl ctl;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int HG = p.Hkv / p.hpc;
+    const int chunk = (int)(blockIdx.x % chunks);
+    const int hg = (int)((blockIdx.x / chunks) % HG);
+    const int b = (int)(blockIdx.x / (chunks * HG));
 
-    uint32_t flags = 0;
-    SeqPlan sp;
-    seq_plan(p, b, sp, flags);
-    const int64_t T = p.prefix[p.B];
-    const int per = sp.gt + sp.lt;
-    const int64_t base = (int64_t)p.prefix[b] + (int64_t)hg * per;
+    // Everything above depends on the launch only; from here on the main kernel's results are read.
+    grid_dependency_wait();
+
+    if (wid == 0) {
+        uint32_t flags = 0;
+        SeqPlan sp;
+        seq_plan(p, b, sp, flags);
+        const int64_t T = p.prefix[p.B];
+        const int nctas = plan_ctas(T, p.num_ctas);
+        const int per = sp.gt + sp.lt;
+        const int64_t base = (int64_t)p.prefix[b] + (int64_t)hg * per;
+        if (lane < 4) {
+            // lane 0/1: first/last block of the shared-cache item; lane 2/3: of the windows item
+            const int kind = lane >> 1;
+            const int64_t s = kind == 0 ? base : base + sp.gt;
+            const int64_t e = kind == 0 ? base + sp.gt : base + per;
+            int c = (lane & 1) ? -1 : 0;
+            if (s < e) c = cta_of(T, (lane & 1) ? e - 1 : s, nctas);
+            if (lane & 1) ctl.c1[kind] = c; else ctl.c0[kind] = c;
+        }
+        if (lane < kMaxLoops) {
+            int cut = 0;
+#pragma unroll
+            for (int k = 0; k < kMaxLoops; ++k)
+                if (k == lane) cut = sp.cut[k];
+            ctl.cut[lane] = cut;
+        }
+    }
+    __syncthreads();
+
+    const int row = chunk * kReduceWarps + wid;   // packed row of this head group: hl * R + r
+    if (row >= p.hpc * p.R) return;
+    const int hl = row / p.R, r = row - hl * p.R;
+    const int l = r / p.G, g = r - l * p.G;
+    const int h = (hg * p.hpc + hl) * p.G + g;
 
     Vec<D> yg, yl;
     float out[Vec<D>::N];
-    int cut = 0;
-#pragma unroll
-    for (int k = 0; k < kMaxLoops; ++k)
-        if (k == l) cut = sp.cut[k];
-    if (cut == 0) {
+    if (ctl.cut[l] == 0) {
 #pragma unroll
         for (int i = 0; i < Vec<D>::N; ++i) out[i] = 0.f;
     } else {
-        const float dg = merge_item<D>(p, item_index(p, b, hg, 0), hl, r, T, base, base + sp.gt, lane, yg);
+        const float dg = merge_item<D>(p, item_index(p, b, hg, 0), hl, r, ctl.c0[0], ctl.c1[0], lane, yg);
         const float ig = dg > 0.f ? 1.f / dg : 0.f;
         if (l == 0) {
 #pragma unroll
             for (int i = 0; i < Vec<D>::N; ++i) out[i] = yg.v[i] * ig;
         } else {
-            const float dl = merge_item<D>(p, item_index(p, b, hg, 1), hl, r, T, base + sp.gt, base + per, lane, yl);
+            const float dl = merge_item<D>(p, item_index(p, b, hg, 1), hl, r, ctl.c0[1], ctl.c1[1], lane, yl);
             const float il = dl > 0.f ? 1.f / dl : 0.f;  // empty window: y_local = 0
             const float x = p.gate_logits[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h];
             const float gate = 1.f / (1.f + expf(-x));
@@ -89,30 +136,55 @@ __global__ void __launch_bounds__(128) plt_decode_reduce(const __grid_constant__
             for (int i = 0; i < Vec<D>::N; ++i) out[i] = gate * (yl.v[i] * il) + (1.f - gate) * (yg.v[i] * ig);
         }
     }
-    const int64_t o = row_id * D + lane * Vec<D>::N;
+    const int64_t o = (((int64_t)b * p.L + l) * p.Hq + h) * D + lane * Vec<D>::N;
     if (BF16) {
         __nv_bfloat16* dst = (__nv_bfloat16*)p.out + o;
-#pragma unroll
-        for (int i = 0; i < Vec<D>::N; i += 2) *(__nv_bfloat162*)(dst + i) = __floats2bfloat162_rn(out[i], out[i + 1]);
+        if constexpr (Vec<D>::N == 4) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(out[0], out[1]), hi = __floats2bfloat162_rn(out[2], out[3]);
+            uint2 u;
+            u.x = *(const uint32_t*)&lo;
+            u.y = *(const uint32_t*)&hi;
+            *(uint2*)dst = u;
+        } else {
+            *(__nv_bfloat162*)dst = __floats2bfloat162_rn(out[0], out[1]);
+        }
     } else {
         float* dst = (float*)p.out + o;
-#pragma unroll
-        for (int i = 0; i < Vec<D>::N; ++i) dst[i] = out[i];
+        if constexpr (Vec<D>::N == 4) *(float4*)dst = make_float4(out[0], out[1], out[2], out[3]);
+        else *(float2*)dst = make_float2(out[0], out[1]);
     }
 }
 
-cudaError_t launch_reduce(const Params& p, bool bf16, cudaStream_t stream) {
-    const int64_t rows = (int64_t)p.B * p.L * p.Hq;
-    if (rows == 0) return cudaSuccess;
-    const unsigned grid = (unsigned)((rows + 3) / 4);
-    if (p.d == 128) {
-        if (bf16) plt_decode_reduce<128, true><<<grid, 128, 0, stream>>>(p);
-        else plt_decode_reduce<128, false><<<grid, 128, 0, stream>>>(p);
-    } else {
-        if (bf16) plt_decode_reduce<64, true><<<grid, 128, 0, stream>>>(p);
-        else plt_decode_reduce<64, false><<<grid, 128, 0, stream>>>(p);
-    }
-    return cudaGetLastError();
+template <int D, bool BF16>
+cudaError_t launch_one(const Params& p, unsigned grid, int chunks, bool overlap, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kReduceWarps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, plt_decode_reduce<D, BF16>, p, chunks);
+}
+
+}  // namespace
+
+// `overlap`: launch with programmatic stream serialisation, so that the blocks of this kernel are
+// set up while the main kernel (the launch before it in the stream) drains; they wait for its
+// completion in grid_dependency_wait() before reading anything it wrote.
+cudaError_t launch_reduce(const Params& p, bool bf16, bool overlap, cudaStream_t stream) {
+    const int rows = p.hpc * p.R;
+    const int chunks = (rows + kReduceWarps - 1) / kReduceWarps;
+    const int64_t blocks = (int64_t)p.B * (p.Hkv / p.hpc) * chunks;
+    if (blocks == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)blocks;
+    if (p.d == 128) return bf16 ? launch_one<128, true>(p, grid, chunks, overlap, stream)
+                                : launch_one<128, false>(p, grid, chunks, overlap, stream);
+    return bf16 ? launch_one<64, true>(p, grid, chunks, overlap, stream)
+                : launch_one<64, false>(p, grid, chunks, overlap, stream);
 }
 
 }  // namespace plt
