@@ -29,6 +29,14 @@ size_t main_f32_smem(int D, int R, int max_batch);
 cudaError_t main_f32_prepare(int D, int R, int max_batch, int* blocks_per_sm);
 cudaError_t launch_main_f32(const Params& p, int grid, size_t smem, cudaStream_t stream);
 
+// tcgen05 / tensor-memory main kernel (bf16, d = 128, one KV head per item, 128-key tiles, one block per SM).
+int main_umma_rows(int R);            // packed rows rounded up to the N of the instruction: 16, 32 or 64
+int main_umma_max_slots();
+size_t main_umma_smem(int R, int nslot, int max_batch);
+cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm);
+cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
+                             int wbox, cudaStream_t stream);
+
 cudaError_t launch_reduce(const Params& p, bool bf16, bool overlap, cudaStream_t stream);
 
 }  // namespace plt

@@ -1,0 +1,593 @@
+// bf16 split-KV main kernel of the CLP decode attention on the 5th-generation tensor cores
+// (tcgen05.mma with accumulators in tensor memory), head dimension 128.
+//
+// Same tile plan and split-partial format as the other main kernels (Algorithm 3 lines 2-3 for all
+// L loops): one persistent block per SM walks its share of the line of 128-key tiles, one KV head
+// per work item. The products are laid out with the KEYS as the M dimension, so that the packed
+// query rows (all L loop-queries times all GQA heads of a KV head, R <= 64) form the N dimension
+// and nothing is padded up to a 64- or 128-row tile:
+//
+//   S^T [128 keys x RP]  = K_tile [128 x 128] . Q^T        A = K tile as TMA wrote it (K-major,
+//                                                          128-byte swizzle), B = packed query rows
+//   O^T [128 dims x RP] += V_tile^T [128 x 128] . P^T      A = V tile as TMA wrote it (MN-major,
+//                                                          128-byte swizzle), B = probabilities
+//
+// RP is R rounded up to 16, 32 or 64. Both operands of both products are read from shared memory by
+// the tensor core itself, once, whatever R is; the 128 softmax threads own one key each (their
+// tensor-memory lane) and the RP scores of that key.
+//
+// Warp roles: warps 0-3 softmax and epilogue (thread = key / output dimension), warp 4 TMA
+// producer, warp 5 MMA issuer and owner of the tensor-memory allocation.
+//
+// Online softmax with a lazily updated reference maximum per row: probabilities are formed against
+// a reference that may lag the true running maximum by up to kSlack powers of two; only when a
+// score exceeds that (a vote over the 128 threads) are the true maxima reduced across threads and
+// the accumulators in tensor memory rescaled. Every wait on an mbarrier is bounded.
+#include <cuda_bf16.h>
+
+#include "plt_common.cuh"
+#include "plt_host.h"
+#include "plt_ptx.cuh"
+
+namespace plt {
+
+namespace {
+
+constexpr int UK = 128;                  // keys per tile
+constexpr int UD = 128;                  // head dimension
+constexpr int kSlotBytes = UK * UD * 2;  // one K tile or one V tile of one KV head
+constexpr int kHalfBytes = UK * 128;     // one 64-element half of a tile: [128 keys][128 bytes]
+constexpr int kMaxSlots = 6;
+constexpr int kSmThreads = 128;          // softmax threads
+constexpr int kUmmaThreads = 192;
+constexpr float kSlack = 8.f;
+constexpr uint64_t kUmmaWaitNs = 1000000000ull;
+
+// mbarrier indices
+constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_PFREE = 19, B_OFULL = 20,
+              B_OFREE = 21, B_QFULL = 22 /* two */, B_DRAIN = 24, B_COUNT = 25;
+
+template <int RP>
+struct UCfg {
+    static constexpr int QLBO = RP * 16 + 16;      // bytes between the 16-byte column chunks of the packed query tile
+    static constexpr int QBUF = 16 * QLBO;         // one packed query tile: [16 chunks][RP rows][16 bytes] (+ pad)
+    static constexpr int PBUF = RP * 256;          // probabilities: [RP / 8][128 keys][16 bytes]
+    static constexpr int TMEM_COLS = 2 * RP < 32 ? 32 : 2 * RP;  // S^T then O^T, RP columns each
+    __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
+        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2) + 64 +
+               (size_t)(max_batch + 4) * 4;
+    }
+};
+
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading and stride byte offsets in
+// 16-byte units, descriptor version 1, swizzle mode (0 = none, 2 = 128 bytes).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle) {
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | ((uint64_t)swizzle << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 A and B, majorness (0 = K-major, 1 = MN-major), N / 8, M / 16.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Bounded wait that also gives up as soon as another thread of the block has given up.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xffu) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kUmmaWaitNs) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Launch-time geometry of the TMA boxes (set by the host from the tensor maps it encoded).
+struct UmmaGeom {
+    int nslot;       // ring slots of kSlotBytes
+    int kbox;        // keys per box of the shared cache (min(128, page size or capacity))
+    int wbox;        // keys per box of a window (min(128, w))
+};
+
+template <int RP>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
+                     const __grid_constant__ Params p, const UmmaGeom geo) {
+    using C = UCfg<RP>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int nslot = geo.nslot;
+    uint8_t* pbuf = smem + (size_t)nslot * kSlotBytes;
+    uint8_t* qbuf = pbuf + C::PBUF;                       // two buffers of QBUF
+    uint64_t* bars = (uint64_t*)(qbuf + 2 * C::QBUF);
+    float* s_negm = (float*)(bars + B_COUNT);             // [RP] minus the reference maximum (1e30 while there is none)
+    float* s_mref = s_negm + RP;                          // [RP] reference maximum, log2 units
+    float* s_alpha = s_mref + RP;                         // [RP] rescale factors of the slow path
+    float* s_red = s_alpha + RP;                          // [4][RP] cross-warp reduction scratch
+    int32_t* s_lim = (int32_t*)(s_red + 4 * RP);          // [RP] keys visible to each row in the current segment
+    int32_t* s_rowloop = s_lim + RP;                      // [RP] loop (0-based) of each packed row
+    int32_t* s_ctl = s_rowloop + RP;                      // [0] abort flag, [1] tensor-memory base, [2] fills issued
+    int32_t* s_prefix = s_ctl + 16;
+    volatile int* abort_flag = (volatile int*)&s_ctl[0];
+
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    uint32_t flags = 0;
+
+    if (tid == 0) {
+        s_ctl[0] = 0;
+        s_ctl[2] = 0;
+        for (int s = 0; s < kMaxSlots; ++s) {
+            mbar_init(&bars[B_FULL + s], 1);
+            mbar_init(&bars[B_EMPTY + s], 1);
+        }
+        mbar_init(&bars[B_SFULL], 1);
+        mbar_init(&bars[B_SFREE], kSmThreads);
+        mbar_init(&bars[B_PFULL], kSmThreads);
+        mbar_init(&bars[B_PFREE], 1);
+        mbar_init(&bars[B_OFULL], 1);
+        mbar_init(&bars[B_OFREE], kSmThreads);
+        mbar_init(&bars[B_QFULL], kSmThreads);
+        mbar_init(&bars[B_QFULL + 1], kSmThreads);
+        mbar_init(&bars[B_DRAIN], 1);
+        mbar_fence_init();
+    }
+    if (tid < RP) s_rowloop[tid] = tid / p.G;
+    if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
+    grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
+    build_prefix(p, s_prefix, flags);  // contains __syncthreads
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = (uint32_t)s_ctl[1];
+    const uint32_t tS = tmem_base, tO = tmem_base + RP;
+
+    const int64_t T = s_prefix[p.B];
+    const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
+    if (cta == 0)
+        for (int b = tid; b <= p.B; b += kUmmaThreads) p.prefix[b] = s_prefix[b];
+    const bool in_plan = cta < nctas;
+    const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
+
+    if (wid == 4) {
+        // ================================ TMA producer (one lane) =================================
+        if (lane == 0 && lo < hi) {
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+            if (p.L > 1) {
+                tma_prefetch_desc(&tmKw);
+                tma_prefetch_desc(&tmVw);
+            }
+            uint32_t fill = 0;   // K tile of the n-th tile is fill 2n, its V tile fill 2n + 1
+            bool ok = true;
+            PieceWalk walk(p, s_prefix, lo, hi);
+            Piece pc;
+            while (ok && walk.next(pc, flags)) {
+                WinCursor cur;
+                if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
+                for (int t = pc.t0; t < pc.t1 && ok; ++t) {
+                    // boxes of this tile: (key coordinate, outermost coordinate), same for K and V
+                    int nbox, c1[UK / 16], c3[UK / 16], box_keys;
+                    const CUtensorMap *mk, *mv;
+                    if (pc.kind == 0) {
+                        const int key0 = t * UK;
+                        mk = &tmK;
+                        mv = &tmV;
+                        box_keys = geo.kbox;
+                        if (p.page_size > 0) {
+                            const int rem = pc.sp.cmax - key0;   // keys that hold data from key0 on (>= 1)
+                            nbox = (min(rem, UK) + box_keys - 1) / box_keys;
+                            for (int i = 0; i < nbox; ++i) {
+                                const int key = key0 + i * box_keys;
+                                int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
+                                if (page < 0 || page >= p.num_pool_pages) {
+                                    flags |= kDevPageIdClamped;
+                                    page = page < 0 ? 0 : p.num_pool_pages - 1;
+                                }
+                                c1[i] = key % p.page_size;
+                                c3[i] = page;
+                            }
+                        } else {
+                            nbox = 1;
+                            c1[0] = key0;
+                            c3[0] = pc.b;
+                        }
+                    } else {
+                        mk = &tmKw;
+                        mv = &tmVw;
+                        box_keys = geo.wbox;
+                        nbox = 1;
+                        c1[0] = cur.key0;
+                        c3[0] = pc.b * (p.L - 1) + (cur.l - 1);
+                        cur.advance(p, pc.sp);
+                    }
+                    const uint32_t bytes = (uint32_t)(nbox * box_keys * 256);
+#pragma unroll
+                    for (int which = 0; which < 2; ++which, ++fill) {
+                        const int slot = (int)(fill % (uint32_t)nslot);
+                        const uint32_t use = fill / (uint32_t)nslot;
+                        if (use > 0) ok = ok && wait_or_abort(&bars[B_EMPTY + slot], (use - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        uint8_t* dst = smem + (size_t)slot * kSlotBytes;
+                        mbar_expect_tx(&bars[B_FULL + slot], bytes);
+                        for (int i = 0; i < nbox; ++i)
+#pragma unroll
+                            for (int hf = 0; hf < 2; ++hf)
+                                tma_load_4d(dst + hf * kHalfBytes + i * box_keys * 128, which == 0 ? mk : mv,
+                                            &bars[B_FULL + slot], hf * 64, c1[i], pc.hg, c3[i]);
+                    }
+                }
+            }
+            s_ctl[2] = (int32_t)fill;
+        }
+    } else if (wid == 5) {
+        // ================================ MMA issuer (one lane) ===================================
+        if (lane == 0 && lo < hi) {
+            constexpr uint32_t idesc_qk = instr_desc(UK, RP, 0, 0);
+            constexpr uint32_t idesc_pv = instr_desc(UD, RP, 1, 1);
+            const uint32_t pbuf_a = smem_u32(pbuf), qbuf_a = smem_u32(qbuf), smem_a = smem_u32(smem);
+            bool ok = true;
+            uint32_t gt = 0, pi = 0;             // tiles and pieces done by this block so far
+            bool have_prev = false;              // a tile whose S^T product is issued but whose PV product is not
+            uint32_t prev_gt = 0, prev_pi = 0;
+            bool prev_first = false, prev_last = false;
+
+            auto issue_pv = [&]() {
+                ok = ok && wait_or_abort(&bars[B_PFULL], prev_gt & 1, abort_flag);
+                const uint32_t fillv = 2 * prev_gt + 1;
+                const int slot = (int)(fillv % (uint32_t)nslot);
+                ok = ok && wait_or_abort(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1, abort_flag);
+                if (prev_first && prev_pi > 0) ok = ok && wait_or_abort(&bars[B_OFREE], (prev_pi - 1) & 1, abort_flag);
+                if (!ok) return;
+                tc_fence_after_sync();
+                const uint32_t vs = smem_a + (uint32_t)slot * kSlotBytes;
+#pragma unroll
+                for (int ks = 0; ks < UK / 16; ++ks)
+                    umma_bf16(tO, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), smem_desc(pbuf_a + ks * 256, 128, 2048, 0),
+                              idesc_pv, (prev_first && ks == 0) ? 0u : 1u);
+                umma_commit(&bars[B_EMPTY + slot]);
+                umma_commit(&bars[B_PFREE]);
+                if (prev_last) umma_commit(&bars[B_OFULL]);
+            };
+
+            PieceWalk walk(p, s_prefix, lo, hi);
+            Piece pc;
+            while (ok && walk.next(pc, flags)) {
+                for (int t = pc.t0; t < pc.t1 && ok; ++t) {
+                    // ---- S^T of tile gt ----
+                    if (t == pc.t0) ok = ok && wait_or_abort(&bars[B_QFULL + (pi & 1)], (pi >> 1) & 1, abort_flag);
+                    const uint32_t fillk = 2 * gt;
+                    const int slot = (int)(fillk % (uint32_t)nslot);
+                    ok = ok && wait_or_abort(&bars[B_FULL + slot], (fillk / (uint32_t)nslot) & 1, abort_flag);
+                    if (gt > 0) ok = ok && wait_or_abort(&bars[B_SFREE], (gt - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
+                    const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
+#pragma unroll
+                    for (int kk = 0; kk < UD / 16; ++kk)
+                        umma_bf16(tS, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
+                                  smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
+                    umma_commit(&bars[B_SFULL]);
+                    umma_commit(&bars[B_EMPTY + slot]);
+                    // ---- O^T += V^T P^T of the tile before, whose probabilities are ready by now ----
+                    if (have_prev) issue_pv();
+                    have_prev = true;
+                    prev_gt = gt;
+                    prev_pi = pi;
+                    prev_first = (t == pc.t0);
+                    prev_last = (t == pc.t1 - 1);
+                    ++gt;
+                }
+                ++pi;
+            }
+            if (ok && have_prev) issue_pv();
+        }
+    } else {
+        // ============================ softmax and epilogue (warps 0-3) ============================
+        // Thread tid owns key tid of every tile (tensor-memory lane tid of S^T) and, in the epilogue,
+        // output dimension tid (lane tid of O^T).
+        const uint32_t lane_off = (uint32_t)(wid * 32) << 16;
+        const float scale = p.scale_log2;
+        const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
+        // `failed`: a wait of this warp ran out; the warp stops touching data but keeps the common control flow.
+        // Kept warp-uniform, because the tensor-memory loads and stores are warp-collective.
+        bool failed = false;
+        auto sm_wait = [&](uint64_t* bar, uint32_t parity) {
+            bool bad = false;
+            if (!failed) bad = !wait_or_abort(bar, parity, abort_flag);
+            failed = __any_sync(0xffffffffu, failed || bad);
+        };
+        bool aborted = false;   // agreed by all 128 threads
+
+        named_barrier_sync(1, kSmThreads);   // s_rowloop visible (written before the block-wide barrier, kept for clarity)
+
+        // Packed query rows of a piece into buffer `buf`: [chunk c][row r][16 bytes], rows >= R zero.
+        auto load_q = [&](const Piece& q_pc, int buf) {
+            uint8_t* dst = qbuf + buf * C::QBUF;
+            for (int id = tid; id < RP * 16; id += kSmThreads) {
+                const int r = id >> 4, c = id & 15;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (r < p.R) {
+                    const int l = s_rowloop[r], g = r - l * p.G;
+                    v = *(const uint4*)(qg + (((int64_t)q_pc.b * p.L + l) * p.Hq + q_pc.hg * p.G + g) * UD + c * 8);
+                }
+                *(uint4*)(dst + c * C::QLBO + r * 16) = v;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars[B_QFULL + buf]);
+        };
+
+        uint32_t gt = 0, pi = 0;
+        PieceWalk walk(p, s_prefix, lo, hi);
+        Piece pc, npc;
+        bool have = walk.next(pc, flags);
+        if (have) load_q(pc, 0);
+        while (have && !aborted) {
+            // The next piece's query rows go into the other buffer now: every product that read it has completed
+            // (this thread has seen the scores of the last tile of the piece before).
+            const bool nhave = walk.next(npc, flags);
+            if (nhave) load_q(npc, (pi + 1) & 1);
+
+            // ---- per-piece state ----
+            int cmin = 0x7fffffff;
+#pragma unroll
+            for (int l = 0; l < kMaxLoops; ++l)
+                if (l < p.L) cmin = min(cmin, pc.sp.cut[l]);
+            if (tid < RP) {
+                s_mref[tid] = -INFINITY;
+                s_negm[tid] = 1e30f;
+                if (pc.kind == 0) {
+                    int cut = 0;
+#pragma unroll
+                    for (int l = 0; l < kMaxLoops; ++l)
+                        if (l == s_rowloop[tid]) cut = pc.sp.cut[l];
+                    s_lim[tid] = tid < p.R ? cut : 0;
+                }
+            }
+            named_barrier_sync(1, kSmThreads);
+            float lsum[RP];
+#pragma unroll
+            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
+            WinCursor cur;
+            cur.l = 0;
+            cur.key0 = 0;
+            if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
+            int seg_l = -1, wl = 0;
+
+            for (int t = pc.t0; t < pc.t1; ++t, ++gt) {
+                int kbase, nvalid;
+                bool masked;
+                if (pc.kind == 0) {
+                    kbase = t * UK;
+                    nvalid = pc.sp.cmax - kbase;
+                    masked = kbase + UK > cmin;
+                } else {
+                    if (cur.l != seg_l) {   // a new window: only the rows of its loop see it
+                        seg_l = cur.l;
+#pragma unroll
+                        for (int k = 1; k < kMaxLoops; ++k)
+                            if (k == cur.l) wl = pc.sp.wl[k];
+                        if (tid < RP) s_lim[tid] = (tid < p.R && s_rowloop[tid] == cur.l) ? wl : 0;
+                        named_barrier_sync(1, kSmThreads);
+                    }
+                    kbase = cur.key0;
+                    nvalid = wl - kbase;
+                    masked = true;
+                }
+                // ---- scores of this thread's key ----
+                sm_wait(&bars[B_SFULL], gt & 1);
+                uint32_t sv[RP];
+                if (!failed) {
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < RP / 16; ++c) tmem_ld16(tS + lane_off + c * 16, sv + c * 16);
+                    tmem_wait_ld();
+                    tc_fence_before_sync();
+                } else {
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) sv[r] = 0xff800000u;
+                }
+                mbar_arrive(&bars[B_SFREE]);
+                if (masked) {
+                    const int key = kbase + tid;
+#pragma unroll
+                    for (int r = 0; r < RP; ++r)
+                        if (key >= s_lim[r]) sv[r] = 0xff800000u;   // -inf; also replaces whatever a stale K row gave
+                }
+                float over = -INFINITY;
+#pragma unroll
+                for (int r = 0; r < RP; ++r)
+                    if (r < p.R) over = fmaxf(over, fmaf(__uint_as_float(sv[r]), scale, s_negm[r]));
+                const bool trouble = failed || (*abort_flag != 0);
+                if (named_barrier_or(1, kSmThreads, over > kSlack || trouble)) {
+                    if (named_barrier_or(1, kSmThreads, trouble)) {
+                        aborted = true;
+                        break;
+                    }
+                    // ---- slow path: true maxima over the 128 keys, new references, rescale O^T ----
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) {
+                        const float v = warp_max(__uint_as_float(sv[r]) * scale);
+                        if (lane == 0) s_red[wid * RP + r] = v;
+                    }
+                    named_barrier_sync(1, kSmThreads);
+                    if (tid < RP) {
+                        const float mo = s_mref[tid];
+                        const float mn = fmaxf(fmaxf(mo, fmaxf(s_red[tid], s_red[RP + tid])),
+                                               fmaxf(s_red[2 * RP + tid], s_red[3 * RP + tid]));
+                        s_alpha[tid] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
+                        s_mref[tid] = mn;
+                        s_negm[tid] = (mn == -INFINITY) ? 1e30f : -mn;
+                    }
+                    named_barrier_sync(1, kSmThreads);
+                    if (t != pc.t0) {
+                        // O^T holds the earlier tiles of this piece; their last product must have completed
+                        sm_wait(&bars[B_PFREE], (gt - 1) & 1);
+                        if (!failed) {
+                            tc_fence_after_sync();
+#pragma unroll
+                            for (int c = 0; c < RP / 16; ++c) {
+                                uint32_t o[16];
+                                tmem_ld16(tO + lane_off + c * 16, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * s_alpha[c * 16 + j]);
+                                tmem_st16(tO + lane_off + c * 16, o);
+                            }
+                            tmem_wait_st();
+                            tc_fence_before_sync();
+                        }
+#pragma unroll
+                        for (int r = 0; r < RP; ++r) lsum[r] *= s_alpha[r];
+                    }
+                }
+                // ---- probabilities (bf16) into shared memory, denominators from the rounded values ----
+                if (gt > 0) sm_wait(&bars[B_PFREE], (gt - 1) & 1);
+#pragma unroll
+                for (int j = 0; j < RP / 8; ++j) {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int r0 = j * 8 + 2 * q;
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[r0]), scale, s_negm[r0]));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[r0 + 1]), scale, s_negm[r0 + 1]));
+                        w4[q] = pack_bf16x2(p0, p1);
+                        lsum[r0] += __uint_as_float(w4[q] << 16);
+                        lsum[r0 + 1] += __uint_as_float(w4[q] & 0xffff0000u);
+                    }
+                    if (!failed) *(uint4*)(pbuf + j * 2048 + tid * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
+                if (masked && nvalid < UK) {
+                    // V rows that hold no data may contain anything: zero them so that 0 * garbage stays 0
+                    const uint32_t fillv = 2 * gt + 1;
+                    const int slot = (int)(fillv % (uint32_t)nslot);
+                    sm_wait(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1);
+                    if (!failed && tid >= nvalid) {
+                        uint8_t* row = smem + (size_t)slot * kSlotBytes + tid * 128;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            *(uint4*)(row + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+                            *(uint4*)(row + kHalfBytes + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[B_PFULL]);
+                if (pc.kind == 1) cur.advance(p, pc.sp);
+            }
+            if (aborted) break;
+
+            // ---- end of piece: denominators across the 128 keys, then O^T out of tensor memory ----
+#pragma unroll
+            for (int r = 0; r < RP; ++r) {
+                const float v = warp_sum(lsum[r]);
+                if (lane == 0) s_red[wid * RP + r] = v;
+            }
+            sm_wait(&bars[B_OFULL], pi & 1);
+            named_barrier_sync(1, kSmThreads);
+            const int64_t prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // hpc == 1 on this path
+            if (tid < p.R)
+                *(float2*)(p.part_ml + (prow + tid) * 2) =
+                    make_float2(s_mref[tid], (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]));
+            uint32_t o[RP];
+            if (!failed) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tO + lane_off + c * 16, o + c * 16);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+            }
+            mbar_arrive(&bars[B_OFREE]);
+            if (!failed) {
+#pragma unroll
+                for (int r = 0; r < RP; ++r)
+                    if (r < p.R) p.part_acc[(prow + r) * UD + tid] = __uint_as_float(o[r]);
+            }
+            named_barrier_sync(1, kSmThreads);   // s_red and s_mref are rewritten by the next piece
+            pc = npc;
+            have = nhave;
+            ++pi;
+        }
+    }
+
+    // ---- common exit: nothing of this block may still be in flight when tensor memory is freed ----
+    __syncthreads();
+    const bool gave_up = *abort_flag != 0;
+    if (wid == 5 && lane == 0) {
+        umma_commit(&bars[B_DRAIN]);   // arrives once every product issued by this thread has completed
+        wait_or_abort(&bars[B_DRAIN], 0, abort_flag);
+    }
+    if (wid == 4 && lane == 0 && gave_up) {
+        // give every copy that was issued a bounded chance to land
+        const uint32_t fills = (uint32_t)s_ctl[2];
+        for (uint32_t f = fills > (uint32_t)nslot ? fills - (uint32_t)nslot : 0; f < fills; ++f)
+            mbar_wait_bounded(&bars[B_FULL + (int)(f % (uint32_t)nslot)], (f / (uint32_t)nslot) & 1, kUmmaWaitNs);
+    }
+    if (gave_up) flags |= kDevWaitTimeout;
+    if (flags) atomicOr(p.status, flags);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (wid == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+template <int RP>
+cudaError_t umma_prepare(size_t smem, int* blocks_per_sm) {
+    auto fn = plt_decode_main_umma<RP>;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, kUmmaThreads, smem);
+}
+
+}  // namespace
+
+int main_umma_rows(int R) { return R <= 16 ? 16 : (R <= 32 ? 32 : 64); }
+
+int main_umma_max_slots() { return kMaxSlots; }
+
+size_t main_umma_smem(int R, int nslot, int max_batch) {
+    const int rp = main_umma_rows(R);
+    return rp == 16 ? UCfg<16>::smem_bytes(nslot, max_batch)
+                    : (rp == 32 ? UCfg<32>::smem_bytes(nslot, max_batch) : UCfg<64>::smem_bytes(nslot, max_batch));
+}
+
+cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm) {
+    const int rp = main_umma_rows(R);
+    return rp == 16 ? umma_prepare<16>(smem, blocks_per_sm)
+                    : (rp == 32 ? umma_prepare<32>(smem, blocks_per_sm) : umma_prepare<64>(smem, blocks_per_sm));
+}
+
+cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
+                             int wbox, cudaStream_t stream) {
+    const UmmaGeom geo{nslot, kbox, wbox};
+    const int rp = main_umma_rows(p.R);
+    if (rp == 16)
+        plt_decode_main_umma<16><<<grid, kUmmaThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo);
+    else if (rp == 32)
+        plt_decode_main_umma<32><<<grid, kUmmaThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo);
+    else
+        plt_decode_main_umma<64><<<grid, kUmmaThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo);
+    return cudaGetLastError();
+}
+
+}  // namespace plt
