@@ -53,6 +53,14 @@ typedef enum {
 
 typedef enum { PLT_F32 = 0, PLT_BF16 = 1 } plt_dtype;
 
+/* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
+typedef enum {
+    PLT_PATH_AUTO = 0,      /* the library chooses */
+    PLT_PATH_WARP_MMA = 1,  /* warp-level tensor-core products (mma.sync); fp32 inputs always use SIMT fp32 */
+    PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16, d = 128, pages that divide
+                               or are a multiple of 128 tokens; anything else is refused with PLT_ERR_UNSUPPORTED */
+} plt_kernel_path;
+
 /* Bits of the device status word reported by plt_decode_attn_check. */
 #define PLT_DEV_SEQ_LEN_CLAMPED 1u  /* a seq_lens entry was outside [0, max_seq_len] */
 #define PLT_DEV_PAGE_ID_CLAMPED 2u  /* a page id was outside [0, num_pool_pages) */
@@ -81,6 +89,8 @@ typedef struct {
     int32_t key_slices;    /* 16-key slices per pipeline tile (bf16 path; 1, 2 or 4) */
     int32_t stages;        /* depth of the shared-memory pipeline (bf16 path) */
     int32_t ctas_per_sm;   /* persistent thread blocks per SM */
+    int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (3..6) and
+                              heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block) */
 } plt_decode_attn_config;
 
 /*
@@ -152,9 +162,10 @@ const char* plt_decode_attn_last_error(plt_decode_attn_t handle);
 plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config* config, size_t* out_bytes);
 
 /* Number of kernels one plt_decode_attn_run launches, and the variant chosen at create
- * (heads_per_cta, key_slices, stages, ctas_per_sm, grid size); any pointer may be NULL. */
+ * (heads_per_cta, key_slices, stages, ctas_per_sm, grid size, plt_kernel_path actually used); any pointer may be NULL. */
 plt_status plt_decode_attn_launch_info(plt_decode_attn_t handle, int32_t* kernels_per_run, int32_t* heads_per_cta,
-                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid);
+                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid,
+                                       int32_t* kernel_path);
 
 /* Measurement aid: when both are non-NULL (cudaEvent_t created by the caller, with timing enabled), every later
  * plt_decode_attn_run records ev_main_begin just before and ev_main_end just after the split-KV main kernel on

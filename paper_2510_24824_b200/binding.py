@@ -16,6 +16,7 @@ LIB_PATH = _PKG / "libplt_decode_attn.so"
 PLT_OK, PLT_ERR_INVALID_ARG, PLT_ERR_UNSUPPORTED, PLT_ERR_OUT_OF_MEMORY, PLT_ERR_CUDA, PLT_ERR_CAPACITY, \
     PLT_ERR_DEVICE_CHECK = range(7)
 PLT_F32, PLT_BF16 = 0, 1
+PLT_PATH_AUTO, PLT_PATH_WARP_MMA, PLT_PATH_TCGEN05 = 0, 1, 2
 PLT_DEV_SEQ_LEN_CLAMPED, PLT_DEV_PAGE_ID_CLAMPED, PLT_DEV_WAIT_TIMEOUT, PLT_DEV_WIN_LEN_CLAMPED = 1, 2, 4, 8
 
 EXPORTS = (
@@ -40,7 +41,7 @@ class Config(ctypes.Structure):
         ("max_seq_len", ctypes.c_int32), ("w", ctypes.c_int32), ("page_size", ctypes.c_int32),
         ("sm_scale", ctypes.c_float), ("device", ctypes.c_int32), ("loop_offset", ctypes.POINTER(ctypes.c_int32)),
         ("heads_per_cta", ctypes.c_int32), ("key_slices", ctypes.c_int32), ("stages", ctypes.c_int32),
-        ("ctas_per_sm", ctypes.c_int32),
+        ("ctas_per_sm", ctypes.c_int32), ("kernel_path", ctypes.c_int32),
     ]
 
 
@@ -76,7 +77,7 @@ def load_library() -> ctypes.CDLL:
         lib.plt_decode_attn_last_error.restype = ctypes.c_char_p
         lib.plt_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(ctypes.c_size_t)]
         i32p = ctypes.POINTER(ctypes.c_int32)
-        lib.plt_decode_attn_launch_info.argtypes = [h, i32p, i32p, i32p, i32p, i32p, i32p]
+        lib.plt_decode_attn_launch_info.argtypes = [h, i32p, i32p, i32p, i32p, i32p, i32p, i32p]
         lib.plt_decode_attn_set_profile_events.argtypes = [h, ctypes.c_void_p, ctypes.c_void_p]
         lib.plt_decode_attn_run_no_alloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Args), ctypes.c_void_p]
         for name in EXPORTS:
@@ -94,7 +95,7 @@ def _raise(status: int, handle) -> None:
 def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_seq_len: int, w: int,
                 page_size: int = 0, sm_scale: float = 0.0, device: int = 0,
                 loop_offset: Optional[Sequence[int]] = None, heads_per_cta: int = 0, key_slices: int = 0,
-                stages: int = 0, ctas_per_sm: int = 0) -> Config:
+                stages: int = 0, ctas_per_sm: int = 0, kernel_path: int = 0) -> Config:
     c = Config()
     c.struct_size = ctypes.sizeof(Config)
     c.dtype = {"f32": PLT_F32, "bf16": PLT_BF16}.get(dtype, dtype)
@@ -106,6 +107,7 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
         c._keep = arr
         c.loop_offset = ctypes.cast(arr, ctypes.POINTER(ctypes.c_int32))
     c.heads_per_cta, c.key_slices, c.stages, c.ctas_per_sm = heads_per_cta, key_slices, stages, ctas_per_sm
+    c.kernel_path = kernel_path
     return c
 
 
@@ -180,11 +182,11 @@ def plt_decode_attn_destroy(handle) -> None:
 
 
 def plt_decode_attn_launch_info(handle) -> dict:
-    vals = [ctypes.c_int32() for _ in range(6)]
+    vals = [ctypes.c_int32() for _ in range(7)]
     st = load_library().plt_decode_attn_launch_info(handle, *[ctypes.byref(v) for v in vals])
     if st != PLT_OK:
         _raise(st, handle)
-    keys = ("kernels_per_run", "heads_per_cta", "key_slices", "stages", "ctas_per_sm", "grid")
+    keys = ("kernels_per_run", "heads_per_cta", "key_slices", "stages", "ctas_per_sm", "grid", "kernel_path")
     return {k: int(v.value) for k, v in zip(keys, vals)}
 
 

@@ -46,6 +46,8 @@ struct plt_decode_attn {
     bool bf16;
     int sm_count;
     MainVariant var;      // bf16: full variant; fp32: only grid/smem used
+    bool umma = false;    // bf16 path on tcgen05 / tensor memory (var.HPC = 1, var.KW = 8, var.stages = ring slots)
+    int kbox = 0, wbox = 0;  // keys per TMA box of the shared cache / of a window on that path
     int ctas_per_sm;
     float scale_log2;
     // workspace
@@ -188,6 +190,83 @@ plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, in
     return PLT_OK;
 }
 
+// Can the tcgen05 kernel take this configuration? (bf16, d = 128, pages that tile or are tiled by 128 keys)
+bool umma_eligible(const plt_decode_attn_config* c) {
+    if (c->dtype != PLT_BF16 || c->d != 128) return false;
+    if (c->page_size > 0 && c->page_size % 128 != 0 && 128 % c->page_size != 0) return false;
+    return true;
+}
+
+bool want_umma(const plt_decode_attn_config* c) {
+    if (c->kernel_path == PLT_PATH_WARP_MMA) return false;
+    if (c->kernel_path == PLT_PATH_TCGEN05) return true;
+    return false;
+}
+
+// Chooses the kernel path and variant, prepares the kernels (shared-memory attribute, occupancy) and fills
+// h->var, h->umma, h->ctas_per_sm. Needs h->bf16, h->sm_count. Errors go to the create-time message.
+plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* config, const Geometry& g) {
+    int blocks = 0;
+    cudaError_t e;
+    h->umma = false;
+    if (config->kernel_path < 0 || config->kernel_path > PLT_PATH_TCGEN05)
+        return fail(nullptr, PLT_ERR_INVALID_ARG, "kernel_path %d outside [0, 2]", config->kernel_path);
+    if (config->kernel_path == PLT_PATH_TCGEN05 && !umma_eligible(config))
+        return fail(nullptr, PLT_ERR_UNSUPPORTED,
+                    "the tcgen05 path needs bf16, d = 128 and a page size that divides or is a multiple of 128");
+    if (h->bf16 && want_umma(config)) {
+        int nslot = config->stages;
+        if (nslot == 0) {
+            nslot = main_umma_max_slots();
+            while (nslot > 3 && main_umma_smem(g.R, nslot, config->max_batch) > 227 * 1024) --nslot;
+        }
+        if (nslot < 3 || nslot > main_umma_max_slots())
+            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [3, %d] on the tcgen05 path", nslot, main_umma_max_slots());
+        const size_t smem = main_umma_smem(g.R, nslot, config->max_batch);
+        if (smem > 227 * 1024)
+            return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 path needs %zu bytes of shared memory (> 227 KB)", smem);
+        e = main_umma_prepare(g.R, smem, &blocks);
+        if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the tcgen05 main kernel", e);
+        if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
+        h->umma = true;
+        h->var = MainVariant{config->d, g.MT, 1, 8, nslot, 0, smem};
+        h->ctas_per_sm = 1;
+        h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)
+                                        : (config->max_seq_len < 128 ? config->max_seq_len : 128);
+        h->wbox = config->w < 128 ? (config->w > 0 ? config->w : 1) : 128;
+    } else if (h->bf16) {
+        int cps = 0;
+        plt_status s = choose_variant(config, g, &h->var, &cps);
+        if (s != PLT_OK) return s;
+        e = main_bf16_prepare(h->var, &blocks);
+        if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the bf16 main kernel", e);
+        if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
+        h->ctas_per_sm = blocks < cps ? blocks : cps;
+    } else {
+        h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
+        e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
+        if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the fp32 main kernel", e);
+        if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM");
+        const int cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
+        h->ctas_per_sm = blocks < cps ? blocks : cps;
+    }
+    h->var.grid = h->sm_count * h->ctas_per_sm;
+    if (h->bf16) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess)
+            return fail(nullptr, PLT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        h->encode = (EncodeTiledFn)fn;
+    }
+    // The tile line must fit 31 bits.
+    const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+    const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
+                         ((double)(config->max_seq_len + tk - 1) / tk + (double)(config->L - 1) * ((config->w + tk - 1) / tk));
+    if (tiles >= 2147483647.0) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan");
+    return PLT_OK;
+}
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 }  // namespace
@@ -205,7 +284,9 @@ PLT_API plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config*
     if (cudaGetDeviceProperties(&prop, config->device) == cudaSuccess) sms = prop.multiProcessorCount;
     else (void)cudaGetLastError();
     int hpc = 1, cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
-    if (config->dtype == PLT_BF16) {
+    if (config->dtype == PLT_BF16 && want_umma(config)) {
+        cps = 1;
+    } else if (config->dtype == PLT_BF16) {
         MainVariant v;
         s = choose_variant(config, g, &v, &cps);
         if (s != PLT_OK) return s;
@@ -245,38 +326,8 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     h->scale_log2 = scale * 1.4426950408889634f;
     h->err[0] = 0;
 
-    int blocks = 0;
-    if (h->bf16) {
-        int cps = 0;
-        s = choose_variant(config, g, &h->var, &cps);
-        if (s != PLT_OK) { delete h; return s; }
-        e = main_bf16_prepare(h->var, &blocks);
-        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, "preparing the bf16 main kernel", e); }
-        if (blocks < 1) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM"); }
-        h->ctas_per_sm = blocks < cps ? blocks : cps;
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) {
-            delete h;
-            return fail(nullptr, PLT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-        }
-        h->encode = (EncodeTiledFn)fn;
-    } else {
-        h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
-        e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
-        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, "preparing the fp32 main kernel", e); }
-        if (blocks < 1) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM"); }
-        const int cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
-        h->ctas_per_sm = blocks < cps ? blocks : cps;
-    }
-    h->var.grid = h->sm_count * h->ctas_per_sm;
-
-    // The tile line must fit 31 bits.
-    const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
-    const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
-                         ((double)(config->max_seq_len + tk - 1) / tk + (double)(config->L - 1) * ((config->w + tk - 1) / tk));
-    if (tiles >= 2147483647.0) { delete h; return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan"); }
+    s = setup_kernels(h, config, g);
+    if (s != PLT_OK) { delete h; return s; }
 
     size_t acc_floats, ml_floats;
     h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
@@ -359,31 +410,37 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     cudaError_t e;
     if (h->bf16) {
-        const int tk = 16 * h->var.KW;
+        // keys and heads per TMA box: the warp-level kernel loads [heads per block][tile keys], the tcgen05 kernel
+        // [1 head][up to 128 keys]
+        const int tk = h->umma ? h->kbox : 16 * h->var.KW;
+        const int tkw = h->umma ? h->wbox : 16 * h->var.KW;
+        const int bh = h->umma ? 1 : h->var.HPC;
         plt_status s;
         if (c.page_size > 0) {
-            s = encode_map(h, 0, a->k_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, h->var.HPC);
+            s = encode_map(h, 0, a->k_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, bh);
             if (s == PLT_OK)
-                s = encode_map(h, 1, a->v_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, h->var.HPC);
+                s = encode_map(h, 1, a->v_cache, es, c.d, c.page_size, c.Hkv, a->num_pool_pages, sn, sh, sb, tk, bh);
         } else {
-            s = encode_map(h, 0, a->k_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, h->var.HPC);
+            s = encode_map(h, 0, a->k_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, bh);
             if (s == PLT_OK)
-                s = encode_map(h, 1, a->v_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, h->var.HPC);
+                s = encode_map(h, 1, a->v_cache, es, c.d, c.max_seq_len, c.Hkv, a->batch, sn, sh, sb, tk, bh);
         }
         if (s != PLT_OK) return s;
         if (c.L > 1) {
             const int64_t wn = (int64_t)c.Hkv * c.d, wb = (int64_t)c.w * wn;
-            s = encode_map(h, 2, a->k_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tk, h->var.HPC);
+            s = encode_map(h, 2, a->k_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tkw, bh);
             if (s == PLT_OK)
-                s = encode_map(h, 3, a->v_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tk,
-                               h->var.HPC);
+                s = encode_map(h, 3, a->v_win, es, c.d, c.w, c.Hkv, (int64_t)a->batch * (c.L - 1), wn, c.d, wb, tkw, bh);
             if (s != PLT_OK) return s;
         } else {
             h->maps[2] = h->maps[0];
             h->maps[3] = h->maps[1];
         }
         if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
-        e = launch_main_bf16(h->var, h->maps, p, stream);
+        if (h->umma)
+            e = launch_main_umma(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox, stream);
+        else
+            e = launch_main_bf16(h->var, h->maps, p, stream);
     } else {
         if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
         e = launch_main_f32(p, h->var.grid, h->var.smem, stream);
@@ -520,7 +577,8 @@ PLT_API plt_status plt_decode_attn_set_profile_events(plt_decode_attn_t h, void*
 }
 
 PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* kernels_per_run, int32_t* heads_per_cta,
-                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid) {
+                                       int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid,
+                                       int32_t* kernel_path) {
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
     if (kernels_per_run) *kernels_per_run = 2;
     if (heads_per_cta) *heads_per_cta = h->var.HPC;
@@ -528,6 +586,7 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
     if (stages) *stages = h->var.stages;
     if (ctas_per_sm) *ctas_per_sm = h->ctas_per_sm;
     if (grid) *grid = h->var.grid;
+    if (kernel_path) *kernel_path = h->umma ? PLT_PATH_TCGEN05 : PLT_PATH_WARP_MMA;
     return PLT_OK;
 }
 
@@ -640,31 +699,9 @@ extern "C" PLT_API plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn
         const float scale = config->sm_scale > 0.f ? config->sm_scale : 1.0f / sqrtf((float)config->d);
         h->scale_log2 = scale * 1.4426950408889634f;
         h->err[0] = 0;
-        h->encode = dv.encode;
         for (bool& v : h->map_valid) v = false;
-        int blocks = 0;
-        if (h->bf16) {
-            int cps = 0;
-            s = choose_variant(config, g, &h->var, &cps);
-            if (s != PLT_OK) return s;
-            e = main_bf16_prepare(h->var, &blocks);
-            if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the bf16 main kernel", e);
-            if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
-            h->ctas_per_sm = blocks < cps ? blocks : cps;
-        } else {
-            h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
-            e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
-            if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the fp32 main kernel", e);
-            if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM");
-            const int cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
-            h->ctas_per_sm = blocks < cps ? blocks : cps;
-        }
-        h->var.grid = h->sm_count * h->ctas_per_sm;
-        const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
-        const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
-                             ((double)(config->max_seq_len + tk - 1) / tk +
-                              (double)(config->L - 1) * ((config->w + tk - 1) / tk));
-        if (tiles >= 2147483647.0) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan");
+        s = setup_kernels(h, config, g);
+        if (s != PLT_OK) return s;
         size_t acc_floats, ml_floats;
         h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
         if (h->ws_bytes > kNoAllocScratchBytes)

@@ -533,7 +533,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const bool gave_up = *abort_flag != 0;
     if (wid == 5 && lane == 0) {
         umma_commit(&bars[B_DRAIN]);   // arrives once every product issued by this thread has completed
-        wait_or_abort(&bars[B_DRAIN], 0, abort_flag);
+        mbar_wait_bounded(&bars[B_DRAIN], 0, kUmmaWaitNs);
     }
     if (wid == 4 && lane == 0 && gave_up) {
         // give every copy that was issued a bounded chance to land
