@@ -60,12 +60,17 @@ struct SeqPlan {
 
 __device__ __forceinline__ int32_t ceil_div(int32_t a, int32_t b) { return (a + b - 1) / b; }
 
-__device__ __forceinline__ void seq_plan(const Params& p, int b, SeqPlan& s, uint32_t& flags) {
+// Length of sequence b, clamped to [0, capacity].
+__device__ __forceinline__ int32_t seq_len_clamped(const Params& p, int b, uint32_t& flags) {
     int32_t n = p.seq_lens[b];
     if (n < 0 || n > p.max_seq_len) {
         flags |= kDevSeqLenClamped;
         n = n < 0 ? 0 : p.max_seq_len;
     }
+    return n;
+}
+
+__device__ __forceinline__ void seq_plan_n(const Params& p, int b, int32_t n, SeqPlan& s, uint32_t& flags) {
     s.n = n;
     s.cmax = 0;
     s.lt = 0;
@@ -93,6 +98,10 @@ __device__ __forceinline__ void seq_plan(const Params& p, int b, SeqPlan& s, uin
         }
     }
     s.gt = ceil_div(s.cmax, p.tile_keys);
+}
+
+__device__ __forceinline__ void seq_plan(const Params& p, int b, SeqPlan& s, uint32_t& flags) {
+    seq_plan_n(p, b, seq_len_clamped(p, b, flags), s, flags);
 }
 
 // Tiles sequence b puts on the line.
@@ -123,9 +132,17 @@ __device__ __forceinline__ int item_index(const Params& p, int b, int hg, int ki
 __device__ __forceinline__ int64_t slot_of(int item, int cta) { return (int64_t)item + cta; }
 
 // Block-wide exclusive prefix of seq_tiles into sp[0..B] (shared memory). All threads of the block call it.
-__device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint32_t& flags) {
+// With `lens` (shared memory, B entries) the clamped lengths are kept for PieceWalk, so that walking the pieces
+// reads no global memory.
+__device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint32_t& flags, int32_t* lens = nullptr) {
     const int tid = threadIdx.x, nt = blockDim.x;
-    for (int b = tid; b < p.B; b += nt) sp[b + 1] = seq_tiles(p, b, flags);
+    for (int b = tid; b < p.B; b += nt) {
+        const int32_t n = seq_len_clamped(p, b, flags);
+        if (lens != nullptr) lens[b] = n;
+        SeqPlan s;
+        seq_plan_n(p, b, n, s, flags);
+        sp[b + 1] = (p.Hkv / p.hpc) * (s.gt + s.lt);
+    }
     if (tid == 0) sp[0] = 0;
     __syncthreads();
     if (tid < 32) {
@@ -170,16 +187,18 @@ struct Piece {
 struct PieceWalk {
     const Params& p;
     const int32_t* sp;
+    const int32_t* lens;   // clamped lengths in shared memory, or null (then seq_lens is read)
     int64_t pos, hi;
     int b;
-    __device__ PieceWalk(const Params& p_, const int32_t* sp_, int64_t lo_, int64_t hi_)
-        : p(p_), sp(sp_), pos(lo_), hi(hi_), b(0) {
+    __device__ PieceWalk(const Params& p_, const int32_t* sp_, int64_t lo_, int64_t hi_, const int32_t* lens_ = nullptr)
+        : p(p_), sp(sp_), lens(lens_), pos(lo_), hi(hi_), b(0) {
         if (pos < hi) b = find_seq(sp, p.B, pos);
     }
     __device__ bool next(Piece& pc, uint32_t& flags) {
         if (pos >= hi) return false;
         while ((int64_t)sp[b + 1] <= pos) ++b;
-        seq_plan(p, b, pc.sp, flags);
+        if (lens != nullptr) seq_plan_n(p, b, lens[b], pc.sp, flags);
+        else seq_plan(p, b, pc.sp, flags);
         const int per = pc.sp.gt + pc.sp.lt;
         const int o = (int)(pos - sp[b]);
         pc.b = b;

@@ -44,18 +44,18 @@ constexpr float kSlack = 8.f;
 constexpr uint64_t kUmmaWaitNs = 1000000000ull;
 
 // mbarrier indices
-constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_PFREE = 19, B_OFULL = 20,
-              B_OFREE = 21, B_QFULL = 22 /* two */, B_DRAIN = 24, B_COUNT = 25;
+constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_PFREE = 19, B_OFULL = 20 /* two */,
+              B_OFREE = 22 /* two */, B_QFULL = 24 /* two */, B_DRAIN = 26, B_COUNT = 27;
 
 template <int RP>
 struct UCfg {
     static constexpr int QLBO = RP * 16 + 16;      // bytes between the 16-byte column chunks of the packed query tile
     static constexpr int QBUF = 16 * QLBO;         // one packed query tile: [16 chunks][RP rows][16 bytes] (+ pad)
     static constexpr int PBUF = RP * 256;          // probabilities: [RP / 8][128 keys][16 bytes]
-    static constexpr int TMEM_COLS = 2 * RP < 32 ? 32 : 2 * RP;  // S^T then O^T, RP columns each
+    static constexpr int TMEM_COLS = 4 * RP;       // S^T, then two O^T buffers, RP columns each (power of two)
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
-        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2) + 64 +
-               (size_t)(max_batch + 4) * 4;
+        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 4) + 64 +
+               (size_t)(2 * max_batch + 4) * 4;
     }
 };
 
@@ -88,15 +88,46 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     return true;
 }
 
-__device__ __forceinline__ float warp_max(float v) {
+// Reduces N values per lane across the 32 lanes of a warp with N - 1 (+ a few) shuffles instead of 5 N: each
+// step halves the values a lane still carries and doubles the lanes they cover. The result of row r goes to
+// dst[r] (shared memory).
+template <int N, bool MAX>
+__device__ __forceinline__ void warp_reduce_rows(float (&v)[N], int lane, float* dst) {
+    static_assert(N == 16 || N == 32 || N == 64, "rows per warp reduction");
+    if constexpr (N == 64) {
+        float a[32], b[32];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-__device__ __forceinline__ float warp_sum(float v) {
+        for (int i = 0; i < 32; ++i) {
+            a[i] = v[i];
+            b[i] = v[32 + i];
+        }
+        warp_reduce_rows<32, MAX>(a, lane, dst);
+        warp_reduce_rows<32, MAX>(b, lane, dst + 32);
+    } else {
+        int n = N;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
+        for (int o = 16; o > 0; o >>= 1) {
+            if (n > 1) {
+                const bool up = (lane & o) != 0;
+                n >>= 1;
+#pragma unroll
+                for (int i = 0; i < N / 2; ++i) {
+                    if (i < n) {
+                        const float keep = up ? v[i + n] : v[i];
+                        const float send = up ? v[i] : v[i + n];
+                        const float got = __shfl_xor_sync(0xffffffffu, send, o);
+                        v[i] = MAX ? fmaxf(keep, got) : keep + got;
+                    }
+                }
+            } else {
+                const float got = __shfl_xor_sync(0xffffffffu, v[0], o);
+                v[0] = MAX ? fmaxf(v[0], got) : v[0] + got;
+            }
+        }
+        // N = 32: lane l holds row l. N = 16: lanes 2r and 2r + 1 both hold row r.
+        if (N == 32) dst[lane] = v[0];
+        else if ((lane & 1) == 0) dst[lane >> 1] = v[0];
+    }
 }
 
 // Launch-time geometry of the TMA boxes (set by the host from the tensor maps it encoded).
@@ -124,8 +155,11 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     float* s_red = s_alpha + RP;                          // [4][RP] cross-warp reduction scratch
     int32_t* s_lim = (int32_t*)(s_red + 4 * RP);          // [RP] keys visible to each row in the current segment
     int32_t* s_rowloop = s_lim + RP;                      // [RP] loop (0-based) of each packed row
-    int32_t* s_ctl = s_rowloop + RP;                      // [0] abort flag, [1] tensor-memory base, [2] fills issued
-    int32_t* s_prefix = s_ctl + 16;
+    float* s_lfin = (float*)(s_rowloop + RP);             // [2][RP] denominators of a finished piece, by O^T buffer
+    float* s_mfin = s_lfin + 2 * RP;                      // [2][RP] its reference maxima
+    int32_t* s_ctl = (int32_t*)(s_mfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] fills issued
+    int32_t* s_prefix = s_ctl + 16;                       // [B + 1] tile prefix
+    int32_t* s_len = s_prefix + p.B + 1;                  // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -143,7 +177,9 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         mbar_init(&bars[B_PFULL], kSmThreads);
         mbar_init(&bars[B_PFREE], 1);
         mbar_init(&bars[B_OFULL], 1);
+        mbar_init(&bars[B_OFULL + 1], 1);
         mbar_init(&bars[B_OFREE], kSmThreads);
+        mbar_init(&bars[B_OFREE + 1], kSmThreads);
         mbar_init(&bars[B_QFULL], kSmThreads);
         mbar_init(&bars[B_QFULL + 1], kSmThreads);
         mbar_init(&bars[B_DRAIN], 1);
@@ -152,7 +188,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     if (tid < RP) s_rowloop[tid] = tid / p.G;
     if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
-    build_prefix(p, s_prefix, flags);  // contains __syncthreads
+    build_prefix(p, s_prefix, flags, s_len);  // contains __syncthreads
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -177,7 +213,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             uint32_t fill = 0;   // K tile of the n-th tile is fill 2n, its V tile fill 2n + 1
             bool ok = true;
-            PieceWalk walk(p, s_prefix, lo, hi);
+            PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
             while (ok && walk.next(pc, flags)) {
                 WinCursor cur;
@@ -254,20 +290,21 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const uint32_t fillv = 2 * prev_gt + 1;
                 const int slot = (int)(fillv % (uint32_t)nslot);
                 ok = ok && wait_or_abort(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1, abort_flag);
-                if (prev_first && prev_pi > 0) ok = ok && wait_or_abort(&bars[B_OFREE], (prev_pi - 1) & 1, abort_flag);
+                if (prev_first && prev_pi >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
+                    ok = ok && wait_or_abort(&bars[B_OFREE + (prev_pi & 1)], ((prev_pi >> 1) - 1) & 1, abort_flag);
                 if (!ok) return;
                 tc_fence_after_sync();
                 const uint32_t vs = smem_a + (uint32_t)slot * kSlotBytes;
 #pragma unroll
                 for (int ks = 0; ks < UK / 16; ++ks)
-                    umma_bf16(tO, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), smem_desc(pbuf_a + ks * 256, 128, 2048, 0),
+                    umma_bf16(tO + (prev_pi & 1) * RP, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), smem_desc(pbuf_a + ks * 256, 128, 2048, 0),
                               idesc_pv, (prev_first && ks == 0) ? 0u : 1u);
                 umma_commit(&bars[B_EMPTY + slot]);
                 umma_commit(&bars[B_PFREE]);
-                if (prev_last) umma_commit(&bars[B_OFULL]);
+                if (prev_last) umma_commit(&bars[B_OFULL + (prev_pi & 1)]);
             };
 
-            PieceWalk walk(p, s_prefix, lo, hi);
+            PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
             while (ok && walk.next(pc, flags)) {
                 for (int t = pc.t0; t < pc.t1 && ok; ++t) {
@@ -317,34 +354,68 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         };
         bool aborted = false;   // agreed by all 128 threads
 
-        named_barrier_sync(1, kSmThreads);   // s_rowloop visible (written before the block-wide barrier, kept for clarity)
+        // Rows R..RP-1 of both packed-query buffers stay zero for the whole kernel.
+        for (int i = tid; i < 2 * C::QBUF / 16; i += kSmThreads) *(uint4*)(qbuf + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+        named_barrier_sync(1, kSmThreads);
 
-        // Packed query rows of a piece into buffer `buf`: [chunk c][row r][16 bytes], rows >= R zero.
-        auto load_q = [&](const Piece& q_pc, int buf) {
-            uint8_t* dst = qbuf + buf * C::QBUF;
-            for (int id = tid; id < RP * 16; id += kSmThreads) {
+        // Packed query rows of a piece into buffer `buf`, [chunk c][row r][16 bytes]: asynchronous copies ...
+        auto load_q_begin = [&](const Piece& q_pc, int buf) {
+            const uint32_t dst = smem_u32(qbuf + buf * C::QBUF);
+            for (int id = tid; id < p.R * 16; id += kSmThreads) {
                 const int r = id >> 4, c = id & 15;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (r < p.R) {
-                    const int l = s_rowloop[r], g = r - l * p.G;
-                    v = *(const uint4*)(qg + (((int64_t)q_pc.b * p.L + l) * p.Hq + q_pc.hg * p.G + g) * UD + c * 8);
-                }
-                *(uint4*)(dst + c * C::QLBO + r * 16) = v;
+                const int l = s_rowloop[r], g = r - l * p.G;
+                const __nv_bfloat16* src = qg + (((int64_t)q_pc.b * p.L + l) * p.Hq + q_pc.hg * p.G + g) * UD + c * 8;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + c * C::QLBO + r * 16), "l"(src) : "memory");
             }
+        };
+        // ... and their completion, handed to the tensor core's view of shared memory.
+        auto load_q_end = [&](int buf) {
+            asm volatile("cp.async.wait_all;" ::: "memory");
             fence_proxy_async_smem();
             mbar_arrive(&bars[B_QFULL + buf]);
         };
 
+        // Epilogue of a finished piece (its denominators and maxima are parked in s_lfin / s_mfin): O^T out of
+        // tensor memory into the split partial. Runs one piece late, while the next piece is already streaming.
+        bool ep_pending = false;
+        uint32_t ep_pi = 0;
+        int64_t ep_prow = 0;
+        auto epilogue = [&]() {
+            const int ob = (int)(ep_pi & 1);
+            sm_wait(&bars[B_OFULL + ob], (ep_pi >> 1) & 1);
+            if (tid < p.R)
+                *(float2*)(p.part_ml + (ep_prow + tid) * 2) = make_float2(s_mfin[ob * RP + tid], s_lfin[ob * RP + tid]);
+            uint32_t o[RP];
+            if (!failed) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tO + ob * RP + lane_off + c * 16, o + c * 16);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+            }
+            mbar_arrive(&bars[B_OFREE + ob]);
+            if (!failed) {
+#pragma unroll
+                for (int r = 0; r < RP; ++r)
+                    if (r < p.R) p.part_acc[(ep_prow + r) * UD + tid] = __uint_as_float(o[r]);
+            }
+            ep_pending = false;
+        };
+
         uint32_t gt = 0, pi = 0;
-        PieceWalk walk(p, s_prefix, lo, hi);
+        PieceWalk walk(p, s_prefix, lo, hi, s_len);
         Piece pc, npc;
         bool have = walk.next(pc, flags);
-        if (have) load_q(pc, 0);
+        if (have) {
+            load_q_begin(pc, 0);
+            load_q_end(0);
+        }
         while (have && !aborted) {
-            // The next piece's query rows go into the other buffer now: every product that read it has completed
+            // The next piece's query rows go into the other buffer: every product that read it has completed
             // (this thread has seen the scores of the last tile of the piece before).
             const bool nhave = walk.next(npc, flags);
-            if (nhave) load_q(npc, (pi + 1) & 1);
+            if (nhave) load_q_begin(npc, (pi + 1) & 1);
+            const uint32_t tOb = tO + (pi & 1) * RP;
 
             // ---- per-piece state ----
             int cmin = 0x7fffffff;
@@ -423,10 +494,11 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         break;
                     }
                     // ---- slow path: true maxima over the 128 keys, new references, rescale O^T ----
+                    {
+                        float v[RP];
 #pragma unroll
-                    for (int r = 0; r < RP; ++r) {
-                        const float v = warp_max(__uint_as_float(sv[r]) * scale);
-                        if (lane == 0) s_red[wid * RP + r] = v;
+                        for (int r = 0; r < RP; ++r) v[r] = __uint_as_float(sv[r]) * scale;
+                        warp_reduce_rows<RP, true>(v, lane, s_red + wid * RP);
                     }
                     named_barrier_sync(1, kSmThreads);
                     if (tid < RP) {
@@ -446,11 +518,11 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
                             for (int c = 0; c < RP / 16; ++c) {
                                 uint32_t o[16];
-                                tmem_ld16(tO + lane_off + c * 16, o);
+                                tmem_ld16(tOb + lane_off + c * 16, o);
                                 tmem_wait_ld();
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * s_alpha[c * 16 + j]);
-                                tmem_st16(tO + lane_off + c * 16, o);
+                                tmem_st16(tOb + lane_off + c * 16, o);
                             }
                             tmem_wait_st();
                             tc_fence_before_sync();
@@ -492,39 +564,32 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 fence_proxy_async_smem();
                 mbar_arrive(&bars[B_PFULL]);
                 if (pc.kind == 1) cur.advance(p, pc.sp);
+                if (t == pc.t0) {
+                    // Work that was put off so that the pipeline restarts first: the partial of the piece before,
+                    // and the hand-over of the next piece's query rows.
+                    if (ep_pending) epilogue();
+                    if (nhave) load_q_end((pi + 1) & 1);
+                }
             }
             if (aborted) break;
 
-            // ---- end of piece: denominators across the 128 keys, then O^T out of tensor memory ----
-#pragma unroll
-            for (int r = 0; r < RP; ++r) {
-                const float v = warp_sum(lsum[r]);
-                if (lane == 0) s_red[wid * RP + r] = v;
-            }
-            sm_wait(&bars[B_OFULL], pi & 1);
+            // ---- end of piece: denominators across the 128 keys; the rest of the epilogue runs one piece late ----
+            warp_reduce_rows<RP, false>(lsum, lane, s_red + wid * RP);
             named_barrier_sync(1, kSmThreads);
-            const int64_t prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // hpc == 1 on this path
-            if (tid < p.R)
-                *(float2*)(p.part_ml + (prow + tid) * 2) =
-                    make_float2(s_mref[tid], (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]));
-            uint32_t o[RP];
-            if (!failed) {
-                tc_fence_after_sync();
-#pragma unroll
-                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tO + lane_off + c * 16, o + c * 16);
-                tmem_wait_ld();
-                tc_fence_before_sync();
+            if (tid < RP) {
+                s_lfin[(pi & 1) * RP + tid] = (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]);
+                s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
             }
-            mbar_arrive(&bars[B_OFREE]);
-            if (!failed) {
-#pragma unroll
-                for (int r = 0; r < RP; ++r)
-                    if (r < p.R) p.part_acc[(prow + r) * UD + tid] = __uint_as_float(o[r]);
-            }
-            named_barrier_sync(1, kSmThreads);   // s_red and s_mref are rewritten by the next piece
+            ep_pending = true;
+            ep_pi = pi;
+            ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // hpc == 1 on this path
             pc = npc;
             have = nhave;
             ++pi;
+            if (!have) {
+                named_barrier_sync(1, kSmThreads);   // s_lfin / s_mfin of the last piece visible to all
+                epilogue();
+            }
         }
     }
 
