@@ -89,8 +89,9 @@ typedef struct {
     int32_t key_slices;    /* 16-key slices per pipeline tile (bf16 path; 1, 2 or 4) */
     int32_t stages;        /* depth of the shared-memory pipeline (bf16 path) */
     int32_t ctas_per_sm;   /* persistent thread blocks per SM */
-    int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (3..6) and
+    int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (4 or 6) and
                               heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block) */
+    int32_t loads_in_flight; /* PLT_PATH_TCGEN05: K tiles (and likewise V tiles) kept in flight at most, clamped to stages / 2; 0 = automatic */
 } plt_decode_attn_config;
 
 /*

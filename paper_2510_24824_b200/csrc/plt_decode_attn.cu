@@ -211,17 +211,16 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
     h->umma = false;
     if (config->kernel_path < 0 || config->kernel_path > PLT_PATH_TCGEN05)
         return fail(nullptr, PLT_ERR_INVALID_ARG, "kernel_path %d outside [0, 2]", config->kernel_path);
+    if (config->loads_in_flight < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "loads_in_flight %d < 0", config->loads_in_flight);
     if (config->kernel_path == PLT_PATH_TCGEN05 && !umma_eligible(config))
         return fail(nullptr, PLT_ERR_UNSUPPORTED,
                     "the tcgen05 path needs bf16, d = 128 and a page size that divides or is a multiple of 128");
     if (h->bf16 && want_umma(config)) {
+        // Ring slots: an even number, so that a slot is always refilled by the stream (K or V) that used it before.
         int nslot = config->stages;
-        if (nslot == 0) {
-            nslot = main_umma_max_slots();
-            while (nslot > 3 && main_umma_smem(g.R, nslot, config->max_batch) > 227 * 1024) --nslot;
-        }
-        if (nslot < 3 || nslot > main_umma_max_slots())
-            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [3, %d] on the tcgen05 path", nslot, main_umma_max_slots());
+        if (nslot == 0) nslot = main_umma_smem(g.R, 6, config->max_batch) <= 227 * 1024 ? 6 : 4;
+        if (nslot != 4 && nslot != 6)
+            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path (supported: 4 or 6 ring slots)", nslot);
         const size_t smem = main_umma_smem(g.R, nslot, config->max_batch);
         if (smem > 227 * 1024)
             return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 path needs %zu bytes of shared memory (> 227 KB)", smem);
@@ -438,7 +437,8 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
         }
         if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
         if (h->umma)
-            e = launch_main_umma(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox, stream);
+            e = launch_main_umma(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox,
+                                 c.loads_in_flight > 0 ? c.loads_in_flight : 2, stream);
         else
             e = launch_main_bf16(h->var, h->maps, p, stream);
     } else {

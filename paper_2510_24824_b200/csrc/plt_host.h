@@ -35,7 +35,7 @@ int main_umma_max_slots();
 size_t main_umma_smem(int R, int nslot, int max_batch);
 cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm);
 cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
-                             int wbox, cudaStream_t stream);
+                             int wbox, int cap, cudaStream_t stream);
 
 cudaError_t launch_reduce(const Params& p, bool bf16, bool overlap, cudaStream_t stream);
 

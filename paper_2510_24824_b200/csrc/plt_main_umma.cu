@@ -16,8 +16,9 @@
 // the tensor core itself, once, whatever R is; the 128 softmax threads own one key each (their
 // tensor-memory lane) and the RP scores of that key.
 //
-// Warp roles: warps 0-3 softmax and epilogue (thread = key / output dimension), warp 4 TMA
-// producer, warp 5 MMA issuer and owner of the tensor-memory allocation.
+// Warp roles: warps 0-3 softmax and epilogue (thread = key / output dimension); warp 4 TMA producer
+// of K tiles, warp 6 of V tiles; warp 5 issues the S^T products and owns the tensor-memory
+// allocation, warp 7 issues the O^T products. One lane works in each of warps 4-7.
 //
 // Online softmax with a lazily updated reference maximum per row: probabilities are formed against
 // a reference that may lag the true running maximum by up to kSlack powers of two; only when a
@@ -39,13 +40,13 @@ constexpr int kSlotBytes = UK * UD * 2;  // one K tile or one V tile of one KV h
 constexpr int kHalfBytes = UK * 128;     // one 64-element half of a tile: [128 keys][128 bytes]
 constexpr int kMaxSlots = 6;
 constexpr int kSmThreads = 128;          // softmax threads
-constexpr int kUmmaThreads = 192;
+constexpr int kUmmaThreads = 256;
 constexpr float kSlack = 8.f;
 constexpr uint64_t kUmmaWaitNs = 1000000000ull;
 
 // mbarrier indices
 constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_PFREE = 19, B_OFULL = 20 /* two */,
-              B_OFREE = 22 /* two */, B_QFULL = 24 /* two */, B_DRAIN = 26, B_COUNT = 27;
+              B_OFREE = 22 /* two */, B_QFULL = 24 /* two */, B_DRAIN = 26 /* two */, B_COUNT = 28;
 
 template <int RP>
 struct UCfg {
@@ -135,6 +136,72 @@ struct UmmaGeom {
     int nslot;       // ring slots of kSlotBytes
     int kbox;        // keys per box of the shared cache (min(128, page size or capacity))
     int wbox;        // keys per box of a window (min(128, w))
+    int cap;         // tiles each of the two producers keeps in flight (issued, not landed) at most; 2 cap <= nslot
+};
+
+// Ring position of the K tile / V tile of the n-th tile a block streams (T tiles in all): K(0), then
+// K(n), V(n-1) for n = 1 .. T-1, then V(T-1).
+__device__ __forceinline__ uint32_t pos_k(uint32_t n) { return n == 0 ? 0u : 2u * n - 1u; }
+__device__ __forceinline__ uint32_t pos_v(uint32_t n, uint32_t T) { return n + 1 == T ? 2u * T - 1u : 2u * n + 2u; }
+
+// TMA boxes of one tile: (key coordinate, outermost coordinate) per box, the same for K and V.
+struct TileCoords {
+    int nbox, box_keys, head;
+    bool window;
+    int c1[UK / 16], c3[UK / 16];
+};
+
+// Walks the tiles of a block's range in order and yields their box coordinates.
+struct TileSource {
+    PieceWalk walk;
+    Piece pc;
+    WinCursor cur;
+    int t;
+    bool have;
+    __device__ TileSource(const Params& p, const int32_t* sp, int64_t lo, int64_t hi, const int32_t* lens)
+        : walk(p, sp, lo, hi, lens), t(0), have(false) {
+        pc.t0 = pc.t1 = 0;
+        cur.l = 0;
+        cur.key0 = 0;
+    }
+    __device__ void next(const Params& p, const UmmaGeom& geo, TileCoords& tc, uint32_t& flags) {
+        if (!have || t == pc.t1) {
+            have = walk.next(pc, flags);
+            t = pc.t0;
+            if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
+        }
+        tc.head = pc.hg;
+        tc.window = pc.kind == 1;
+        if (pc.kind == 0) {
+            const int key0 = t * UK;
+            tc.box_keys = geo.kbox;
+            if (p.page_size > 0) {
+                const int rem = pc.sp.cmax - key0;   // keys that hold data from key0 on (>= 1)
+                tc.nbox = (min(rem, UK) + tc.box_keys - 1) / tc.box_keys;
+                for (int i = 0; i < tc.nbox; ++i) {
+                    const int key = key0 + i * tc.box_keys;
+                    int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
+                    if (page < 0 || page >= p.num_pool_pages) {
+                        flags |= kDevPageIdClamped;
+                        page = page < 0 ? 0 : p.num_pool_pages - 1;
+                    }
+                    tc.c1[i] = key % p.page_size;
+                    tc.c3[i] = page;
+                }
+            } else {
+                tc.nbox = 1;
+                tc.c1[0] = key0;
+                tc.c3[0] = pc.b;
+            }
+        } else {
+            tc.box_keys = geo.wbox;
+            tc.nbox = 1;
+            tc.c1[0] = cur.key0;
+            tc.c3[0] = pc.b * (p.L - 1) + (cur.l - 1);
+            cur.advance(p, pc.sp);
+        }
+        ++t;
+    }
 };
 
 template <int RP>
@@ -168,6 +235,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     if (tid == 0) {
         s_ctl[0] = 0;
         s_ctl[2] = 0;
+        s_ctl[3] = 0;
         for (int s = 0; s < kMaxSlots; ++s) {
             mbar_init(&bars[B_FULL + s], 1);
             mbar_init(&bars[B_EMPTY + s], 1);
@@ -183,6 +251,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         mbar_init(&bars[B_QFULL], kSmThreads);
         mbar_init(&bars[B_QFULL + 1], kSmThreads);
         mbar_init(&bars[B_DRAIN], 1);
+        mbar_init(&bars[B_DRAIN + 1], 1);
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
@@ -202,140 +271,119 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const bool in_plan = cta < nctas;
     const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
 
-    if (wid == 4) {
-        // ================================ TMA producer (one lane) =================================
+    if (wid == 4 || wid == 6) {
+        // ========================= TMA producers: warp 4 streams K tiles, warp 6 V tiles ==========
+        // Ring positions follow the order of use: K(0), then K(n), V(n-1) for n = 1.., then the last V, so a
+        // V tile (needed one softmax later than its K tile) does not sit in its slot longer than a K tile.
+        // Each producer keeps at most `cap` of its copies in flight: more outstanding requests make the
+        // memory system slower, not faster.
         if (lane == 0 && lo < hi) {
-            tma_prefetch_desc(&tmK);
-            tma_prefetch_desc(&tmV);
-            if (p.L > 1) {
-                tma_prefetch_desc(&tmKw);
-                tma_prefetch_desc(&tmVw);
+            const bool is_v = wid == 6;
+            tma_prefetch_desc(is_v ? &tmV : &tmK);
+            if (p.L > 1) tma_prefetch_desc(is_v ? &tmVw : &tmKw);
+            const uint32_t T = (uint32_t)(hi - lo);
+            const uint32_t cap = (uint32_t)geo.cap;
+            bool ok = true;
+            uint32_t issued = 0;
+            TileSource src(p, s_prefix, lo, hi, s_len);
+            TileCoords tc;
+            for (uint32_t n = 0; n < T && ok; ++n) {
+                src.next(p, geo, tc, flags);
+                const uint32_t pos = is_v ? pos_v(n, T) : pos_k(n);
+                const int slot = (int)(pos % (uint32_t)nslot);
+                const uint32_t use = pos / (uint32_t)nslot;
+                // The copy issued `cap` tiles ago must have landed. With 2 cap <= slots, the slot of that copy
+                // cannot have been refilled and landed again by now, so its phase parity is unambiguous; the one
+                // exception, ring position 0 (which the V stream reuses early), is skipped.
+                if (n >= cap && (is_v || n > cap)) {
+                    const uint32_t q = is_v ? pos_v(n - cap, T) : pos_k(n - cap);
+                    ok = wait_or_abort(&bars[B_FULL + (int)(q % (uint32_t)nslot)], (q / (uint32_t)nslot) & 1, abort_flag);
+                }
+                if (ok && use > 0) ok = wait_or_abort(&bars[B_EMPTY + slot], (use - 1) & 1, abort_flag);
+                if (!ok) break;
+                const CUtensorMap* map = tc.window ? (is_v ? &tmVw : &tmKw) : (is_v ? &tmV : &tmK);
+                uint8_t* dst = smem + (size_t)slot * kSlotBytes;
+                mbar_expect_tx(&bars[B_FULL + slot], (uint32_t)(tc.nbox * tc.box_keys * 256));
+                for (int i = 0; i < tc.nbox; ++i)
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf)
+                        tma_load_4d(dst + hf * kHalfBytes + i * tc.box_keys * 128, map, &bars[B_FULL + slot], hf * 64,
+                                    tc.c1[i], tc.head, tc.c3[i]);
+                ++issued;
             }
-            uint32_t fill = 0;   // K tile of the n-th tile is fill 2n, its V tile fill 2n + 1
+            s_ctl[is_v ? 3 : 2] = (int32_t)issued;
+        }
+    } else if (wid == 5) {
+        // ====================== S^T = K Q^T issuer (one lane); owner of tensor memory ==============
+        if (lane == 0 && lo < hi) {
+            constexpr uint32_t idesc_qk = instr_desc(UK, RP, 0, 0);
+            const uint32_t qbuf_a = smem_u32(qbuf), smem_a = smem_u32(smem);
+            const uint32_t T = (uint32_t)(hi - lo);
             bool ok = true;
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
-            while (ok && walk.next(pc, flags)) {
-                WinCursor cur;
-                if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
-                for (int t = pc.t0; t < pc.t1 && ok; ++t) {
-                    // boxes of this tile: (key coordinate, outermost coordinate), same for K and V
-                    int nbox, c1[UK / 16], c3[UK / 16], box_keys;
-                    const CUtensorMap *mk, *mv;
-                    if (pc.kind == 0) {
-                        const int key0 = t * UK;
-                        mk = &tmK;
-                        mv = &tmV;
-                        box_keys = geo.kbox;
-                        if (p.page_size > 0) {
-                            const int rem = pc.sp.cmax - key0;   // keys that hold data from key0 on (>= 1)
-                            nbox = (min(rem, UK) + box_keys - 1) / box_keys;
-                            for (int i = 0; i < nbox; ++i) {
-                                const int key = key0 + i * box_keys;
-                                int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
-                                if (page < 0 || page >= p.num_pool_pages) {
-                                    flags |= kDevPageIdClamped;
-                                    page = page < 0 ? 0 : p.num_pool_pages - 1;
-                                }
-                                c1[i] = key % p.page_size;
-                                c3[i] = page;
-                            }
-                        } else {
-                            nbox = 1;
-                            c1[0] = key0;
-                            c3[0] = pc.b;
-                        }
-                    } else {
-                        mk = &tmKw;
-                        mv = &tmVw;
-                        box_keys = geo.wbox;
-                        nbox = 1;
-                        c1[0] = cur.key0;
-                        c3[0] = pc.b * (p.L - 1) + (cur.l - 1);
-                        cur.advance(p, pc.sp);
-                    }
-                    const uint32_t bytes = (uint32_t)(nbox * box_keys * 256);
+            walk.next(pc, flags);
+            int t = pc.t0;
+            uint32_t pi = 0;
+            for (uint32_t g = 0; g < T && ok; ++g) {
+                const uint32_t pos = pos_k(g);
+                const int slot = (int)(pos % (uint32_t)nslot);
+                if (t == pc.t0) ok = wait_or_abort(&bars[B_QFULL + (pi & 1)], (pi >> 1) & 1, abort_flag);
+                if (ok && g > 0) ok = wait_or_abort(&bars[B_SFREE], (g - 1) & 1, abort_flag);   // scores of the tile before read out
+                if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
+                const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
 #pragma unroll
-                    for (int which = 0; which < 2; ++which, ++fill) {
-                        const int slot = (int)(fill % (uint32_t)nslot);
-                        const uint32_t use = fill / (uint32_t)nslot;
-                        if (use > 0) ok = ok && wait_or_abort(&bars[B_EMPTY + slot], (use - 1) & 1, abort_flag);
-                        if (!ok) break;
-                        uint8_t* dst = smem + (size_t)slot * kSlotBytes;
-                        mbar_expect_tx(&bars[B_FULL + slot], bytes);
-                        for (int i = 0; i < nbox; ++i)
-#pragma unroll
-                            for (int hf = 0; hf < 2; ++hf)
-                                tma_load_4d(dst + hf * kHalfBytes + i * box_keys * 128, which == 0 ? mk : mv,
-                                            &bars[B_FULL + slot], hf * 64, c1[i], pc.hg, c3[i]);
-                    }
+                for (int kk = 0; kk < UD / 16; ++kk)
+                    umma_bf16(tS, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
+                              smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
+                umma_commit(&bars[B_SFULL]);
+                umma_commit(&bars[B_EMPTY + slot]);
+                if (++t == pc.t1 && g + 1 < T) {
+                    walk.next(pc, flags);
+                    t = pc.t0;
+                    ++pi;
                 }
             }
-            s_ctl[2] = (int32_t)fill;
         }
-    } else if (wid == 5) {
-        // ================================ MMA issuer (one lane) ===================================
+    } else if (wid == 7) {
+        // ============================ O^T += V^T P^T issuer (one lane) ============================
         if (lane == 0 && lo < hi) {
-            constexpr uint32_t idesc_qk = instr_desc(UK, RP, 0, 0);
             constexpr uint32_t idesc_pv = instr_desc(UD, RP, 1, 1);
-            const uint32_t pbuf_a = smem_u32(pbuf), qbuf_a = smem_u32(qbuf), smem_a = smem_u32(smem);
+            const uint32_t pbuf_a = smem_u32(pbuf), smem_a = smem_u32(smem);
+            const uint32_t T = (uint32_t)(hi - lo);
             bool ok = true;
-            uint32_t gt = 0, pi = 0;             // tiles and pieces done by this block so far
-            bool have_prev = false;              // a tile whose S^T product is issued but whose PV product is not
-            uint32_t prev_gt = 0, prev_pi = 0;
-            bool prev_first = false, prev_last = false;
-
-            auto issue_pv = [&]() {
-                ok = ok && wait_or_abort(&bars[B_PFULL], prev_gt & 1, abort_flag);
-                const uint32_t fillv = 2 * prev_gt + 1;
-                const int slot = (int)(fillv % (uint32_t)nslot);
-                ok = ok && wait_or_abort(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1, abort_flag);
-                if (prev_first && prev_pi >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
-                    ok = ok && wait_or_abort(&bars[B_OFREE + (prev_pi & 1)], ((prev_pi >> 1) - 1) & 1, abort_flag);
-                if (!ok) return;
+            PieceWalk walk(p, s_prefix, lo, hi, s_len);
+            Piece pc;
+            walk.next(pc, flags);
+            int t = pc.t0;
+            uint32_t pi = 0;
+            for (uint32_t g = 0; g < T && ok; ++g) {
+                const uint32_t pos = pos_v(g, T);
+                const int slot = (int)(pos % (uint32_t)nslot);
+                const bool first = t == pc.t0, last = t == pc.t1 - 1;
+                if (first && pi >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
+                    ok = wait_or_abort(&bars[B_OFREE + (pi & 1)], ((pi >> 1) - 1) & 1, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[B_PFULL], g & 1, abort_flag);
+                if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t vs = smem_a + (uint32_t)slot * kSlotBytes;
 #pragma unroll
                 for (int ks = 0; ks < UK / 16; ++ks)
-                    umma_bf16(tO + (prev_pi & 1) * RP, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), smem_desc(pbuf_a + ks * 256, 128, 2048, 0),
-                              idesc_pv, (prev_first && ks == 0) ? 0u : 1u);
-                umma_commit(&bars[B_EMPTY + slot]);
+                    umma_bf16(tO + (pi & 1) * RP, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2),
+                              smem_desc(pbuf_a + ks * 256, 128, 2048, 0), idesc_pv, (first && ks == 0) ? 0u : 1u);
                 umma_commit(&bars[B_PFREE]);
-                if (prev_last) umma_commit(&bars[B_OFULL + (prev_pi & 1)]);
-            };
-
-            PieceWalk walk(p, s_prefix, lo, hi, s_len);
-            Piece pc;
-            while (ok && walk.next(pc, flags)) {
-                for (int t = pc.t0; t < pc.t1 && ok; ++t) {
-                    // ---- S^T of tile gt ----
-                    if (t == pc.t0) ok = ok && wait_or_abort(&bars[B_QFULL + (pi & 1)], (pi >> 1) & 1, abort_flag);
-                    const uint32_t fillk = 2 * gt;
-                    const int slot = (int)(fillk % (uint32_t)nslot);
-                    ok = ok && wait_or_abort(&bars[B_FULL + slot], (fillk / (uint32_t)nslot) & 1, abort_flag);
-                    if (gt > 0) ok = ok && wait_or_abort(&bars[B_SFREE], (gt - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
-                    const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
-#pragma unroll
-                    for (int kk = 0; kk < UD / 16; ++kk)
-                        umma_bf16(tS, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
-                                  smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
-                    umma_commit(&bars[B_SFULL]);
-                    umma_commit(&bars[B_EMPTY + slot]);
-                    // ---- O^T += V^T P^T of the tile before, whose probabilities are ready by now ----
-                    if (have_prev) issue_pv();
-                    have_prev = true;
-                    prev_gt = gt;
-                    prev_pi = pi;
-                    prev_first = (t == pc.t0);
-                    prev_last = (t == pc.t1 - 1);
-                    ++gt;
+                umma_commit(&bars[B_EMPTY + slot]);
+                if (last) umma_commit(&bars[B_OFULL + (pi & 1)]);
+                if (++t == pc.t1 && g + 1 < T) {
+                    walk.next(pc, flags);
+                    t = pc.t0;
+                    ++pi;
                 }
-                ++pi;
             }
-            if (ok && have_prev) issue_pv();
         }
     } else {
         // ============================ softmax and epilogue (warps 0-3) ============================
@@ -549,7 +597,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 }
                 if (masked && nvalid < UK) {
                     // V rows that hold no data may contain anything: zero them so that 0 * garbage stays 0
-                    const uint32_t fillv = 2 * gt + 1;
+                    const uint32_t fillv = pos_v(gt, (uint32_t)(hi - lo));
                     const int slot = (int)(fillv % (uint32_t)nslot);
                     sm_wait(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1);
                     if (!failed && tid >= nvalid) {
@@ -596,15 +644,20 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     // ---- common exit: nothing of this block may still be in flight when tensor memory is freed ----
     __syncthreads();
     const bool gave_up = *abort_flag != 0;
-    if (wid == 5 && lane == 0) {
-        umma_commit(&bars[B_DRAIN]);   // arrives once every product issued by this thread has completed
-        mbar_wait_bounded(&bars[B_DRAIN], 0, kUmmaWaitNs);
+    if ((wid == 5 || wid == 7) && lane == 0) {
+        uint64_t* drain = &bars[wid == 5 ? B_DRAIN : B_DRAIN + 1];
+        umma_commit(drain);   // arrives once every product issued by this thread has completed
+        mbar_wait_bounded(drain, 0, kUmmaWaitNs);
     }
-    if (wid == 4 && lane == 0 && gave_up) {
+    if ((wid == 4 || wid == 6) && lane == 0 && gave_up) {
         // give every copy that was issued a bounded chance to land
-        const uint32_t fills = (uint32_t)s_ctl[2];
-        for (uint32_t f = fills > (uint32_t)nslot ? fills - (uint32_t)nslot : 0; f < fills; ++f)
-            mbar_wait_bounded(&bars[B_FULL + (int)(f % (uint32_t)nslot)], (f / (uint32_t)nslot) & 1, kUmmaWaitNs);
+        const bool is_v = wid == 6;
+        const uint32_t T = (uint32_t)(hi - lo);
+        const uint32_t issued = (uint32_t)s_ctl[is_v ? 3 : 2];
+        for (uint32_t n = issued > (uint32_t)nslot ? issued - (uint32_t)nslot : 0; n < issued; ++n) {
+            const uint32_t pos = is_v ? pos_v(n, T) : pos_k(n);
+            mbar_wait_bounded(&bars[B_FULL + (int)(pos % (uint32_t)nslot)], (pos / (uint32_t)nslot) & 1, kUmmaWaitNs);
+        }
     }
     if (gave_up) flags |= kDevWaitTimeout;
     if (flags) atomicOr(p.status, flags);
@@ -643,8 +696,8 @@ cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm) {
 }
 
 cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
-                             int wbox, cudaStream_t stream) {
-    const UmmaGeom geo{nslot, kbox, wbox};
+                             int wbox, int cap, cudaStream_t stream) {
+    const UmmaGeom geo{nslot, kbox, wbox, cap < 1 ? 1 : (2 * cap > nslot ? nslot / 2 : cap)};
     const int rp = main_umma_rows(p.R);
     if (rp == 16)
         plt_decode_main_umma<16><<<grid, kUmmaThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo);
