@@ -45,17 +45,20 @@ constexpr float kSlack = 8.f;
 constexpr uint64_t kUmmaWaitNs = 1000000000ull;
 
 // mbarrier indices
-constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_PFREE = 19, B_OFULL = 20 /* two */,
-              B_OFREE = 22 /* two */, B_QFULL = 24 /* two */, B_DRAIN = 26 /* two */, B_COUNT = 28;
+constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16 /* two */, B_SFREE = 18 /* two */, B_PFULL = 20, B_PFREE = 21,
+              B_OFULL = 22 /* two */, B_OFREE = 24 /* two */, B_DRAIN = 26 /* two */, B_COUNT = 28;
 
 template <int RP>
 struct UCfg {
     static constexpr int QLBO = RP * 16 + 16;      // bytes between the 16-byte column chunks of the packed query tile
     static constexpr int QBUF = 16 * QLBO;         // one packed query tile: [16 chunks][RP rows][16 bytes] (+ pad)
     static constexpr int PBUF = RP * 256;          // probabilities: [RP / 8][128 keys][16 bytes]
-    static constexpr int TMEM_COLS = 4 * RP;       // S^T, then two O^T buffers, RP columns each (power of two)
+    // Tensor memory: two S^T buffers (tile parity), then per piece parity an O^T buffer followed by the denominators (every lane of
+    // the latter holds the same RP row sums), RP columns each; rounded up to a power of two.
+    static constexpr int TMEM_COLS = RP == 16 ? 128 : (RP == 32 ? 256 : 512);
+    static constexpr int ONES_BYTES = 128 * 32;    // A operand of the denominator product: 128 x 16 ones
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
-        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 4) + 64 +
+        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + ONES_BYTES + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 2) + 64 +
                (size_t)(2 * max_batch + 4) * 4;
     }
 };
@@ -72,9 +75,9 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, 
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Bounded wait that also gives up as soon as another thread of the block has given up.
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait that also gives up as soon as another thread of the block has given up. The slow part is kept
+// out of line: this kernel has eight warps in different loops, and its instruction footprint decides its speed.
+__device__ __noinline__ bool wait_or_abort_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -88,6 +91,12 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     }
     return true;
 }
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_or_abort_slow(bar, parity, abort_flag);
+}
+// Out-of-line step of the piece walk (the plan arithmetic is long once unrolled over the loops).
+__device__ __noinline__ bool walk_next(PieceWalk& walk, Piece& pc, uint32_t& flags) { return walk.next(pc, flags); }
 
 // Reduces N values per lane across the 32 lanes of a warp with N - 1 (+ a few) shuffles instead of 5 N: each
 // step halves the values a lane still carries and doubles the lanes they cover. The result of row r goes to
@@ -164,7 +173,7 @@ struct TileSource {
         cur.l = 0;
         cur.key0 = 0;
     }
-    __device__ void next(const Params& p, const UmmaGeom& geo, TileCoords& tc, uint32_t& flags) {
+    __device__ __noinline__ void next(const Params& p, const UmmaGeom& geo, TileCoords& tc, uint32_t& flags) {
         if (!have || t == pc.t1) {
             have = walk.next(pc, flags);
             t = pc.t0;
@@ -215,15 +224,15 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int nslot = geo.nslot;
     uint8_t* pbuf = smem + (size_t)nslot * kSlotBytes;
     uint8_t* qbuf = pbuf + C::PBUF;                       // two buffers of QBUF
-    uint64_t* bars = (uint64_t*)(qbuf + 2 * C::QBUF);
+    uint8_t* ones = qbuf + 2 * C::QBUF;                   // 128 x 16 bf16 ones
+    uint64_t* bars = (uint64_t*)(ones + C::ONES_BYTES);
     float* s_negm = (float*)(bars + B_COUNT);             // [RP] minus the reference maximum (1e30 while there is none)
     float* s_mref = s_negm + RP;                          // [RP] reference maximum, log2 units
     float* s_alpha = s_mref + RP;                         // [RP] rescale factors of the slow path
     float* s_red = s_alpha + RP;                          // [4][RP] cross-warp reduction scratch
     int32_t* s_lim = (int32_t*)(s_red + 4 * RP);          // [RP] keys visible to each row in the current segment
     int32_t* s_rowloop = s_lim + RP;                      // [RP] loop (0-based) of each packed row
-    float* s_lfin = (float*)(s_rowloop + RP);             // [2][RP] denominators of a finished piece, by O^T buffer
-    float* s_mfin = s_lfin + 2 * RP;                      // [2][RP] its reference maxima
+    float* s_mfin = (float*)(s_rowloop + RP);             // [2][RP] reference maxima of a finished piece, by O^T buffer
     int32_t* s_ctl = (int32_t*)(s_mfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] fills issued
     int32_t* s_prefix = s_ctl + 16;                       // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                  // [B] clamped sequence lengths
@@ -241,20 +250,24 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             mbar_init(&bars[B_EMPTY + s], 1);
         }
         mbar_init(&bars[B_SFULL], 1);
+        mbar_init(&bars[B_SFULL + 1], 1);
         mbar_init(&bars[B_SFREE], kSmThreads);
+        mbar_init(&bars[B_SFREE + 1], kSmThreads);
         mbar_init(&bars[B_PFULL], kSmThreads);
         mbar_init(&bars[B_PFREE], 1);
         mbar_init(&bars[B_OFULL], 1);
         mbar_init(&bars[B_OFULL + 1], 1);
         mbar_init(&bars[B_OFREE], kSmThreads);
         mbar_init(&bars[B_OFREE + 1], kSmThreads);
-        mbar_init(&bars[B_QFULL], kSmThreads);
-        mbar_init(&bars[B_QFULL + 1], kSmThreads);
         mbar_init(&bars[B_DRAIN], 1);
         mbar_init(&bars[B_DRAIN + 1], 1);
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
+    for (int i = tid; i < C::ONES_BYTES / 4; i += kUmmaThreads) ((uint32_t*)ones)[i] = 0x3f803f80u;
+    // Rows R..RP-1 of both packed-query buffers stay zero for the whole kernel.
+    for (int i = tid; i < 2 * C::QBUF / 16; i += kUmmaThreads) *(uint4*)(qbuf + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
     if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags, s_len);  // contains __syncthreads
@@ -262,7 +275,8 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = (uint32_t)s_ctl[1];
-    const uint32_t tS = tmem_base, tO = tmem_base + RP;
+    // S^T of tile parity g at tS + g RP; O^T of piece parity b at tO + 2 b RP, its denominators RP further
+    const uint32_t tS = tmem_base, tO = tmem_base + 2 * RP;
 
     const int64_t T = s_prefix[p.B];
     const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
@@ -314,50 +328,86 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             s_ctl[is_v ? 3 : 2] = (int32_t)issued;
         }
     } else if (wid == 5) {
-        // ====================== S^T = K Q^T issuer (one lane); owner of tensor memory ==============
-        if (lane == 0 && lo < hi) {
+        // ============ S^T = K Q^T issuer (lane 0 issues); owner of tensor memory ==================
+        // The whole warp also copies the packed query rows of each piece into shared memory,
+        // [16-byte column chunk c][row r], one piece ahead of the products that read them.
+        if (lo < hi) {
             constexpr uint32_t idesc_qk = instr_desc(UK, RP, 0, 0);
             const uint32_t qbuf_a = smem_u32(qbuf), smem_a = smem_u32(smem);
             const uint32_t T = (uint32_t)(hi - lo);
+            const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
+            auto load_q = [&](const Piece& q_pc, int buf) {
+                const uint32_t dst = qbuf_a + buf * C::QBUF;
+                for (int id = lane; id < p.R * 16; id += 32) {
+                    const int r = id >> 4, c = id & 15;
+                    const int l = s_rowloop[r], g = r - l * p.G;
+                    const __nv_bfloat16* src = qg + (((int64_t)q_pc.b * p.L + l) * p.Hq + q_pc.hg * p.G + g) * UD + c * 8;
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + c * C::QLBO + r * 16), "l"(src) : "memory");
+                }
+            };
             bool ok = true;
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
-            Piece pc;
-            walk.next(pc, flags);
+            Piece pc, npc;
+            walk_next(walk, pc, flags);
+            bool nhave = false;
+            load_q(pc, 0);
             int t = pc.t0;
             uint32_t pi = 0;
-            for (uint32_t g = 0; g < T && ok; ++g) {
+            for (uint32_t g = 0; g < T; ++g) {
                 const uint32_t pos = pos_k(g);
                 const int slot = (int)(pos % (uint32_t)nslot);
-                if (t == pc.t0) ok = wait_or_abort(&bars[B_QFULL + (pi & 1)], (pi >> 1) & 1, abort_flag);
-                if (ok && g > 0) ok = wait_or_abort(&bars[B_SFREE], (g - 1) & 1, abort_flag);   // scores of the tile before read out
-                if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
-                const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
+                if (t == pc.t0) {
+                    // this piece's rows have arrived; hand them to the tensor core's view of shared memory
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    if (g >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
+                        ok = wait_or_abort(&bars[B_SFREE + (g & 1)], ((g >> 1) - 1) & 1, abort_flag);
+                    if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
+                        const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
 #pragma unroll
-                for (int kk = 0; kk < UD / 16; ++kk)
-                    umma_bf16(tS, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
-                              smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
-                umma_commit(&bars[B_SFULL]);
-                umma_commit(&bars[B_EMPTY + slot]);
+                        for (int kk = 0; kk < UD / 16; ++kk)
+                            umma_bf16(tS + (g & 1) * RP, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
+                                      smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
+                        umma_commit(&bars[B_SFULL + (g & 1)]);
+                        umma_commit(&bars[B_EMPTY + slot]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (t == pc.t0) {
+                    // The other buffer was last read by the products of the piece before this one; the last of
+                    // them (tile g - 1) must have completed before the next piece's rows are fetched into it.
+                    if (lane == 0 && g > 0) ok = wait_or_abort(&bars[B_SFULL + ((g - 1) & 1)], ((g - 1) >> 1) & 1, abort_flag);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    nhave = walk_next(walk, npc, flags);
+                    if (nhave) load_q(npc, (pi + 1) & 1);
+                }
                 if (++t == pc.t1 && g + 1 < T) {
-                    walk.next(pc, flags);
+                    pc = npc;
                     t = pc.t0;
                     ++pi;
                 }
             }
         }
     } else if (wid == 7) {
-        // ============================ O^T += V^T P^T issuer (one lane) ============================
+        // ================= O^T += V^T P^T and denominators += 1 P^T issuer (one lane) ==============
         if (lane == 0 && lo < hi) {
             constexpr uint32_t idesc_pv = instr_desc(UD, RP, 1, 1);
+            constexpr uint32_t idesc_l = instr_desc(128, RP, 0, 1);
             const uint32_t pbuf_a = smem_u32(pbuf), smem_a = smem_u32(smem);
+            const uint64_t ones_desc = smem_desc(smem_u32(ones), 2048, 128, 0);   // K-major, no swizzle: all ones anyway
             const uint32_t T = (uint32_t)(hi - lo);
             bool ok = true;
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
-            walk.next(pc, flags);
+            walk_next(walk, pc, flags);
             int t = pc.t0;
             uint32_t pi = 0;
             for (uint32_t g = 0; g < T && ok; ++g) {
@@ -371,15 +421,19 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t vs = smem_a + (uint32_t)slot * kSlotBytes;
+                const uint32_t tOb = tO + (pi & 1) * 2 * RP;
 #pragma unroll
-                for (int ks = 0; ks < UK / 16; ++ks)
-                    umma_bf16(tO + (pi & 1) * RP, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2),
-                              smem_desc(pbuf_a + ks * 256, 128, 2048, 0), idesc_pv, (first && ks == 0) ? 0u : 1u);
+                for (int ks = 0; ks < UK / 16; ++ks) {
+                    const uint64_t pd = smem_desc(pbuf_a + ks * 256, 128, 2048, 0);
+                    const uint32_t acc = (first && ks == 0) ? 0u : 1u;
+                    umma_bf16(tOb, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), pd, idesc_pv, acc);
+                    umma_bf16(tOb + RP, ones_desc, pd, idesc_l, acc);
+                }
                 umma_commit(&bars[B_PFREE]);
                 umma_commit(&bars[B_EMPTY + slot]);
                 if (last) umma_commit(&bars[B_OFULL + (pi & 1)]);
                 if (++t == pc.t1 && g + 1 < T) {
-                    walk.next(pc, flags);
+                    walk_next(walk, pc, flags);
                     t = pc.t0;
                     ++pi;
                 }
@@ -391,7 +445,6 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // output dimension tid (lane tid of O^T).
         const uint32_t lane_off = (uint32_t)(wid * 32) << 16;
         const float scale = p.scale_log2;
-        const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
         // `failed`: a wait of this warp ran out; the warp stops touching data but keeps the common control flow.
         // Kept warp-uniform, because the tensor-memory loads and stores are warp-collective.
         bool failed = false;
@@ -402,47 +455,33 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         };
         bool aborted = false;   // agreed by all 128 threads
 
-        // Rows R..RP-1 of both packed-query buffers stay zero for the whole kernel.
-        for (int i = tid; i < 2 * C::QBUF / 16; i += kSmThreads) *(uint4*)(qbuf + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-        named_barrier_sync(1, kSmThreads);
-
-        // Packed query rows of a piece into buffer `buf`, [chunk c][row r][16 bytes]: asynchronous copies ...
-        auto load_q_begin = [&](const Piece& q_pc, int buf) {
-            const uint32_t dst = smem_u32(qbuf + buf * C::QBUF);
-            for (int id = tid; id < p.R * 16; id += kSmThreads) {
-                const int r = id >> 4, c = id & 15;
-                const int l = s_rowloop[r], g = r - l * p.G;
-                const __nv_bfloat16* src = qg + (((int64_t)q_pc.b * p.L + l) * p.Hq + q_pc.hg * p.G + g) * UD + c * 8;
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + c * C::QLBO + r * 16), "l"(src) : "memory");
-            }
-        };
-        // ... and their completion, handed to the tensor core's view of shared memory.
-        auto load_q_end = [&](int buf) {
-            asm volatile("cp.async.wait_all;" ::: "memory");
-            fence_proxy_async_smem();
-            mbar_arrive(&bars[B_QFULL + buf]);
-        };
-
-        // Epilogue of a finished piece (its denominators and maxima are parked in s_lfin / s_mfin): O^T out of
+        // Epilogue of a finished piece (its reference maxima are parked in s_mfin): O^T out of
         // tensor memory into the split partial. Runs one piece late, while the next piece is already streaming.
         bool ep_pending = false;
         uint32_t ep_pi = 0;
         int64_t ep_prow = 0;
         auto epilogue = [&]() {
             const int ob = (int)(ep_pi & 1);
+            const uint32_t tOb = tO + ob * 2 * RP + lane_off;
             sm_wait(&bars[B_OFULL + ob], (ep_pi >> 1) & 1);
-            if (tid < p.R)
-                *(float2*)(p.part_ml + (ep_prow + tid) * 2) = make_float2(s_mfin[ob * RP + tid], s_lfin[ob * RP + tid]);
             uint32_t o[RP];
+            float lmine = 0.f;   // denominator of row tid: every lane of the denominator buffer holds all RP of them
             if (!failed) {
                 tc_fence_after_sync();
 #pragma unroll
-                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tO + ob * RP + lane_off + c * 16, o + c * 16);
+                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tOb + RP + c * 16, o + c * 16);
+                tmem_wait_ld();
+#pragma unroll
+                for (int r = 0; r < RP; ++r)
+                    if (r == tid) lmine = __uint_as_float(o[r]);
+#pragma unroll
+                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tOb + c * 16, o + c * 16);
                 tmem_wait_ld();
                 tc_fence_before_sync();
             }
             mbar_arrive(&bars[B_OFREE + ob]);
             if (!failed) {
+                if (tid < p.R) *(float2*)(p.part_ml + (ep_prow + tid) * 2) = make_float2(s_mfin[ob * RP + tid], lmine);
 #pragma unroll
                 for (int r = 0; r < RP; ++r)
                     if (r < p.R) p.part_acc[(ep_prow + r) * UD + tid] = __uint_as_float(o[r]);
@@ -453,17 +492,10 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         uint32_t gt = 0, pi = 0;
         PieceWalk walk(p, s_prefix, lo, hi, s_len);
         Piece pc, npc;
-        bool have = walk.next(pc, flags);
-        if (have) {
-            load_q_begin(pc, 0);
-            load_q_end(0);
-        }
+        bool have = walk_next(walk, pc, flags);
         while (have && !aborted) {
-            // The next piece's query rows go into the other buffer: every product that read it has completed
-            // (this thread has seen the scores of the last tile of the piece before).
-            const bool nhave = walk.next(npc, flags);
-            if (nhave) load_q_begin(npc, (pi + 1) & 1);
-            const uint32_t tOb = tO + (pi & 1) * RP;
+            const bool nhave = walk_next(walk, npc, flags);
+            const uint32_t tOb = tO + (pi & 1) * 2 * RP;   // O^T of this piece, its denominators RP columns further
 
             // ---- per-piece state ----
             int cmin = 0x7fffffff;
@@ -482,9 +514,6 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 }
             }
             named_barrier_sync(1, kSmThreads);
-            float lsum[RP];
-#pragma unroll
-            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
             WinCursor cur;
             cur.l = 0;
             cur.key0 = 0;
@@ -512,19 +541,19 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     masked = true;
                 }
                 // ---- scores of this thread's key ----
-                sm_wait(&bars[B_SFULL], gt & 1);
+                sm_wait(&bars[B_SFULL + (gt & 1)], (gt >> 1) & 1);
                 uint32_t sv[RP];
                 if (!failed) {
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int c = 0; c < RP / 16; ++c) tmem_ld16(tS + lane_off + c * 16, sv + c * 16);
+                    for (int c = 0; c < RP / 16; ++c) tmem_ld16(tS + (gt & 1) * RP + lane_off + c * 16, sv + c * 16);
                     tmem_wait_ld();
                     tc_fence_before_sync();
                 } else {
 #pragma unroll
                     for (int r = 0; r < RP; ++r) sv[r] = 0xff800000u;
                 }
-                mbar_arrive(&bars[B_SFREE]);
+                mbar_arrive(&bars[B_SFREE + (gt & 1)]);
                 if (masked) {
                     const int key = kbase + tid;
 #pragma unroll
@@ -564,22 +593,21 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         if (!failed) {
                             tc_fence_after_sync();
 #pragma unroll
-                            for (int c = 0; c < RP / 16; ++c) {
+                            for (int c = 0; c < 2 * RP / 16; ++c) {   // O^T, then the denominators
                                 uint32_t o[16];
                                 tmem_ld16(tOb + lane_off + c * 16, o);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * s_alpha[c * 16 + j]);
+                                for (int j = 0; j < 16; ++j)
+                                    o[j] = __float_as_uint(__uint_as_float(o[j]) * s_alpha[(c * 16 + j) % RP]);
                                 tmem_st16(tOb + lane_off + c * 16, o);
                             }
                             tmem_wait_st();
                             tc_fence_before_sync();
                         }
-#pragma unroll
-                        for (int r = 0; r < RP; ++r) lsum[r] *= s_alpha[r];
                     }
                 }
-                // ---- probabilities (bf16) into shared memory, denominators from the rounded values ----
+                // ---- probabilities (bf16) into shared memory; the tensor core sums these rounded values into the denominators ----
                 if (gt > 0) sm_wait(&bars[B_PFREE], (gt - 1) & 1);
 #pragma unroll
                 for (int j = 0; j < RP / 8; ++j) {
@@ -590,8 +618,6 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         const float p0 = fast_exp2(fmaf(__uint_as_float(sv[r0]), scale, s_negm[r0]));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(sv[r0 + 1]), scale, s_negm[r0 + 1]));
                         w4[q] = pack_bf16x2(p0, p1);
-                        lsum[r0] += __uint_as_float(w4[q] << 16);
-                        lsum[r0 + 1] += __uint_as_float(w4[q] & 0xffff0000u);
                     }
                     if (!failed) *(uint4*)(pbuf + j * 2048 + tid * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                 }
@@ -613,21 +639,14 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 mbar_arrive(&bars[B_PFULL]);
                 if (pc.kind == 1) cur.advance(p, pc.sp);
                 if (t == pc.t0) {
-                    // Work that was put off so that the pipeline restarts first: the partial of the piece before,
-                    // and the hand-over of the next piece's query rows.
+                    // Work that was put off so that the pipeline restarts first: the partial of the piece before.
                     if (ep_pending) epilogue();
-                    if (nhave) load_q_end((pi + 1) & 1);
                 }
             }
             if (aborted) break;
 
-            // ---- end of piece: denominators across the 128 keys; the rest of the epilogue runs one piece late ----
-            warp_reduce_rows<RP, false>(lsum, lane, s_red + wid * RP);
-            named_barrier_sync(1, kSmThreads);
-            if (tid < RP) {
-                s_lfin[(pi & 1) * RP + tid] = (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]);
-                s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
-            }
+            // ---- end of piece: park its reference maxima; the epilogue proper runs one piece late ----
+            if (tid < RP) s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
             ep_pending = true;
             ep_pi = pi;
             ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // hpc == 1 on this path
@@ -635,7 +654,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             have = nhave;
             ++pi;
             if (!have) {
-                named_barrier_sync(1, kSmThreads);   // s_lfin / s_mfin of the last piece visible to all
+                named_barrier_sync(1, kSmThreads);   // s_mfin of the last piece visible to all
                 epilogue();
             }
         }
