@@ -70,33 +70,47 @@ __device__ __forceinline__ int32_t seq_len_clamped(const Params& p, int b, uint3
     return n;
 }
 
+// One loop's share of the plan of sequence b (length n).
+__device__ __forceinline__ void seq_plan_step(const Params& p, int b, int32_t n, int l, SeqPlan& s, uint32_t& flags) {
+    s.cut[l] = 0;
+    s.wl[l] = 0;
+    if (l < p.L) {
+        int32_t c = n - p.delta[l];
+        c = c > 0 ? c : 0;
+        s.cut[l] = c;
+        s.cmax = c > s.cmax ? c : s.cmax;
+        if (l >= 1) {
+            int32_t wl = c < p.w ? c : p.w;
+            if (p.win_lens != nullptr && c > 0) {
+                wl = p.win_lens[b * (p.L - 1) + (l - 1)];
+                if (wl < 0 || wl > p.w) {
+                    flags |= kDevWinLenClamped;
+                    wl = wl < 0 ? 0 : p.w;
+                }
+            }
+            s.wl[l] = wl;
+            s.lt += ceil_div(wl, p.tile_keys);
+        }
+    }
+}
+
 __device__ __forceinline__ void seq_plan_n(const Params& p, int b, int32_t n, SeqPlan& s, uint32_t& flags) {
     s.n = n;
     s.cmax = 0;
     s.lt = 0;
 #pragma unroll
-    for (int l = 0; l < kMaxLoops; ++l) {
-        s.cut[l] = 0;
-        s.wl[l] = 0;
-        if (l < p.L) {
-            int32_t c = n - p.delta[l];
-            c = c > 0 ? c : 0;
-            s.cut[l] = c;
-            s.cmax = c > s.cmax ? c : s.cmax;
-            if (l >= 1) {
-                int32_t wl = c < p.w ? c : p.w;
-                if (p.win_lens != nullptr && c > 0) {
-                    wl = p.win_lens[b * (p.L - 1) + (l - 1)];
-                    if (wl < 0 || wl > p.w) {
-                        flags |= kDevWinLenClamped;
-                        wl = wl < 0 ? 0 : p.w;
-                    }
-                }
-                s.wl[l] = wl;
-                s.lt += ceil_div(wl, p.tile_keys);
-            }
-        }
-    }
+    for (int l = 0; l < kMaxLoops; ++l) seq_plan_step(p, b, n, l, s, flags);
+    s.gt = ceil_div(s.cmax, p.tile_keys);
+}
+
+// The same plan, compiled small (a rolled loop, out of line) for kernels whose instruction footprint matters
+// more than the few cycles this costs per piece.
+static __device__ __noinline__ void seq_plan_small(const Params& p, int b, int32_t n, SeqPlan& s, uint32_t& flags) {
+    s.n = n;
+    s.cmax = 0;
+    s.lt = 0;
+#pragma unroll 1
+    for (int l = 0; l < kMaxLoops; ++l) seq_plan_step(p, b, n, l, s, flags);
     s.gt = ceil_div(s.cmax, p.tile_keys);
 }
 
@@ -134,13 +148,15 @@ __device__ __forceinline__ int64_t slot_of(int item, int cta) { return (int64_t)
 // Block-wide exclusive prefix of seq_tiles into sp[0..B] (shared memory). All threads of the block call it.
 // With `lens` (shared memory, B entries) the clamped lengths are kept for PieceWalk, so that walking the pieces
 // reads no global memory.
-__device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint32_t& flags, int32_t* lens = nullptr) {
+__device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint32_t& flags, int32_t* lens = nullptr,
+                                             bool small = false) {
     const int tid = threadIdx.x, nt = blockDim.x;
     for (int b = tid; b < p.B; b += nt) {
         const int32_t n = seq_len_clamped(p, b, flags);
         if (lens != nullptr) lens[b] = n;
         SeqPlan s;
-        seq_plan_n(p, b, n, s, flags);
+        if (small) seq_plan_small(p, b, n, s, flags);
+        else seq_plan_n(p, b, n, s, flags);
         sp[b + 1] = (p.Hkv / p.hpc) * (s.gt + s.lt);
     }
     if (tid == 0) sp[0] = 0;
@@ -194,10 +210,15 @@ struct PieceWalk {
         : p(p_), sp(sp_), lens(lens_), pos(lo_), hi(hi_), b(0) {
         if (pos < hi) b = find_seq(sp, p.B, pos);
     }
-    __device__ bool next(Piece& pc, uint32_t& flags) {
+    __device__ bool next(Piece& pc, uint32_t& flags) { return next_impl<false>(pc, flags); }
+    // The same step compiled small; needs the cached lengths.
+    __device__ bool next_small(Piece& pc, uint32_t& flags) { return next_impl<true>(pc, flags); }
+    template <bool SMALL>
+    __device__ __forceinline__ bool next_impl(Piece& pc, uint32_t& flags) {
         if (pos >= hi) return false;
         while ((int64_t)sp[b + 1] <= pos) ++b;
-        if (lens != nullptr) seq_plan_n(p, b, lens[b], pc.sp, flags);
+        if (SMALL) seq_plan_small(p, b, lens[b], pc.sp, flags);
+        else if (lens != nullptr) seq_plan_n(p, b, lens[b], pc.sp, flags);
         else seq_plan(p, b, pc.sp, flags);
         const int per = pc.sp.gt + pc.sp.lt;
         const int o = (int)(pos - sp[b]);

@@ -12,9 +12,11 @@
 //   O^T [128 dims x RP] += V_tile^T [128 x 128] . P^T      A = V tile as TMA wrote it (MN-major,
 //                                                          128-byte swizzle), B = probabilities
 //
-// RP is R rounded up to 16, 32 or 64. Both operands of both products are read from shared memory by
-// the tensor core itself, once, whatever R is; the 128 softmax threads own one key each (their
-// tensor-memory lane) and the RP scores of that key.
+//   l   [128 x RP]      += ones [128 x 128] . P^T          every lane gets the RP denominators
+//
+// RP is R rounded up to 16, 32 or 64. All operands are read from shared memory by the tensor core
+// itself, once, whatever R is; the 128 softmax threads own one key each (their tensor-memory lane)
+// and the RP scores of that key.
 //
 // Warp roles: warps 0-3 softmax and epilogue (thread = key / output dimension); warp 4 TMA producer
 // of K tiles, warp 6 of V tiles; warp 5 issues the S^T products and owns the tensor-memory
@@ -24,6 +26,10 @@
 // a reference that may lag the true running maximum by up to kSlack powers of two; only when a
 // score exceeds that (a vote over the 128 threads) are the true maxima reduced across threads and
 // the accumulators in tensor memory rescaled. Every wait on an mbarrier is bounded.
+//
+// Eight warps run eight different loops here, so the instruction working set decides the speed:
+// everything that is not on the per-tile path (waits that actually wait, plan arithmetic, the
+// rescale, the epilogue) is kept out of line.
 #include <cuda_bf16.h>
 
 #include "plt_common.cuh"
@@ -38,28 +44,29 @@ constexpr int UK = 128;                  // keys per tile
 constexpr int UD = 128;                  // head dimension
 constexpr int kSlotBytes = UK * UD * 2;  // one K tile or one V tile of one KV head
 constexpr int kHalfBytes = UK * 128;     // one 64-element half of a tile: [128 keys][128 bytes]
-constexpr int kMaxSlots = 6;
+constexpr int kMaxRing = 3;              // slots per ring (one ring for K tiles, one for V tiles)
 constexpr int kSmThreads = 128;          // softmax threads
 constexpr int kUmmaThreads = 256;
 constexpr float kSlack = 8.f;
 constexpr uint64_t kUmmaWaitNs = 1000000000ull;
 
 // mbarrier indices
-constexpr int B_FULL = 0, B_EMPTY = 8, B_SFULL = 16 /* two */, B_SFREE = 18 /* two */, B_PFULL = 20, B_PFREE = 21,
-              B_OFULL = 22 /* two */, B_OFREE = 24 /* two */, B_DRAIN = 26 /* two */, B_COUNT = 28;
+constexpr int B_KFULL = 0, B_KEMPTY = 3, B_VFULL = 6, B_VEMPTY = 9, B_SFULL = 12 /* two */, B_SFREE = 14 /* two */,
+              B_PFULL = 16, B_PFREE = 17, B_OFULL = 18 /* two */, B_OFREE = 20 /* two */, B_DRAIN = 22 /* two */,
+              B_COUNT = 24;
 
 template <int RP>
 struct UCfg {
     static constexpr int QLBO = RP * 16 + 16;      // bytes between the 16-byte column chunks of the packed query tile
     static constexpr int QBUF = 16 * QLBO;         // one packed query tile: [16 chunks][RP rows][16 bytes] (+ pad)
     static constexpr int PBUF = RP * 256;          // probabilities: [RP / 8][128 keys][16 bytes]
-    // Tensor memory: two S^T buffers (tile parity), then per piece parity an O^T buffer followed by the denominators (every lane of
-    // the latter holds the same RP row sums), RP columns each; rounded up to a power of two.
-    static constexpr int TMEM_COLS = RP == 16 ? 128 : (RP == 32 ? 256 : 512);
     static constexpr int ONES_BYTES = 128 * 32;    // A operand of the denominator product: 128 x 16 ones
+    // Tensor memory: two S^T buffers (tile parity), then per piece parity an O^T buffer followed by the
+    // denominators, RP columns each; rounded up to a power of two.
+    static constexpr int TMEM_COLS = RP == 16 ? 128 : (RP == 32 ? 256 : 512);
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
-        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + ONES_BYTES + B_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 2) + 64 +
-               (size_t)(2 * max_batch + 4) * 4;
+        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + ONES_BYTES + B_COUNT * 8 +
+               (size_t)RP * 4 * (3 + 4 + 2 + 2) + 64 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
 
@@ -75,13 +82,12 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, 
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Bounded wait that also gives up as soon as another thread of the block has given up. The slow part is kept
-// out of line: this kernel has eight warps in different loops, and its instruction footprint decides its speed.
-__device__ __noinline__ bool wait_or_abort_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait that also gives up as soon as another thread of the block has given up.
+__device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xffu) == 0) {
+    while (!mbar_try_wait_for(bar, parity, 2000)) {
+        if ((++spins & 0x3fu) == 0) {
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kUmmaWaitNs) {
                 *abort_flag = 1;
@@ -92,11 +98,25 @@ __device__ __noinline__ bool wait_or_abort_slow(uint64_t* bar, uint32_t parity, 
     return true;
 }
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_or_abort_slow(bar, parity, abort_flag);
+    if (mbar_test_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, abort_flag);
 }
+
 // Out-of-line step of the piece walk (the plan arithmetic is long once unrolled over the loops).
-__device__ __noinline__ bool walk_next(PieceWalk& walk, Piece& pc, uint32_t& flags) { return walk.next(pc, flags); }
+__device__ __noinline__ bool walk_next(PieceWalk& walk, Piece& pc, uint32_t& flags) { return walk.next_small(pc, flags); }
+
+// Position in a ring of `size` slots: slot index and the parity of its current use.
+struct Ring {
+    int slot;
+    uint32_t parity;
+    __device__ Ring() : slot(0), parity(0) {}
+    __device__ __forceinline__ void advance(int size) {
+        if (++slot == size) {
+            slot = 0;
+            parity ^= 1u;
+        }
+    }
+};
 
 // Reduces N values per lane across the 32 lanes of a warp with N - 1 (+ a few) shuffles instead of 5 N: each
 // step halves the values a lane still carries and doubles the lanes they cover. The result of row r goes to
@@ -140,18 +160,13 @@ __device__ __forceinline__ void warp_reduce_rows(float (&v)[N], int lane, float*
     }
 }
 
-// Launch-time geometry of the TMA boxes (set by the host from the tensor maps it encoded).
+// Launch-time geometry (set by the host from the tensor maps it encoded).
 struct UmmaGeom {
-    int nslot;       // ring slots of kSlotBytes
-    int kbox;        // keys per box of the shared cache (min(128, page size or capacity))
-    int wbox;        // keys per box of a window (min(128, w))
-    int cap;         // tiles each of the two producers keeps in flight (issued, not landed) at most; 2 cap <= nslot
+    int ring;        // slots in the K ring and in the V ring
+    int kbox;        // keys per TMA box of the shared cache (min(128, page size or capacity))
+    int wbox;        // keys per TMA box of a window (min(128, w))
+    int cap;         // tiles each producer keeps in flight (issued, not landed) at most; <= ring
 };
-
-// Ring position of the K tile / V tile of the n-th tile a block streams (T tiles in all): K(0), then
-// K(n), V(n-1) for n = 1 .. T-1, then V(T-1).
-__device__ __forceinline__ uint32_t pos_k(uint32_t n) { return n == 0 ? 0u : 2u * n - 1u; }
-__device__ __forceinline__ uint32_t pos_v(uint32_t n, uint32_t T) { return n + 1 == T ? 2u * T - 1u : 2u * n + 2u; }
 
 // TMA boxes of one tile: (key coordinate, outermost coordinate) per box, the same for K and V.
 struct TileCoords {
@@ -175,7 +190,7 @@ struct TileSource {
     }
     __device__ __noinline__ void next(const Params& p, const UmmaGeom& geo, TileCoords& tc, uint32_t& flags) {
         if (!have || t == pc.t1) {
-            have = walk.next(pc, flags);
+            have = walk_next(walk, pc, flags);
             t = pc.t0;
             if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
         }
@@ -213,6 +228,154 @@ struct TileSource {
     }
 };
 
+// ---- softmax side: per-block context and the pieces of work that are off the per-tile path ----------
+struct SmCtx {
+    float* negm;       // [RP] minus the reference maximum of each row (1e30 while the row has none)
+    float* mref;       // [RP] reference maximum, log2 units
+    float* alpha;      // [RP] rescale factors of the slow path
+    float* red;        // [4][RP] cross-warp reduction scratch
+    float* mfin;       // [2][RP] reference maxima of a finished piece, by O^T buffer
+    int32_t* lim;      // [RP] keys visible to each row in the current segment
+    int32_t* rowloop;  // [RP] loop (0-based) of each packed row
+    uint64_t* bars;
+    volatile int* abort_flag;
+    uint32_t lane_off;  // this warp's lane quarter in a tensor-memory address
+    float scale;
+    int tid, lane, wid;
+};
+
+// Waits as a warp: `failed` (a wait of this warp ran out) stays warp-uniform, because the tensor-memory
+// loads and stores that depend on it are warp-collective.
+__device__ __noinline__ bool sm_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool failed) {
+    bool bad = false;
+    if (!failed) bad = !wait_or_abort(bar, parity, abort_flag);
+    return __any_sync(0xffffffffu, failed || bad);
+}
+__device__ __forceinline__ bool sm_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool failed) {
+    if (__all_sync(0xffffffffu, !failed && mbar_test_wait(bar, parity))) return false;
+    return sm_wait_slow(bar, parity, abort_flag, failed);
+}
+
+// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima, and
+// (unless this is the first tile of the piece) the rescale of O^T and of the denominators in tensor memory.
+// All 128 softmax threads call it together. `pfree_bar` / `pfree_parity`: completion of the last product
+// that accumulated into O^T.
+template <int RP>
+__device__ __noinline__ bool slow_path(const uint32_t (&sv)[RP], const SmCtx& cx, bool rescale, uint32_t tOb,
+                                       uint64_t* pfree_bar, uint32_t pfree_parity, bool failed) {
+    {
+        float v[RP];
+#pragma unroll
+        for (int r = 0; r < RP; ++r) v[r] = __uint_as_float(sv[r]) * cx.scale;
+        warp_reduce_rows<RP, true>(v, cx.lane, cx.red + cx.wid * RP);
+    }
+    named_barrier_sync(1, kSmThreads);
+    if (cx.tid < RP) {
+        const int t = cx.tid;
+        const float mo = cx.mref[t];
+        const float mn = fmaxf(fmaxf(mo, fmaxf(cx.red[t], cx.red[RP + t])), fmaxf(cx.red[2 * RP + t], cx.red[3 * RP + t]));
+        cx.alpha[t] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
+        cx.mref[t] = mn;
+        cx.negm[t] = (mn == -INFINITY) ? 1e30f : -mn;
+    }
+    named_barrier_sync(1, kSmThreads);
+    if (rescale) {
+        failed = sm_wait(pfree_bar, pfree_parity, cx.abort_flag, failed);
+        if (!failed) {
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 2 * RP / 16; ++c) {   // O^T, then the denominators
+                uint32_t o[16];
+                tmem_ld16(tOb + cx.lane_off + c * 16, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[(c * 16 + j) % RP]);
+                tmem_st16(tOb + cx.lane_off + c * 16, o);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+        }
+    }
+    return failed;
+}
+
+// Epilogue of a finished piece: O^T and the denominators out of tensor memory into the split partial.
+template <int RP>
+__device__ __noinline__ bool epilogue(const Params& p, const SmCtx& cx, uint32_t tOb, int ob, uint32_t parity,
+                                      int64_t prow, bool failed) {
+    failed = sm_wait(&cx.bars[B_OFULL + ob], parity, cx.abort_flag, failed);
+    // 16 columns (packed rows) at a time, rolled: this runs once per piece and must stay small.
+    float lmine = 0.f;   // denominator of row tid: every lane of the denominator buffer holds all RP of them
+#pragma unroll 1
+    for (int c = 0; c < 2 * RP / 16; ++c) {
+        const bool denoms = c < RP / 16;
+        const int r0 = (denoms ? c : c - RP / 16) * 16;
+        uint32_t o[16];
+        if (!failed) {
+            tc_fence_after_sync();
+            tmem_ld16(tOb + cx.lane_off + (denoms ? RP : 0) + r0, o);
+            tmem_wait_ld();
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) o[j] = 0u;
+        }
+        if (denoms) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (r0 + j == cx.tid) lmine = __uint_as_float(o[j]);
+        } else if (!failed) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (r0 + j < p.R) p.part_acc[(prow + r0 + j) * UD + cx.tid] = __uint_as_float(o[j]);
+        }
+    }
+    tc_fence_before_sync();
+    mbar_arrive(&cx.bars[B_OFREE + ob]);
+    if (!failed && cx.tid < p.R) *(float2*)(p.part_ml + (prow + cx.tid) * 2) = make_float2(cx.mfin[ob * RP + cx.tid], lmine);
+    return failed;
+}
+
+// V rows of a boundary tile that hold no data may contain anything: zero them so that 0 * garbage stays 0.
+__device__ __noinline__ bool zero_v_rows(uint8_t* vslot, int nvalid, uint64_t* vfull_bar, uint32_t parity, const SmCtx& cx,
+                                         bool failed) {
+    failed = sm_wait(vfull_bar, parity, cx.abort_flag, failed);
+    if (!failed && cx.tid >= nvalid) {
+        uint8_t* row = vslot + cx.tid * 128;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            *(uint4*)(row + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *(uint4*)(row + kHalfBytes + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    return failed;
+}
+
+// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of each row.
+__device__ __noinline__ void set_limits(const Params& p, const SmCtx& cx, const Piece& pc, int RP, int win_loop, int wl,
+                                        bool new_piece) {
+    // Threads still forming the probabilities of the tile before read negm and lim: nobody rewrites them earlier.
+    named_barrier_sync(1, kSmThreads);
+    if (cx.tid < RP) {
+        const int t = cx.tid;
+        if (new_piece) {
+            cx.mref[t] = -INFINITY;
+            cx.negm[t] = 1e30f;
+        }
+        int lim = 0;
+        if (t < p.R) {
+            if (pc.kind == 0) {
+#pragma unroll
+                for (int l = 0; l < kMaxLoops; ++l)
+                    if (l == cx.rowloop[t]) lim = pc.sp.cut[l];
+            } else if (cx.rowloop[t] == win_loop) {
+                lim = wl;
+            }
+        }
+        cx.lim[t] = lim;
+    }
+    named_barrier_sync(1, kSmThreads);
+}
+
 template <int RP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -221,19 +384,21 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     using C = UCfg<RP>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int nslot = geo.nslot;
-    uint8_t* pbuf = smem + (size_t)nslot * kSlotBytes;
+    const int ring = geo.ring;
+    uint8_t* kslots = smem;                                // K ring, then V ring
+    uint8_t* vslots = smem + (size_t)ring * kSlotBytes;
+    uint8_t* pbuf = smem + (size_t)2 * ring * kSlotBytes;
     uint8_t* qbuf = pbuf + C::PBUF;                       // two buffers of QBUF
     uint8_t* ones = qbuf + 2 * C::QBUF;                   // 128 x 16 bf16 ones
     uint64_t* bars = (uint64_t*)(ones + C::ONES_BYTES);
-    float* s_negm = (float*)(bars + B_COUNT);             // [RP] minus the reference maximum (1e30 while there is none)
-    float* s_mref = s_negm + RP;                          // [RP] reference maximum, log2 units
-    float* s_alpha = s_mref + RP;                         // [RP] rescale factors of the slow path
-    float* s_red = s_alpha + RP;                          // [4][RP] cross-warp reduction scratch
-    int32_t* s_lim = (int32_t*)(s_red + 4 * RP);          // [RP] keys visible to each row in the current segment
-    int32_t* s_rowloop = s_lim + RP;                      // [RP] loop (0-based) of each packed row
-    float* s_mfin = (float*)(s_rowloop + RP);             // [2][RP] reference maxima of a finished piece, by O^T buffer
-    int32_t* s_ctl = (int32_t*)(s_mfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] fills issued
+    float* s_negm = (float*)(bars + B_COUNT);
+    float* s_mref = s_negm + RP;
+    float* s_alpha = s_mref + RP;
+    float* s_red = s_alpha + RP;                          // [4][RP]
+    int32_t* s_lim = (int32_t*)(s_red + 4 * RP);
+    int32_t* s_rowloop = s_lim + RP;
+    float* s_mfin = (float*)(s_rowloop + RP);             // [2][RP]
+    int32_t* s_ctl = (int32_t*)(s_mfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued
     int32_t* s_prefix = s_ctl + 16;                       // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                  // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
@@ -245,22 +410,21 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         s_ctl[0] = 0;
         s_ctl[2] = 0;
         s_ctl[3] = 0;
-        for (int s = 0; s < kMaxSlots; ++s) {
-            mbar_init(&bars[B_FULL + s], 1);
-            mbar_init(&bars[B_EMPTY + s], 1);
+        for (int s = 0; s < kMaxRing; ++s) {
+            mbar_init(&bars[B_KFULL + s], 1);
+            mbar_init(&bars[B_KEMPTY + s], 1);
+            mbar_init(&bars[B_VFULL + s], 1);
+            mbar_init(&bars[B_VEMPTY + s], 1);
         }
-        mbar_init(&bars[B_SFULL], 1);
-        mbar_init(&bars[B_SFULL + 1], 1);
-        mbar_init(&bars[B_SFREE], kSmThreads);
-        mbar_init(&bars[B_SFREE + 1], kSmThreads);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars[B_SFULL + i], 1);
+            mbar_init(&bars[B_SFREE + i], kSmThreads);
+            mbar_init(&bars[B_OFULL + i], 1);
+            mbar_init(&bars[B_OFREE + i], kSmThreads);
+            mbar_init(&bars[B_DRAIN + i], 1);
+        }
         mbar_init(&bars[B_PFULL], kSmThreads);
         mbar_init(&bars[B_PFREE], 1);
-        mbar_init(&bars[B_OFULL], 1);
-        mbar_init(&bars[B_OFULL + 1], 1);
-        mbar_init(&bars[B_OFREE], kSmThreads);
-        mbar_init(&bars[B_OFREE + 1], kSmThreads);
-        mbar_init(&bars[B_DRAIN], 1);
-        mbar_init(&bars[B_DRAIN + 1], 1);
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
@@ -270,7 +434,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     fence_proxy_async_smem();
     if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
-    build_prefix(p, s_prefix, flags, s_len);  // contains __syncthreads
+    build_prefix(p, s_prefix, flags, s_len, /*small=*/true);  // contains __syncthreads
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -278,63 +442,58 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     // S^T of tile parity g at tS + g RP; O^T of piece parity b at tO + 2 b RP, its denominators RP further
     const uint32_t tS = tmem_base, tO = tmem_base + 2 * RP;
 
-    const int64_t T = s_prefix[p.B];
-    const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
+    const int64_t T64 = s_prefix[p.B];
+    const int cta = blockIdx.x, nctas = plan_ctas(T64, (int)gridDim.x);
     if (cta == 0)
         for (int b = tid; b <= p.B; b += kUmmaThreads) p.prefix[b] = s_prefix[b];
     const bool in_plan = cta < nctas;
-    const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
+    const int64_t lo = in_plan ? cta_begin(T64, cta, nctas) : 0, hi = in_plan ? cta_begin(T64, cta + 1, nctas) : 0;
+    const uint32_t T = (uint32_t)(hi - lo);   // tiles this block streams
 
     if (wid == 4 || wid == 6) {
         // ========================= TMA producers: warp 4 streams K tiles, warp 6 V tiles ==========
-        // Ring positions follow the order of use: K(0), then K(n), V(n-1) for n = 1.., then the last V, so a
-        // V tile (needed one softmax later than its K tile) does not sit in its slot longer than a K tile.
-        // Each producer keeps at most `cap` of its copies in flight: more outstanding requests make the
-        // memory system slower, not faster.
-        if (lane == 0 && lo < hi) {
+        // Each keeps at most `cap` of its tiles in flight: more outstanding requests make the memory system
+        // slower, not faster. (cap <= ring, so the slot of the tile issued `cap` tiles ago has not been refilled
+        // and its phase parity is unambiguous.)
+        if (lane == 0 && T > 0) {
             const bool is_v = wid == 6;
+            uint8_t* slots = is_v ? vslots : kslots;
+            uint64_t* full = &bars[is_v ? B_VFULL : B_KFULL];
+            uint64_t* empty = &bars[is_v ? B_VEMPTY : B_KEMPTY];
             tma_prefetch_desc(is_v ? &tmV : &tmK);
             if (p.L > 1) tma_prefetch_desc(is_v ? &tmVw : &tmKw);
-            const uint32_t T = (uint32_t)(hi - lo);
-            const uint32_t cap = (uint32_t)geo.cap;
             bool ok = true;
-            uint32_t issued = 0;
+            uint32_t n = 0;
+            Ring cur, old;   // slot of tile n, slot of tile n - cap
             TileSource src(p, s_prefix, lo, hi, s_len);
             TileCoords tc;
-            for (uint32_t n = 0; n < T && ok; ++n) {
+            for (; n < T && ok; ++n) {
                 src.next(p, geo, tc, flags);
-                const uint32_t pos = is_v ? pos_v(n, T) : pos_k(n);
-                const int slot = (int)(pos % (uint32_t)nslot);
-                const uint32_t use = pos / (uint32_t)nslot;
-                // The copy issued `cap` tiles ago must have landed. With 2 cap <= slots, the slot of that copy
-                // cannot have been refilled and landed again by now, so its phase parity is unambiguous; the one
-                // exception, ring position 0 (which the V stream reuses early), is skipped.
-                if (n >= cap && (is_v || n > cap)) {
-                    const uint32_t q = is_v ? pos_v(n - cap, T) : pos_k(n - cap);
-                    ok = wait_or_abort(&bars[B_FULL + (int)(q % (uint32_t)nslot)], (q / (uint32_t)nslot) & 1, abort_flag);
+                if (n >= (uint32_t)geo.cap) {
+                    ok = wait_or_abort(&full[old.slot], old.parity, abort_flag);
+                    old.advance(ring);
                 }
-                if (ok && use > 0) ok = wait_or_abort(&bars[B_EMPTY + slot], (use - 1) & 1, abort_flag);
+                if (ok && n >= (uint32_t)ring) ok = wait_or_abort(&empty[cur.slot], cur.parity ^ 1u, abort_flag);
                 if (!ok) break;
                 const CUtensorMap* map = tc.window ? (is_v ? &tmVw : &tmKw) : (is_v ? &tmV : &tmK);
-                uint8_t* dst = smem + (size_t)slot * kSlotBytes;
-                mbar_expect_tx(&bars[B_FULL + slot], (uint32_t)(tc.nbox * tc.box_keys * 256));
+                uint8_t* dst = slots + (size_t)cur.slot * kSlotBytes;
+                mbar_expect_tx(&full[cur.slot], (uint32_t)(tc.nbox * tc.box_keys * 256));
                 for (int i = 0; i < tc.nbox; ++i)
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf)
-                        tma_load_4d(dst + hf * kHalfBytes + i * tc.box_keys * 128, map, &bars[B_FULL + slot], hf * 64,
-                                    tc.c1[i], tc.head, tc.c3[i]);
-                ++issued;
+                        tma_load_4d(dst + hf * kHalfBytes + i * tc.box_keys * 128, map, &full[cur.slot], hf * 64, tc.c1[i],
+                                    tc.head, tc.c3[i]);
+                cur.advance(ring);
             }
-            s_ctl[is_v ? 3 : 2] = (int32_t)issued;
+            s_ctl[is_v ? 3 : 2] = (int32_t)n;
         }
     } else if (wid == 5) {
         // ============ S^T = K Q^T issuer (lane 0 issues); owner of tensor memory ==================
         // The whole warp also copies the packed query rows of each piece into shared memory,
         // [16-byte column chunk c][row r], one piece ahead of the products that read them.
-        if (lo < hi) {
+        if (T > 0) {
             constexpr uint32_t idesc_qk = instr_desc(UK, RP, 0, 0);
-            const uint32_t qbuf_a = smem_u32(qbuf), smem_a = smem_u32(smem);
-            const uint32_t T = (uint32_t)(hi - lo);
+            const uint32_t qbuf_a = smem_u32(qbuf), kslots_a = smem_u32(kslots);
             const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
             auto load_q = [&](const Piece& q_pc, int buf) {
                 const uint32_t dst = qbuf_a + buf * C::QBUF;
@@ -349,13 +508,13 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc, npc;
             walk_next(walk, pc, flags);
-            bool nhave = false;
             load_q(pc, 0);
             int t = pc.t0;
             uint32_t pi = 0;
+            Ring kr;
             for (uint32_t g = 0; g < T; ++g) {
-                const uint32_t pos = pos_k(g);
-                const int slot = (int)(pos % (uint32_t)nslot);
+                const int sb = (int)(g & 1);           // score buffer
+                const uint32_t sph = (g >> 1) & 1;     // parity of this use of it
                 if (t == pc.t0) {
                     // this piece's rows have arrived; hand them to the tensor core's view of shared memory
                     asm volatile("cp.async.wait_all;" ::: "memory");
@@ -364,31 +523,29 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 }
                 if (lane == 0) {
                     if (g >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
-                        ok = wait_or_abort(&bars[B_SFREE + (g & 1)], ((g >> 1) - 1) & 1, abort_flag);
-                    if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
+                        ok = wait_or_abort(&bars[B_SFREE + sb], sph ^ 1u, abort_flag);
+                    if (ok) ok = wait_or_abort(&bars[B_KFULL + kr.slot], kr.parity, abort_flag);
                     if (ok) {
                         tc_fence_after_sync();
-                        const uint32_t ks_a = smem_a + (uint32_t)slot * kSlotBytes;
+                        const uint32_t ks_a = kslots_a + (uint32_t)kr.slot * kSlotBytes;
                         const uint32_t q_a = qbuf_a + (pi & 1) * C::QBUF;
 #pragma unroll
                         for (int kk = 0; kk < UD / 16; ++kk)
-                            umma_bf16(tS + (g & 1) * RP, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
+                            umma_bf16(tS + sb * RP, smem_desc(ks_a + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024, 2),
                                       smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
-                        umma_commit(&bars[B_SFULL + (g & 1)]);
-                        umma_commit(&bars[B_EMPTY + slot]);
+                        umma_commit(&bars[B_SFULL + sb]);
+                        umma_commit(&bars[B_KEMPTY + kr.slot]);
                     }
                 }
+                kr.advance(ring);
+                const bool first = t == pc.t0;
+                // The other query buffer was last read by the products of the piece before this one; the last of
+                // them (tile g - 1) must have completed before the next piece's rows are fetched into it.
+                if (first && lane == 0 && ok && g > 0)
+                    ok = wait_or_abort(&bars[B_SFULL + (sb ^ 1)], ((g - 1) >> 1) & 1, abort_flag);
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
-                if (t == pc.t0) {
-                    // The other buffer was last read by the products of the piece before this one; the last of
-                    // them (tile g - 1) must have completed before the next piece's rows are fetched into it.
-                    if (lane == 0 && g > 0) ok = wait_or_abort(&bars[B_SFULL + ((g - 1) & 1)], ((g - 1) >> 1) & 1, abort_flag);
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) break;
-                    nhave = walk_next(walk, npc, flags);
-                    if (nhave) load_q(npc, (pi + 1) & 1);
-                }
+                if (first && walk_next(walk, npc, flags)) load_q(npc, (pi + 1) & 1);
                 if (++t == pc.t1 && g + 1 < T) {
                     pc = npc;
                     t = pc.t0;
@@ -398,30 +555,29 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
     } else if (wid == 7) {
         // ================= O^T += V^T P^T and denominators += 1 P^T issuer (one lane) ==============
-        if (lane == 0 && lo < hi) {
+        if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_pv = instr_desc(UD, RP, 1, 1);
             constexpr uint32_t idesc_l = instr_desc(128, RP, 0, 1);
-            const uint32_t pbuf_a = smem_u32(pbuf), smem_a = smem_u32(smem);
+            const uint32_t pbuf_a = smem_u32(pbuf), vslots_a = smem_u32(vslots);
             const uint64_t ones_desc = smem_desc(smem_u32(ones), 2048, 128, 0);   // K-major, no swizzle: all ones anyway
-            const uint32_t T = (uint32_t)(hi - lo);
             bool ok = true;
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
             walk_next(walk, pc, flags);
             int t = pc.t0;
             uint32_t pi = 0;
+            Ring vr;
             for (uint32_t g = 0; g < T && ok; ++g) {
-                const uint32_t pos = pos_v(g, T);
-                const int slot = (int)(pos % (uint32_t)nslot);
                 const bool first = t == pc.t0, last = t == pc.t1 - 1;
+                const int ob = (int)(pi & 1);
                 if (first && pi >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
-                    ok = wait_or_abort(&bars[B_OFREE + (pi & 1)], ((pi >> 1) - 1) & 1, abort_flag);
-                if (ok) ok = wait_or_abort(&bars[B_FULL + slot], (pos / (uint32_t)nslot) & 1, abort_flag);
+                    ok = wait_or_abort(&bars[B_OFREE + ob], ((pi >> 1) & 1) ^ 1u, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[B_VFULL + vr.slot], vr.parity, abort_flag);
                 if (ok) ok = wait_or_abort(&bars[B_PFULL], g & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t vs = smem_a + (uint32_t)slot * kSlotBytes;
-                const uint32_t tOb = tO + (pi & 1) * 2 * RP;
+                const uint32_t vs = vslots_a + (uint32_t)vr.slot * kSlotBytes;
+                const uint32_t tOb = tO + ob * 2 * RP;
 #pragma unroll
                 for (int ks = 0; ks < UK / 16; ++ks) {
                     const uint64_t pd = smem_desc(pbuf_a + ks * 256, 128, 2048, 0);
@@ -430,8 +586,9 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     umma_bf16(tOb + RP, ones_desc, pd, idesc_l, acc);
                 }
                 umma_commit(&bars[B_PFREE]);
-                umma_commit(&bars[B_EMPTY + slot]);
-                if (last) umma_commit(&bars[B_OFULL + (pi & 1)]);
+                umma_commit(&bars[B_VEMPTY + vr.slot]);
+                if (last) umma_commit(&bars[B_OFULL + ob]);
+                vr.advance(ring);
                 if (++t == pc.t1 && g + 1 < T) {
                     walk_next(walk, pc, flags);
                     t = pc.t0;
@@ -443,82 +600,44 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // ============================ softmax and epilogue (warps 0-3) ============================
         // Thread tid owns key tid of every tile (tensor-memory lane tid of S^T) and, in the epilogue,
         // output dimension tid (lane tid of O^T).
-        const uint32_t lane_off = (uint32_t)(wid * 32) << 16;
+        SmCtx cx;
+        cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lim = s_lim;
+        cx.rowloop = s_rowloop; cx.bars = bars; cx.abort_flag = abort_flag;
+        cx.lane_off = (uint32_t)(wid * 32) << 16;
+        cx.scale = p.scale_log2;
+        cx.tid = tid; cx.lane = lane; cx.wid = wid;
         const float scale = p.scale_log2;
-        // `failed`: a wait of this warp ran out; the warp stops touching data but keeps the common control flow.
-        // Kept warp-uniform, because the tensor-memory loads and stores are warp-collective.
-        bool failed = false;
-        auto sm_wait = [&](uint64_t* bar, uint32_t parity) {
-            bool bad = false;
-            if (!failed) bad = !wait_or_abort(bar, parity, abort_flag);
-            failed = __any_sync(0xffffffffu, failed || bad);
-        };
+        bool failed = false;    // a wait of this warp ran out; it stops touching data but keeps the common control flow
         bool aborted = false;   // agreed by all 128 threads
 
-        // Epilogue of a finished piece (its reference maxima are parked in s_mfin): O^T out of
-        // tensor memory into the split partial. Runs one piece late, while the next piece is already streaming.
+        // The epilogue of a piece runs one piece late, while the next piece is already streaming.
         bool ep_pending = false;
         uint32_t ep_pi = 0;
         int64_t ep_prow = 0;
-        auto epilogue = [&]() {
-            const int ob = (int)(ep_pi & 1);
-            const uint32_t tOb = tO + ob * 2 * RP + lane_off;
-            sm_wait(&bars[B_OFULL + ob], (ep_pi >> 1) & 1);
-            uint32_t o[RP];
-            float lmine = 0.f;   // denominator of row tid: every lane of the denominator buffer holds all RP of them
-            if (!failed) {
-                tc_fence_after_sync();
-#pragma unroll
-                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tOb + RP + c * 16, o + c * 16);
-                tmem_wait_ld();
-#pragma unroll
-                for (int r = 0; r < RP; ++r)
-                    if (r == tid) lmine = __uint_as_float(o[r]);
-#pragma unroll
-                for (int c = 0; c < RP / 16; ++c) tmem_ld16(tOb + c * 16, o + c * 16);
-                tmem_wait_ld();
-                tc_fence_before_sync();
-            }
-            mbar_arrive(&bars[B_OFREE + ob]);
-            if (!failed) {
-                if (tid < p.R) *(float2*)(p.part_ml + (ep_prow + tid) * 2) = make_float2(s_mfin[ob * RP + tid], lmine);
-#pragma unroll
-                for (int r = 0; r < RP; ++r)
-                    if (r < p.R) p.part_acc[(ep_prow + r) * UD + tid] = __uint_as_float(o[r]);
-            }
-            ep_pending = false;
-        };
 
         uint32_t gt = 0, pi = 0;
+        Ring vr;   // V slot of tile gt (only boundary tiles look at it)
         PieceWalk walk(p, s_prefix, lo, hi, s_len);
-        Piece pc, npc;
+        Piece pc;
         bool have = walk_next(walk, pc, flags);
         while (have && !aborted) {
-            const bool nhave = walk_next(walk, npc, flags);
             const uint32_t tOb = tO + (pi & 1) * 2 * RP;   // O^T of this piece, its denominators RP columns further
-
-            // ---- per-piece state ----
             int cmin = 0x7fffffff;
 #pragma unroll
             for (int l = 0; l < kMaxLoops; ++l)
                 if (l < p.L) cmin = min(cmin, pc.sp.cut[l]);
-            if (tid < RP) {
-                s_mref[tid] = -INFINITY;
-                s_negm[tid] = 1e30f;
-                if (pc.kind == 0) {
-                    int cut = 0;
-#pragma unroll
-                    for (int l = 0; l < kMaxLoops; ++l)
-                        if (l == s_rowloop[tid]) cut = pc.sp.cut[l];
-                    s_lim[tid] = tid < p.R ? cut : 0;
-                }
-            }
-            named_barrier_sync(1, kSmThreads);
             WinCursor cur;
             cur.l = 0;
             cur.key0 = 0;
-            if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
             int seg_l = -1, wl = 0;
+            if (pc.kind == 1) {
+                cur.seek(p, pc.sp, pc.t0);
+                seg_l = cur.l;
+#pragma unroll
+                for (int k = 1; k < kMaxLoops; ++k)
+                    if (k == cur.l) wl = pc.sp.wl[k];
+            }
+            set_limits(p, cx, pc, RP, seg_l, wl, true);
 
             for (int t = pc.t0; t < pc.t1; ++t, ++gt) {
                 int kbase, nvalid;
@@ -533,27 +652,27 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
                         for (int k = 1; k < kMaxLoops; ++k)
                             if (k == cur.l) wl = pc.sp.wl[k];
-                        if (tid < RP) s_lim[tid] = (tid < p.R && s_rowloop[tid] == cur.l) ? wl : 0;
-                        named_barrier_sync(1, kSmThreads);
+                        set_limits(p, cx, pc, RP, seg_l, wl, false);
                     }
                     kbase = cur.key0;
                     nvalid = wl - kbase;
                     masked = true;
                 }
                 // ---- scores of this thread's key ----
-                sm_wait(&bars[B_SFULL + (gt & 1)], (gt >> 1) & 1);
+                const int sb = (int)(gt & 1);
+                failed = sm_wait(&bars[B_SFULL + sb], (gt >> 1) & 1, abort_flag, failed);
                 uint32_t sv[RP];
                 if (!failed) {
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int c = 0; c < RP / 16; ++c) tmem_ld16(tS + (gt & 1) * RP + lane_off + c * 16, sv + c * 16);
+                    for (int c = 0; c < RP / 16; ++c) tmem_ld16(tS + sb * RP + cx.lane_off + c * 16, sv + c * 16);
                     tmem_wait_ld();
                     tc_fence_before_sync();
                 } else {
 #pragma unroll
                     for (int r = 0; r < RP; ++r) sv[r] = 0xff800000u;
                 }
-                mbar_arrive(&bars[B_SFREE + (gt & 1)]);
+                mbar_arrive(&bars[B_SFREE + sb]);
                 if (masked) {
                     const int key = kbase + tid;
 #pragma unroll
@@ -570,45 +689,11 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         aborted = true;
                         break;
                     }
-                    // ---- slow path: true maxima over the 128 keys, new references, rescale O^T ----
-                    {
-                        float v[RP];
-#pragma unroll
-                        for (int r = 0; r < RP; ++r) v[r] = __uint_as_float(sv[r]) * scale;
-                        warp_reduce_rows<RP, true>(v, lane, s_red + wid * RP);
-                    }
-                    named_barrier_sync(1, kSmThreads);
-                    if (tid < RP) {
-                        const float mo = s_mref[tid];
-                        const float mn = fmaxf(fmaxf(mo, fmaxf(s_red[tid], s_red[RP + tid])),
-                                               fmaxf(s_red[2 * RP + tid], s_red[3 * RP + tid]));
-                        s_alpha[tid] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
-                        s_mref[tid] = mn;
-                        s_negm[tid] = (mn == -INFINITY) ? 1e30f : -mn;
-                    }
-                    named_barrier_sync(1, kSmThreads);
-                    if (t != pc.t0) {
-                        // O^T holds the earlier tiles of this piece; their last product must have completed
-                        sm_wait(&bars[B_PFREE], (gt - 1) & 1);
-                        if (!failed) {
-                            tc_fence_after_sync();
-#pragma unroll
-                            for (int c = 0; c < 2 * RP / 16; ++c) {   // O^T, then the denominators
-                                uint32_t o[16];
-                                tmem_ld16(tOb + lane_off + c * 16, o);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int j = 0; j < 16; ++j)
-                                    o[j] = __float_as_uint(__uint_as_float(o[j]) * s_alpha[(c * 16 + j) % RP]);
-                                tmem_st16(tOb + lane_off + c * 16, o);
-                            }
-                            tmem_wait_st();
-                            tc_fence_before_sync();
-                        }
-                    }
+                    failed = slow_path<RP>(sv, cx, t != pc.t0, tOb, &bars[B_PFREE], (gt - 1) & 1, failed);
                 }
-                // ---- probabilities (bf16) into shared memory; the tensor core sums these rounded values into the denominators ----
-                if (gt > 0) sm_wait(&bars[B_PFREE], (gt - 1) & 1);
+                // ---- probabilities (bf16) into shared memory; the tensor core sums these rounded values
+                //      into the denominators ----
+                if (gt > 0) failed = sm_wait(&bars[B_PFREE], (gt - 1) & 1, abort_flag, failed);
 #pragma unroll
                 for (int j = 0; j < RP / 8; ++j) {
                     uint32_t w4[4];
@@ -621,26 +706,17 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     }
                     if (!failed) *(uint4*)(pbuf + j * 2048 + tid * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                 }
-                if (masked && nvalid < UK) {
-                    // V rows that hold no data may contain anything: zero them so that 0 * garbage stays 0
-                    const uint32_t fillv = pos_v(gt, (uint32_t)(hi - lo));
-                    const int slot = (int)(fillv % (uint32_t)nslot);
-                    sm_wait(&bars[B_FULL + slot], (fillv / (uint32_t)nslot) & 1);
-                    if (!failed && tid >= nvalid) {
-                        uint8_t* row = smem + (size_t)slot * kSlotBytes + tid * 128;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            *(uint4*)(row + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-                            *(uint4*)(row + kHalfBytes + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-                        }
-                    }
-                }
+                if (masked && nvalid < UK)
+                    failed = zero_v_rows(vslots + (size_t)vr.slot * kSlotBytes, nvalid, &bars[B_VFULL + vr.slot], vr.parity, cx,
+                                         failed);
                 fence_proxy_async_smem();
                 mbar_arrive(&bars[B_PFULL]);
+                vr.advance(ring);
                 if (pc.kind == 1) cur.advance(p, pc.sp);
-                if (t == pc.t0) {
-                    // Work that was put off so that the pipeline restarts first: the partial of the piece before.
-                    if (ep_pending) epilogue();
+                if (t == pc.t0 && ep_pending) {
+                    // put off so that the pipeline restarts first: the partial of the piece before
+                    failed = epilogue<RP>(p, cx, tO + (ep_pi & 1) * 2 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, failed);
+                    ep_pending = false;
                 }
             }
             if (aborted) break;
@@ -649,14 +725,13 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (tid < RP) s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
             ep_pending = true;
             ep_pi = pi;
-            ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // hpc == 1 on this path
-            pc = npc;
-            have = nhave;
+            ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // one KV head per item on this path
+            have = walk_next(walk, pc, flags);
             ++pi;
-            if (!have) {
-                named_barrier_sync(1, kSmThreads);   // s_mfin of the last piece visible to all
-                epilogue();
-            }
+        }
+        if (ep_pending && !aborted) {
+            named_barrier_sync(1, kSmThreads);   // s_mfin of the last piece visible to all
+            failed = epilogue<RP>(p, cx, tO + (ep_pi & 1) * 2 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, failed);
         }
     }
 
@@ -671,12 +746,10 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     if ((wid == 4 || wid == 6) && lane == 0 && gave_up) {
         // give every copy that was issued a bounded chance to land
         const bool is_v = wid == 6;
-        const uint32_t T = (uint32_t)(hi - lo);
         const uint32_t issued = (uint32_t)s_ctl[is_v ? 3 : 2];
-        for (uint32_t n = issued > (uint32_t)nslot ? issued - (uint32_t)nslot : 0; n < issued; ++n) {
-            const uint32_t pos = is_v ? pos_v(n, T) : pos_k(n);
-            mbar_wait_bounded(&bars[B_FULL + (int)(pos % (uint32_t)nslot)], (pos / (uint32_t)nslot) & 1, kUmmaWaitNs);
-        }
+        for (uint32_t m = issued > (uint32_t)ring ? issued - (uint32_t)ring : 0; m < issued; ++m)
+            mbar_wait_bounded(&bars[(is_v ? B_VFULL : B_KFULL) + (int)(m % (uint32_t)ring)], (m / (uint32_t)ring) & 1,
+                              kUmmaWaitNs);
     }
     if (gave_up) flags |= kDevWaitTimeout;
     if (flags) atomicOr(p.status, flags);
@@ -700,7 +773,7 @@ cudaError_t umma_prepare(size_t smem, int* blocks_per_sm) {
 
 int main_umma_rows(int R) { return R <= 16 ? 16 : (R <= 32 ? 32 : 64); }
 
-int main_umma_max_slots() { return kMaxSlots; }
+int main_umma_max_slots() { return 2 * kMaxRing; }
 
 size_t main_umma_smem(int R, int nslot, int max_batch) {
     const int rp = main_umma_rows(R);
@@ -716,7 +789,7 @@ cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm) {
 
 cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                              int wbox, int cap, cudaStream_t stream) {
-    const UmmaGeom geo{nslot, kbox, wbox, cap < 1 ? 1 : (2 * cap > nslot ? nslot / 2 : cap)};
+    const UmmaGeom geo{nslot / 2, kbox, wbox, cap < 1 ? 1 : (2 * cap > nslot ? nslot / 2 : cap)};
     const int rp = main_umma_rows(p.R);
     if (rp == 16)
         plt_decode_main_umma<16><<<grid, kUmmaThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo);
