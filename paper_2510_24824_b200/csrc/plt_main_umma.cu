@@ -12,8 +12,6 @@
 //   O^T [128 dims x RP] += V_tile^T [128 x 128] . P^T      A = V tile as TMA wrote it (MN-major,
 //                                                          128-byte swizzle), B = probabilities
 //
-//   l   [128 x RP]      += ones [128 x 128] . P^T          every lane gets the RP denominators
-//
 // RP is R rounded up to 16, 32 or 64. All operands are read from shared memory by the tensor core
 // itself, once, whatever R is; the 128 softmax threads own one key each (their tensor-memory lane)
 // and the RP scores of that key.
@@ -60,13 +58,12 @@ struct UCfg {
     static constexpr int QLBO = RP * 16 + 16;      // bytes between the 16-byte column chunks of the packed query tile
     static constexpr int QBUF = 16 * QLBO;         // one packed query tile: [16 chunks][RP rows][16 bytes] (+ pad)
     static constexpr int PBUF = RP * 256;          // probabilities: [RP / 8][128 keys][16 bytes]
-    static constexpr int ONES_BYTES = 128 * 32;    // A operand of the denominator product: 128 x 16 ones
-    // Tensor memory: two S^T buffers (tile parity), then per piece parity an O^T buffer followed by the
-    // denominators, RP columns each; rounded up to a power of two.
+    // Tensor memory: two S^T buffers (tile parity), then two O^T buffers (piece parity, each with RP spare
+    // columns after it), RP columns each; rounded up to a power of two.
     static constexpr int TMEM_COLS = RP == 16 ? 128 : (RP == 32 ? 256 : 512);
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
-        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + ONES_BYTES + B_COUNT * 8 +
-               (size_t)RP * 4 * (3 + 4 + 2 + 2) + 64 + (size_t)(2 * max_batch + 4) * 4;
+        return 1024 + (size_t)nslot * kSlotBytes + PBUF + 2 * QBUF + B_COUNT * 8 +
+               (size_t)RP * 4 * (3 + 4 + 2 + 4) + 64 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
 
@@ -86,7 +83,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, 
 __device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
-    while (!mbar_try_wait_for(bar, parity, 2000)) {
+    while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3fu) == 0) {
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kUmmaWaitNs) {
@@ -235,6 +232,7 @@ struct SmCtx {
     float* alpha;      // [RP] rescale factors of the slow path
     float* red;        // [4][RP] cross-warp reduction scratch
     float* mfin;       // [2][RP] reference maxima of a finished piece, by O^T buffer
+    float* lfin;       // [2][RP] its denominators
     int32_t* lim;      // [RP] keys visible to each row in the current segment
     int32_t* rowloop;  // [RP] loop (0-based) of each packed row
     uint64_t* bars;
@@ -261,8 +259,8 @@ __device__ __forceinline__ bool sm_wait(uint64_t* bar, uint32_t parity, volatile
 // All 128 softmax threads call it together. `pfree_bar` / `pfree_parity`: completion of the last product
 // that accumulated into O^T.
 template <int RP>
-__device__ __noinline__ bool slow_path(const uint32_t (&sv)[RP], const SmCtx& cx, bool rescale, uint32_t tOb,
-                                       uint64_t* pfree_bar, uint32_t pfree_parity, bool failed) {
+__device__ __noinline__ bool slow_path(const uint32_t (&sv)[RP], float (&lsum)[RP], const SmCtx& cx, bool rescale,
+                                       uint32_t tOb, uint64_t* pfree_bar, uint32_t pfree_parity, bool failed) {
     {
         float v[RP];
 #pragma unroll
@@ -284,17 +282,19 @@ __device__ __noinline__ bool slow_path(const uint32_t (&sv)[RP], const SmCtx& cx
         if (!failed) {
             tc_fence_after_sync();
 #pragma unroll 1
-            for (int c = 0; c < 2 * RP / 16; ++c) {   // O^T, then the denominators
+            for (int c = 0; c < RP / 16; ++c) {
                 uint32_t o[16];
                 tmem_ld16(tOb + cx.lane_off + c * 16, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[(c * 16 + j) % RP]);
+                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[c * 16 + j]);
                 tmem_st16(tOb + cx.lane_off + c * 16, o);
             }
             tmem_wait_st();
             tc_fence_before_sync();
         }
+#pragma unroll
+        for (int r = 0; r < RP; ++r) lsum[r] *= cx.alpha[r];
     }
     return failed;
 }
@@ -305,33 +305,22 @@ __device__ __noinline__ bool epilogue(const Params& p, const SmCtx& cx, uint32_t
                                       int64_t prow, bool failed) {
     failed = sm_wait(&cx.bars[B_OFULL + ob], parity, cx.abort_flag, failed);
     // 16 columns (packed rows) at a time, rolled: this runs once per piece and must stay small.
-    float lmine = 0.f;   // denominator of row tid: every lane of the denominator buffer holds all RP of them
 #pragma unroll 1
-    for (int c = 0; c < 2 * RP / 16; ++c) {
-        const bool denoms = c < RP / 16;
-        const int r0 = (denoms ? c : c - RP / 16) * 16;
+    for (int c = 0; c < RP / 16; ++c) {
         uint32_t o[16];
         if (!failed) {
             tc_fence_after_sync();
-            tmem_ld16(tOb + cx.lane_off + (denoms ? RP : 0) + r0, o);
+            tmem_ld16(tOb + cx.lane_off + c * 16, o);
             tmem_wait_ld();
-        } else {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) o[j] = 0u;
-        }
-        if (denoms) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (r0 + j == cx.tid) lmine = __uint_as_float(o[j]);
-        } else if (!failed) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (r0 + j < p.R) p.part_acc[(prow + r0 + j) * UD + cx.tid] = __uint_as_float(o[j]);
+                if (c * 16 + j < p.R) p.part_acc[(prow + c * 16 + j) * UD + cx.tid] = __uint_as_float(o[j]);
         }
     }
     tc_fence_before_sync();
     mbar_arrive(&cx.bars[B_OFREE + ob]);
-    if (!failed && cx.tid < p.R) *(float2*)(p.part_ml + (prow + cx.tid) * 2) = make_float2(cx.mfin[ob * RP + cx.tid], lmine);
+    if (!failed && cx.tid < p.R)
+        *(float2*)(p.part_ml + (prow + cx.tid) * 2) = make_float2(cx.mfin[ob * RP + cx.tid], cx.lfin[ob * RP + cx.tid]);
     return failed;
 }
 
@@ -389,8 +378,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     uint8_t* vslots = smem + (size_t)ring * kSlotBytes;
     uint8_t* pbuf = smem + (size_t)2 * ring * kSlotBytes;
     uint8_t* qbuf = pbuf + C::PBUF;                       // two buffers of QBUF
-    uint8_t* ones = qbuf + 2 * C::QBUF;                   // 128 x 16 bf16 ones
-    uint64_t* bars = (uint64_t*)(ones + C::ONES_BYTES);
+    uint64_t* bars = (uint64_t*)(qbuf + 2 * C::QBUF);
     float* s_negm = (float*)(bars + B_COUNT);
     float* s_mref = s_negm + RP;
     float* s_alpha = s_mref + RP;
@@ -398,7 +386,8 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
     int32_t* s_lim = (int32_t*)(s_red + 4 * RP);
     int32_t* s_rowloop = s_lim + RP;
     float* s_mfin = (float*)(s_rowloop + RP);             // [2][RP]
-    int32_t* s_ctl = (int32_t*)(s_mfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued
+    float* s_lfin = s_mfin + 2 * RP;                      // [2][RP]
+    int32_t* s_ctl = (int32_t*)(s_lfin + 2 * RP);         // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued
     int32_t* s_prefix = s_ctl + 16;                       // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                  // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
@@ -428,7 +417,6 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
-    for (int i = tid; i < C::ONES_BYTES / 4; i += kUmmaThreads) ((uint32_t*)ones)[i] = 0x3f803f80u;
     // Rows R..RP-1 of both packed-query buffers stay zero for the whole kernel.
     for (int i = tid; i < 2 * C::QBUF / 16; i += kUmmaThreads) *(uint4*)(qbuf + i * 16) = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
@@ -557,9 +545,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // ================= O^T += V^T P^T and denominators += 1 P^T issuer (one lane) ==============
         if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_pv = instr_desc(UD, RP, 1, 1);
-            constexpr uint32_t idesc_l = instr_desc(128, RP, 0, 1);
             const uint32_t pbuf_a = smem_u32(pbuf), vslots_a = smem_u32(vslots);
-            const uint64_t ones_desc = smem_desc(smem_u32(ones), 2048, 128, 0);   // K-major, no swizzle: all ones anyway
             bool ok = true;
             PieceWalk walk(p, s_prefix, lo, hi, s_len);
             Piece pc;
@@ -583,7 +569,6 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     const uint64_t pd = smem_desc(pbuf_a + ks * 256, 128, 2048, 0);
                     const uint32_t acc = (first && ks == 0) ? 0u : 1u;
                     umma_bf16(tOb, smem_desc(vs + ks * 2048, kHalfBytes, 1024, 2), pd, idesc_pv, acc);
-                    umma_bf16(tOb + RP, ones_desc, pd, idesc_l, acc);
                 }
                 umma_commit(&bars[B_PFREE]);
                 umma_commit(&bars[B_VEMPTY + vr.slot]);
@@ -601,7 +586,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // Thread tid owns key tid of every tile (tensor-memory lane tid of S^T) and, in the epilogue,
         // output dimension tid (lane tid of O^T).
         SmCtx cx;
-        cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lim = s_lim;
+        cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lfin = s_lfin; cx.lim = s_lim;
         cx.rowloop = s_rowloop; cx.bars = bars; cx.abort_flag = abort_flag;
         cx.lane_off = (uint32_t)(wid * 32) << 16;
         cx.scale = p.scale_log2;
@@ -638,6 +623,9 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     if (k == cur.l) wl = pc.sp.wl[k];
             }
             set_limits(p, cx, pc, RP, seg_l, wl, true);
+            float lsum[RP];   // this key's share of the denominators
+#pragma unroll
+            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
 
             for (int t = pc.t0; t < pc.t1; ++t, ++gt) {
                 int kbase, nvalid;
@@ -689,10 +677,20 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         aborted = true;
                         break;
                     }
-                    failed = slow_path<RP>(sv, cx, t != pc.t0, tOb, &bars[B_PFREE], (gt - 1) & 1, failed);
+                    // Copies, so that the arrays of the per-tile path stay in registers (the out-of-line call takes
+                    // the addresses of its arguments).
+                    uint32_t sv_c[RP];
+                    float ls_c[RP];
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) {
+                        sv_c[r] = sv[r];
+                        ls_c[r] = lsum[r];
+                    }
+                    failed = slow_path<RP>(sv_c, ls_c, cx, t != pc.t0, tOb, &bars[B_PFREE], (gt - 1) & 1, failed);
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
                 }
-                // ---- probabilities (bf16) into shared memory; the tensor core sums these rounded values
-                //      into the denominators ----
+                // ---- probabilities (bf16) into shared memory; denominators from the rounded values ----
                 if (gt > 0) failed = sm_wait(&bars[B_PFREE], (gt - 1) & 1, abort_flag, failed);
 #pragma unroll
                 for (int j = 0; j < RP / 8; ++j) {
@@ -703,6 +701,8 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         const float p0 = fast_exp2(fmaf(__uint_as_float(sv[r0]), scale, s_negm[r0]));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(sv[r0 + 1]), scale, s_negm[r0 + 1]));
                         w4[q] = pack_bf16x2(p0, p1);
+                        lsum[r0] += __uint_as_float(w4[q] << 16);            // the rounded values, as the product uses them
+                        lsum[r0 + 1] += __uint_as_float(w4[q] & 0xffff0000u);
                     }
                     if (!failed) *(uint4*)(pbuf + j * 2048 + tid * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                 }
@@ -721,8 +721,14 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             if (aborted) break;
 
-            // ---- end of piece: park its reference maxima; the epilogue proper runs one piece late ----
-            if (tid < RP) s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
+            // ---- end of piece: denominators across the 128 keys, parked with the reference maxima; the epilogue
+            //      proper runs one piece late ----
+            warp_reduce_rows<RP, false>(lsum, lane, s_red + wid * RP);
+            named_barrier_sync(1, kSmThreads);
+            if (tid < RP) {
+                s_lfin[(pi & 1) * RP + tid] = (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]);
+                s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
+            }
             ep_pending = true;
             ep_pi = pi;
             ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // one KV head per item on this path
