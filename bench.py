@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--kw", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--cps", type=int, default=0)
+    ap.add_argument("--loops", type=int, default=0, help="override the workload's number of loops L (for the traffic-vs-L sweep)")
+    ap.add_argument("--path", type=int, default=0, help="kernel path: 0 automatic, 1 warp-level mma, 2 tcgen05")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
@@ -72,12 +74,13 @@ def peak_hbm():
     return FALLBACK_HBM_GBS, "fallback (6650 GB/s, earlier measurement on this pool)"
 
 
-def recorded_traffic(name: str):
-    """DRAM bytes per launch of the main kernel from the committed ncu capture of this workload, or None."""
+def recorded_traffic(name: str, kernel: str):
+    """DRAM bytes per launch of the main kernel from the committed ncu capture of this workload and kernel, or None."""
     f = ROOT / "profiles" / "main_kernel_dram_traffic.json"
     if f.exists():
         try:
-            return json.loads(f.read_text()).get(name, {}).get("dram_bytes_per_launch")
+            entry = json.loads(f.read_text()).get(name, {})
+            return entry.get("dram_bytes_per_launch") if entry.get("kernel") == kernel else None
         except Exception:
             return None
     return None
@@ -137,11 +140,14 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def replica_spec(index: int, rank: int) -> dict:
+def replica_spec(index: int, rank: int, loops: int = 0) -> dict:
     """Workload of one replica: every rank streams its own data (seed offset by rank), same shapes."""
     from paper_2510_24824_b200.inputs import workload
     spec = workload(index)
     spec["seed"] = spec["seed"] + 1000 * rank
+    if loops > 0:
+        spec["L"] = loops
+        spec["name"] = f"{spec['name']}_L{loops}"
     return spec
 
 
@@ -185,12 +191,18 @@ def time_oracle(p, cpu_seconds: float):
     per_row = t_probe / len(probe)  # wall seconds per row with all cores busy
     n = int(min(total_rows, max(len(probe), cpu_seconds / cores / max(per_row, 1e-9))))
     rows = all_rows if n >= total_rows else all_rows[rng.choice(total_rows, size=n, replace=False)]
+    # A workload the oracle finishes in well under the budget is repeated whole, so that the sample is
+    # about cpu_seconds core-seconds of work either way.
+    reps = 1
+    if len(rows) == total_rows:
+        reps = int(max(1, min(50, round(cpu_seconds / cores / max(per_row * total_rows, 1e-9)))))
     t0 = time.perf_counter()
-    oracle.decode_attn_rows(p, rows)
+    for _ in range(reps):
+        oracle.decode_attn_rows(p, rows)
     t = time.perf_counter() - t0
-    step_seconds = t * total_rows / len(rows)
+    step_seconds = t / reps * total_rows / len(rows)
     sample = (f"{len(rows)} of {total_rows} output rows (b, loop, head) of the same workload, drawn uniformly"
-              if len(rows) < total_rows else f"all {total_rows} output rows of the workload (one full step)")
+              if len(rows) < total_rows else f"all {total_rows} output rows of the workload, {reps} full step(s)")
     return 1.0 / step_seconds, {"cores": cores, "kind": "oracle", "sample": sample, "sample_seconds": t}
 
 
@@ -258,9 +270,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    p = make_problem(replica_spec(args.workload, rank))
+    p = make_problem(replica_spec(args.workload, rank, args.loops))
     dp = DeviceProblem(p, dev)
-    tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps)
+    tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
+                  kernel_path=args.path)
     op = DecodeAttn(p, device_index=local_rank, **tuning)
     stream = torch.cuda.current_stream().cuda_stream
     cfg, by = workload_config(p, {"launch": op.info, "parallelism": f"replicas x{world} (no collective)"})
@@ -334,6 +347,7 @@ def main():
         peak, peak_src = peak_hbm()
         main_bytes = by["shared_kv"] + by["window_kv"] + by["q_o"] // 2 + by["index"]
         achieved = main_bytes / (main_avg_ms * 1e-3) / 1e9
+        kernel_name = {1: "plt_decode_main_" + p.dtype, 2: "plt_decode_main_umma"}[op.info["kernel_path"]]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -344,10 +358,10 @@ def main():
             "clocks": sampler.summary(),
             "gpu_launches": int(op.info["kernels_per_run"]) * args.steps,
             "roofline": {
-                "bound": "hbm", "kernel": "plt_decode_main_" + p.dtype, "achieved": achieved, "peak": peak,
+                "bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": main_bytes, "avg_launch_ms": main_avg_ms,
-                "launches_timed": n_prof, "traffic": recorded_traffic(p.name),
+                "launches_timed": n_prof, "traffic": recorded_traffic(p.name, kernel_name),
             },
         }
         if e2e is not None:
