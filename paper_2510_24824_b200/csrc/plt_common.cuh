@@ -32,6 +32,8 @@ struct Params {
     float* part_acc;           // [slots][hpc][R][d]  unnormalised sum of p * V
     float* part_ml;            // [slots][hpc][R][2]  running max (log2 units) and sum of p
     int32_t* prefix;           // [B + 1] tile prefix written by block 0 of the main kernel
+    int32_t* item_blocks;      // [items][2] first and last main-kernel block holding a piece of the item (written by
+                               // the blocks that own the item's first / last tile; items without tiles are not written)
     uint32_t* status;          // device status word
 #ifdef PLT_TIMELINE
     void* timeline;            // [grid][8] u64, instrumentation builds only
@@ -145,6 +147,7 @@ __device__ __forceinline__ int item_index(const Params& p, int b, int hg, int ki
 // A piece (the part of an item done by one block) stores its partial in slot item + block.
 __device__ __forceinline__ int64_t slot_of(int item, int cta) { return (int64_t)item + cta; }
 
+
 // Block-wide exclusive prefix of seq_tiles into sp[0..B] (shared memory). All threads of the block call it.
 // With `lens` (shared memory, B entries) the clamped lengths are kept for PieceWalk, so that walking the pieces
 // reads no global memory.
@@ -241,6 +244,12 @@ struct PieceWalk {
         return true;
     }
 };
+
+__device__ __forceinline__ void note_piece(const Params& p, const Piece& pc, int cta) {
+    const int item = item_index(p, pc.b, pc.hg, pc.kind);
+    if (pc.t0 == 0) p.item_blocks[2 * item] = cta;
+    if (pc.t1 == (pc.kind == 0 ? pc.sp.gt : pc.sp.lt)) p.item_blocks[2 * item + 1] = cta;
+}
 
 // Window tile cursor: maps the running tile index of a windows item to (loop, first key in that window).
 struct WinCursor {

@@ -54,6 +54,7 @@ struct plt_decode_attn {
     float* part_acc = nullptr;
     float* part_ml = nullptr;
     int32_t* prefix = nullptr;
+    int32_t* item_blocks = nullptr;
     uint32_t* status = nullptr;
     size_t ws_bytes = 0;
     // TMA descriptors, re-encoded only when a base pointer, stride or extent changes
@@ -167,7 +168,8 @@ size_t workspace_bytes_for(const plt_decode_attn_config* c, const Geometry& g, i
     const size_t slots = (size_t)c->max_batch * (c->Hkv / hpc) * 2 + (size_t)grid;
     *acc_floats = slots * hpc * g.R * c->d;
     *ml_floats = slots * hpc * g.R * 2;
-    return (*acc_floats + *ml_floats) * 4 + (size_t)(c->max_batch + 1) * 4 + 256;
+    const size_t items = (size_t)c->max_batch * (c->Hkv / hpc) * 2;
+    return (*acc_floats + *ml_floats) * 4 + items * 8 + (size_t)(c->max_batch + 1) * 4 + 256;
 }
 
 plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, int D, int64_t d1, int64_t d2, int64_t d3,
@@ -344,7 +346,8 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     }
     h->part_acc = (float*)ws;
     h->part_ml = h->part_acc + acc_floats;
-    h->prefix = (int32_t*)(h->part_ml + ml_floats);
+    h->item_blocks = (int32_t*)(h->part_ml + ml_floats);   // 16-byte aligned: both float counts are multiples of 4
+    h->prefix = h->item_blocks + (size_t)config->max_batch * (config->Hkv / h->var.HPC) * 4;
     h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
     e = cudaMemset(h->status, 0, 4);
     if (e != cudaSuccess) { cudaFree(ws); delete h; return cuda_fail(nullptr, "cudaMemset", e); }
@@ -397,7 +400,8 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     p.q = a->q; p.k_cache = a->k_cache; p.v_cache = a->v_cache; p.k_win = a->k_win; p.v_win = a->v_win;
     p.seq_lens = a->seq_lens; p.win_lens = a->win_lens; p.page_table = a->page_table; p.gate_logits = a->gate_logits;
     p.out = a->out;
-    p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.status = h->status;
+    p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.item_blocks = h->item_blocks;
+    p.status = h->status;
 #ifdef PLT_TIMELINE
     p.timeline = h->timeline;
 #endif
@@ -716,7 +720,8 @@ extern "C" PLT_API plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn
                         h->ws_bytes, kNoAllocScratchBytes);
         h->part_acc = (float*)dv.scratch;
         h->part_ml = h->part_acc + acc_floats;
-        h->prefix = (int32_t*)(h->part_ml + ml_floats);
+        h->item_blocks = (int32_t*)(h->part_ml + ml_floats);
+        h->prefix = h->item_blocks + (size_t)config->max_batch * (config->Hkv / h->var.HPC) * 4;
         h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
         dv.cfg = *config;
         for (int l = 0; l < kMaxLoops; ++l) dv.offsets[l] = h->delta[l];

@@ -351,6 +351,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             const int64_t slot = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta);
             const int64_t prow = (slot * HPC + h_local) * p.R;
+            if (tid == 0) note_piece(p, pc, cta);
             if (KW == 1) {
 #pragma unroll
                 for (int nd = 0; nd < D / 8; ++nd) {

@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(NT) plt_decode_main_f32(const __grid_constant_
         // ---- store the split partial ------------------------------------------------------------------
         const int64_t slot = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta);
         const int64_t prow = slot * R;
+        if (tid == 0) note_piece(p, pc, cta);
 #pragma unroll
         for (int k = 0; k < C::MAXK; ++k) {
             const int r = pc_rg + k * C::RG;

@@ -732,6 +732,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
             ep_pending = true;
             ep_pi = pi;
             ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // one KV head per item on this path
+            if (tid == 0) note_piece(p, pc, cta);
             have = walk_next(walk, pc, flags);
             ++pi;
         }

@@ -2,8 +2,8 @@
 // attention (y_global, Algorithm 3 line 2) and of the window attention (y_local, line 3) by their
 // running maxima, normalises each, and applies the sigmoid gate mix of Eq. 2 (lines 4-5):
 //   O = g * y_local + (1 - g) * y_global for loops 2..L,  O = y_global for loop 1.
-// One block per (sequence, KV-head group, chunk of 8 packed rows); one warp per output row. The
-// first warp works out once per block which blocks of the main kernel hold pieces of the two items.
+// One block per (sequence, KV-head group, chunk of 8 packed rows); one warp per output row. Which
+// blocks of the main kernel hold pieces of an item is read from the table those blocks left.
 #include <cuda_bf16.h>
 
 #include "plt_common.cuh"
@@ -15,11 +15,6 @@ namespace plt {
 namespace {
 
 constexpr int kReduceWarps = 8;
-
-struct ReduceCtl {
-    int32_t c0[2], c1[2];        // first and last main-kernel block of the shared-cache item [0] and the windows item [1]
-    int32_t cut[kMaxLoops];
-};
 
 template <int D>
 struct Vec {
@@ -73,62 +68,47 @@ __device__ __forceinline__ float merge_item(const Params& p, int item, int hl, i
 
 template <int D, bool BF16>
 __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __grid_constant__ Params p, const int chunks) {
-    __shared__ ReduceCtl ctl;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int HG = p.Hkv / p.hpc;
     const int chunk = (int)(blockIdx.x % chunks);
     const int hg = (int)((blockIdx.x / chunks) % HG);
     const int b = (int)(blockIdx.x / (chunks * HG));
-
-    // Everything above depends on the launch only; from here on the main kernel's results are read.
-    grid_dependency_wait();
-
-    if (wid == 0) {
-        uint32_t flags = 0;
-        SeqPlan sp;
-        seq_plan(p, b, sp, flags);
-        const int64_t T = p.prefix[p.B];
-        const int nctas = plan_ctas(T, p.num_ctas);
-        const int per = sp.gt + sp.lt;
-        const int64_t base = (int64_t)p.prefix[b] + (int64_t)hg * per;
-        if (lane < 4) {
-            // lane 0/1: first/last block of the shared-cache item; lane 2/3: of the windows item
-            const int kind = lane >> 1;
-            const int64_t s = kind == 0 ? base : base + sp.gt;
-            const int64_t e = kind == 0 ? base + sp.gt : base + per;
-            int c = (lane & 1) ? -1 : 0;
-            if (s < e) c = cta_of(T, (lane & 1) ? e - 1 : s, nctas);
-            if (lane & 1) ctl.c1[kind] = c; else ctl.c0[kind] = c;
-        }
-        if (lane < kMaxLoops) {
-            int cut = 0;
-#pragma unroll
-            for (int k = 0; k < kMaxLoops; ++k)
-                if (k == lane) cut = sp.cut[k];
-            ctl.cut[lane] = cut;
-        }
-    }
-    __syncthreads();
-
     const int row = chunk * kReduceWarps + wid;   // packed row of this head group: hl * R + r
     if (row >= p.hpc * p.R) return;
     const int hl = row / p.R, r = row - hl * p.R;
     const int l = r / p.G, g = r - l * p.G;
     const int h = (hg * p.hpc + hl) * p.G + g;
 
+    // Everything above depends on the launch only; from here on the main kernel's results are read.
+    grid_dependency_wait();
+
+    // Each warp works out its own row: the plan of the sequence (is there anything to merge?) and, from the table
+    // the main kernel's blocks left, which of them hold the pieces of the two items.
+    uint32_t flags = 0;
+    SeqPlan sp;
+    seq_plan(p, b, sp, flags);
+    int cut = 0;
+#pragma unroll
+    for (int k = 0; k < kMaxLoops; ++k)
+        if (k == l) cut = sp.cut[k];
+    const int item_g = item_index(p, b, hg, 0), item_l = item_index(p, b, hg, 1);
+    int2 rg = make_int2(0, -1), rl = make_int2(0, -1);
+    if (sp.gt > 0) rg = *(const int2*)(p.item_blocks + 2 * item_g);
+    if (sp.lt > 0 && l > 0) rl = *(const int2*)(p.item_blocks + 2 * item_l);
+
     Vec<D> yg, yl;
     float out[Vec<D>::N];
-    if (ctl.cut[l] == 0) {
+    if (cut == 0) {
 #pragma unroll
         for (int i = 0; i < Vec<D>::N; ++i) out[i] = 0.f;
     } else {
-        const float dg = merge_item<D>(p, item_index(p, b, hg, 0), hl, r, ctl.c0[0], ctl.c1[0], lane, yg);
+        const float dg = merge_item<D>(p, item_g, hl, r, rg.x, rg.y, lane, yg);
         const float ig = dg > 0.f ? 1.f / dg : 0.f;
         if (l == 0) {
 #pragma unroll
             for (int i = 0; i < Vec<D>::N; ++i) out[i] = yg.v[i] * ig;
         } else {
-            const float dl = merge_item<D>(p, item_index(p, b, hg, 1), hl, r, ctl.c0[1], ctl.c1[1], lane, yl);
+            const float dl = merge_item<D>(p, item_l, hl, r, rl.x, rl.y, lane, yl);
             const float il = dl > 0.f ? 1.f / dl : 0.f;  // empty window: y_local = 0
             const float x = p.gate_logits[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h];
             const float gate = 1.f / (1.f + expf(-x));
