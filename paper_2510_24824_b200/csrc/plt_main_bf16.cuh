@@ -198,6 +198,15 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int head0 = pc.hg * HPC;
                 WinCursor cur;
                 if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
+                // Paged cache: the id of the page in use and, loaded one page early so that its latency is off the
+                // issue path, the id of the page after it.
+                const int32_t* ptab = p.page_table + (int64_t)pc.b * p.max_pages;
+                int pg = 0, page_id = 0, page_next = 0;
+                if (pc.kind == 0 && p.page_size > 0) {
+                    pg = (pc.t0 * C::TK) / p.page_size;
+                    page_id = ptab[pg];
+                    page_next = ptab[min(pg + 1, p.max_pages - 1)];
+                }
                 for (int t = pc.t0; t < pc.t1; ++t, ++it) {
                     const CUtensorMap *mk, *mv;
                     int c1, c3;
@@ -206,12 +215,18 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         mk = &tmK;
                         mv = &tmV;
                         if (p.page_size > 0) {
-                            int page = p.page_table[(int64_t)pc.b * p.max_pages + key0 / p.page_size];
+                            const int in_page = key0 % p.page_size;
+                            if (in_page == 0 && t != pc.t0) {
+                                ++pg;
+                                page_id = page_next;
+                                page_next = ptab[min(pg + 1, p.max_pages - 1)];
+                            }
+                            int page = page_id;
                             if (page < 0 || page >= p.num_pool_pages) {
                                 flags |= kDevPageIdClamped;
                                 page = page < 0 ? 0 : p.num_pool_pages - 1;
                             }
-                            c1 = key0 % p.page_size;
+                            c1 = in_page;
                             c3 = page;
                         } else {
                             c1 = key0;
@@ -264,13 +279,17 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
 
         int stage = 0;
         uint32_t use = 0;
+        int q_b = -1, q_hg = -1;   // (sequence, head group) whose query rows are in qf
+        uint32_t qf[D / 16][4];
         PieceWalk walk(p, s_prefix, lo, hi);
         Piece pc;
         while (walk.next(pc, flags)) {
             const int kvh = pc.hg * HPC + h_local;
             // ---- packed query rows of this KV head: row r = loop * G + head-in-group --------------
-            uint32_t qf[D / 16][4];
-            {
+            // (the windows item of a head group follows its shared-cache item: same rows, kept)
+            if (pc.b != q_b || pc.hg != q_hg) {
+                q_b = pc.b;
+                q_hg = pc.hg;
                 const int64_t q0 = (((int64_t)pc.b * p.L + l0) * p.Hq + kvh * p.G + (r0 - l0 * p.G)) * D;
                 const int64_t q1 = (((int64_t)pc.b * p.L + l1) * p.Hq + kvh * p.G + (r1 - l1 * p.G)) * D;
 #pragma unroll
