@@ -86,12 +86,16 @@ typedef struct {
     const int32_t* loop_offset; /* host, L entries delta_l >= 0; NULL: delta_l = l-1. Copied at create. */
     /* Launch tuning, 0 = automatic. Results do not depend on these beyond rounding order. */
     int32_t heads_per_cta; /* KV heads one thread block streams together (bf16 path; divides Hkv) */
-    int32_t key_slices;    /* 16-key slices per pipeline tile (bf16 path; 1, 2 or 4) */
+    int32_t key_slices;    /* warps that split the keys of a pipeline tile (bf16 path; 1, 2, 4 or 8) */
     int32_t stages;        /* depth of the shared-memory pipeline (bf16 path) */
     int32_t ctas_per_sm;   /* persistent thread blocks per SM */
     int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (4 or 6) and
                               heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block) */
     int32_t loads_in_flight; /* PLT_PATH_TCGEN05: K tiles (and likewise V tiles) kept in flight at most, clamped to stages / 2; 0 = automatic */
+    int32_t slices_per_warp; /* PLT_PATH_WARP_MMA: 16-key slices each of those warps takes per tile (1 or 2); a tile holds
+                              16 * key_slices * slices_per_warp keys */
+    int32_t row_warps;     /* PLT_PATH_WARP_MMA: warps that split the L * Hq/Hkv packed rows of a KV head (1 or 2; each
+                              takes at most 32 rows) */
 } plt_decode_attn_config;
 
 /*

@@ -42,7 +42,7 @@ class Config(ctypes.Structure):
         ("sm_scale", ctypes.c_float), ("device", ctypes.c_int32), ("loop_offset", ctypes.POINTER(ctypes.c_int32)),
         ("heads_per_cta", ctypes.c_int32), ("key_slices", ctypes.c_int32), ("stages", ctypes.c_int32),
         ("ctas_per_sm", ctypes.c_int32), ("kernel_path", ctypes.c_int32),
-        ("loads_in_flight", ctypes.c_int32),
+        ("loads_in_flight", ctypes.c_int32), ("slices_per_warp", ctypes.c_int32), ("row_warps", ctypes.c_int32),
     ]
 
 
@@ -96,7 +96,8 @@ def _raise(status: int, handle) -> None:
 def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_seq_len: int, w: int,
                 page_size: int = 0, sm_scale: float = 0.0, device: int = 0,
                 loop_offset: Optional[Sequence[int]] = None, heads_per_cta: int = 0, key_slices: int = 0,
-                stages: int = 0, ctas_per_sm: int = 0, kernel_path: int = 0, loads_in_flight: int = 0) -> Config:
+                stages: int = 0, ctas_per_sm: int = 0, kernel_path: int = 0, loads_in_flight: int = 0,
+                row_warps: int = 0, slices_per_warp: int = 0) -> Config:
     c = Config()
     c.struct_size = ctypes.sizeof(Config)
     c.dtype = {"f32": PLT_F32, "bf16": PLT_BF16}.get(dtype, dtype)
@@ -110,6 +111,8 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
     c.heads_per_cta, c.key_slices, c.stages, c.ctas_per_sm = heads_per_cta, key_slices, stages, ctas_per_sm
     c.kernel_path = kernel_path
     c.loads_in_flight = loads_in_flight
+    c.row_warps = row_warps
+    c.slices_per_warp = slices_per_warp
     return c
 
 

@@ -89,7 +89,7 @@ plt_status cuda_fail(plt_decode_attn_t h, const char* what, cudaError_t e) {
 int elem_size(bool bf16) { return bf16 ? 2 : 4; }
 
 struct Geometry {
-    int G, R, MT;
+    int G, R;
 };
 
 plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
@@ -109,7 +109,6 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
     g->R = c->L * g->G;
     if (g->R > kMaxRows)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "L * Hq/Hkv = %d packed rows > %d", g->R, kMaxRows);
-    g->MT = g->R <= 16 ? 1 : (g->R <= 32 ? 2 : 4);
     if (c->page_size > 0 && c->page_size % 16 != 0)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "page_size %d is not a multiple of 16", c->page_size);
     if (c->loop_offset)
@@ -118,45 +117,59 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
     return PLT_OK;
 }
 
-// Picks (heads per block, key slices, stages, blocks per SM) for the bf16 kernel.
+// Picks (rows per warp, heads per block, key slices, stages, blocks per SM) for the warp-level bf16 kernel.
 plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, MainVariant* v, int* want_ctas_per_sm) {
     v->D = c->d;
-    v->MT = g.MT;
+    int rw = c->row_warps;
+    if (rw == 0) rw = g.R > 24 ? 2 : 1;   // 32 rows in one warp leave room for one warp per scheduler only: measured slower
+    if (rw != 1 && rw != 2) return fail(nullptr, PLT_ERR_INVALID_ARG, "row_warps %d (supported: 1 or 2)", rw);
+    int nt = (g.R + 8 * rw - 1) / (8 * rw);   // 8-row groups per warp
+    if (rw == 2 && nt < 2) nt = 2;
+    if (nt > 4) return fail(nullptr, PLT_ERR_UNSUPPORTED, "%d packed rows need row_warps = 2", g.R);
+    v->NT = nt;
+    v->RW = rw;
+    // Up to 16 rows per warp the kernel fits 168 registers and two blocks of 4 consumer warps share an SM; above that
+    // one block of 4 warps has the SM to itself.
+    const bool small = nt <= 2;
     int hpc = c->heads_per_cta, kw = c->key_slices;
+    int ks = c->slices_per_warp;
+    if (ks == 0) ks = (rw == 2 && nt <= 2) ? 2 : 1;
+    if (ks != 1 && ks != 2) return fail(nullptr, PLT_ERR_INVALID_ARG, "slices_per_warp %d (supported: 1 or 2)", ks);
     if (hpc == 0) {
         hpc = 1;
-        const int cap = g.MT >= 4 ? 1 : (g.MT == 2 ? 2 : 4);
+        const int cap = 4 / rw;
         for (int h = cap; h >= 1; h >>= 1)
             if (c->Hkv % h == 0) { hpc = h; break; }
     }
     if (kw == 0) {
-        kw = 4 / (hpc * g.MT);
+        kw = 4 / (hpc * rw);
         if (kw < 1) kw = 1;
-        if (kw > 4) kw = 4;
     }
     if (c->Hkv % hpc != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "heads_per_cta %d does not divide Hkv %d", hpc, c->Hkv);
-    while (c->page_size > 0 && c->page_size % (16 * kw) != 0 && kw > 1) kw >>= 1;
-    if (!main_bf16_exists(v->D, v->MT, hpc, kw))
-        return fail(nullptr, PLT_ERR_UNSUPPORTED, "no bf16 kernel for heads_per_cta=%d key_slices=%d with %d row tiles", hpc,
-                    kw, g.MT);
+    while (c->page_size > 0 && c->page_size % (16 * kw * ks) != 0 && kw > 1) kw >>= 1;
+    if (c->page_size > 0 && c->page_size % (16 * kw * ks) != 0) ks = 1;
+    if (!main_bf16_exists(v->D, nt, rw, hpc, kw, ks))
+        return fail(nullptr, PLT_ERR_UNSUPPORTED,
+                    "no bf16 kernel for heads_per_cta=%d key_slices=%d slices_per_warp=%d row_warps=%d", hpc, kw, ks, rw);
     v->HPC = hpc;
     v->KW = kw;
-    const int ncw = hpc * kw * g.MT;
-    int cps = c->ctas_per_sm > 0 ? c->ctas_per_sm : (ncw <= 4 ? 2 : 1);
+    v->KS = ks;
+    const int ncw = hpc * kw * rw;
+    int cps = c->ctas_per_sm > 0 ? c->ctas_per_sm : (small && ncw <= 4 ? 2 : 1);
     const size_t budget = (size_t)(cps >= 2 ? 227 * 1024 / cps - 1024 : 227 * 1024);
     int stages = c->stages;
     if (stages == 0) {
         // About 128 KB of loads in flight per SM measured fastest on B200; more only delays the first data.
-        const size_t stage_bytes = main_bf16_smem(v->D, v->MT, hpc, kw, 3, c->max_batch) -
-                                   main_bf16_smem(v->D, v->MT, hpc, kw, 2, c->max_batch);
+        const size_t stage_bytes = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 3, c->max_batch) -
+                                   main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 2, c->max_batch);
         stages = (int)((128 * 1024) / (stage_bytes * (size_t)cps));
         if (stages < 2) stages = 2;
-        while (stages > 2 && main_bf16_smem(v->D, v->MT, hpc, kw, stages, c->max_batch) > budget) --stages;
+        while (stages > 2 && main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch) > budget) --stages;
         if (stages > 8) stages = 8;
     }
     if (stages < 2 || stages > 12) return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [2, 12]", stages);
     v->stages = stages;
-    v->smem = main_bf16_smem(v->D, v->MT, hpc, kw, stages, c->max_batch);
+    v->smem = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch);
     if (v->smem > 227 * 1024)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "variant needs %zu bytes of shared memory (> 227 KB)", v->smem);
     *want_ctas_per_sm = cps;
@@ -235,7 +248,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the tcgen05 main kernel", e);
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
         h->umma = true;
-        h->var = MainVariant{config->d, g.MT, 1, 8, nslot, 0, smem};
+        h->var = MainVariant{config->d, 0, 0, 1, 8, 1, nslot, 0, smem};
         h->ctas_per_sm = 1;
         h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)
                                         : (config->max_seq_len < 128 ? config->max_seq_len : 128);
@@ -249,7 +262,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
         h->ctas_per_sm = blocks < cps ? blocks : cps;
     } else {
-        h->var = MainVariant{config->d, g.MT, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
+        h->var = MainVariant{config->d, 0, 0, 1, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
         e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
         if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the fp32 main kernel", e);
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM");
@@ -266,7 +279,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         h->encode = (EncodeTiledFn)fn;
     }
     // The tile line must fit 31 bits.
-    const int tk = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+    const int tk = h->bf16 ? 16 * h->var.KW * h->var.KS : kF32TileKeys;
     const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
                          ((double)(config->max_seq_len + tk - 1) / tk + (double)(config->L - 1) * ((config->w + tk - 1) / tk));
     if (tiles >= 2147483647.0) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan");
@@ -410,7 +423,7 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
     p.num_pool_pages = a->num_pool_pages;
     p.hpc = h->var.HPC;
-    p.tile_keys = h->bf16 ? 16 * h->var.KW : kF32TileKeys;
+    p.tile_keys = h->bf16 ? 16 * h->var.KW * h->var.KS : kF32TileKeys;
     p.num_ctas = h->var.grid;
     p.scale_log2 = h->scale_log2;
     for (int l = 0; l < kMaxLoops; ++l) p.delta[l] = h->delta[l];
@@ -420,8 +433,8 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     if (h->bf16) {
         // keys and heads per TMA box: the warp-level kernel loads [heads per block][tile keys], the tcgen05 kernel
         // [1 head][up to 128 keys]
-        const int tk = h->umma ? h->kbox : 16 * h->var.KW;
-        const int tkw = h->umma ? h->wbox : 16 * h->var.KW;
+        const int tk = h->umma ? h->kbox : 16 * h->var.KW * h->var.KS;
+        const int tkw = h->umma ? h->wbox : 16 * h->var.KW * h->var.KS;
         const int bh = h->umma ? 1 : h->var.HPC;
         plt_status s;
         if (c.page_size > 0) {
@@ -591,7 +604,7 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
     if (kernels_per_run) *kernels_per_run = 2;
     if (heads_per_cta) *heads_per_cta = h->var.HPC;
-    if (key_slices) *key_slices = h->bf16 ? h->var.KW : kF32TileKeys / 16;
+    if (key_slices) *key_slices = h->bf16 ? h->var.KW * h->var.KS : kF32TileKeys / 16;
     if (stages) *stages = h->var.stages;
     if (ctas_per_sm) *ctas_per_sm = h->ctas_per_sm;
     if (grid) *grid = h->var.grid;

@@ -10,14 +10,15 @@ namespace plt {
 
 // Variant of the bf16 main kernel.
 struct MainVariant {
-    int D, MT, HPC, KW;  // head dim, 16-row tiles, KV heads per block, 16-key slices per tile
+    int D, NT, RW;       // head dim, 8-row groups per warp, warps along the packed rows
+    int HPC, KW, KS;     // KV heads per block, warps along the keys of a tile, 16-key slices per warp
     int stages;          // ring depth
     int grid;            // persistent blocks
     size_t smem;         // dynamic shared memory per block
 };
 
-bool main_bf16_exists(int D, int MT, int HPC, int KW);
-size_t main_bf16_smem(int D, int MT, int HPC, int KW, int stages, int max_batch);
+bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS);
+size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch);
 // Sets the shared-memory attribute and reports how many blocks fit one SM.
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
 cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, cudaStream_t stream);

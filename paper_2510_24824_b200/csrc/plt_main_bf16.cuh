@@ -1,12 +1,21 @@
-// bf16 split-KV main kernel of the CLP decode attention (Algorithm 3 lines 2-3 for all L loops).
+// bf16 split-KV main kernel of the CLP decode attention (Algorithm 3 lines 2-3 for all L loops),
+// warp-level tensor-core products with the KEYS as the M dimension.
 //
-// One persistent thread block owns an equal share of the line of key tiles of all sequences.
-// A producer warp streams K/V tiles of the shared first-loop cache (and of the windows of loops
-// 2..L) into a shared-memory ring with tiled TMA loads (128-byte swizzle); consumer warps run
-// S = Q K^T and acc += P V on the tensor cores with all L loop-queries and all GQA heads of a KV
-// head packed as the 16*MT rows of one tile, so every K/V byte is read from HBM once and used by
-// every loop. Softmax state is kept online in fp32 per row. Each consumer warp owns one 16-key
-// slice of a tile for one KV head and 16 packed rows; slices are merged once per piece.
+// One persistent thread block owns an equal share of the line of key tiles of all sequences. A
+// producer warp streams K/V tiles of the shared first-loop cache (and of the windows of loops 2..L)
+// into a shared-memory ring with tiled TMA loads (128-byte swizzle). Each consumer warp owns KS
+// 16-key slices of a tile for one KV head and ALL packed query rows of that head (all L loop-queries
+// times all GQA heads, 8 NT rows; RW warps split the rows when there are more than 32):
+//
+//   S^T [16 keys x 8 NT]   = K_slice [16 x d] . Q^T          A = K via ldmatrix, B = query rows in registers
+//   O^T [d x 8 NT]        += V_slice^T [d x 16] . P^T         A = V via ldmatrix.trans, B = P^T via movmatrix
+//   l   [. x 8 NT]        += ones [16 x 16] . P^T             softmax denominators, every row alike
+//
+// With the rows in the N dimension (granularity 8) nothing is padded to 16-row tiles, the K and V
+// fragments are loaded once for all rows, and the softmax needs no shuffles on the per-tile path:
+// the reference maximum of a row is updated lazily (a warp vote triggers the true row maxima and the
+// rescale of the accumulators only when a score exceeds the reference by more than kSlack powers
+// of two). Every K/V byte is read from HBM once and used by every loop.
 #pragma once
 #include <cuda_bf16.h>
 #include "plt_common.cuh"
@@ -15,20 +24,25 @@
 namespace plt {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every barrier wait gives up after ~2 s
+constexpr float kSlack = 8.f;
+constexpr float kNoMax = -1e30f;   // reference maximum of a row that has seen no key yet (finite, so that no select is needed)
+constexpr uint32_t kOnesBf16x2 = 0x3f803f80u;
 
-template <int D, int MT, int HPC, int KW>
-struct MainCfg {
+template <int D, int NT, int RW, int HPC, int KW, int KS>
+struct TCfg {
     static constexpr int NH = D / 64;               // 64-element (128-byte) halves of a head row
-    static constexpr int TK = 16 * KW;              // keys per tile
-    static constexpr int NCW = HPC * KW * MT;       // consumer warps
+    static constexpr int TK = 16 * KW * KS;         // keys per tile: KW warps along the keys, KS 16-key slices each
+    static constexpr int NCW = HPC * KW * RW;       // consumer warps
     static constexpr int NTHREADS = (NCW + 1) * 32;
-    static constexpr int MIN_BLOCKS = NCW <= 2 ? 4 : (NCW <= 4 ? 2 : 1);  // register budget: blocks per SM aimed at
+    static constexpr int ROWS_W = 8 * NT;           // packed rows per warp
+    // register budget: up to 16 rows per warp two to four blocks share an SM, above that one block has it all
+    static constexpr int MIN_BLOCKS = NT <= 2 ? (NCW <= 2 ? 4 : (NCW <= 4 ? 2 : 1)) : 1;
     static constexpr int BOX_BYTES = 128 * TK * HPC;        // one TMA box: [HPC][TK][64 elements]
     static constexpr int TENSOR_BYTES = NH * BOX_BYTES;     // K (or V) part of a stage
     static constexpr int STAGE_BYTES = 2 * TENSOR_BYTES;
-    static constexpr int MROW = D + 8;                      // padded row of the merge buffer (floats)
-    static constexpr int MERGE_ACC_FLOATS = KW > 1 ? HPC * MT * 16 * MROW : 0;
-    static constexpr int MERGE_ML_FLOATS = KW > 1 ? HPC * MT * KW * 32 : 0;
+    static constexpr int MROW = D + 4;                      // padded row of the merge buffer (floats): no bank conflicts
+    static constexpr int MERGE_ACC_FLOATS = KW > 1 ? HPC * RW * ROWS_W * MROW : 0;
+    static constexpr int MERGE_ML_FLOATS = KW > 1 ? HPC * RW * KW * ROWS_W * 2 : 0;
     static constexpr int kMaxStages = 12;
     __host__ __device__ static constexpr size_t smem_bytes(int stages, int max_batch) {
         return 1024 /* alignment slack */ + (size_t)stages * STAGE_BYTES + 2 * kMaxStages * 8 +
@@ -36,106 +50,154 @@ struct MainCfg {
     }
 };
 
-template <int D, int MT, int HPC, int KW, bool MASKED>
-__device__ __forceinline__ void process_slice(uint32_t sK, uint32_t sV, const uint32_t (&qf)[D / 16][4],
-                                              float (&acc)[D / 8][4], float (&m)[2], float (&lsum)[2],
-                                              int lim0, int lim1, int nvalid, float scale_log2, int lane,
-                                              int kw, int h_local) {
-    using C = MainCfg<D, MT, HPC, KW>;
-    const int tq = lane & 3;
-    // ---- S = Q K^T for this warp's 16 keys -------------------------------------------------------
-    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+// One consumer-warp step: this warp's 16 KS keys of a tile against its 8 NT packed rows.
+// Thread (grp = lane / 4, tq = lane % 4) holds of S^T, per 16-key slice ki, the keys grp and grp + 8 and, per 8-row
+// group nt, the rows 2 tq and 2 tq + 1: s[ki][nt][0..1] = key grp, s[ki][nt][2..3] = key grp + 8. lim[nt][j] (keys
+// visible to row 8 nt + 2 tq + j) and nvalid (keys that hold data) count from the first key of the tile and are used
+// only when MASKED. mref[nt][j] is the reference maximum (log2 units; kNoMax while the row has seen no key) the
+// accumulators of that row are scaled to; lacc[nt][j] the row's softmax denominator, accumulated on the tensor cores
+// from exactly the bf16-rounded weights that multiply V.
+template <int D, int NT, int KS, int HPC, int KW, int TKEYS, int BOXB, bool MASKED>
+__device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uint32_t (&qb)[D / 16][NT][2],
+                                             float (&acc)[D / 16][NT][4], float (&mref)[NT][2], float (&lacc)[NT][4],
+                                             const int (&lim)[NT][2], int nvalid, float scale_log2, int lane, int kw,
+                                             int h_local) {
+    const int grp = lane >> 2, tq = lane & 3;
+    const int kbase = kw * 16 * KS;   // first key of this warp in the tile
+    // ---- S^T = K Q^T ---------------------------------------------------------------------------------
+    // Shared-memory rows are 128 bytes (64 elements) with the 16-byte chunks XOR-swizzled by (row & 7); the two
+    // 64-element halves of a 128-wide head are BOXB bytes apart. Chunk (2 k + dhalf) ^ x of a row = base ^ (k << 5).
+    float s[KS][NT][4];
+#pragma unroll
+    for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) s[ki][nt][0] = s[ki][nt][1] = s[ki][nt][2] = s[ki][nt][3] = 0.f;
     {
-        const int key = kw * 16 + ((lane >> 4) << 3) + (lane & 7);
-        const int dhalf = (lane >> 3) & 1;
-        const uint32_t row = sK + (uint32_t)((h_local * C::TK + key) * 128);
-        const int x = key & 7;
+        const int key = kbase + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const uint32_t base = sK + (uint32_t)((h_local * TKEYS + key) * 128 + (((lane >> 4) ^ (key & 7)) << 4));
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-            const int cin = ((ks & 3) * 2 + dhalf) ^ x;
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4(row + (uint32_t)((ks >> 2) * C::BOX_BYTES + cin * 16), b0, b1, b2, b3);
-            mma_bf16_16816(s[0], qf[ks], b0, b1);
-            mma_bf16_16816(s[1], qf[ks], b2, b3);
+            const uint32_t addr = (base ^ (uint32_t)((ks & 3) << 5)) + (uint32_t)((ks >> 2) * BOXB);
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                uint32_t a[4];
+                ldmatrix_x4(addr + (uint32_t)(ki * 16 * 128), a[0], a[1], a[2], a[3]);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(s[ki][nt], a, qb[ks][nt][0], qb[ks][nt][1]);
+            }
         }
     }
-    // ---- per-loop causal cutoff / window length (only on boundary tiles) --------------------------
+    // ---- per-loop causal cutoff / window length (only on boundary tiles) ------------------------------
     if (MASKED) {
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+        for (int ki = 0; ki < KS; ++ki)
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int kk = kw * 16 + nt * 8 + 2 * tq + e;
-                if (kk >= lim0) s[nt][e] = -INFINITY;
-                if (kk >= lim1) s[nt][2 + e] = -INFINITY;
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int kk = kbase + ki * 16 + grp + (e >= 2 ? 8 : 0);
+                    if (kk >= lim[nt][e & 1]) s[ki][nt][e] = -INFINITY;
+                }
+    }
+    // ---- lazily updated reference maxima ----------------------------------------------------------------
+    bool grow = false;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
+#pragma unroll
+            for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
+            grow = grow || (fmaf(mx, scale_log2, -mref[nt][j]) > kSlack);  // true for a row's first visible key
+        }
+    if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
+#pragma unroll
+                for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                const float m_new = fmaxf(mref[nt][j], mx * scale_log2);
+                const float alpha = fast_exp2(mref[nt][j] - m_new);   // 1 while the row is empty, 0 at its first key
+                mref[nt][j] = m_new;
+                lacc[nt][j] *= alpha;
+                lacc[nt][2 + j] *= alpha;
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) {
+                    acc[mt][nt][j] *= alpha;
+                    acc[mt][nt][2 + j] *= alpha;
+                }
             }
     }
-    // ---- online softmax, fp32, rows grp (i = 0) and grp + 8 (i = 1) ------------------------------
-    uint32_t pa[4];
+    // ---- probabilities, transposed into the B operand of the second product --------------------------
+    uint32_t pb[KS][NT][2];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        float mx = fmaxf(fmaxf(s[0][2 * i], s[0][2 * i + 1]), fmaxf(s[1][2 * i], s[1][2 * i + 1]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m[i], mx * scale_log2);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = fast_exp2(m[i] - m_use);
-        m[i] = m_new;
-        const float p00 = fast_exp2(fmaf(s[0][2 * i], scale_log2, -m_use));
-        const float p01 = fast_exp2(fmaf(s[0][2 * i + 1], scale_log2, -m_use));
-        const float p10 = fast_exp2(fmaf(s[1][2 * i], scale_log2, -m_use));
-        const float p11 = fast_exp2(fmaf(s[1][2 * i + 1], scale_log2, -m_use));
-        pa[i] = pack_bf16x2(p00, p01);       // keys 2tq, 2tq+1
-        pa[2 + i] = pack_bf16x2(p10, p11);   // keys 8 + 2tq, 9 + 2tq
-        // The denominator sums the probabilities as rounded to bf16, i.e. exactly the weights the P V
-        // product uses: numerator and denominator then carry the same rounding, which cancels when a few
-        // keys dominate the softmax.
-        const float r00 = __uint_as_float(pa[i] << 16), r01 = __uint_as_float(pa[i] & 0xffff0000u);
-        const float r10 = __uint_as_float(pa[2 + i] << 16), r11 = __uint_as_float(pa[2 + i] & 0xffff0000u);
-        lsum[i] = fmaf(lsum[i], alpha, (r00 + r01) + (r10 + r11));
+    for (int ki = 0; ki < KS; ++ki)
 #pragma unroll
-        for (int nd = 0; nd < D / 8; ++nd) {
-            acc[nd][2 * i] *= alpha;
-            acc[nd][2 * i + 1] *= alpha;
+        for (int nt = 0; nt < NT; ++nt) {
+            const float p0 = fast_exp2(fmaf(s[ki][nt][0], scale_log2, -mref[nt][0]));
+            const float p1 = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
+            const float p2 = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
+            const float p3 = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
+            pb[ki][nt][0] = movmatrix_trans(pack_bf16x2(p0, p1));   // keys 0-7 of the slice
+            pb[ki][nt][1] = movmatrix_trans(pack_bf16x2(p2, p3));   // keys 8-15
         }
-    }
-    // ---- acc += P V ------------------------------------------------------------------------------
+    // ---- O^T += V^T P^T, denominators += 1 P^T --------------------------------------------------------
     {
-        const int mi = lane >> 3;
-        const int key = kw * 16 + ((mi & 1) << 3) + (lane & 7);
-        const uint32_t row = sV + (uint32_t)((h_local * C::TK + key) * 128);
-        const int x = key & 7;
-        uint32_t mask_lo = 0xffffffffu, mask_hi = 0xffffffffu;
+        const int key = kbase + (lane & 7) + (lane >> 4) * 8;
+        const uint32_t base = sV + (uint32_t)((h_local * TKEYS + key) * 128 + ((((lane >> 3) & 1) ^ (key & 7)) << 4));
+        uint32_t mask_lo[KS], mask_hi[KS];
         if (MASKED) {
-            // Rows at or beyond nvalid may hold anything (uninitialised cache slots): force them to 0
-            // so that 0 * garbage cannot produce NaN.
-            const int k0 = kw * 16 + 2 * tq;
-            mask_lo = (k0 < nvalid ? 0x0000ffffu : 0u) | (k0 + 1 < nvalid ? 0xffff0000u : 0u);
-            mask_hi = (k0 + 8 < nvalid ? 0x0000ffffu : 0u) | (k0 + 9 < nvalid ? 0xffff0000u : 0u);
+            // Rows at or beyond nvalid may hold anything (uninitialised cache slots): force them to 0 so that
+            // 0 * garbage cannot produce NaN.
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                const int k0 = kbase + ki * 16 + 2 * tq;
+                mask_lo[ki] = (k0 < nvalid ? 0x0000ffffu : 0u) | (k0 + 1 < nvalid ? 0xffff0000u : 0u);
+                mask_hi[ki] = (k0 + 8 < nvalid ? 0x0000ffffu : 0u) | (k0 + 9 < nvalid ? 0xffff0000u : 0u);
+            }
         }
 #pragma unroll
-        for (int j = 0; j < D / 16; ++j) {
-            const int cin = ((j & 3) * 2 + (mi >> 1)) ^ x;
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(row + (uint32_t)((j >> 2) * C::BOX_BYTES + cin * 16), b0, b1, b2, b3);
-            if (MASKED) {
-                b0 &= mask_lo;
-                b2 &= mask_lo;
-                b1 &= mask_hi;
-                b3 &= mask_hi;
+        for (int mt = 0; mt < D / 16; ++mt) {
+            const uint32_t addr = (base ^ (uint32_t)((mt & 3) << 5)) + (uint32_t)((mt >> 2) * BOXB);
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(addr + (uint32_t)(ki * 16 * 128), a[0], a[1], a[2], a[3]);
+                if (MASKED) {
+                    a[0] &= mask_lo[ki];
+                    a[1] &= mask_lo[ki];
+                    a[2] &= mask_hi[ki];
+                    a[3] &= mask_hi[ki];
+                }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(acc[mt][nt], a, pb[ki][nt][0], pb[ki][nt][1]);
             }
-            mma_bf16_16816(acc[2 * j], pa, b0, b1);
-            mma_bf16_16816(acc[2 * j + 1], pa, b2, b3);
         }
+        const uint32_t ones[4] = {kOnesBf16x2, kOnesBf16x2, kOnesBf16x2, kOnesBf16x2};
+#pragma unroll
+        for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(lacc[nt], ones, pb[ki][nt][0], pb[ki][nt][1]);
     }
 }
 
-template <int D, int MT, int HPC, int KW>
-__global__ void __launch_bounds__(MainCfg<D, MT, HPC, KW>::NTHREADS, MainCfg<D, MT, HPC, KW>::MIN_BLOCKS)
+template <int D, int NT, int RW, int HPC, int KW, int KS>
+__global__ void __launch_bounds__(TCfg<D, NT, RW, HPC, KW, KS>::NTHREADS, TCfg<D, NT, RW, HPC, KW, KS>::MIN_BLOCKS)
 plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
                      const __grid_constant__ Params p, const int stages) {
-    using C = MainCfg<D, MT, HPC, KW>;
+    using C = TCfg<D, NT, RW, HPC, KW, KS>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* full_bar = (uint64_t*)(smem + (size_t)stages * C::STAGE_BYTES);
@@ -148,15 +210,6 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
     bool ok = true;
-#ifdef PLT_TIMELINE
-    unsigned long long* tl = (unsigned long long*)p.timeline + (size_t)blockIdx.x * 8;
-    if (tid == 0) {
-        unsigned smid;
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        tl[0] = smid;
-        tl[1] = global_timer_ns();
-    }
-#endif
 
     if (tid == 0) {
         s_ctl[0] = 0;
@@ -175,10 +228,6 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         for (int b = tid; b <= p.B; b += C::NTHREADS) p.prefix[b] = s_prefix[b];
     const bool in_plan = cta < nctas;
     const int64_t lo = in_plan ? cta_begin(T, cta, nctas) : 0, hi = in_plan ? cta_begin(T, cta + 1, nctas) : 0;
-#ifdef PLT_TIMELINE
-    if (tid == 0) { tl[2] = global_timer_ns(); tl[7] = (unsigned long long)(hi - lo); }
-    bool tl_first = true;
-#endif
 
     if (wid == C::NCW) {
         // =========================== producer warp (one lane issues) ==============================
@@ -243,9 +292,6 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         ok = mbar_wait_bounded(&empty_bar[stage], (use - 1) & 1, kWaitLimitNs);
                         if (!ok) flags |= kDevWaitTimeout;
                     }
-#ifdef PLT_TIMELINE
-                    if (tl_first) { tl[3] = global_timer_ns(); tl_first = false; }
-#endif
                     if (ok) {
                         uint8_t* dst = smem + (size_t)stage * C::STAGE_BYTES;
                         mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
@@ -268,51 +314,70 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
     } else {
         // ================================= consumer warps =========================================
-        const int h_local = wid / (KW * MT);
-        const int mt = (wid % (KW * MT)) / KW;
+        const int h_local = wid / (KW * RW);
+        const int rw = (wid % (KW * RW)) / KW;
         const int kw = wid % KW;
         const int grp = lane >> 2, tq = lane & 3;
-        const int r0 = mt * 16 + grp, r1 = r0 + 8;
-        const int l0 = r0 / p.G, l1 = r1 / p.G;     // loop (0-based) of each row
-        const bool v0 = r0 < p.R, v1 = r1 < p.R;
+        const int rb = rw * C::ROWS_W;              // first packed row of this warp
         const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
+        // Rows as the accumulator fragments see them: column 2 tq + j of 8-row group nt.
+        int lc[NT][2];                               // loop (0-based) of the row, kMaxLoops for rows beyond R
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int r = rb + nt * 8 + 2 * tq + j;
+                lc[nt][j] = r < p.R ? r / p.G : kMaxLoops;
+            }
 
         int stage = 0;
         uint32_t use = 0;
-        int q_b = -1, q_hg = -1;   // (sequence, head group) whose query rows are in qf
-        uint32_t qf[D / 16][4];
+        int q_b = -1, q_hg = -1;   // (sequence, head group) whose query rows are in qb
+        uint32_t qb[D / 16][NT][2];
         PieceWalk walk(p, s_prefix, lo, hi);
         Piece pc;
         while (walk.next(pc, flags)) {
             const int kvh = pc.hg * HPC + h_local;
-            // ---- packed query rows of this KV head: row r = loop * G + head-in-group --------------
+            // ---- packed query rows of this KV head: row r = loop * G + head-in-group, as B fragments (row = lane / 4)
             // (the windows item of a head group follows its shared-cache item: same rows, kept)
             if (pc.b != q_b || pc.hg != q_hg) {
                 q_b = pc.b;
                 q_hg = pc.hg;
-                const int64_t q0 = (((int64_t)pc.b * p.L + l0) * p.Hq + kvh * p.G + (r0 - l0 * p.G)) * D;
-                const int64_t q1 = (((int64_t)pc.b * p.L + l1) * p.Hq + kvh * p.G + (r1 - l1 * p.G)) * D;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const int c = ks * 16 + 2 * tq;
-                    qf[ks][0] = v0 ? *(const uint32_t*)(qg + q0 + c) : 0u;
-                    qf[ks][1] = v1 ? *(const uint32_t*)(qg + q1 + c) : 0u;
-                    qf[ks][2] = v0 ? *(const uint32_t*)(qg + q0 + c + 8) : 0u;
-                    qf[ks][3] = v1 ? *(const uint32_t*)(qg + q1 + c + 8) : 0u;
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int r = rb + nt * 8 + grp;
+                    const bool v = r < p.R;
+                    const int l = v ? r / p.G : 0;
+                    const int64_t q0 = (((int64_t)pc.b * p.L + l) * p.Hq + kvh * p.G + (r - l * p.G)) * D + 2 * tq;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        qb[ks][nt][0] = v ? *(const uint32_t*)(qg + q0 + ks * 16) : 0u;
+                        qb[ks][nt][1] = v ? *(const uint32_t*)(qg + q0 + ks * 16 + 8) : 0u;
+                    }
                 }
             }
-            int cut0 = 0, cut1 = 0, cmin = 0x7fffffff;
+            int cutr[NT][2], cmin = 0x7fffffff;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) cutr[nt][0] = cutr[nt][1] = 0;
 #pragma unroll
             for (int l = 0; l < kMaxLoops; ++l)
                 if (l < p.L) {
-                    if (v0 && l == l0) cut0 = pc.sp.cut[l];
-                    if (v1 && l == l1) cut1 = pc.sp.cut[l];
-                    cmin = min(cmin, pc.sp.cut[l]);
-                }
-            float acc[D / 8][4];
+                    const int c = pc.sp.cut[l];
+                    cmin = min(cmin, c);
 #pragma unroll
-            for (int nd = 0; nd < D / 8; ++nd) acc[nd][0] = acc[nd][1] = acc[nd][2] = acc[nd][3] = 0.f;
-            float m[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
+                    for (int nt = 0; nt < NT; ++nt) {
+                        if (lc[nt][0] == l) cutr[nt][0] = c;
+                        if (lc[nt][1] == l) cutr[nt][1] = c;
+                    }
+                }
+            float acc[D / 16][NT][4], mref[NT][2], lacc[NT][4];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mref[nt][0] = mref[nt][1] = kNoMax;
+                lacc[nt][0] = lacc[nt][1] = lacc[nt][2] = lacc[nt][3] = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
+            }
 
             WinCursor cur;
             if (pc.kind == 1) cur.seek(p, pc.sp, pc.t0);
@@ -321,21 +386,25 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     ok = mbar_wait_bounded(&full_bar[stage], use & 1, kWaitLimitNs);
                     if (!ok) flags |= kDevWaitTimeout;
                 }
-#ifdef PLT_TIMELINE
-                if (tl_first && tid == 0) { tl[4] = global_timer_ns(); }
-                tl_first = false;
-#endif
                 const uint32_t sK = smem_u32(smem + (size_t)stage * C::STAGE_BYTES);
                 const uint32_t sV = sK + C::TENSOR_BYTES;
+                int lim[NT][2];
                 if (pc.kind == 0) {
                     const int key0 = t * C::TK;
                     if (ok) {
-                        if (key0 + C::TK <= cmin)
-                            process_slice<D, MT, HPC, KW, false>(sK, sV, qf, acc, m, lsum, 0, 0, 0, p.scale_log2, lane,
-                                                                 kw, h_local);
-                        else
-                            process_slice<D, MT, HPC, KW, true>(sK, sV, qf, acc, m, lsum, cut0 - key0, cut1 - key0,
-                                                                pc.sp.cmax - key0, p.scale_log2, lane, kw, h_local);
+                        if (key0 + C::TK <= cmin) {
+                            process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, false>(sK, sV, qb, acc, mref, lacc, cutr,
+                                                                                         0, p.scale_log2, lane, kw, h_local);
+                        } else {
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                lim[nt][0] = cutr[nt][0] - key0;
+                                lim[nt][1] = cutr[nt][1] - key0;
+                            }
+                            process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim,
+                                                                                        pc.sp.cmax - key0, p.scale_log2,
+                                                                                        lane, kw, h_local);
+                        }
                     }
                 } else {
                     // Window of loop cur.l: only the rows of that loop take part.
@@ -345,12 +414,16 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     for (int k = 1; k < kMaxLoops; ++k)
                         if (k == l) wl = pc.sp.wl[k];
                     const int row_lo = l * p.G, row_hi = row_lo + p.G;
-                    const bool any = row_lo < mt * 16 + 16 && row_hi > mt * 16;
+                    const bool any = row_lo < rb + C::ROWS_W && row_hi > rb;
                     if (ok && any) {
                         const int n = wl - cur.key0;
-                        process_slice<D, MT, HPC, KW, true>(sK, sV, qf, acc, m, lsum, (v0 && l0 == l) ? n : 0,
-                                                            (v1 && l1 == l) ? n : 0, n, p.scale_log2, lane, kw,
-                                                            h_local);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            lim[nt][0] = lc[nt][0] == l ? n : 0;
+                            lim[nt][1] = lc[nt][1] == l ? n : 0;
+                        }
+                        process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim, n,
+                                                                                    p.scale_log2, lane, kw, h_local);
                     }
                     cur.advance(p, pc.sp);
                 }
@@ -364,92 +437,96 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
 
             // ---- end of piece: merge the key slices and store the split partial ------------------
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                lsum[i] += __shfl_xor_sync(0xffffffffu, lsum[i], 1);
-                lsum[i] += __shfl_xor_sync(0xffffffffu, lsum[i], 2);
-            }
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    if (mref[nt][j] == kNoMax) mref[nt][j] = -INFINITY;   // the partial's "saw no key" mark
             const int64_t slot = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta);
-            const int64_t prow = (slot * HPC + h_local) * p.R;
+            const int64_t prow = (slot * HPC + h_local) * p.R + rb;
             if (tid == 0) note_piece(p, pc, cta);
             if (KW == 1) {
 #pragma unroll
-                for (int nd = 0; nd < D / 8; ++nd) {
-                    const int c = nd * 8 + 2 * tq;
-                    if (v0) *(float2*)(p.part_acc + (prow + r0) * D + c) = make_float2(acc[nd][0], acc[nd][1]);
-                    if (v1) *(float2*)(p.part_acc + (prow + r1) * D + c) = make_float2(acc[nd][2], acc[nd][3]);
-                }
-                if (tq == 0) {
-                    if (v0) *(float2*)(p.part_ml + (prow + r0) * 2) = make_float2(m[0], lsum[0]);
-                    if (v1) *(float2*)(p.part_ml + (prow + r1) * 2) = make_float2(m[1], lsum[1]);
-                }
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        if (lc[nt][j] == kMaxLoops) continue;
+                        const int64_t row = prow + nt * 8 + 2 * tq + j;
+                        float* dst = p.part_acc + row * D + grp;
+#pragma unroll
+                        for (int mt = 0; mt < D / 16; ++mt) {
+                            dst[mt * 16] = acc[mt][nt][j];
+                            dst[mt * 16 + 8] = acc[mt][nt][2 + j];
+                        }
+                        if (grp == 0) *(float2*)(p.part_ml + row * 2) = make_float2(mref[nt][j], lacc[nt][j]);
+                    }
             } else {
-                const int gidx = h_local * MT + mt;
-                float* macc = merge_acc + gidx * 16 * C::MROW;
-                float* mml = merge_ml + gidx * KW * 32;
-                if (tq == 0) {
-                    *(float2*)(mml + (kw * 16 + grp) * 2) = make_float2(m[0], lsum[0]);
-                    *(float2*)(mml + (kw * 16 + grp + 8) * 2) = make_float2(m[1], lsum[1]);
+                const int gidx = h_local * RW + rw;
+                float* macc = merge_acc + gidx * C::ROWS_W * C::MROW;
+                float* mml = merge_ml + gidx * KW * C::ROWS_W * 2;
+                if (grp == 0) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)
+                            *(float2*)(mml + (kw * C::ROWS_W + nt * 8 + 2 * tq + j) * 2) = make_float2(mref[nt][j], lacc[nt][j]);
                 }
                 named_barrier_sync(1, C::NCW * 32);
-                float mstar[2], lstar[2], sc[2];
+                float sc[NT][2];
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    float mm = -INFINITY;
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int k = 0; k < KW; ++k) mm = fmaxf(mm, mml[(k * 16 + grp + 8 * i) * 2]);
-                    const float ms = (mm == -INFINITY) ? 0.f : mm;
-                    float ll = 0.f;
+                    for (int j = 0; j < 2; ++j) {
+                        const int lr = nt * 8 + 2 * tq + j;
+                        float mm = -INFINITY;
 #pragma unroll
-                    for (int k = 0; k < KW; ++k) {
-                        const float2 v = *(const float2*)(mml + (k * 16 + grp + 8 * i) * 2);
-                        ll = fmaf(v.y, fast_exp2(v.x - ms), ll);
+                        for (int k = 0; k < KW; ++k) mm = fmaxf(mm, mml[(k * C::ROWS_W + lr) * 2]);
+                        const float ms = (mm == -INFINITY) ? 0.f : mm;
+                        sc[nt][j] = fast_exp2(mref[nt][j] - ms);
+                        if (kw == 0 && grp == 0 && lc[nt][j] != kMaxLoops) {
+                            float ll = 0.f;
+#pragma unroll
+                            for (int k = 0; k < KW; ++k) {
+                                const float2 v = *(const float2*)(mml + (k * C::ROWS_W + lr) * 2);
+                                ll = fmaf(v.y, fast_exp2(v.x - ms), ll);
+                            }
+                            *(float2*)(p.part_ml + (prow + lr) * 2) = make_float2(mm, ll);
+                        }
                     }
-                    mstar[i] = mm;
-                    lstar[i] = ll;
-                    sc[i] = fast_exp2(m[i] - ms);
-                }
 #pragma unroll
                 for (int k = 0; k < KW; ++k) {
                     if (kw == k) {
 #pragma unroll
-                        for (int nd = 0; nd < D / 8; ++nd) {
-                            float2* a0 = (float2*)(macc + grp * C::MROW + nd * 8 + 2 * tq);
-                            float2* a1 = (float2*)(macc + (grp + 8) * C::MROW + nd * 8 + 2 * tq);
-                            float2 x0 = make_float2(acc[nd][0] * sc[0], acc[nd][1] * sc[0]);
-                            float2 x1 = make_float2(acc[nd][2] * sc[1], acc[nd][3] * sc[1]);
-                            if (k > 0) {
-                                const float2 y0 = *a0, y1 = *a1;
-                                x0.x += y0.x; x0.y += y0.y; x1.x += y1.x; x1.y += y1.y;
+                        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                float* a = macc + (nt * 8 + 2 * tq + j) * C::MROW + grp;
+#pragma unroll
+                                for (int mt = 0; mt < D / 16; ++mt) {
+                                    float x0 = acc[mt][nt][j] * sc[nt][j], x1 = acc[mt][nt][2 + j] * sc[nt][j];
+                                    if (k > 0) {
+                                        x0 += a[mt * 16];
+                                        x1 += a[mt * 16 + 8];
+                                    }
+                                    a[mt * 16] = x0;
+                                    a[mt * 16 + 8] = x1;
+                                }
                             }
-                            *a0 = x0;
-                            *a1 = x1;
-                        }
                     }
                     named_barrier_sync(1, C::NCW * 32);
                 }
                 // The KW warps of the group copy the merged rows out, 16 bytes per thread per step.
-                for (int i4 = kw * 32 + lane; i4 < 16 * (D / 4); i4 += KW * 32) {
+                for (int i4 = kw * 32 + lane; i4 < C::ROWS_W * (D / 4); i4 += KW * 32) {
                     const int row = i4 / (D / 4), c = (i4 % (D / 4)) * 4;
-                    if (mt * 16 + row < p.R)
-                        *(float4*)(p.part_acc + (prow + mt * 16 + row) * D + c) = *(const float4*)(macc + row * C::MROW + c);
-                }
-                if (kw == 0 && tq == 0) {
-                    if (v0) *(float2*)(p.part_ml + (prow + r0) * 2) = make_float2(mstar[0], lstar[0]);
-                    if (v1) *(float2*)(p.part_ml + (prow + r1) * 2) = make_float2(mstar[1], lstar[1]);
+                    if (rb + row < p.R)
+                        *(float4*)(p.part_acc + (prow + row) * D + c) = *(const float4*)(macc + row * C::MROW + c);
                 }
                 named_barrier_sync(1, C::NCW * 32);
             }
         }
     }
-#ifdef PLT_TIMELINE
-    if (tid == 0) tl[5] = global_timer_ns();
-#endif
     if (flags) atomicOr(p.status, flags);
     if (flags & kDevWaitTimeout) s_ctl[0] = 1;
     __syncthreads();
-#ifdef PLT_TIMELINE
-    if (tid == 0) tl[6] = global_timer_ns();
-#endif
     // A wait ran out somewhere: before the block retires, give every copy that was issued a bounded
     // chance to land (in the normal path the consumers have waited for all of them already).
     if (s_ctl[0] != 0 && tid == 0) {

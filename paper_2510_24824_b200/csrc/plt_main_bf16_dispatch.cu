@@ -3,27 +3,29 @@
 
 namespace plt {
 
-#define PLT_DECL(D, MT) \
-    cudaError_t main_bf16_d##D##_mt##MT(int, const MainVariant&, const CUtensorMap*, const Params*, cudaStream_t, int*);
-PLT_DECL(64, 1) PLT_DECL(64, 2) PLT_DECL(64, 4) PLT_DECL(128, 1) PLT_DECL(128, 2) PLT_DECL(128, 4)
+#define PLT_ALL(X, D) X(D, 1, 1) X(D, 2, 1) X(D, 3, 1) X(D, 4, 1) X(D, 2, 2) X(D, 3, 2) X(D, 4, 2)
+#define PLT_DECL(D, NT, RW) \
+    cudaError_t main_bf16_d##D##_n##NT##r##RW(int, const MainVariant&, const CUtensorMap*, const Params*, cudaStream_t, int*);
+PLT_ALL(PLT_DECL, 64) PLT_ALL(PLT_DECL, 128)
 #undef PLT_DECL
 
 static cudaError_t dispatch(int op, const MainVariant& v, const CUtensorMap* maps, const Params* p, cudaStream_t s,
                             int* out) {
-#define PLT_GO(D_, MT_) \
-    if (v.D == D_ && v.MT == MT_) return main_bf16_d##D_##_mt##MT_(op, v, maps, p, s, out);
-    PLT_GO(64, 1) PLT_GO(64, 2) PLT_GO(64, 4) PLT_GO(128, 1) PLT_GO(128, 2) PLT_GO(128, 4)
+#define PLT_GO(D_, NT_, RW_) \
+    if (v.D == D_ && v.NT == NT_ && v.RW == RW_) return main_bf16_d##D_##_n##NT_##r##RW_(op, v, maps, p, s, out);
+    PLT_ALL(PLT_GO, 64) PLT_ALL(PLT_GO, 128)
 #undef PLT_GO
+#undef PLT_ALL
     return cudaErrorInvalidValue;
 }
 
-bool main_bf16_exists(int D, int MT, int HPC, int KW) {
-    MainVariant v{D, MT, HPC, KW, 1, 1, 0};
+bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, 1, 1, 0};
     return dispatch(0, v, nullptr, nullptr, nullptr, nullptr) == cudaSuccess;
 }
 
-size_t main_bf16_smem(int D, int MT, int HPC, int KW, int stages, int max_batch) {
-    MainVariant v{D, MT, HPC, KW, stages, max_batch, 0};
+size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, stages, max_batch, 0};
     int out = 0;
     if (dispatch(3, v, nullptr, nullptr, nullptr, &out) != cudaSuccess) return 0;
     return (size_t)out;

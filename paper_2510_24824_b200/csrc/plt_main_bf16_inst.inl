@@ -1,6 +1,7 @@
-// Instantiates the bf16 main kernel for one (head dim, row tiles) pair and the (KV heads per block,
-// key slices) variants that fit 8 consumer warps. Included by the plt_main_bf16_d*_mt*.cu files,
-// which define PLT_INST_D, PLT_INST_MT and PLT_INST_NAME.
+// Instantiates the bf16 main kernel for one (head dim, 8-row groups per warp, warps along the rows)
+// triple and the (KV heads per block, warps along the keys, slices per warp) variants that fit 8
+// consumer warps. Included by the plt_main_bf16_d*_n*r*.cu files, which define PLT_INST_D,
+// PLT_INST_NT, PLT_INST_RW and PLT_INST_NAME.
 #include "plt_host.h"
 #include "plt_main_bf16.cuh"
 
@@ -8,12 +9,12 @@ namespace plt {
 
 namespace {
 
-template <int HPC, int KW>
+template <int HPC, int KW, int KS>
 cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const Params* p, cudaStream_t stream,
                    int* out) {
-    constexpr int D = PLT_INST_D, MT = PLT_INST_MT;
-    using C = MainCfg<D, MT, HPC, KW>;
-    auto fn = plt_decode_main_bf16<D, MT, HPC, KW>;
+    constexpr int D = PLT_INST_D, NT = PLT_INST_NT, RW = PLT_INST_RW;
+    using C = TCfg<D, NT, RW, HPC, KW, KS>;
+    auto fn = plt_decode_main_bf16<D, NT, RW, HPC, KW, KS>;
     if (op == 0) return cudaSuccess;
     if (op == 1) {
         cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)v.smem);
@@ -32,12 +33,13 @@ cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const 
 
 cudaError_t PLT_INST_NAME(int op, const MainVariant& v, const CUtensorMap* maps, const Params* p, cudaStream_t stream,
                           int* out) {
-#define PLT_CASE(H, K)                                               \
-    if (v.HPC == H && v.KW == K) {                                   \
-        if constexpr (H * K * PLT_INST_MT <= 8) return run_op<H, K>(op, v, maps, p, stream, out); \
+#define PLT_CASE(H, K, S)                                            \
+    if (v.HPC == H && v.KW == K && v.KS == S) {                      \
+        if constexpr (H * K * PLT_INST_RW <= 8) return run_op<H, K, S>(op, v, maps, p, stream, out); \
     }
-    PLT_CASE(1, 1) PLT_CASE(1, 2) PLT_CASE(1, 4) PLT_CASE(2, 1) PLT_CASE(2, 2) PLT_CASE(2, 4)
-    PLT_CASE(4, 1) PLT_CASE(4, 2) PLT_CASE(8, 1)
+    PLT_CASE(1, 1, 1) PLT_CASE(1, 2, 1) PLT_CASE(1, 4, 1) PLT_CASE(2, 1, 1) PLT_CASE(2, 2, 1) PLT_CASE(2, 4, 1)
+    PLT_CASE(1, 8, 1) PLT_CASE(4, 1, 1) PLT_CASE(4, 2, 1) PLT_CASE(8, 1, 1)
+    PLT_CASE(1, 1, 2) PLT_CASE(1, 2, 2) PLT_CASE(1, 4, 2) PLT_CASE(2, 1, 2) PLT_CASE(2, 2, 2) PLT_CASE(4, 1, 2)
 #undef PLT_CASE
     return cudaErrorInvalidValue;
 }
