@@ -146,14 +146,16 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
         if (kw < 1) kw = 1;
     }
     if (c->Hkv % hpc != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "heads_per_cta %d does not divide Hkv %d", hpc, c->Hkv);
-    while (c->page_size > 0 && c->page_size % (16 * kw * ks) != 0 && kw > 1) kw >>= 1;
-    if (c->page_size > 0 && c->page_size % (16 * kw * ks) != 0) ks = 1;
+    auto tile = [&]() { return main_bf16_tile_keys(v->D, nt, rw, hpc, kw, ks); };
+    while (c->page_size > 0 && tile() > 0 && c->page_size % tile() != 0 && kw > 1) kw >>= 1;
+    if (c->page_size > 0 && tile() > 0 && c->page_size % tile() != 0) ks = 1;
     if (!main_bf16_exists(v->D, nt, rw, hpc, kw, ks))
         return fail(nullptr, PLT_ERR_UNSUPPORTED,
                     "no bf16 kernel for heads_per_cta=%d key_slices=%d slices_per_warp=%d row_warps=%d", hpc, kw, ks, rw);
     v->HPC = hpc;
     v->KW = kw;
     v->KS = ks;
+    v->tile_keys = tile();
     const int ncw = hpc * kw * rw;
     int cps = c->ctas_per_sm > 0 ? c->ctas_per_sm : (small && ncw <= 4 ? 2 : 1);
     const size_t budget = (size_t)(cps >= 2 ? 227 * 1024 / cps - 1024 : 227 * 1024);
@@ -248,7 +250,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the tcgen05 main kernel", e);
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
         h->umma = true;
-        h->var = MainVariant{config->d, 0, 0, 1, 8, 1, nslot, 0, smem};
+        h->var = MainVariant{config->d, 0, 0, 1, 8, 1, 128, nslot, 0, smem};
         h->ctas_per_sm = 1;
         h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)
                                         : (config->max_seq_len < 128 ? config->max_seq_len : 128);
@@ -262,7 +264,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
         h->ctas_per_sm = blocks < cps ? blocks : cps;
     } else {
-        h->var = MainVariant{config->d, 0, 0, 1, 1, 1, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
+        h->var = MainVariant{config->d, 0, 0, 1, 1, 1, kF32TileKeys, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
         e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
         if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the fp32 main kernel", e);
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "fp32 main kernel does not fit an SM");
@@ -279,7 +281,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         h->encode = (EncodeTiledFn)fn;
     }
     // The tile line must fit 31 bits.
-    const int tk = h->bf16 ? 16 * h->var.KW * h->var.KS : kF32TileKeys;
+    const int tk = h->var.tile_keys;
     const double tiles = (double)config->max_batch * (config->Hkv / h->var.HPC) *
                          ((double)(config->max_seq_len + tk - 1) / tk + (double)(config->L - 1) * ((config->w + tk - 1) / tk));
     if (tiles >= 2147483647.0) return fail(nullptr, PLT_ERR_UNSUPPORTED, "max_batch * max_seq_len too large for the tile plan");
@@ -423,7 +425,7 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
     p.num_pool_pages = a->num_pool_pages;
     p.hpc = h->var.HPC;
-    p.tile_keys = h->bf16 ? 16 * h->var.KW * h->var.KS : kF32TileKeys;
+    p.tile_keys = h->var.tile_keys;
     p.num_ctas = h->var.grid;
     p.scale_log2 = h->scale_log2;
     for (int l = 0; l < kMaxLoops; ++l) p.delta[l] = h->delta[l];
@@ -433,8 +435,8 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     if (h->bf16) {
         // keys and heads per TMA box: the warp-level kernel loads [heads per block][tile keys], the tcgen05 kernel
         // [1 head][up to 128 keys]
-        const int tk = h->umma ? h->kbox : 16 * h->var.KW * h->var.KS;
-        const int tkw = h->umma ? h->wbox : 16 * h->var.KW * h->var.KS;
+        const int tk = h->umma ? h->kbox : h->var.tile_keys;
+        const int tkw = h->umma ? h->wbox : h->var.tile_keys;
         const int bh = h->umma ? 1 : h->var.HPC;
         plt_status s;
         if (c.page_size > 0) {
@@ -604,7 +606,7 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
     if (kernels_per_run) *kernels_per_run = 2;
     if (heads_per_cta) *heads_per_cta = h->var.HPC;
-    if (key_slices) *key_slices = h->bf16 ? h->var.KW * h->var.KS : kF32TileKeys / 16;
+    if (key_slices) *key_slices = h->var.tile_keys / 16;
     if (stages) *stages = h->var.stages;
     if (ctas_per_sm) *ctas_per_sm = h->ctas_per_sm;
     if (grid) *grid = h->var.grid;

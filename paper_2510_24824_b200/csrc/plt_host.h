@@ -12,6 +12,7 @@ namespace plt {
 struct MainVariant {
     int D, NT, RW;       // head dim, 8-row groups per warp, warps along the packed rows
     int HPC, KW, KS;     // KV heads per block, warps along the keys of a tile, 16-key slices per warp
+    int tile_keys;       // keys per pipeline tile
     int stages;          // ring depth
     int grid;            // persistent blocks
     size_t smem;         // dynamic shared memory per block
@@ -19,6 +20,8 @@ struct MainVariant {
 
 bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS);
 size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch);
+// Keys per pipeline tile of a variant (0 if it does not exist): the warps along the keys split a tile or take turns.
+int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS);
 // Sets the shared-memory attribute and reports how many blocks fit one SM.
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
 cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, cudaStream_t stream);

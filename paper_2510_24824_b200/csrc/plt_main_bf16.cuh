@@ -250,9 +250,10 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 // Paged cache: the id of the page in use and, loaded one page early so that its latency is off the
                 // issue path, the id of the page after it.
                 const int32_t* ptab = p.page_table + (int64_t)pc.b * p.max_pages;
-                int pg = 0, page_id = 0, page_next = 0;
+                int pg = 0, in_page = 0, page_id = 0, page_next = 0;
                 if (pc.kind == 0 && p.page_size > 0) {
                     pg = (pc.t0 * C::TK) / p.page_size;
+                    in_page = pc.t0 * C::TK - pg * p.page_size;   // advanced by a tile per step: no division per tile
                     page_id = ptab[pg];
                     page_next = ptab[min(pg + 1, p.max_pages - 1)];
                 }
@@ -264,8 +265,8 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         mk = &tmK;
                         mv = &tmV;
                         if (p.page_size > 0) {
-                            const int in_page = key0 % p.page_size;
-                            if (in_page == 0 && t != pc.t0) {
+                            if (in_page == p.page_size) {
+                                in_page = 0;
                                 ++pg;
                                 page_id = page_next;
                                 page_next = ptab[min(pg + 1, p.max_pages - 1)];
@@ -277,6 +278,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                             }
                             c1 = in_page;
                             c3 = page;
+                            in_page += C::TK;
                         } else {
                             c1 = key0;
                             c3 = pc.b;

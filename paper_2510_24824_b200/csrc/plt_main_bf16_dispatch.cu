@@ -20,15 +20,22 @@ static cudaError_t dispatch(int op, const MainVariant& v, const CUtensorMap* map
 }
 
 bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS) {
-    MainVariant v{D, NT, RW, HPC, KW, KS, 1, 1, 0};
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0};
     return dispatch(0, v, nullptr, nullptr, nullptr, nullptr) == cudaSuccess;
 }
 
 size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch) {
-    MainVariant v{D, NT, RW, HPC, KW, KS, stages, max_batch, 0};
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, stages, max_batch, 0};
     int out = 0;
     if (dispatch(3, v, nullptr, nullptr, nullptr, &out) != cudaSuccess) return 0;
     return (size_t)out;
+}
+
+int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0};
+    int out = 0;
+    if (dispatch(4, v, nullptr, nullptr, nullptr, &out) != cudaSuccess) return 0;
+    return out;
 }
 
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm) {

@@ -21,6 +21,10 @@ cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const 
         if (e != cudaSuccess) return e;
         return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, fn, C::NTHREADS, v.smem);
     }
+    if (op == 4) {
+        *out = C::TK;
+        return cudaSuccess;
+    }
     if (op == 3) {
         *out = (int)C::smem_bytes(v.stages, v.grid /* max_batch passed in grid for this query */);
         return cudaSuccess;
@@ -35,7 +39,8 @@ cudaError_t PLT_INST_NAME(int op, const MainVariant& v, const CUtensorMap* maps,
                           int* out) {
 #define PLT_CASE(H, K, S)                                            \
     if (v.HPC == H && v.KW == K && v.KS == S) {                      \
-        if constexpr (H * K * PLT_INST_RW <= 8) return run_op<H, K, S>(op, v, maps, p, stream, out); \
+        if constexpr (H * K * PLT_INST_RW <= (PLT_INST_NT <= 2 ? 8 : 4))                          \
+            return run_op<H, K, S>(op, v, maps, p, stream, out);                              \
     }
     PLT_CASE(1, 1, 1) PLT_CASE(1, 2, 1) PLT_CASE(1, 4, 1) PLT_CASE(2, 1, 1) PLT_CASE(2, 2, 1) PLT_CASE(2, 4, 1)
     PLT_CASE(1, 8, 1) PLT_CASE(4, 1, 1) PLT_CASE(4, 2, 1) PLT_CASE(8, 1, 1)

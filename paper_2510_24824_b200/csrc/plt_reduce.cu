@@ -79,28 +79,58 @@ __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __g
     const int l = r / p.G, g = r - l * p.G;
     const int h = (hg * p.hpc + hl) * p.G + g;
 
-    // Everything above depends on the launch only; from here on the main kernel's results are read.
-    grid_dependency_wait();
-
-    // Each warp works out its own row: the plan of the sequence (is there anything to merge?) and, from the table
-    // the main kernel's blocks left, which of them hold the pieces of the two items.
+    // What the caller passed (length, window length, gate logit) is read while the main kernel still drains; this
+    // row's loop alone decides what is merged: cut = keys of the shared cache it may see, wl = its window's valid slots.
     uint32_t flags = 0;
-    SeqPlan sp;
-    seq_plan(p, b, sp, flags);
-    int cut = 0;
-#pragma unroll
-    for (int k = 0; k < kMaxLoops; ++k)
-        if (k == l) cut = sp.cut[k];
+    const int32_t n = seq_len_clamped(p, b, flags);
+    int cut = n - p.delta[l];
+    cut = cut > 0 ? cut : 0;
+    int wl = 0;
+    float x = 0.f;
+    if (l > 0) {
+        wl = cut < p.w ? cut : p.w;
+        if (p.win_lens != nullptr && cut > 0) {
+            wl = p.win_lens[b * (p.L - 1) + (l - 1)];
+            wl = wl < 0 ? 0 : (wl > p.w ? p.w : wl);
+        }
+        x = p.gate_logits[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h];
+    }
     const int item_g = item_index(p, b, hg, 0), item_l = item_index(p, b, hg, 1);
+
+    // From here on the main kernel's results are read: first which of its blocks hold the pieces of the two items
+    // (the table those blocks left), then the pieces. Both items' loads are issued together.
+    grid_dependency_wait();
     int2 rg = make_int2(0, -1), rl = make_int2(0, -1);
-    if (sp.gt > 0) rg = *(const int2*)(p.item_blocks + 2 * item_g);
-    if (sp.lt > 0 && l > 0) rl = *(const int2*)(p.item_blocks + 2 * item_l);
+    if (cut > 0) rg = *(const int2*)(p.item_blocks + 2 * item_g);
+    if (wl > 0) rl = *(const int2*)(p.item_blocks + 2 * item_l);
 
     Vec<D> yg, yl;
     float out[Vec<D>::N];
     if (cut == 0) {
 #pragma unroll
         for (int i = 0; i < Vec<D>::N; ++i) out[i] = 0.f;
+    } else if (rg.x == rg.y && rl.x >= rl.y) {
+        // The usual case: each item was done by one block (or the window is empty); nothing to rescale.
+        const int64_t row_g = (slot_of(item_g, rg.x) * p.hpc + hl) * p.R + r;
+        const int64_t row_l = (slot_of(item_l, rl.x) * p.hpc + hl) * p.R + r;
+        const bool has_l = rl.x == rl.y;
+        float2 mg = *(const float2*)(p.part_ml + row_g * 2), ml = make_float2(-INFINITY, 0.f);
+        load_vec<D>(p.part_acc + row_g * D + lane * Vec<D>::N, yg);
+        if (has_l) {
+            ml = *(const float2*)(p.part_ml + row_l * 2);
+            load_vec<D>(p.part_acc + row_l * D + lane * Vec<D>::N, yl);
+        }
+        const float ig = (mg.x != -INFINITY && mg.y > 0.f) ? 1.f / mg.y : 0.f;
+        if (l == 0) {
+#pragma unroll
+            for (int i = 0; i < Vec<D>::N; ++i) out[i] = yg.v[i] * ig;
+        } else {
+            const float il = (has_l && ml.x != -INFINITY && ml.y > 0.f) ? 1.f / ml.y : 0.f;  // empty window: y_local = 0
+            const float gate = 1.f / (1.f + expf(-x));
+#pragma unroll
+            for (int i = 0; i < Vec<D>::N; ++i)
+                out[i] = gate * (has_l ? yl.v[i] * il : 0.f) + (1.f - gate) * (yg.v[i] * ig);
+        }
     } else {
         const float dg = merge_item<D>(p, item_g, hl, r, rg.x, rg.y, lane, yg);
         const float ig = dg > 0.f ? 1.f / dg : 0.f;
@@ -110,7 +140,6 @@ __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __g
         } else {
             const float dl = merge_item<D>(p, item_l, hl, r, rl.x, rl.y, lane, yl);
             const float il = dl > 0.f ? 1.f / dl : 0.f;  // empty window: y_local = 0
-            const float x = p.gate_logits[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h];
             const float gate = 1.f / (1.f + expf(-x));
 #pragma unroll
             for (int i = 0; i < Vec<D>::N; ++i) out[i] = gate * (yl.v[i] * il) + (1.f - gate) * (yg.v[i] * ig);
