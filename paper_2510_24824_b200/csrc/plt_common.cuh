@@ -44,6 +44,7 @@ struct Params {
     int32_t hpc;               // KV heads per work item
     int32_t tile_keys;         // keys per plan tile
     int32_t num_ctas;          // persistent grid size of the main kernel
+    int32_t piece_cost;        // what starting and finishing an item costs a block, in tiles (balances the plan)
     float scale_log2;          // sm_scale * log2(e)
     int32_t delta[kMaxLoops];  // per-loop causal offset
 };
@@ -120,11 +121,16 @@ __device__ __forceinline__ void seq_plan(const Params& p, int b, SeqPlan& s, uin
     seq_plan_n(p, b, seq_len_clamped(p, b, flags), s, flags);
 }
 
-// Tiles sequence b puts on the line.
+// Positions an item of `tiles` tiles takes on the line: its tiles preceded by piece_cost positions that stand for the
+// work of starting and finishing it (query rows, plan step, partial store). A block whose share of an item holds
+// none of its tiles skips it. Blocks with many short items thus get fewer tiles than blocks inside a long one.
+__device__ __forceinline__ int32_t line_len(const Params& p, int32_t tiles) { return tiles > 0 ? tiles + p.piece_cost : 0; }
+
+// Positions sequence b puts on the line.
 __device__ __forceinline__ int32_t seq_tiles(const Params& p, int b, uint32_t& flags) {
     SeqPlan s;
     seq_plan(p, b, s, flags);
-    return (p.Hkv / p.hpc) * (s.gt + s.lt);
+    return (p.Hkv / p.hpc) * (line_len(p, s.gt) + line_len(p, s.lt));
 }
 
 // Blocks that take part in the plan: never more than there are tiles, so that every taking-part
@@ -160,7 +166,7 @@ __device__ __forceinline__ void build_prefix(const Params& p, int32_t* sp, uint3
         SeqPlan s;
         if (small) seq_plan_small(p, b, n, s, flags);
         else seq_plan_n(p, b, n, s, flags);
-        sp[b + 1] = (p.Hkv / p.hpc) * (s.gt + s.lt);
+        sp[b + 1] = (p.Hkv / p.hpc) * (line_len(p, s.gt) + line_len(p, s.lt));
     }
     if (tid == 0) sp[0] = 0;
     __syncthreads();
@@ -218,30 +224,35 @@ struct PieceWalk {
     __device__ bool next_small(Piece& pc, uint32_t& flags) { return next_impl<true>(pc, flags); }
     template <bool SMALL>
     __device__ __forceinline__ bool next_impl(Piece& pc, uint32_t& flags) {
-        if (pos >= hi) return false;
-        while ((int64_t)sp[b + 1] <= pos) ++b;
-        if (SMALL) seq_plan_small(p, b, lens[b], pc.sp, flags);
-        else if (lens != nullptr) seq_plan_n(p, b, lens[b], pc.sp, flags);
-        else seq_plan(p, b, pc.sp, flags);
-        const int per = pc.sp.gt + pc.sp.lt;
-        const int o = (int)(pos - sp[b]);
-        pc.b = b;
-        pc.hg = o / per;
-        const int o2 = o - pc.hg * per;
-        int64_t item_end;
-        if (o2 < pc.sp.gt) {
-            pc.kind = 0;
-            pc.t0 = o2;
-            item_end = pos + (pc.sp.gt - o2);
-        } else {
-            pc.kind = 1;
-            pc.t0 = o2 - pc.sp.gt;
-            item_end = pos + (per - o2);
+        for (;;) {
+            if (pos >= hi) return false;
+            while ((int64_t)sp[b + 1] <= pos) ++b;
+            if (SMALL) seq_plan_small(p, b, lens[b], pc.sp, flags);
+            else if (lens != nullptr) seq_plan_n(p, b, lens[b], pc.sp, flags);
+            else seq_plan(p, b, pc.sp, flags);
+            const int vg = line_len(p, pc.sp.gt), per = vg + line_len(p, pc.sp.lt);
+            const int o = (int)(pos - sp[b]);
+            pc.b = b;
+            pc.hg = o / per;
+            const int o2 = o - pc.hg * per;
+            int v0;   // position inside the item
+            int64_t item_end;
+            if (o2 < vg) {
+                pc.kind = 0;
+                v0 = o2;
+                item_end = pos + (vg - o2);
+            } else {
+                pc.kind = 1;
+                v0 = o2 - vg;
+                item_end = pos + (per - o2);
+            }
+            const int64_t end = item_end < hi ? item_end : hi;
+            const int v1 = v0 + (int)(end - pos);
+            pos = end;
+            pc.t0 = v0 > p.piece_cost ? v0 - p.piece_cost : 0;
+            pc.t1 = v1 > p.piece_cost ? v1 - p.piece_cost : 0;
+            if (pc.t1 > pc.t0) return true;   // else: only the item's lead-in positions fell to this block
         }
-        const int64_t end = item_end < hi ? item_end : hi;
-        pc.t1 = pc.t0 + (int)(end - pos);
-        pos = end;
-        return true;
     }
 };
 

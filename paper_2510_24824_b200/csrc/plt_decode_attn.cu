@@ -49,6 +49,7 @@ struct plt_decode_attn {
     bool umma = false;    // bf16 path on tcgen05 / tensor memory (var.HPC = 1, var.KW = 8, var.stages = ring slots)
     int kbox = 0, wbox = 0;  // keys per TMA box of the shared cache / of a window on that path
     int ctas_per_sm;
+    int piece_cost = 0;   // Params::piece_cost of the main kernel in use
     float scale_log2;
     // workspace
     float* part_acc = nullptr;
@@ -231,6 +232,7 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
     int blocks = 0;
     cudaError_t e;
     h->umma = false;
+    h->piece_cost = 0;
     if (config->kernel_path < 0 || config->kernel_path > PLT_PATH_TCGEN05)
         return fail(nullptr, PLT_ERR_INVALID_ARG, "kernel_path %d outside [0, 2]", config->kernel_path);
     if (config->loads_in_flight < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "loads_in_flight %d < 0", config->loads_in_flight);
@@ -263,6 +265,13 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the bf16 main kernel", e);
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "bf16 main kernel does not fit an SM");
         h->ctas_per_sm = blocks < cps ? blocks : cps;
+        // Starting and finishing an item (plan step, query rows, first load latency, partial store) stalls a block for
+        // about as long as streaming 192 KB takes it (measured on B200 on a batch of short sequences: 4-5 us);
+        // the plan charges every item that much, in tiles, so that blocks with many short items get fewer tiles.
+        const size_t stage_bytes = main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 3, 1) -
+                                   main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 2, 1);
+        h->piece_cost = (int)((192 * 1024) / (stage_bytes * (size_t)h->ctas_per_sm));
+        if (h->piece_cost < 1) h->piece_cost = 1;
     } else {
         h->var = MainVariant{config->d, 0, 0, 1, 1, 1, kF32TileKeys, 0, 0, main_f32_smem(config->d, g.R, config->max_batch)};
         e = main_f32_prepare(config->d, g.R, config->max_batch, &blocks);
@@ -426,6 +435,7 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     p.num_pool_pages = a->num_pool_pages;
     p.hpc = h->var.HPC;
     p.tile_keys = h->var.tile_keys;
+    p.piece_cost = h->piece_cost;
     p.num_ctas = h->var.grid;
     p.scale_log2 = h->scale_log2;
     for (int l = 0; l < kMaxLoops; ++l) p.delta[l] = h->delta[l];

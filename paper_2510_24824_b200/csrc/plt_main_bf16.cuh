@@ -46,7 +46,7 @@ struct TCfg {
     static constexpr int kMaxStages = 12;
     __host__ __device__ static constexpr size_t smem_bytes(int stages, int max_batch) {
         return 1024 /* alignment slack */ + (size_t)stages * STAGE_BYTES + 2 * kMaxStages * 8 +
-               (size_t)(MERGE_ACC_FLOATS + MERGE_ML_FLOATS) * 4 + (size_t)(max_batch + 4) * 4;
+               (size_t)(MERGE_ACC_FLOATS + MERGE_ML_FLOATS) * 4 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
 
@@ -205,7 +205,8 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
     float* merge_acc = (float*)(empty_bar + C::kMaxStages);
     float* merge_ml = merge_acc + C::MERGE_ACC_FLOATS;
     int32_t* s_ctl = (int32_t*)(merge_ml + C::MERGE_ML_FLOATS);  // [0] abort flag, [1] tiles issued
-    int32_t* s_prefix = s_ctl + 2;
+    int32_t* s_prefix = s_ctl + 2;                      // [B + 1] tile prefix
+    int32_t* s_lens = s_prefix + p.B + 2;               // [B] clamped lengths, so that walking the pieces reads no global memory
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
@@ -221,7 +222,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         mbar_fence_init();
     }
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
-    build_prefix(p, s_prefix, flags);  // contains __syncthreads
+    build_prefix(p, s_prefix, flags, s_lens);  // contains __syncthreads
     const int64_t T = s_prefix[p.B];
     const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
     if (cta == 0)
@@ -241,7 +242,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t it = 0;
             int stage = 0;
             uint32_t use = 0;  // how many times `stage` has been filled before
-            PieceWalk walk(p, s_prefix, lo, hi);
+            PieceWalk walk(p, s_prefix, lo, hi, s_lens);
             Piece pc;
             while (walk.next(pc, flags)) {
                 const int head0 = pc.hg * HPC;
@@ -336,7 +337,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         uint32_t use = 0;
         int q_b = -1, q_hg = -1;   // (sequence, head group) whose query rows are in qb
         uint32_t qb[D / 16][NT][2];
-        PieceWalk walk(p, s_prefix, lo, hi);
+        PieceWalk walk(p, s_prefix, lo, hi, s_lens);
         Piece pc;
         while (walk.next(pc, flags)) {
             const int kvh = pc.hg * HPC + h_local;
