@@ -4,6 +4,7 @@ import pytest
 import torch
 
 import oracle
+from paper_2510_24824_b200 import binding as B
 from paper_2510_24824_b200.inputs import make_problem, shrunk_workload, workload
 from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
 
@@ -33,8 +34,9 @@ def test_tiny_fp32_config_exact_shape():
 
 
 # ---- every launch variant must give the same answer (split invariance) --------------------------------------
-@pytest.mark.parametrize("hpc,kw", [(1, 1), (1, 2), (1, 4), (2, 1), (2, 2), (2, 4), (4, 1), (4, 2), (8, 1)])
-def test_bf16_variants_one_row_tile(hpc, kw):
+# heads_per_cta x key_slices (warps along the keys) x slices_per_warp x row_warps; R = packed rows per KV head.
+@pytest.mark.parametrize("hpc,kw", [(1, 1), (1, 2), (1, 4), (2, 1), (2, 2), (2, 4), (4, 1), (4, 2), (8, 1), (1, 8)])
+def test_bf16_variants_12_rows(hpc, kw):
     p = make_problem(custom(B=4, L=3, Hq=32, Hkv=8, w=70, lens=("list", [513, 64, 2, 1000])))
     ref = oracle.decode_attn(p)
     for cps, stages in ((1, 2), (2, 0)):
@@ -42,16 +44,37 @@ def test_bf16_variants_one_row_tile(hpc, kw):
                       f"hpc={hpc} kw={kw} cps={cps}")
 
 
-@pytest.mark.parametrize("hpc,kw", [(1, 1), (1, 2), (1, 4), (2, 1), (2, 2), (4, 1)])
-def test_bf16_variants_two_row_tiles(hpc, kw):
-    p = make_problem(custom(B=3, L=3, Hq=32, Hkv=4, w=50, lens=("list", [700, 65, 3])))  # 24 packed rows
-    assert_parity(run_gpu(p, heads_per_cta=hpc, key_slices=kw), oracle.decode_attn(p), "bf16", f"hpc={hpc} kw={kw}")
+@pytest.mark.parametrize("hpc,kw,ks,rw", [(1, 1, 1, 1), (1, 2, 1, 1), (1, 4, 1, 1), (2, 1, 1, 1), (2, 2, 1, 1), (4, 1, 1, 1),
+                                          (1, 1, 2, 1), (2, 2, 2, 1), (4, 1, 2, 1), (1, 1, 1, 2), (2, 2, 1, 2), (2, 1, 2, 2),
+                                          (1, 4, 2, 2)])
+def test_bf16_variants_24_rows(hpc, kw, ks, rw):
+    """24 packed rows: one warp with three 8-row groups, or two warps with two groups each (the second half empty)."""
+    p = make_problem(custom(B=3, L=3, Hq=32, Hkv=4, w=50, lens=("list", [700, 65, 3])))
+    got = run_gpu(p, heads_per_cta=hpc, key_slices=kw, slices_per_warp=ks, row_warps=rw)
+    assert_parity(got, oracle.decode_attn(p), "bf16", f"hpc={hpc} kw={kw} ks={ks} rw={rw}")
 
 
-@pytest.mark.parametrize("hpc,kw", [(1, 1), (1, 2), (2, 1)])
-def test_bf16_variants_four_row_tiles(hpc, kw):
-    p = make_problem(custom(B=2, L=4, Hq=32, Hkv=2, w=33, lens=("list", [400, 5])))  # 64 packed rows
-    assert_parity(run_gpu(p, heads_per_cta=hpc, key_slices=kw), oracle.decode_attn(p), "bf16", f"hpc={hpc} kw={kw}")
+@pytest.mark.parametrize("hpc,kw,ks,rw", [(1, 1, 1, 1), (2, 2, 1, 1), (1, 2, 2, 1), (2, 1, 2, 2), (1, 2, 1, 2), (4, 1, 1, 2)])
+def test_bf16_variants_32_rows(hpc, kw, ks, rw):
+    """32 packed rows: four 8-row groups in one warp, or two in each of two warps (the automatic choice)."""
+    p = make_problem(custom(B=3, L=4, Hq=32, Hkv=4, w=90, lens=("list", [900, 130, 2])))
+    got = run_gpu(p, heads_per_cta=hpc, key_slices=kw, slices_per_warp=ks, row_warps=rw)
+    assert_parity(got, oracle.decode_attn(p), "bf16", f"hpc={hpc} kw={kw} ks={ks} rw={rw}")
+
+
+@pytest.mark.parametrize("hpc,kw,ks", [(1, 1, 1), (1, 2, 1), (2, 1, 1), (1, 1, 2), (2, 2, 1)])
+def test_bf16_variants_64_rows(hpc, kw, ks):
+    p = make_problem(custom(B=2, L=4, Hq=32, Hkv=2, w=33, lens=("list", [400, 5])))  # two warps of 32 rows
+    got = run_gpu(p, heads_per_cta=hpc, key_slices=kw, slices_per_warp=ks)
+    assert_parity(got, oracle.decode_attn(p), "bf16", f"hpc={hpc} kw={kw} ks={ks}")
+
+
+def test_variant_arguments_are_checked():
+    p = make_problem(custom(B=2, L=4, Hq=32, Hkv=2, w=33, lens=("list", [400, 5])))   # 64 packed rows
+    for bad in (dict(row_warps=3), dict(slices_per_warp=3), dict(row_warps=1, heads_per_cta=1),   # 64 rows need 2 warps
+                dict(heads_per_cta=3), dict(heads_per_cta=1, key_slices=3)):
+        with pytest.raises(B.PltError):
+            DecodeAttn(p, **bad)
 
 
 @pytest.mark.parametrize("d", [64, 128])
