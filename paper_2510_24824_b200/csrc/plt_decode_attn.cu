@@ -218,11 +218,12 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 // Automatic choice: the tcgen05 kernel where the packed rows exceed 32 (there the warp-level products, not HBM,
 // bound the other kernel: measured 14-19 % faster at 48 and 64 rows on long sequences); the warp-level kernel
 // elsewhere (it is the faster one up to 32 rows, and by far on batches of short sequences). An explicit
-// heads_per_cta / key_slices / ctas_per_sm asks for the warp-level kernel's variants.
+// heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
     if (c->kernel_path == PLT_PATH_WARP_MMA) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
-    if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0) return false;
+    if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
+        return false;
     return umma_eligible(c) && c->L * (c->Hq / c->Hkv) > 32 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
