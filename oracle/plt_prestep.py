@@ -1,0 +1,73 @@
+"""fp64 / byte-exact CPU oracle of the step that precedes the CLP decode attention (test infrastructure only).
+
+One decode step runs L loops side by side (Algorithm 1: first loop on token i, second loop on token i-1, ...).
+Before the attention of Algorithm 3 lines 2-3 can run, the K and V that line 1 (f_qkv) produced for this step have
+to be where the attention reads them, and line 4 needs the gate logits:
+
+  * the first loop's K, V row is appended to the shared cache (Algorithm 1 line 7 returns the updated cache);
+  * every later loop keeps "the most recent w KV entries" (Sec. 2.2.2): its row replaces the oldest entry of its
+    window, i.e. goes to slot (index of its token in its own stream) mod w;
+  * f_gate is head-wise with one scalar per head (Sec. 2.2.2): logit[h] = <w_gate[h], Q[h]> + b_gate[h].
+
+With the convention of the attention oracle (seq_lens counts the current token, loop l sees
+cut_l = max(0, N - delta_l) keys) the token loop l handles in this step has index cut_l - 1 in its stream.
+Plain numpy and Python loops, copies of the inputs, nothing shared with the CUDA path.
+"""
+from __future__ import annotations
+
+from dataclasses import replace
+
+import numpy as np
+
+
+def _to_f64(a: np.ndarray) -> np.ndarray:
+    """Stored values (float32, or bfloat16 bit patterns in uint16) as float64."""
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+def gate_logits(q: np.ndarray, w_gate: np.ndarray, b_gate: np.ndarray) -> np.ndarray:
+    """[B, L-1, Hq] float64: the head-wise gate linear of Algorithm 3 line 4 (before the sigmoid) for loops 2..L."""
+    qf = _to_f64(q)                                    # [B, L, Hq, d]
+    B, L, Hq, d = qf.shape
+    out = np.zeros((B, max(L - 1, 0), Hq), dtype=np.float64)
+    for b in range(B):
+        for l in range(1, L):
+            for h in range(Hq):
+                acc = 0.0
+                for j in range(d):
+                    acc += float(w_gate[h, j]) * qf[b, l, h, j]
+                out[b, l - 1, h] = acc + float(b_gate[h])
+    return out
+
+
+def prestep(p, k_new: np.ndarray, v_new: np.ndarray, w_gate: np.ndarray, b_gate: np.ndarray):
+    """Returns (problem after the step's cache updates with the new gate logits stored as float32, logits in float64).
+
+    p: the synthetic-input container with the caches as they were BEFORE this step and seq_lens already counting the
+    current token. k_new, v_new: [B, L, Hkv, d] in the storage type of the caches (row l = what loop l+1 produced).
+    """
+    kc, vc = p.k_cache.copy(), p.v_cache.copy()
+    kw, vw = p.k_win.copy(), p.v_win.copy()
+    cuts = p.cuts()                                    # [B, L]
+    for b in range(p.B):
+        c0 = int(cuts[b, 0])
+        if c0 > 0:                                     # first loop: append at position c0 - 1 of the shared cache
+            pos = c0 - 1
+            if p.page_size:
+                page = int(p.page_table[b, pos // p.page_size])
+                kc[page, pos % p.page_size] = k_new[b, 0]
+                vc[page, pos % p.page_size] = v_new[b, 0]
+            else:
+                kc[b, pos] = k_new[b, 0]
+                vc[b, pos] = v_new[b, 0]
+        for l in range(1, p.L):                        # later loops: overwrite the oldest window entry
+            c = int(cuts[b, l])
+            if c > 0:
+                slot = (c - 1) % p.w
+                kw[b, l - 1, slot] = k_new[b, l]
+                vw[b, l - 1, slot] = v_new[b, l]
+    g = gate_logits(p.q, w_gate, b_gate)
+    g32 = g.astype(np.float32) if p.L > 1 else p.gate_logits
+    return replace(p, k_cache=kc, v_cache=vc, k_win=kw, v_win=vw, gate_logits=g32), g
