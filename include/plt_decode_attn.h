@@ -151,6 +151,35 @@ plt_status plt_decode_attn_run(plt_decode_attn_t handle, const plt_decode_attn_a
  */
 plt_status plt_decode_attn_run_host(plt_decode_attn_t handle, const plt_decode_attn_args* host_args, void* cuda_stream);
 
+/*
+ * What one decode step hands to plt_decode_attn_step besides plt_decode_attn_args: the K and V rows that line 1 of
+ * Algorithm 3 (f_qkv) produced for this step, and the head-wise gate linear f_gate of line 4 (Sec. 2.2.2: one
+ * scalar per head).  All pointers are device memory; k_new / v_new 16-byte aligned.
+ */
+typedef struct {
+    uint32_t struct_size;
+    const void* k_new;        /* [B, L, Hkv, d], dtype of the caches: row l-1 = keys of the token loop l handles now */
+    const void* v_new;        /* [B, L, Hkv, d] */
+    const float* w_gate;      /* [Hq, d] fp32 (ignored when L == 1) */
+    const float* b_gate;      /* [Hq] fp32 */
+    float* gate_logits;       /* [B, L-1, Hq] fp32, written by the call and then used by the attention */
+} plt_decode_attn_step_args;
+
+/*
+ * One whole decode step of the path: the pre-step and then the attention of plt_decode_attn_run, three launches.
+ * Pre-step (one kernel), with cut(b,l) = max(0, N_b - delta_l) and N_b counting the current token:
+ *   - loop 1: k_new/v_new[b, 0] are stored at position cut(b,1) - 1 of the shared cache (Algorithm 1 line 7: the
+ *     step returns the updated cache);
+ *   - loops 2..L: k_new/v_new[b, l-1] are stored in slot (cut(b,l) - 1) mod w of that loop's window, so that the window
+ *     holds the most recent w entries (Sec. 2.2.2); nothing is written where cut(b,l) = 0;
+ *   - step->gate_logits[b, l-2, h] = sum_j w_gate[h, j] * q[b, l-1, h, j] + b_gate[h]  (fp32 accumulation).
+ * This call therefore WRITES through args->k_cache, v_cache, k_win and v_win although the struct declares them
+ * const; args->gate_logits is ignored and args->win_lens must be NULL (the window length is min(w, cut)).  Errors and
+ * stream semantics as plt_decode_attn_run; out-of-range page ids are clamped and flagged in the status word.
+ */
+plt_status plt_decode_attn_step(plt_decode_attn_t handle, const plt_decode_attn_args* args,
+                                const plt_decode_attn_step_args* step, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, reads the device status word and clears it.
  * PLT_OK if it was 0; else PLT_ERR_DEVICE_CHECK with *out_bits (optional) = PLT_DEV_* bits. */
 plt_status plt_decode_attn_check(plt_decode_attn_t handle, void* cuda_stream, uint32_t* out_bits);

@@ -23,6 +23,7 @@ EXPORTS = (
     "plt_decode_attn_create", "plt_decode_attn_run", "plt_decode_attn_run_host", "plt_decode_attn_check",
     "plt_decode_attn_destroy", "plt_decode_attn_last_error", "plt_decode_attn_workspace_bytes",
     "plt_decode_attn_launch_info", "plt_decode_attn_set_profile_events", "plt_decode_attn_run_no_alloc",
+    "plt_decode_attn_step",
 )
 PLT_NO_ALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -58,6 +59,13 @@ class Args(ctypes.Structure):
     ]
 
 
+class StepArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
+        ("w_gate", ctypes.c_void_p), ("b_gate", ctypes.c_void_p), ("gate_logits", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -72,6 +80,7 @@ def load_library() -> ctypes.CDLL:
         lib.plt_decode_attn_create.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(h)]
         lib.plt_decode_attn_run.argtypes = [h, ctypes.POINTER(Args), ctypes.c_void_p]
         lib.plt_decode_attn_run_host.argtypes = [h, ctypes.POINTER(Args), ctypes.c_void_p]
+        lib.plt_decode_attn_step.argtypes = [h, ctypes.POINTER(Args), ctypes.POINTER(StepArgs), ctypes.c_void_p]
         lib.plt_decode_attn_check.argtypes = [h, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
         lib.plt_decode_attn_destroy.argtypes = [h]
         lib.plt_decode_attn_last_error.argtypes = [h]
@@ -163,6 +172,20 @@ def make_args(batch: int, q, k_cache, v_cache, seq_lens, out, k_win=None, v_win=
 
 def plt_decode_attn_run(handle, args: Args, stream: int = 0) -> None:
     st = load_library().plt_decode_attn_run(handle, ctypes.byref(args), ctypes.c_void_p(stream))
+    if st != PLT_OK:
+        _raise(st, handle)
+
+
+def make_step_args(k_new, v_new, w_gate=None, b_gate=None, gate_logits=None) -> StepArgs:
+    s = StepArgs()
+    s.struct_size = ctypes.sizeof(StepArgs)
+    s.k_new, s.v_new = _ptr(k_new), _ptr(v_new)
+    s.w_gate, s.b_gate, s.gate_logits = _ptr(w_gate), _ptr(b_gate), _ptr(gate_logits)
+    return s
+
+
+def plt_decode_attn_step(handle, args: Args, step: StepArgs, stream: int = 0) -> None:
+    st = load_library().plt_decode_attn_step(handle, ctypes.byref(args), ctypes.byref(step), ctypes.c_void_p(stream))
     if st != PLT_OK:
         _raise(st, handle)
 

@@ -384,7 +384,38 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     return PLT_OK;
 }
 
+namespace {
+plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream,
+                    const plt_decode_attn_step_args* step);
+}
+
 PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream) {
+    return run_impl(h, a, cuda_stream, nullptr);
+}
+
+PLT_API plt_status plt_decode_attn_step(plt_decode_attn_t h, const plt_decode_attn_args* a,
+                                        const plt_decode_attn_step_args* step, void* cuda_stream) {
+    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if (!a) return fail(h, PLT_ERR_INVALID_ARG, "args is NULL");
+    if (!step) return fail(h, PLT_ERR_INVALID_ARG, "step is NULL");
+    if (step->struct_size != sizeof(plt_decode_attn_step_args))
+        return fail(h, PLT_ERR_INVALID_ARG, "step.struct_size %u != %zu", step->struct_size, sizeof(plt_decode_attn_step_args));
+    if (a->struct_size != sizeof(plt_decode_attn_args))
+        return fail(h, PLT_ERR_INVALID_ARG, "args.struct_size %u != %zu", a->struct_size, sizeof(plt_decode_attn_args));
+    if (!step->k_new || !step->v_new) return fail(h, PLT_ERR_INVALID_ARG, "k_new and v_new must not be NULL");
+    if (!aligned16(step->k_new) || !aligned16(step->v_new))
+        return fail(h, PLT_ERR_INVALID_ARG, "k_new and v_new must be 16-byte aligned");
+    if (h->cfg.L > 1 && (!step->w_gate || !step->b_gate || !step->gate_logits))
+        return fail(h, PLT_ERR_INVALID_ARG, "w_gate, b_gate and gate_logits must not be NULL when L > 1");
+    if (a->win_lens) return fail(h, PLT_ERR_INVALID_ARG, "win_lens must be NULL: the ring update fixes wl = min(w, cut)");
+    plt_decode_attn_args a2 = *a;
+    a2.gate_logits = step->gate_logits;
+    return run_impl(h, &a2, cuda_stream, step);
+}
+
+namespace {
+plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream,
+                    const plt_decode_attn_step_args* step) {
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
     if (!a) return fail(h, PLT_ERR_INVALID_ARG, "args is NULL");
     if (a->struct_size != sizeof(plt_decode_attn_args))
@@ -443,6 +474,10 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     cudaError_t e;
+    if (step) {
+        e = launch_prestep(p, h->bf16, step->k_new, step->v_new, step->w_gate, step->b_gate, step->gate_logits, stream);
+        if (e != cudaSuccess) return cuda_fail(h, "launching the pre-step kernel", e);
+    }
     if (h->bf16) {
         // keys and heads per TMA box: the warp-level kernel loads [heads per block][tile keys], the tcgen05 kernel
         // [1 head][up to 128 keys]
@@ -487,6 +522,7 @@ PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_att
     if (e != cudaSuccess) return cuda_fail(h, "launching the merge kernel", e);
     return PLT_OK;
 }
+}  // namespace
 
 static plt_status stage_in(plt_decode_attn_t h, int idx, const void* host, size_t bytes, cudaStream_t stream,
                            const void** dev) {

@@ -41,6 +41,11 @@ cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm);
 cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                              int wbox, int cap, cudaStream_t stream);
 
+// Pre-step of a decode step: shared-cache append, window ring update, gate linear (writes through p.k_cache,
+// p.v_cache, p.k_win, p.v_win, which the attention kernels only read).
+cudaError_t launch_prestep(const Params& p, bool bf16, const void* k_new, const void* v_new, const float* w_gate,
+                           const float* b_gate, float* gate_out, cudaStream_t stream);
+
 cudaError_t launch_reduce(const Params& p, bool bf16, bool overlap, cudaStream_t stream);
 
 }  // namespace plt

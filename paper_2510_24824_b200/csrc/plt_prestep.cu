@@ -1,0 +1,99 @@
+// Pre-step kernel of a CLP decode step: puts what line 1 of Algorithm 3 (f_qkv) produced for this step where the
+// attention reads it, and evaluates the head-wise gate linear of line 4.
+//   * the first loop's K, V row is appended to the shared cache at position cut_1 - 1 (Algorithm 1 line 7);
+//   * each later loop's row replaces the oldest entry of its window, slot (cut_l - 1) mod w ("the most recent w
+//     KV entries", Sec. 2.2.2);
+//   * gate_logits[b, l, h] = <w_gate[h], Q[b, l, h]> + b_gate[h] for loops 2..L (one scalar per head).
+// One block per (sequence, loop): 16-byte copies of the two rows, then one warp per query head for the dot products.
+// One launch instead of three; the attention kernels follow in the same stream.
+#include <cuda_bf16.h>
+
+#include "plt_common.cuh"
+#include "plt_host.h"
+
+namespace plt {
+
+namespace {
+
+constexpr int kPreThreads = 128;
+
+template <bool BF16>
+__global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_constant__ Params p, const void* k_new,
+                                                                  const void* v_new, const float* w_gate,
+                                                                  const float* b_gate, float* gate_out) {
+    using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+    const int b = blockIdx.x / p.L, l = blockIdx.x % p.L;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    uint32_t flags = 0;
+    const int32_t n = seq_len_clamped(p, b, flags);
+    int cut = n - p.delta[l];
+    cut = cut > 0 ? cut : 0;
+
+    if (cut > 0) {
+        // destination rows of this loop's K and V: [Hkv] rows of d elements, kd elements apart
+        T *kd, *vd;
+        int64_t head_stride;
+        if (l == 0) {
+            const int pos = cut - 1;
+            int64_t base;
+            if (p.page_size > 0) {
+                int page = p.page_table[(int64_t)b * p.max_pages + pos / p.page_size];
+                if (page < 0 || page >= p.num_pool_pages) {
+                    flags |= kDevPageIdClamped;
+                    page = page < 0 ? 0 : p.num_pool_pages - 1;
+                }
+                base = (int64_t)page * p.kv_stride_b + (int64_t)(pos % p.page_size) * p.kv_stride_n;
+            } else {
+                base = (int64_t)b * p.kv_stride_b + (int64_t)pos * p.kv_stride_n;
+            }
+            kd = (T*)p.k_cache + base;
+            vd = (T*)p.v_cache + base;
+            head_stride = p.kv_stride_h;
+        } else {
+            const int slot = (cut - 1) % p.w;
+            const int64_t base = ((((int64_t)b * (p.L - 1) + (l - 1)) * p.w + slot) * p.Hkv) * p.d;
+            kd = (T*)p.k_win + base;
+            vd = (T*)p.v_win + base;
+            head_stride = p.d;
+        }
+        const int64_t src = (((int64_t)b * p.L + l) * p.Hkv) * p.d;
+        const int per_row = p.d * (int)sizeof(T) / 16;   // 16-byte chunks per head row
+        for (int i = tid; i < p.Hkv * per_row; i += kPreThreads) {
+            const int h = i / per_row, c = i - h * per_row;
+            const uint4 kk = *((const uint4*)((const T*)k_new + src + (int64_t)h * p.d) + c);
+            const uint4 vv = *((const uint4*)((const T*)v_new + src + (int64_t)h * p.d) + c);
+            *((uint4*)(kd + h * head_stride) + c) = kk;
+            *((uint4*)(vd + h * head_stride) + c) = vv;
+        }
+    }
+    if (l > 0) {
+        // head-wise gate linear; written for every sequence and loop (the attention ignores it where cut = 0)
+        for (int h = wid; h < p.Hq; h += kPreThreads / 32) {
+            const T* q = (const T*)p.q + (((int64_t)b * p.L + l) * p.Hq + h) * p.d;
+            float acc = 0.f;
+            for (int j = lane; j < p.d; j += 32) {
+                float x;
+                if constexpr (BF16) x = __bfloat162float(q[j]);
+                else x = q[j];
+                acc = fmaf(w_gate[(int64_t)h * p.d + j], x, acc);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) gate_out[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h] = acc + b_gate[h];
+        }
+    }
+    if (flags && tid == 0) atomicOr(p.status, flags);
+}
+
+}  // namespace
+
+cudaError_t launch_prestep(const Params& p, bool bf16, const void* k_new, const void* v_new, const float* w_gate,
+                           const float* b_gate, float* gate_out, cudaStream_t stream) {
+    const unsigned grid = (unsigned)(p.B * p.L);
+    if (grid == 0) return cudaSuccess;
+    if (bf16) plt_decode_prestep<true><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
+    else plt_decode_prestep<false><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
+    return cudaGetLastError();
+}
+
+}  // namespace plt

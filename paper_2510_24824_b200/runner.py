@@ -12,7 +12,8 @@ import torch
 from . import binding as B
 
 
-def _to_torch(a: Optional[np.ndarray], dtype: str, device, pin: bool = False):
+def to_torch(a: Optional[np.ndarray], dtype: str, device, pin: bool = False):
+    """Host array (float32 / int32, or bf16 bit patterns when dtype == 'bf16') as a torch tensor on `device`."""
     if a is None:
         return None
     t = torch.from_numpy(np.ascontiguousarray(a))
@@ -34,7 +35,7 @@ class DeviceProblem:
         for f in self.FIELDS:
             a = getattr(p, f)
             is_data = f in ("q", "k_cache", "v_cache", "k_win", "v_win")
-            setattr(self, f, _to_torch(a, p.dtype if is_data else "", device, pin))
+            setattr(self, f, to_torch(a, p.dtype if is_data else "", device, pin))
         tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
         if device is None:
             self.out = torch.empty((p.B, p.L, p.Hq, p.d), dtype=tdt)
@@ -79,6 +80,15 @@ class DecodeAttn:
             stream = torch.cuda.current_stream().cuda_stream
         B.plt_decode_attn_run(self.handle, dp.args(out), stream)
         return dp.out if out is None else out
+
+    def step(self, dp: DeviceProblem, k_new, v_new, w_gate, b_gate, stream: Optional[int] = None):
+        """Pre-step (cache append, window ring update, gate linear into dp.gate_logits) and attention in one call.
+        k_new, v_new, w_gate, b_gate: device tensors."""
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        st = B.make_step_args(k_new, v_new, w_gate, b_gate, dp.gate_logits if dp.problem.L > 1 else None)
+        B.plt_decode_attn_step(self.handle, dp.args(), st, stream)
+        return dp.out
 
     def run_host(self, hp: DeviceProblem, stream: Optional[int] = None):
         if stream is None:
