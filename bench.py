@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--cps", type=int, default=0)
     ap.add_argument("--loops", type=int, default=0, help="override the workload's number of loops L (for the traffic-vs-L sweep)")
     ap.add_argument("--path", type=int, default=0, help="kernel path: 0 automatic, 1 warp-level mma, 2 tcgen05")
+    ap.add_argument("--prestep", action="store_true",
+                    help="time plt_decode_attn_step: the pre-step kernel (cache append, window ring update, gate linear) "
+                         "ahead of the attention, three launches per step")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
@@ -284,9 +287,28 @@ def main():
         torch.cuda.synchronize()
 
     run_args = dp.args()
+    launches_per_step = int(op.info["kernels_per_run"])
+    if args.prestep:
+        # Synthetic rows of this step: the same K/V rows and gate weights every step (the lengths do not advance, so
+        # the same cache positions are rewritten: a timing stand-in for consecutive decode steps).
+        from paper_2510_24824_b200.runner import to_torch
+        from paper_2510_24824_b200.inputs import f32_to_bf16_bits
+        rng = np.random.default_rng(1000 + rank)
+        rows = [rng.standard_normal((p.B, p.L, p.Hkv, p.d)).astype(np.float32) for _ in range(2)]
+        if p.dtype == "bf16":
+            rows = [f32_to_bf16_bits(x) for x in rows]
+        k_new, v_new = (to_torch(x, p.dtype, dev) for x in rows)
+        w_gate = to_torch((rng.standard_normal((p.Hq, p.d)) / np.sqrt(p.d)).astype(np.float32), "", dev)
+        b_gate = to_torch(rng.standard_normal(p.Hq).astype(np.float32), "", dev)
+        step_args = B.make_step_args(k_new, v_new, w_gate, b_gate, dp.gate_logits if p.L > 1 else None)
+        launches_per_step += 1
+        cfg["prestep"] = "plt_decode_attn_step: pre-step kernel + attention"
 
     def step():
-        B.plt_decode_attn_run(op.handle, run_args, stream)
+        if args.prestep:
+            B.plt_decode_attn_step(op.handle, run_args, step_args, stream)
+        else:
+            B.plt_decode_attn_run(op.handle, run_args, stream)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -356,7 +378,7 @@ def main():
             "hbm_gbs_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9,
             "hbm_frac_of_8tbs": by["total"] / (ms_per_step * 1e-3) / 8e12,
             "clocks": sampler.summary(),
-            "gpu_launches": int(op.info["kernels_per_run"]) * args.steps,
+            "gpu_launches": launches_per_step * args.steps,
             "roofline": {
                 "bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,

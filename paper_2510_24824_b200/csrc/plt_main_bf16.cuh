@@ -221,8 +221,13 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         mbar_fence_init();
     }
-    grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags, s_lens);  // contains __syncthreads
+    // Everything above reads only what the caller passed. If this grid was launched to overlap the pre-step kernel,
+    // the caches, windows and query rows may be read only from here on (a no-op for an ordinary launch).
+    grid_dependency_wait();
+    // The merge kernel may be set up from now on (it reads the gate logits, which the pre-step may have written, before
+    // its own wait, hence not earlier); it waits for this grid to complete before it reads the partials.
+    grid_launch_dependents();
     const int64_t T = s_prefix[p.B];
     const int cta = blockIdx.x, nctas = plan_ctas(T, (int)gridDim.x);
     if (cta == 0)

@@ -42,8 +42,9 @@ cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm) {
     return dispatch(1, v, nullptr, nullptr, nullptr, blocks_per_sm);
 }
 
-cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, cudaStream_t stream) {
-    return dispatch(2, v, maps, &p, stream, nullptr);
+cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, bool after_prestep,
+                             cudaStream_t stream) {
+    return dispatch(after_prestep ? 5 : 2, v, maps, &p, stream, nullptr);
 }
 
 }  // namespace plt

@@ -29,8 +29,19 @@ cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const 
         *out = (int)C::smem_bytes(v.stages, v.grid /* max_batch passed in grid for this query */);
         return cudaSuccess;
     }
-    fn<<<v.grid, C::NTHREADS, v.smem, stream>>>(maps[0], maps[1], maps[2], maps[3], *p, v.stages);
-    return cudaGetLastError();
+    // op 2: plain launch; op 5: launch with programmatic stream serialisation (the kernel before it in the stream is the
+    // pre-step kernel: this grid's blocks are set up while it runs and wait for its results in grid_dependency_wait()).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)v.grid);
+    cfg.blockDim = dim3(C::NTHREADS);
+    cfg.dynamicSmemBytes = v.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = op == 5 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, fn, maps[0], maps[1], maps[2], maps[3], *p, v.stages);
 }
 
 }  // namespace

@@ -10,6 +10,7 @@
 
 #include "plt_common.cuh"
 #include "plt_host.h"
+#include "plt_ptx.cuh"
 
 namespace plt {
 
@@ -22,6 +23,7 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
                                                                   const void* v_new, const float* w_gate,
                                                                   const float* b_gate, float* gate_out) {
     using T = typename std::conditional<BF16, __nv_bfloat16, float>::type;
+    grid_launch_dependents();   // the attention kernel's blocks may be set up meanwhile; they wait for this grid
     const int b = blockIdx.x / p.L, l = blockIdx.x % p.L;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
