@@ -171,7 +171,7 @@ typedef struct {
  *   - loop 1: k_new/v_new[b, 0] are stored at position cut(b,1) - 1 of the shared cache (Algorithm 1 line 7: the
  *     step returns the updated cache);
  *   - loops 2..L: k_new/v_new[b, l-1] are stored in slot (cut(b,l) - 1) mod w of that loop's window, so that the window
- *     holds the most recent w entries (Sec. 2.2.2); nothing is written where cut(b,l) = 0;
+ *     holds the w newest entries of that loop (Sec. 2.2.2); nothing is written where cut(b,l) = 0;
  *   - step->gate_logits[b, l-2, h] = sum_j w_gate[h, j] * q[b, l-1, h, j] + b_gate[h]  (fp32 accumulation).
  * This call therefore WRITES through args->k_cache, v_cache, k_win and v_win although the struct declares them
  * const; args->gate_logits is ignored and args->win_lens must be NULL (the window length is min(w, cut)).  Errors and

@@ -5,9 +5,9 @@ Before the attention of Algorithm 3 lines 2-3 can run, the K and V that line 1 (
 to be where the attention reads them, and line 4 needs the gate logits:
 
   * the first loop's K, V row is appended to the shared cache (Algorithm 1 line 7 returns the updated cache);
-  * every later loop keeps "the most recent w KV entries" (Sec. 2.2.2): its row replaces the oldest entry of its
+  * every later loop keeps only its w newest K/V entries (Sec. 2.2.2): its row replaces the oldest entry of its
     window, i.e. goes to slot (index of its token in its own stream) mod w;
-  * f_gate is head-wise with one scalar per head (Sec. 2.2.2): logit[h] = <w_gate[h], Q[h]> + b_gate[h].
+  * f_gate maps each head's query to a single number for that head (Sec. 2.2.2): logit[h] = <w_gate[h], Q[h]> + b_gate[h].
 
 With the convention of the attention oracle (seq_lens counts the current token, loop l sees
 cut_l = max(0, N - delta_l) keys) the token loop l handles in this step has index cut_l - 1 in its stream.

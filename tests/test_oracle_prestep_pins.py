@@ -2,7 +2,7 @@
 
 The decisive pin replays a whole decode of a tiny model-free stream: T steps of pre-step + attention must equal,
 at every step, attention computed directly from the lists of everything each loop has produced so far
-("all first-loop K/V" and "the most recent w K/V of this loop", Sec. 2.2.2), with no cache and no ring at all.
+(all first-loop K/V rows, and the w newest K/V rows of the loop itself, Sec. 2.2.2), with no cache and no ring at all.
 """
 import math
 
@@ -72,7 +72,7 @@ def test_replayed_decode_equals_attention_over_plain_token_lists(dtype, page_siz
                     if l == 0:
                         want = yg
                     else:
-                        Kl = np.array([r[kv] for r in hist_k[b][l][-w:]])   # the most recent w rows of this loop
+                        Kl = np.array([r[kv] for r in hist_k[b][l][-w:]])   # the w newest rows of this loop
                         Vl = np.array([r[kv] for r in hist_v[b][l][-w:]])
                         yl = softmax_attend(qv, Kl, Vl, p.scale())
                         x = float(np.float32(float(np.dot(w_gate[h], qv)) + b_gate[h]))
