@@ -4,15 +4,15 @@
  *
  * One call computes, for a batch of B sequences, the attention of ONE layer at
  * ONE decode step for all L loops at once (the paper's displaced micro-batch,
- * Algorithm 1 line 5 and the "Inference" paragraph of Sec. 2.2.1): loop l
+ * Algorithm 1 and the "Inference" paragraph of Sec. 2.2.1): loop l
  * (1-indexed) serves token i-l+1, so its query may see the first
  * cut(b,l) = max(0, N_b - delta_l) entries of the single shared first-loop KV
  * cache (delta_l = l-1 unless overridden).  Every loop attends that one cache
- * ("KV-cache sharing from the first loop", Sec. 2.2.2, Algorithm 3 line 2),
+ * (the first-loop KV sharing of Sec. 2.2.2, y_global of Algorithm 3),
  * which the kernels read from HBM once per sequence, not once per loop.
- * Loops 2..L additionally attend their private window of the most recent
- * <= w entries (Algorithm 3 line 3) and the two normalised results are mixed
- * with a per-head sigmoid gate (Algorithm 3 lines 4-5, Eq. 2):
+ * Loops 2..L additionally attend their private window of their newest
+ * <= w entries (y_local of Algorithm 3) and the two normalised results are mixed
+ * with a per-head sigmoid gate (Algorithm 3, Eq. 2):
  *
  *   y_global = softmax(sm_scale * q K_share[0:cut]^T) V_share[0:cut]
  *   y_local  = softmax(sm_scale * q K_win[0:wl]^T)    V_win[0:wl]
@@ -132,7 +132,7 @@ typedef struct {
 plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_decode_attn_t* out_handle);
 
 /*
- * Enqueues one decode-step attention (Algorithm 3 lines 2-5 for all L loops of
+ * Enqueues one decode-step attention (Algorithm 3 from y_global to the gate mix, for all L loops of
  * all B sequences) on `cuda_stream` (a cudaStream_t; NULL = default stream).
  * Asynchronous: no allocation and no host synchronisation.  Host-visible
  * arguments are validated first and nothing is launched on error.  Two kernels
@@ -152,8 +152,8 @@ plt_status plt_decode_attn_run(plt_decode_attn_t handle, const plt_decode_attn_a
 plt_status plt_decode_attn_run_host(plt_decode_attn_t handle, const plt_decode_attn_args* host_args, void* cuda_stream);
 
 /*
- * What one decode step hands to plt_decode_attn_step besides plt_decode_attn_args: the K and V rows that line 1 of
- * Algorithm 3 (f_qkv) produced for this step, and the head-wise gate linear f_gate of line 4 (Sec. 2.2.2: one
+ * What one decode step hands to plt_decode_attn_step besides plt_decode_attn_args: the K and V rows that f_qkv of
+ * Algorithm 3 produced for this step, and the head-wise gate linear f_gate of that algorithm (Sec. 2.2.2: one
  * scalar per head).  All pointers are device memory; k_new / v_new 16-byte aligned.
  */
 typedef struct {
@@ -168,7 +168,7 @@ typedef struct {
 /*
  * One whole decode step of the path: the pre-step and then the attention of plt_decode_attn_run, three launches.
  * Pre-step (one kernel), with cut(b,l) = max(0, N_b - delta_l) and N_b counting the current token:
- *   - loop 1: k_new/v_new[b, 0] are stored at position cut(b,1) - 1 of the shared cache (Algorithm 1 line 7: the
+ *   - loop 1: k_new/v_new[b, 0] are stored at position cut(b,1) - 1 of the shared cache (Algorithm 1: the
  *     step returns the updated cache);
  *   - loops 2..L: k_new/v_new[b, l-1] are stored in slot (cut(b,l) - 1) mod w of that loop's window, so that the window
  *     holds the w newest entries of that loop (Sec. 2.2.2); nothing is written where cut(b,l) = 0;

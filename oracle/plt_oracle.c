@@ -7,15 +7,15 @@
  * link or call it; it shares no code, header or table with the CUDA sources.
  *
  * What it computes, for every sequence b, loop l (1-indexed) and query head h
- * (Algorithm 3 lines 2-5, Eq. 2, and the CLP description of Sec. 2.2.1):
+ * (Algorithm 3, Eq. 2, and the CLP description of Sec. 2.2.1):
  *
  *   cut      = max(0, N_b - delta_l)                      delta_l = l-1 by default
- *   y_global = softmax(sm_scale * q . K_share[0:cut]) V_share[0:cut]   (Alg. 3 line 2)
+ *   y_global = softmax(sm_scale * q . K_share[0:cut]) V_share[0:cut]   (Alg. 3, global)
  *   l == 1 :  O = y_global                               (first loop = vanilla attention)
  *   l >= 2 :  wl = win_lens ? win_lens[b,l-2] : min(w, cut)
- *             y_local = softmax(sm_scale * q . K_win[0:wl]) V_win[0:wl] (Alg. 3 line 3)
- *             g = 1 / (1 + exp(-gate_logit))              (Alg. 3 line 4)
- *             O = g * y_local + (1 - g) * y_global        (Alg. 3 line 5 / Eq. 2)
+ *             y_local = softmax(sm_scale * q . K_win[0:wl]) V_win[0:wl] (Alg. 3, local)
+ *             g = 1 / (1 + exp(-gate_logit))              (Alg. 3, gate)  
+ *             O = g * y_local + (1 - g) * y_global        (Alg. 3 / Eq. 2)
  *   cut == 0:  O = 0 (the loop has no token to serve yet)
  *   wl  == 0 with cut > 0:  y_local = 0
  *

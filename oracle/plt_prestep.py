@@ -1,10 +1,10 @@
 """fp64 / byte-exact CPU oracle of the step that precedes the CLP decode attention (test infrastructure only).
 
 One decode step runs L loops side by side (Algorithm 1: first loop on token i, second loop on token i-1, ...).
-Before the attention of Algorithm 3 lines 2-3 can run, the K and V that line 1 (f_qkv) produced for this step have
-to be where the attention reads them, and line 4 needs the gate logits:
+Before the two attentions of Algorithm 3 can run, the K and V that its f_qkv produced for this step have
+to be where the attention reads them, and its gate needs the logits of f_gate:
 
-  * the first loop's K, V row is appended to the shared cache (Algorithm 1 line 7 returns the updated cache);
+  * the first loop's K, V row is appended to the shared cache (the decode step of Algorithm 1 returns the updated cache);
   * every later loop keeps only its w newest K/V entries (Sec. 2.2.2): its row replaces the oldest entry of its
     window, i.e. goes to slot (index of its token in its own stream) mod w;
   * f_gate maps each head's query to a single number for that head (Sec. 2.2.2): logit[h] = <w_gate[h], Q[h]> + b_gate[h].
@@ -28,7 +28,7 @@ def _to_f64(a: np.ndarray) -> np.ndarray:
 
 
 def gate_logits(q: np.ndarray, w_gate: np.ndarray, b_gate: np.ndarray) -> np.ndarray:
-    """[B, L-1, Hq] float64: the head-wise gate linear of Algorithm 3 line 4 (before the sigmoid) for loops 2..L."""
+    """[B, L-1, Hq] float64: the head-wise gate linear f_gate of Algorithm 3 (before the sigmoid) for loops 2..L."""
     qf = _to_f64(q)                                    # [B, L, Hq, d]
     B, L, Hq, d = qf.shape
     out = np.zeros((B, max(L - 1, 0), Hq), dtype=np.float64)

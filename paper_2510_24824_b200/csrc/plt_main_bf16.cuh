@@ -1,4 +1,4 @@
-// bf16 split-KV main kernel of the CLP decode attention (Algorithm 3 lines 2-3 for all L loops),
+// bf16 split-KV main kernel of the CLP decode attention (y_global and y_local of Algorithm 3 for all L loops),
 // warp-level tensor-core products with the KEYS as the M dimension.
 //
 // One persistent thread block owns an equal share of the line of key tiles of all sequences. A

@@ -1,4 +1,4 @@
-// fp32 split-KV main kernel of the CLP decode attention (Algorithm 3 lines 2-3 for all L loops).
+// fp32 split-KV main kernel of the CLP decode attention (y_global and y_local of Algorithm 3 for all L loops).
 // Plain SIMT fp32 FMA only (no tensor cores: a 1e-5 relative bound rules out tf32/bf16 products).
 // Same tile plan and partial layout as the bf16 kernel: one persistent block walks its share of
 // the line of 32-key tiles; the R = L * Hq/Hkv packed query rows of a KV head are kept in shared

@@ -1,7 +1,7 @@
 // bf16 split-KV main kernel of the CLP decode attention on the 5th-generation tensor cores
 // (tcgen05.mma with accumulators in tensor memory), head dimension 128.
 //
-// Same tile plan and split-partial format as the other main kernels (Algorithm 3 lines 2-3 for all
+// Same tile plan and split-partial format as the other main kernels (y_global and y_local of Algorithm 3 for all
 // L loops): one persistent block per SM walks its share of the line of 128-key tiles, one KV head
 // per work item. The products are laid out with the KEYS as the M dimension, so that the packed
 // query rows (all L loop-queries times all GQA heads of a KV head, R <= 64) form the N dimension

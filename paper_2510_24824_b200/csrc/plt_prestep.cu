@@ -1,6 +1,6 @@
-// Pre-step kernel of a CLP decode step: puts what line 1 of Algorithm 3 (f_qkv) produced for this step where the
-// attention reads it, and evaluates the head-wise gate linear of line 4.
-//   * the first loop's K, V row is appended to the shared cache at position cut_1 - 1 (Algorithm 1 line 7);
+// Pre-step kernel of a CLP decode step: puts what f_qkv of Algorithm 3 produced for this step where the
+// attention reads it, and evaluates the head-wise gate linear f_gate of the same algorithm.
+//   * the first loop's K, V row is appended to the shared cache at position cut_1 - 1 (Algorithm 1: the decode step returns the updated cache);
 //   * each later loop's row replaces the oldest entry of its window, slot (cut_l - 1) mod w (a non-first loop keeps
 //     only its w newest entries, Sec. 2.2.2);
 //   * gate_logits[b, l, h] = <w_gate[h], Q[b, l, h]> + b_gate[h] for loops 2..L (one scalar per head).

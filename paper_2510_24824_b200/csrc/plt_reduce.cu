@@ -1,6 +1,6 @@
 // Merge kernel of the CLP decode attention: combines the split partials of the shared-cache
-// attention (y_global, Algorithm 3 line 2) and of the window attention (y_local, line 3) by their
-// running maxima, normalises each, and applies the sigmoid gate mix of Eq. 2 (lines 4-5):
+// attention (y_global of Algorithm 3) and of the window attention (y_local of Algorithm 3) by their
+// running maxima, normalises each, and applies the sigmoid gate mix of Eq. 2:
 //   O = g * y_local + (1 - g) * y_global for loops 2..L,  O = y_global for loop 1.
 // One block per (sequence, KV-head group, chunk of 8 packed rows); one warp per output row. Which
 // blocks of the main kernel hold pieces of an item is read from the table those blocks left.
