@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--prestep", action="store_true",
                     help="time plt_decode_attn_step: the pre-step kernel (cache append, window ring update, gate linear) "
                          "ahead of the attention, three launches per step")
+    ap.add_argument("--ablation", action="store_true",
+                    help="also time the same queries as L sequential single-loop calls, each scanning the shared cache "
+                         "again (the vanilla loop order of Table 1), and report the ratio")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
@@ -344,6 +347,41 @@ def main():
     main_ms = [a.elapsed_time(b) for a, b in raw]
     main_avg_ms = float(np.mean(main_ms))
 
+    # ---- ablation: the L loops one after the other, every loop scanning the shared cache again ---------------
+    ablation = None
+    if args.ablation and p.L > 1:
+        from paper_2510_24824_b200.runner import to_torch
+        p1 = p.with_(L=1, w=0, q=np.ascontiguousarray(p.q[:, :1]), loop_offset=None, win_lens=None)
+        op1 = DecodeAttn(p1, device_index=local_rank, kernel_path=args.path)
+        calls = []
+        for l in range(p.L):
+            ql = to_torch(np.ascontiguousarray(p.q[:, l:l + 1]), p.dtype, dev)
+            nl = to_torch(np.maximum(p.seq_lens - int(p.offsets()[l]), 0).astype(np.int32), "", dev)
+            ol = torch.empty_like(ql)
+            calls.append((ql, nl, ol, B.make_args(p.B, ql, dp.k_cache, dp.v_cache, nl, ol, page_table=dp.page_table,
+                                                  max_pages=p.max_pages, num_pool_pages=p.num_pool_pages)))
+
+        def seq_step():
+            for c in calls:
+                B.plt_decode_attn_run(op1.handle, c[3], stream)
+
+        for _ in range(5):
+            seq_step()
+        torch.cuda.synchronize()
+        n_abl = min(args.steps, 300)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(n_abl):
+            seq_step()
+        a1.record()
+        torch.cuda.synchronize()
+        seq_ms = a0.elapsed_time(a1) / n_abl
+        assert op1.check(stream) == 0
+        op1.close()
+        ablation = {"sequential_single_loop_calls_ms": seq_ms, "calls_per_step": p.L, "steps_timed": n_abl,
+                    "note": "global attention only (no window, no gate): a lower bound of the sequential loop order; "
+                            "ratio = this / ms_per_step of the cross-loop-parallel step"}
+
     # ---- end to end: host buffers through plt_decode_attn_run_host ------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -388,6 +426,9 @@ def main():
         }
         if e2e is not None:
             line["e2e"] = e2e
+        if ablation is not None:
+            ablation["ratio"] = ablation["sequential_single_loop_calls_ms"] / ms_per_step
+            line["ablation"] = ablation
         if not args.no_cpu:
             v, info = time_oracle(p, args.cpu_seconds)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, **info}
