@@ -55,7 +55,8 @@ typedef enum { PLT_F32 = 0, PLT_BF16 = 1 } plt_dtype;
 
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
 typedef enum {
-    PLT_PATH_AUTO = 0,      /* the library chooses: tcgen05 above 32 packed rows (L * Hq / Hkv) where it applies */
+    PLT_PATH_AUTO = 0,      /* the library chooses: tcgen05 above 48 packed rows (L * Hq / Hkv) when max_seq_len >= 16384
+                               and it applies, else the warp-level kernel */
     PLT_PATH_WARP_MMA = 1,  /* warp-level tensor-core products (mma.sync); fp32 inputs always use SIMT fp32 */
     PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16, d = 128, pages that divide
                                or are a multiple of 128 tokens; anything else is refused with PLT_ERR_UNSUPPORTED */

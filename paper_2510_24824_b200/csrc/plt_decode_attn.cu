@@ -134,7 +134,7 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
     const bool small = nt <= 2;
     int hpc = c->heads_per_cta, kw = c->key_slices;
     int ks = c->slices_per_warp;
-    if (ks == 0) ks = (rw == 2 && nt <= 2) ? 2 : 1;
+    if (ks == 0) ks = rw == 2 ? 2 : 1;   // two warps per head: 32 keys each per tile (measured 25-35 % faster at 48 and 64 rows)
     if (ks != 1 && ks != 2) return fail(nullptr, PLT_ERR_INVALID_ARG, "slices_per_warp %d (supported: 1 or 2)", ks);
     if (hpc == 0) {
         hpc = 1;
@@ -215,16 +215,18 @@ bool umma_eligible(const plt_decode_attn_config* c) {
     return true;
 }
 
-// Automatic choice: the tcgen05 kernel where the packed rows exceed 32 (there the warp-level products, not HBM,
-// bound the other kernel: measured 14-19 % faster at 48 and 64 rows on long sequences); the warp-level kernel
-// elsewhere (it is the faster one up to 32 rows, and by far on batches of short sequences). An explicit
-// heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level kernel's variants.
+// Automatic choice: the warp-level kernel, except above 48 packed rows on long-context configurations, where the
+// tcgen05 kernel measured 8 % faster (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches
+// of short sequences at any row count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one.
+// An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
+// kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
     if (c->kernel_path == PLT_PATH_WARP_MMA) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
-    return umma_eligible(c) && c->L * (c->Hq / c->Hkv) > 32 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
+    return umma_eligible(c) && c->L * (c->Hq / c->Hkv) > 48 && c->max_seq_len >= 16384 &&
+           (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
 // Chooses the kernel path and variant, prepares the kernels (shared-memory attribute, occupancy) and fills

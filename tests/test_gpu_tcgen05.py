@@ -28,6 +28,12 @@ def test_path_is_reported_and_unsupported_shapes_are_refused():
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05 and op.info["grid"] >= 1 and op.info["stages"] in (4, 6)
     with DecodeAttn(p) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
+    # automatic choice: tcgen05 only above 48 packed rows on long-context configurations
+    wide = custom(B=1, L=4, Hq=32, Hkv=2, w=33, lens=("list", [400]))
+    with DecodeAttn(make_problem(dict(wide, max_seq_len=16384))) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
+    with DecodeAttn(make_problem(dict(wide, max_seq_len=4096))) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
     for bad in (custom(d=64), custom(dtype="f32"), custom(page_size=48, lens=("list", [300, 77, 1]))):
         with pytest.raises(B.PltError) as e:
             DecodeAttn(make_problem(bad), **TC)
