@@ -30,6 +30,11 @@
  *
  * Storage types: inputs are float32 or bfloat16 (passed as uint16 bit
  * patterns, widened exactly); all arithmetic and the output are fp64.
+ * The caches and windows may instead hold 8-bit E4M3 codes (OCP 8-bit floating
+ * point: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities,
+ * S.1111.111 is NaN) with one fp32 scale per KV head for K and one for V; the
+ * attention is then the same definition applied to the dequantised values
+ * code_value * scale, formed in fp64.
  */
 #include <math.h>
 #include <stdint.h>
@@ -38,6 +43,7 @@
 
 #define PLT_ORACLE_F32 0
 #define PLT_ORACLE_BF16 1
+#define PLT_ORACLE_E4M3 3
 
 typedef struct {
     int32_t dtype;            /* PLT_ORACLE_F32 or PLT_ORACLE_BF16: type of q, caches, windows */
@@ -45,7 +51,7 @@ typedef struct {
     int32_t w;                /* window capacity (slots per non-first loop) */
     int32_t page_size;        /* 0: contiguous cache; >0: tokens per page */
     int32_t max_pages;        /* row length of page_table (paged only) */
-    int32_t pad_;
+    int32_t kv_dtype;         /* 0: caches and windows stored like q; PLT_ORACLE_E4M3: 8-bit codes */
     int64_t kv_stride_b;      /* contiguous cache strides in elements */
     int64_t kv_stride_n;      /* contiguous: token stride; paged: token-in-page stride */
     int64_t kv_stride_h;      /* KV-head stride */
@@ -61,6 +67,8 @@ typedef struct {
     const int32_t* win_lens;  /* [B, L-1] or NULL */
     const float* gate_logits; /* [B, L-1, Hq] pre-sigmoid */
     const int32_t* loop_offset; /* [L] delta_l, or NULL for delta_l = l-1 */
+    const float* k_scale;     /* [Hkv] dequantisation scale of K codes, or NULL (= 1) */
+    const float* v_scale;     /* [Hkv] dequantisation scale of V codes, or NULL (= 1) */
 } plt_oracle_problem;
 
 static double load_elem(const void* base, int64_t idx, int dtype) {
@@ -71,6 +79,23 @@ static double load_elem(const void* base, int64_t idx, int dtype) {
         return (double)f;
     }
     return (double)((const float*)base)[idx];
+}
+
+/* Value of an E4M3 code, from the format's definition. */
+double plt_oracle_e4m3_value(uint8_t code) {
+    const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);            /* subnormal: 0.m * 2^(1-bias) */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* Element of a cache or window: stored like q, or an E4M3 code times the KV head's scale. */
+static double load_kv(const plt_oracle_problem* p, const void* base, int64_t idx, const float* scale, int kvh) {
+    if (p->kv_dtype == PLT_ORACLE_E4M3)
+        return plt_oracle_e4m3_value(((const uint8_t*)base)[idx]) * (scale ? (double)scale[kvh] : 1.0);
+    return load_elem(base, idx, p->dtype);
 }
 
 /* Element offset of the shared cache row (b, token j, KV head kvh). */
@@ -103,7 +128,7 @@ static void attend(const plt_oracle_problem* p, const double* qv, const void* kb
     for (int j = 0; j < n; ++j) {
         int64_t off = rowfn(p, b, l, j, kvh);
         double s = 0.0;
-        for (int c = 0; c < d; ++c) s += qv[c] * load_elem(kbase, off + c, p->dtype);
+        for (int c = 0; c < d; ++c) s += qv[c] * load_kv(p, kbase, off + c, p->k_scale, kvh);
         s *= p->sm_scale;
         scores[j] = s;
         if (s > smax) smax = s;
@@ -116,7 +141,7 @@ static void attend(const plt_oracle_problem* p, const double* qv, const void* kb
     for (int j = 0; j < n; ++j) {
         int64_t off = rowfn(p, b, l, j, kvh);
         double pj = scores[j] / denom;
-        for (int c = 0; c < d; ++c) y[c] += pj * load_elem(vbase, off + c, p->dtype);
+        for (int c = 0; c < d; ++c) y[c] += pj * load_kv(p, vbase, off + c, p->v_scale, kvh);
     }
 }
 

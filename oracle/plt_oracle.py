@@ -24,13 +24,13 @@ class _Problem(ctypes.Structure):
     _fields_ = [
         ("dtype", ctypes.c_int32), ("B", ctypes.c_int32), ("L", ctypes.c_int32), ("Hq", ctypes.c_int32),
         ("Hkv", ctypes.c_int32), ("d", ctypes.c_int32), ("w", ctypes.c_int32), ("page_size", ctypes.c_int32),
-        ("max_pages", ctypes.c_int32), ("pad_", ctypes.c_int32),
+        ("max_pages", ctypes.c_int32), ("kv_dtype", ctypes.c_int32),
         ("kv_stride_b", ctypes.c_int64), ("kv_stride_n", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64),
         ("kv_stride_page", ctypes.c_int64), ("sm_scale", ctypes.c_double),
         ("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("seq_lens", ctypes.c_void_p), ("page_table", ctypes.c_void_p), ("k_win", ctypes.c_void_p),
         ("v_win", ctypes.c_void_p), ("win_lens", ctypes.c_void_p), ("gate_logits", ctypes.c_void_p),
-        ("loop_offset", ctypes.c_void_p),
+        ("loop_offset", ctypes.c_void_p), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -79,12 +79,15 @@ def _marshal(p):
         return a.ctypes.data
 
     st = np.uint16 if p.dtype == "bf16" else np.float32
+    e4m3 = getattr(p, "kv_dtype", "") == "e4m3"
+    kst = np.uint8 if e4m3 else st     # storage type of the caches and windows
     s = _Problem()
     s.dtype = 1 if p.dtype == "bf16" else 0
     s.B, s.L, s.Hq, s.Hkv, s.d, s.w = p.B, p.L, p.Hq, p.Hkv, p.d, p.w
     s.page_size = int(p.page_size)
     s.max_pages = 0 if p.page_table is None else int(p.page_table.shape[1])
-    kc = np.ascontiguousarray(p.k_cache, dtype=st)
+    s.kv_dtype = 3 if e4m3 else 0
+    kc = np.ascontiguousarray(p.k_cache, dtype=kst)
     # dense [B, N, Hkv, d] or pool [P, page, Hkv, d]
     s.kv_stride_h = p.d
     s.kv_stride_n = p.Hkv * p.d
@@ -92,12 +95,14 @@ def _marshal(p):
     s.kv_stride_page = s.kv_stride_b
     s.sm_scale = float(p.sm_scale) if p.sm_scale > 0 else 1.0 / float(np.sqrt(np.float64(p.d)))
     s.q = ptr(p.q, st)
-    s.k_cache = ptr(kc, st)
-    s.v_cache = ptr(p.v_cache, st)
+    s.k_cache = ptr(kc, kst)
+    s.v_cache = ptr(p.v_cache, kst)
     s.seq_lens = ptr(p.seq_lens, np.int32)
     s.page_table = ptr(p.page_table, np.int32)
-    s.k_win = ptr(p.k_win, st)
-    s.v_win = ptr(p.v_win, st)
+    s.k_win = ptr(p.k_win, kst)
+    s.v_win = ptr(p.v_win, kst)
+    s.k_scale = ptr(getattr(p, "k_scale", None), np.float32) if e4m3 else None
+    s.v_scale = ptr(getattr(p, "v_scale", None), np.float32) if e4m3 else None
     s.win_lens = ptr(p.win_lens, np.int32)
     s.gate_logits = ptr(p.gate_logits, np.float32)
     s.loop_offset = ptr(p.loop_offset, np.int32)

@@ -70,11 +70,18 @@ class ClpProblem:
     win_lens: Optional[np.ndarray] = None  # [B, L-1] int32 or None (= min(w, cut))
     loop_offset: Optional[np.ndarray] = None  # [L] int32 or None (= l-1)
     sm_scale: float = 0.0  # <= 0: 1/sqrt(d)
+    kv_dtype: str = ""  # "": caches and windows stored like q; "e4m3": uint8 E4M3 codes with per-KV-head scales
+    k_scale: Optional[np.ndarray] = None  # [Hkv] float32 (e4m3 only): value = code value * scale
+    v_scale: Optional[np.ndarray] = None
     meta: dict = field(default_factory=dict)
 
     @property
     def elem_size(self) -> int:
         return 2 if self.dtype == "bf16" else 4
+
+    @property
+    def kv_elem_size(self) -> int:
+        return 1 if self.kv_dtype == "e4m3" else self.elem_size
 
     @property
     def max_pages(self) -> int:
@@ -111,7 +118,7 @@ class ClpProblem:
 def algorithmic_bytes(p: ClpProblem) -> dict:
     """Bytes one decode step must move, each tensor counted once (no partials, padding or re-reads)."""
     s = p.elem_size
-    row = p.Hkv * p.d * 2 * s  # K and V of one token, all KV heads
+    row = p.Hkv * p.d * 2 * p.kv_elem_size  # K and V of one token, all KV heads
     shared = int(np.max(p.cuts(), axis=1).sum()) * row if p.B else 0
     window = int(p.window_lengths().sum()) * row
     qo = 2 * p.B * p.L * p.Hq * p.d * s
@@ -277,4 +284,40 @@ def make_problem(spec: dict, seed: Optional[int] = None, tail_fill: Optional[flo
             for l in range(L - 1):
                 prob.k_win[b, l, int(wl[b, l]):] = fill
                 prob.v_win[b, l, int(wl[b, l]):] = fill
+    if spec.get("kv_dtype") == "e4m3":
+        prob = quantize_kv_e4m3(prob)
     return prob
+
+
+def quantize_kv_e4m3(p: ClpProblem) -> ClpProblem:
+    """The same problem with the shared cache and the windows stored as E4M3 codes (uint8) and one scale per KV head
+    for K and one for V (largest magnitude of that head over cache and windows / 448). Input preparation only: the
+    rounding is torch's float32 -> float8_e4m3fn cast (round to nearest even)."""
+    import torch
+
+    def f32(a):
+        return bf16_bits_to_f32(a) if a.dtype == np.uint16 else a.astype(np.float32, copy=False)
+
+    def amax(a, b):  # per KV head (axis -2) over everything else, NaN-free inputs
+        m = np.zeros(p.Hkv, dtype=np.float32)
+        for x in (a, b):
+            for i in range(x.shape[0]):     # chunked over the leading axis to bound the float32 temporaries
+                v = np.abs(f32(x[i])).reshape(-1, p.Hkv, p.d)
+                if v.size:
+                    m = np.maximum(m, v.max(axis=(0, 2)))
+        return m
+
+    def codes(a, scale):
+        out = np.empty(a.shape, dtype=np.uint8)
+        inv = (1.0 / scale).astype(np.float32).reshape(1, p.Hkv, 1)
+        for i in range(a.shape[0]):
+            x = torch.from_numpy(np.ascontiguousarray(f32(a[i]).reshape(-1, p.Hkv, p.d) * inv))
+            x = torch.clamp(x, -448.0, 448.0)
+            out[i] = x.to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(a[i].shape)
+        return out
+
+    k_scale = np.maximum(amax(p.k_cache, p.k_win), 1e-12).astype(np.float32) / np.float32(448.0)
+    v_scale = np.maximum(amax(p.v_cache, p.v_win), 1e-12).astype(np.float32) / np.float32(448.0)
+    return replace(p, kv_dtype="e4m3", k_scale=k_scale.astype(np.float32), v_scale=v_scale.astype(np.float32),
+                   k_cache=codes(p.k_cache, k_scale), v_cache=codes(p.v_cache, v_scale),
+                   k_win=codes(p.k_win, k_scale), v_win=codes(p.v_win, v_scale))
