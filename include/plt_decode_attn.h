@@ -53,6 +53,17 @@ typedef enum {
 
 typedef enum { PLT_F32 = 0, PLT_BF16 = 1 } plt_dtype;
 
+/* Storage of the shared cache and the windows (plt_decode_attn_config.kv_dtype). */
+typedef enum {
+    PLT_KV_SAME = 0,   /* like q and out (config.dtype) */
+    PLT_KV_E4M3 = 1    /* 8-bit E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) with one
+                          fp32 scale per KV head for K and one for V: value = code value * scale.  The attention is the
+                          same definition on those dequantised values (the paper's efficiency runs use FP8 attention,
+                          Sec. 3.2).  Needs dtype = PLT_BF16 and d = 128; q and out stay bf16; softmax and
+                          accumulation stay fp32.  Served by the warp-level kernel; plt_decode_attn_run_host and
+                          plt_decode_attn_step refuse it. */
+} plt_kv_dtype;
+
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
 typedef enum {
     PLT_PATH_AUTO = 0,      /* the library chooses: tcgen05 above 48 packed rows (L * Hq / Hkv) when max_seq_len >= 16384
@@ -97,6 +108,7 @@ typedef struct {
                               16 * key_slices * slices_per_warp keys */
     int32_t row_warps;     /* PLT_PATH_WARP_MMA: warps that split the L * Hq/Hkv packed rows of a KV head (1 or 2; each
                               takes at most 32 rows) */
+    int32_t kv_dtype;      /* plt_kv_dtype of k_cache, v_cache, k_win, v_win; strides are then in bytes (= elements) */
 } plt_decode_attn_config;
 
 /*
@@ -123,6 +135,8 @@ typedef struct {
     const int32_t* win_lens;       /* optional [B, L-1]; NULL: wl = min(w, cut(b,l)) */
     const float* gate_logits;      /* [B, L-1, Hq] pre-sigmoid; +-inf allowed (NULL allowed when L == 1) */
     void* out;                     /* [B, L, Hq, d], same dtype as q */
+    const float* k_scale;          /* PLT_KV_E4M3 only: [Hkv] fp32 scales of the K codes (cache and windows); else ignored */
+    const float* v_scale;          /* PLT_KV_E4M3 only: [Hkv] fp32 scales of the V codes */
 } plt_decode_attn_args;
 
 /*

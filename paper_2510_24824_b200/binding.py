@@ -17,6 +17,7 @@ PLT_OK, PLT_ERR_INVALID_ARG, PLT_ERR_UNSUPPORTED, PLT_ERR_OUT_OF_MEMORY, PLT_ERR
     PLT_ERR_DEVICE_CHECK = range(7)
 PLT_F32, PLT_BF16 = 0, 1
 PLT_PATH_AUTO, PLT_PATH_WARP_MMA, PLT_PATH_TCGEN05 = 0, 1, 2
+PLT_KV_SAME, PLT_KV_E4M3 = 0, 1
 PLT_DEV_SEQ_LEN_CLAMPED, PLT_DEV_PAGE_ID_CLAMPED, PLT_DEV_WAIT_TIMEOUT, PLT_DEV_WIN_LEN_CLAMPED = 1, 2, 4, 8
 
 EXPORTS = (
@@ -44,6 +45,7 @@ class Config(ctypes.Structure):
         ("heads_per_cta", ctypes.c_int32), ("key_slices", ctypes.c_int32), ("stages", ctypes.c_int32),
         ("ctas_per_sm", ctypes.c_int32), ("kernel_path", ctypes.c_int32),
         ("loads_in_flight", ctypes.c_int32), ("slices_per_warp", ctypes.c_int32), ("row_warps", ctypes.c_int32),
+        ("kv_dtype", ctypes.c_int32),
     ]
 
 
@@ -56,6 +58,7 @@ class Args(ctypes.Structure):
         ("max_pages", ctypes.c_int32), ("num_pool_pages", ctypes.c_int32),
         ("k_win", ctypes.c_void_p), ("v_win", ctypes.c_void_p), ("win_lens", ctypes.c_void_p),
         ("gate_logits", ctypes.c_void_p), ("out", ctypes.c_void_p),
+        ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -106,7 +109,7 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
                 page_size: int = 0, sm_scale: float = 0.0, device: int = 0,
                 loop_offset: Optional[Sequence[int]] = None, heads_per_cta: int = 0, key_slices: int = 0,
                 stages: int = 0, ctas_per_sm: int = 0, kernel_path: int = 0, loads_in_flight: int = 0,
-                row_warps: int = 0, slices_per_warp: int = 0) -> Config:
+                row_warps: int = 0, slices_per_warp: int = 0, kv_dtype: int = 0) -> Config:
     c = Config()
     c.struct_size = ctypes.sizeof(Config)
     c.dtype = {"f32": PLT_F32, "bf16": PLT_BF16}.get(dtype, dtype)
@@ -122,6 +125,7 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
     c.loads_in_flight = loads_in_flight
     c.row_warps = row_warps
     c.slices_per_warp = slices_per_warp
+    c.kv_dtype = {"": PLT_KV_SAME, "e4m3": PLT_KV_E4M3}.get(kv_dtype, kv_dtype)
     return c
 
 
@@ -157,7 +161,7 @@ def _ptr(x) -> Optional[int]:
 
 def make_args(batch: int, q, k_cache, v_cache, seq_lens, out, k_win=None, v_win=None, gate_logits=None,
               page_table=None, max_pages: int = 0, num_pool_pages: int = 0, win_lens=None,
-              kv_strides=(0, 0, 0)) -> Args:
+              kv_strides=(0, 0, 0), k_scale=None, v_scale=None) -> Args:
     a = Args()
     a.struct_size = ctypes.sizeof(Args)
     a.batch = batch
@@ -167,6 +171,7 @@ def make_args(batch: int, q, k_cache, v_cache, seq_lens, out, k_win=None, v_win=
     a.max_pages, a.num_pool_pages = max_pages, num_pool_pages
     a.k_win, a.v_win, a.win_lens = _ptr(k_win), _ptr(v_win), _ptr(win_lens)
     a.gate_logits, a.out = _ptr(gate_logits), _ptr(out)
+    a.k_scale, a.v_scale = _ptr(k_scale), _ptr(v_scale)
     return a
 
 

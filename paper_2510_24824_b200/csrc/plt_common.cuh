@@ -28,6 +28,8 @@ struct Params {
     const int32_t* win_lens;   // [B, L-1] or null
     const int32_t* page_table; // [B, max_pages] or null
     const float* gate_logits;  // [B, L-1, Hq]
+    const float* k_scale;      // [Hkv] dequantisation scales of E4M3 caches and windows, else null
+    const float* v_scale;
     void* out;                 // [B, L, Hq, d]
     float* part_acc;           // [slots][hpc][R][d]  unnormalised sum of p * V
     float* part_ml;            // [slots][hpc][R][2]  running max (log2 units) and sum of p

@@ -106,6 +106,14 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
     if (c->Hq % c->Hkv != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "Hq %d is not a multiple of Hkv %d", c->Hq, c->Hkv);
     if (c->d != 64 && c->d != 128) return fail(nullptr, PLT_ERR_UNSUPPORTED, "head dim %d (supported: 64, 128)", c->d);
     if (c->L > 1 && c->w < 1) return fail(nullptr, PLT_ERR_INVALID_ARG, "w must be >= 1 when L > 1");
+    if (c->kv_dtype != PLT_KV_SAME && c->kv_dtype != PLT_KV_E4M3)
+        return fail(nullptr, PLT_ERR_INVALID_ARG, "unknown kv_dtype %d", c->kv_dtype);
+    if (c->kv_dtype == PLT_KV_E4M3) {
+        if (c->dtype != PLT_BF16 || c->d != 128)
+            return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches need bf16 queries and head dim 128");
+        if (c->kernel_path == PLT_PATH_TCGEN05)
+            return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches are served by the warp-level kernel only");
+    }
     g->G = c->Hq / c->Hkv;
     g->R = c->L * g->G;
     if (g->R > kMaxRows)
@@ -121,6 +129,8 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
 // Picks (rows per warp, heads per block, key slices, stages, blocks per SM) for the warp-level bf16 kernel.
 plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, MainVariant* v, int* want_ctas_per_sm) {
     v->D = c->d;
+    const bool fp8 = c->kv_dtype == PLT_KV_E4M3;
+    v->fp8 = fp8;
     int rw = c->row_warps;
     if (rw == 0) rw = g.R > 24 ? 2 : 1;   // 32 rows in one warp leave room for one warp per scheduler only: measured slower
     if (rw != 1 && rw != 2) return fail(nullptr, PLT_ERR_INVALID_ARG, "row_warps %d (supported: 1 or 2)", rw);
@@ -134,7 +144,7 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
     const bool small = nt <= 2;
     int hpc = c->heads_per_cta, kw = c->key_slices;
     int ks = c->slices_per_warp;
-    if (ks == 0) ks = rw == 2 ? 2 : 1;   // two warps per head: 32 keys each per tile (measured 25-35 % faster at 48 and 64 rows)
+    if (ks == 0) ks = (rw == 2 || fp8) ? 2 : 1;   // two warps per head: 32 keys each per tile (measured 25-35 % faster at 48 and 64 rows)
     if (ks != 1 && ks != 2) return fail(nullptr, PLT_ERR_INVALID_ARG, "slices_per_warp %d (supported: 1 or 2)", ks);
     if (hpc == 0) {
         hpc = 1;
@@ -147,10 +157,10 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
         if (kw < 1) kw = 1;
     }
     if (c->Hkv % hpc != 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "heads_per_cta %d does not divide Hkv %d", hpc, c->Hkv);
-    auto tile = [&]() { return main_bf16_tile_keys(v->D, nt, rw, hpc, kw, ks); };
+    auto tile = [&]() { return main_bf16_tile_keys(v->D, nt, rw, hpc, kw, ks, fp8); };
     while (c->page_size > 0 && tile() > 0 && c->page_size % tile() != 0 && kw > 1) kw >>= 1;
-    if (c->page_size > 0 && tile() > 0 && c->page_size % tile() != 0) ks = 1;
-    if (!main_bf16_exists(v->D, nt, rw, hpc, kw, ks))
+    if (c->page_size > 0 && tile() > 0 && c->page_size % tile() != 0 && !fp8) ks = 1;
+    if (!main_bf16_exists(v->D, nt, rw, hpc, kw, ks, fp8) || (c->page_size > 0 && c->page_size % tile() != 0))
         return fail(nullptr, PLT_ERR_UNSUPPORTED,
                     "no bf16 kernel for heads_per_cta=%d key_slices=%d slices_per_warp=%d row_warps=%d", hpc, kw, ks, rw);
     v->HPC = hpc;
@@ -163,16 +173,16 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
     int stages = c->stages;
     if (stages == 0) {
         // About 128 KB of loads in flight per SM measured fastest on B200; more only delays the first data.
-        const size_t stage_bytes = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 3, c->max_batch) -
-                                   main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 2, c->max_batch);
+        const size_t stage_bytes = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 3, c->max_batch, fp8) -
+                                   main_bf16_smem(v->D, nt, rw, hpc, kw, ks, 2, c->max_batch, fp8);
         stages = (int)((128 * 1024) / (stage_bytes * (size_t)cps));
         if (stages < 2) stages = 2;
-        while (stages > 2 && main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch) > budget) --stages;
+        while (stages > 2 && main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch, fp8) > budget) --stages;
         if (stages > 8) stages = 8;
     }
     if (stages < 2 || stages > 12) return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d outside [2, 12]", stages);
     v->stages = stages;
-    v->smem = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch);
+    v->smem = main_bf16_smem(v->D, nt, rw, hpc, kw, ks, stages, c->max_batch, fp8);
     if (v->smem > 227 * 1024)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "variant needs %zu bytes of shared memory (> 227 KB)", v->smem);
     *want_ctas_per_sm = cps;
@@ -194,9 +204,9 @@ plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, in
     if (h->map_valid[idx] && h->keys[idx] == key) return PLT_OK;
     cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)d1, (cuuint64_t)d2, (cuuint64_t)d3};
     cuuint64_t strides[3] = {(cuuint64_t)(s1 * es), (cuuint64_t)(s2 * es), (cuuint64_t)(s3 * es)};
-    cuuint32_t box[4] = {64u, (cuuint32_t)box_keys, (cuuint32_t)box_heads, 1u};
+    cuuint32_t box[4] = {(cuuint32_t)(128 / es), (cuuint32_t)box_keys, (cuuint32_t)box_heads, 1u};   // 128-byte rows
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    CUresult r = h->encode(&h->maps[idx], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+    CUresult r = h->encode(&h->maps[idx], es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -221,7 +231,7 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
-    if (c->kernel_path == PLT_PATH_WARP_MMA) return false;
+    if (c->kernel_path == PLT_PATH_WARP_MMA || c->kv_dtype == PLT_KV_E4M3) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
@@ -271,8 +281,8 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         // Starting and finishing an item (plan step, query rows, first load latency, partial store) stalls a block for
         // about as long as streaming 192 KB takes it (measured on B200 on a batch of short sequences: 4-5 us);
         // the plan charges every item that much, in tiles, so that blocks with many short items get fewer tiles.
-        const size_t stage_bytes = main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 3, 1) -
-                                   main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 2, 1);
+        const size_t stage_bytes = main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 3, 1, h->var.fp8) -
+                                   main_bf16_smem(h->var.D, h->var.NT, h->var.RW, h->var.HPC, h->var.KW, h->var.KS, 2, 1, h->var.fp8);
         h->piece_cost = (int)((192 * 1024) / (stage_bytes * (size_t)h->ctas_per_sm));
         if (h->piece_cost < 1) h->piece_cost = 1;
     } else {
@@ -433,7 +443,10 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
     if (!aligned16(a->q) || !aligned16(a->k_cache) || !aligned16(a->v_cache) || !aligned16(a->out) ||
         (c.L > 1 && (!aligned16(a->k_win) || !aligned16(a->v_win))))
         return fail(h, PLT_ERR_INVALID_ARG, "tensor base pointers must be 16-byte aligned");
-    const int es = elem_size(h->bf16);
+    const bool fp8 = h->cfg.kv_dtype == PLT_KV_E4M3;
+    const int es = fp8 ? 1 : elem_size(h->bf16);   // element size of the caches and windows
+    if (fp8 && (!a->k_scale || !a->v_scale)) return fail(h, PLT_ERR_INVALID_ARG, "k_scale and v_scale must not be NULL with E4M3 caches");
+    if (fp8 && step) return fail(h, PLT_ERR_UNSUPPORTED, "plt_decode_attn_step with E4M3 caches");
     int64_t sb = a->kv_stride_b, sn = a->kv_stride_n, sh = a->kv_stride_h;
     if (sb == 0 && sn == 0 && sh == 0) {
         sh = c.d;
@@ -458,6 +471,8 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
     p.q = a->q; p.k_cache = a->k_cache; p.v_cache = a->v_cache; p.k_win = a->k_win; p.v_win = a->v_win;
     p.seq_lens = a->seq_lens; p.win_lens = a->win_lens; p.page_table = a->page_table; p.gate_logits = a->gate_logits;
     p.out = a->out;
+    p.k_scale = fp8 ? a->k_scale : nullptr;
+    p.v_scale = fp8 ? a->v_scale : nullptr;
     p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.item_blocks = h->item_blocks;
     p.status = h->status;
 #ifdef PLT_TIMELINE
@@ -557,6 +572,7 @@ PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decod
     if (a->batch < 0) return fail(h, PLT_ERR_INVALID_ARG, "batch %d < 0", a->batch);
     if (a->batch > c.max_batch) return fail(h, PLT_ERR_CAPACITY, "batch %d > max_batch %d", a->batch, c.max_batch);
     if (a->batch == 0) return PLT_OK;
+    if (c.kv_dtype == PLT_KV_E4M3) return fail(h, PLT_ERR_UNSUPPORTED, "run_host with E4M3 caches");
     if (a->kv_stride_b || a->kv_stride_n || a->kv_stride_h)
         return fail(h, PLT_ERR_UNSUPPORTED, "run_host takes dense shared caches only (strides must be 0)");
     if (!a->q || !a->k_cache || !a->v_cache || !a->seq_lens || !a->out)

@@ -16,12 +16,13 @@ struct MainVariant {
     int stages;          // ring depth
     int grid;            // persistent blocks
     size_t smem;         // dynamic shared memory per block
+    bool fp8;            // caches and windows hold E4M3 codes (the f16-product kernel)
 };
 
-bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS);
-size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch);
+bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8 = false);
+size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch, bool fp8 = false);
 // Keys per pipeline tile of a variant (0 if it does not exist): the warps along the keys split a tile or take turns.
-int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS);
+int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8 = false);
 // Sets the shared-memory attribute and reports how many blocks fit one SM.
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
 // after_prestep: the launch before it in the stream is the pre-step kernel; overlap this grid's set-up with it.

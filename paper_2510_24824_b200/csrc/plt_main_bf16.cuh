@@ -28,9 +28,10 @@ constexpr float kSlack = 8.f;
 constexpr float kNoMax = -1e30f;   // reference maximum of a row that has seen no key yet (finite, so that no select is needed)
 constexpr uint32_t kOnesBf16x2 = 0x3f803f80u;
 
-template <int D, int NT, int RW, int HPC, int KW, int KS>
+template <int D, int NT, int RW, int HPC, int KW, int KS, bool FP8 = false>
 struct TCfg {
-    static constexpr int NH = D / 64;               // 64-element (128-byte) halves of a head row
+    static constexpr int ES = FP8 ? 1 : 2;          // bytes per cache element: E4M3 codes or bf16
+    static constexpr int NH = D * ES / 128;         // 128-byte pieces of a head row (one TMA box each)
     static constexpr int TK = 16 * KW * KS;         // keys per tile: KW warps along the keys, KS 16-key slices each
     static constexpr int NCW = HPC * KW * RW;       // consumer warps
     static constexpr int NTHREADS = (NCW + 1) * 32;
@@ -192,12 +193,154 @@ __device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uin
     }
 }
 
-template <int D, int NT, int RW, int HPC, int KW, int KS>
-__global__ void __launch_bounds__(TCfg<D, NT, RW, HPC, KW, KS>::NTHREADS, TCfg<D, NT, RW, HPC, KW, KS>::MIN_BLOCKS)
+// The same step for caches of E4M3 codes (d = 128: one 128-byte row per key). The codes convert exactly to f16, so the
+// products run as f16 mma with the query rows and the probabilities in f16. ldmatrix moves 16-bit units, i.e. PAIRS of
+// codes, so the fragments come out permuted; both permutations are absorbed without data movement:
+//   S^T: a thread gets d = 16 c + 4 tq .. + 3 of key grp (chunk c of 16 codes). The contraction index may be permuted
+//        freely as long as B uses the same order: the query fragments qb are loaded in that order (see the caller).
+//   O^T: ldmatrix.trans hands a thread the 2 x 2 block keys (2 tq, 2 tq + 1) x d (2 grp, 2 grp + 1); one byte
+//        permute splits it into the rows d = 2 grp and d = 2 grp + 1, so accumulator row grp is d = 16 mt + 2 grp and
+//        row grp + 8 is d = 16 mt + 2 grp + 1 (the caller stores accordingly).
+// scale_log2 already contains the K scale of the head; the V scale is applied when the piece is stored.
+template <int D, int NT, int KS, int HPC, int KW, int TKEYS, bool MASKED>
+__device__ __forceinline__ void process_keys_fp8(uint32_t sK, uint32_t sV, const uint32_t (&qb)[D / 16][NT][2],
+                                                 float (&acc)[D / 16][NT][4], float (&mref)[NT][2], float (&lacc)[NT][4],
+                                                 const int (&lim)[NT][2], int nvalid, float scale_log2, int lane, int kw,
+                                                 int h_local) {
+    static_assert(D == 128, "E4M3 caches: head dimension 128 only");
+    const int grp = lane >> 2, tq = lane & 3;
+    const int kbase = kw * 16 * KS;
+    float s[KS][NT][4];
+#pragma unroll
+    for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) s[ki][nt][0] = s[ki][nt][1] = s[ki][nt][2] = s[ki][nt][3] = 0.f;
+    {
+        const int key = kbase + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const uint32_t base = sK + (uint32_t)((h_local * TKEYS + key) * 128 + (((lane >> 4) ^ (key & 7)) << 4));
+#pragma unroll
+        for (int j = 0; j < D / 32; ++j) {          // chunks 2 j and 2 j + 1 (16 codes each) of every key
+            const uint32_t addr = base ^ (uint32_t)(j << 5);
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                uint32_t r[4];   // keys 0-7 / 8-15 of chunk 2 j, keys 0-7 / 8-15 of chunk 2 j + 1
+                ldmatrix_x4(addr + (uint32_t)(ki * 16 * 128), r[0], r[1], r[2], r[3]);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const uint32_t a[4] = {e4m3x2_to_f16x2(r[2 * c]), e4m3x2_to_f16x2(r[2 * c + 1]),
+                                           e4m3x2_to_f16x2(r[2 * c] >> 16), e4m3x2_to_f16x2(r[2 * c + 1] >> 16)};
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma_f16_16816(s[ki][nt], a, qb[2 * j + c][nt][0], qb[2 * j + c][nt][1]);
+                }
+            }
+        }
+    }
+    if (MASKED) {
+#pragma unroll
+        for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int kk = kbase + ki * 16 + grp + (e >= 2 ? 8 : 0);
+                    if (kk >= lim[nt][e & 1]) s[ki][nt][e] = -INFINITY;
+                }
+    }
+    bool grow = false;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
+#pragma unroll
+            for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
+            grow = grow || (fmaf(mx, scale_log2, -mref[nt][j]) > kSlack);
+        }
+    if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
+#pragma unroll
+                for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                const float m_new = fmaxf(mref[nt][j], mx * scale_log2);
+                const float alpha = fast_exp2(mref[nt][j] - m_new);
+                mref[nt][j] = m_new;
+                lacc[nt][j] *= alpha;
+                lacc[nt][2 + j] *= alpha;
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) {
+                    acc[mt][nt][j] *= alpha;
+                    acc[mt][nt][2 + j] *= alpha;
+                }
+            }
+    }
+    uint32_t pb[KS][NT][2];
+#pragma unroll
+    for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const float p0 = fast_exp2(fmaf(s[ki][nt][0], scale_log2, -mref[nt][0]));
+            const float p1 = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
+            const float p2 = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
+            const float p3 = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
+            pb[ki][nt][0] = movmatrix_trans(pack_f16x2(p0, p1));
+            pb[ki][nt][1] = movmatrix_trans(pack_f16x2(p2, p3));
+        }
+    {
+        const int key = kbase + (lane & 7) + (lane >> 4) * 8;
+        const uint32_t base = sV + (uint32_t)((h_local * TKEYS + key) * 128 + ((((lane >> 3) & 1) ^ (key & 7)) << 4));
+        uint32_t mask_lo[KS], mask_hi[KS];
+        if (MASKED) {
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                const int k0 = kbase + ki * 16 + 2 * tq;
+                mask_lo[ki] = (k0 < nvalid ? 0x0000ffffu : 0u) | (k0 + 1 < nvalid ? 0xffff0000u : 0u);
+                mask_hi[ki] = (k0 + 8 < nvalid ? 0x0000ffffu : 0u) | (k0 + 9 < nvalid ? 0xffff0000u : 0u);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < D / 32; ++j) {
+            const uint32_t addr = base ^ (uint32_t)(j << 5);
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                uint32_t r[4];   // keys 0-7 of chunks 2 j, 2 j + 1, then keys 8-15 of chunks 2 j, 2 j + 1
+                ldmatrix_x4_trans(addr + (uint32_t)(ki * 16 * 128), r[0], r[1], r[2], r[3]);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    // bytes (k0 d0, k0 d1, k1 d0, k1 d1) -> (k0 d0, k1 d0 | k0 d1, k1 d1)
+                    const uint32_t lo = byte_perm(r[c], 0u, 0x3120u), hi = byte_perm(r[2 + c], 0u, 0x3120u);
+                    uint32_t a[4] = {e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(lo >> 16), e4m3x2_to_f16x2(hi),
+                                     e4m3x2_to_f16x2(hi >> 16)};
+                    if (MASKED) {
+                        a[0] &= mask_lo[ki];
+                        a[1] &= mask_lo[ki];
+                        a[2] &= mask_hi[ki];
+                        a[3] &= mask_hi[ki];
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma_f16_16816(acc[2 * j + c][nt], a, pb[ki][nt][0], pb[ki][nt][1]);
+                }
+            }
+        }
+        const uint32_t ones[4] = {0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u};   // f16 1.0
+#pragma unroll
+        for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) mma_f16_16816(lacc[nt], ones, pb[ki][nt][0], pb[ki][nt][1]);
+    }
+}
+
+template <int D, int NT, int RW, int HPC, int KW, int KS, bool FP8>
+__global__ void __launch_bounds__(TCfg<D, NT, RW, HPC, KW, KS, FP8>::NTHREADS, TCfg<D, NT, RW, HPC, KW, KS, FP8>::MIN_BLOCKS)
 plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
                      const __grid_constant__ Params p, const int stages) {
-    using C = TCfg<D, NT, RW, HPC, KW, KS>;
+    using C = TCfg<D, NT, RW, HPC, KW, KS, FP8>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* full_bar = (uint64_t*)(smem + (size_t)stages * C::STAGE_BYTES);
@@ -356,11 +499,23 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     const int r = rb + nt * 8 + grp;
                     const bool v = r < p.R;
                     const int l = v ? r / p.G : 0;
-                    const int64_t q0 = (((int64_t)pc.b * p.L + l) * p.Hq + kvh * p.G + (r - l * p.G)) * D + 2 * tq;
+                    const int64_t qrow = (((int64_t)pc.b * p.L + l) * p.Hq + kvh * p.G + (r - l * p.G)) * D;
+                    if constexpr (FP8) {
+                        // contraction order of process_keys_fp8: k-step ks takes d = 16 ks + 4 tq .. + 3; bf16 -> f16
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        qb[ks][nt][0] = v ? *(const uint32_t*)(qg + q0 + ks * 16) : 0u;
-                        qb[ks][nt][1] = v ? *(const uint32_t*)(qg + q0 + ks * 16 + 8) : 0u;
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            uint2 u = make_uint2(0u, 0u);
+                            if (v) u = *(const uint2*)(qg + qrow + ks * 16 + 4 * tq);
+                            qb[ks][nt][0] = pack_f16x2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+                            qb[ks][nt][1] = pack_f16x2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+                        }
+                    } else {
+                        const int64_t q0 = qrow + 2 * tq;
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            qb[ks][nt][0] = v ? *(const uint32_t*)(qg + q0 + ks * 16) : 0u;
+                            qb[ks][nt][1] = v ? *(const uint32_t*)(qg + q0 + ks * 16 + 8) : 0u;
+                        }
                     }
                 }
             }
@@ -379,6 +534,8 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     }
                 }
             float acc[D / 16][NT][4], mref[NT][2], lacc[NT][4];
+            // E4M3 caches: the K scale of the head is a score scale, the V scale is applied to the finished partial
+            const float sc2 = FP8 ? p.scale_log2 * p.k_scale[kvh] : p.scale_log2;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 mref[nt][0] = mref[nt][1] = kNoMax;
@@ -401,17 +558,25 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     const int key0 = t * C::TK;
                     if (ok) {
                         if (key0 + C::TK <= cmin) {
-                            process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, false>(sK, sV, qb, acc, mref, lacc, cutr,
-                                                                                         0, p.scale_log2, lane, kw, h_local);
+                            if constexpr (FP8)
+                                process_keys_fp8<D, NT, KS, HPC, KW, C::TK, false>(sK, sV, qb, acc, mref, lacc, cutr, 0, sc2,
+                                                                                   lane, kw, h_local);
+                            else
+                                process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, false>(sK, sV, qb, acc, mref, lacc,
+                                                                                             cutr, 0, sc2, lane, kw, h_local);
                         } else {
 #pragma unroll
                             for (int nt = 0; nt < NT; ++nt) {
                                 lim[nt][0] = cutr[nt][0] - key0;
                                 lim[nt][1] = cutr[nt][1] - key0;
                             }
-                            process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim,
-                                                                                        pc.sp.cmax - key0, p.scale_log2,
-                                                                                        lane, kw, h_local);
+                            if constexpr (FP8)
+                                process_keys_fp8<D, NT, KS, HPC, KW, C::TK, true>(sK, sV, qb, acc, mref, lacc, lim,
+                                                                                  pc.sp.cmax - key0, sc2, lane, kw, h_local);
+                            else
+                                process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim,
+                                                                                            pc.sp.cmax - key0, sc2, lane, kw,
+                                                                                            h_local);
                         }
                     }
                 } else {
@@ -430,8 +595,12 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                             lim[nt][0] = lc[nt][0] == l ? n : 0;
                             lim[nt][1] = lc[nt][1] == l ? n : 0;
                         }
-                        process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim, n,
-                                                                                    p.scale_log2, lane, kw, h_local);
+                        if constexpr (FP8)
+                            process_keys_fp8<D, NT, KS, HPC, KW, C::TK, true>(sK, sV, qb, acc, mref, lacc, lim, n, sc2, lane, kw,
+                                                                              h_local);
+                        else
+                            process_keys<D, NT, KS, HPC, KW, C::TK, C::BOX_BYTES, true>(sK, sV, qb, acc, mref, lacc, lim, n, sc2,
+                                                                                        lane, kw, h_local);
                     }
                     cur.advance(p, pc.sp);
                 }
@@ -449,6 +618,18 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
                 for (int j = 0; j < 2; ++j)
                     if (mref[nt][j] == kNoMax) mref[nt][j] = -INFINITY;   // the partial's "saw no key" mark
+            // Accumulator fragment rows (lane / 4, lane / 4 + 8) of 16-row group mt are the head dimensions
+            // 16 mt + dA and 16 mt + dB (E4M3 caches: see process_keys_fp8).
+            const int dA = FP8 ? 2 * grp : grp, dB = FP8 ? 2 * grp + 1 : grp + 8;
+            if constexpr (FP8) {
+                const float vs = p.v_scale[kvh];
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[mt][nt][e] *= vs;
+            }
             const int64_t slot = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta);
             const int64_t prow = (slot * HPC + h_local) * p.R + rb;
             if (tid == 0) note_piece(p, pc, cta);
@@ -459,11 +640,11 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     for (int j = 0; j < 2; ++j) {
                         if (lc[nt][j] == kMaxLoops) continue;
                         const int64_t row = prow + nt * 8 + 2 * tq + j;
-                        float* dst = p.part_acc + row * D + grp;
+                        float* dst = p.part_acc + row * D;
 #pragma unroll
                         for (int mt = 0; mt < D / 16; ++mt) {
-                            dst[mt * 16] = acc[mt][nt][j];
-                            dst[mt * 16 + 8] = acc[mt][nt][2 + j];
+                            dst[mt * 16 + dA] = acc[mt][nt][j];
+                            dst[mt * 16 + dB] = acc[mt][nt][2 + j];
                         }
                         if (grp == 0) *(float2*)(p.part_ml + row * 2) = make_float2(mref[nt][j], lacc[nt][j]);
                     }
@@ -507,16 +688,16 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                             for (int j = 0; j < 2; ++j) {
-                                float* a = macc + (nt * 8 + 2 * tq + j) * C::MROW + grp;
+                                float* a = macc + (nt * 8 + 2 * tq + j) * C::MROW;
 #pragma unroll
                                 for (int mt = 0; mt < D / 16; ++mt) {
                                     float x0 = acc[mt][nt][j] * sc[nt][j], x1 = acc[mt][nt][2 + j] * sc[nt][j];
                                     if (k > 0) {
-                                        x0 += a[mt * 16];
-                                        x1 += a[mt * 16 + 8];
+                                        x0 += a[mt * 16 + dA];
+                                        x1 += a[mt * 16 + dB];
                                     }
-                                    a[mt * 16] = x0;
-                                    a[mt * 16 + 8] = x1;
+                                    a[mt * 16 + dA] = x0;
+                                    a[mt * 16 + dB] = x1;
                                 }
                             }
                     }

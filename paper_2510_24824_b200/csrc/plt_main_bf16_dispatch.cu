@@ -8,31 +8,42 @@ namespace plt {
     cudaError_t main_bf16_d##D##_n##NT##r##RW(int, const MainVariant&, const CUtensorMap*, const Params*, cudaStream_t, int*);
 PLT_ALL(PLT_DECL, 64) PLT_ALL(PLT_DECL, 128)
 #undef PLT_DECL
+#define PLT_DECL8(D, NT, RW) \
+    cudaError_t main_fp8_d##D##_n##NT##r##RW(int, const MainVariant&, const CUtensorMap*, const Params*, cudaStream_t, int*);
+PLT_ALL(PLT_DECL8, 128)
+#undef PLT_DECL8
 
 static cudaError_t dispatch(int op, const MainVariant& v, const CUtensorMap* maps, const Params* p, cudaStream_t s,
                             int* out) {
 #define PLT_GO(D_, NT_, RW_) \
     if (v.D == D_ && v.NT == NT_ && v.RW == RW_) return main_bf16_d##D_##_n##NT_##r##RW_(op, v, maps, p, s, out);
+#define PLT_GO8(D_, NT_, RW_) \
+    if (v.D == D_ && v.NT == NT_ && v.RW == RW_) return main_fp8_d##D_##_n##NT_##r##RW_(op, v, maps, p, s, out);
+    if (v.fp8) {
+        PLT_ALL(PLT_GO8, 128)
+        return cudaErrorInvalidValue;
+    }
     PLT_ALL(PLT_GO, 64) PLT_ALL(PLT_GO, 128)
 #undef PLT_GO
+#undef PLT_GO8
 #undef PLT_ALL
     return cudaErrorInvalidValue;
 }
 
-bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS) {
-    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0};
+bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0, fp8};
     return dispatch(0, v, nullptr, nullptr, nullptr, nullptr) == cudaSuccess;
 }
 
-size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch) {
-    MainVariant v{D, NT, RW, HPC, KW, KS, 0, stages, max_batch, 0};
+size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch, bool fp8) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, stages, max_batch, 0, fp8};
     int out = 0;
     if (dispatch(3, v, nullptr, nullptr, nullptr, &out) != cudaSuccess) return 0;
     return (size_t)out;
 }
 
-int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS) {
-    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0};
+int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8) {
+    MainVariant v{D, NT, RW, HPC, KW, KS, 0, 1, 1, 0, fp8};
     int out = 0;
     if (dispatch(4, v, nullptr, nullptr, nullptr, &out) != cudaSuccess) return 0;
     return out;

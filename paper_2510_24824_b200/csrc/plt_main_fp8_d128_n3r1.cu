@@ -1,0 +1,6 @@
+#define PLT_INST_D 128
+#define PLT_INST_NT 3
+#define PLT_INST_RW 1
+#define PLT_INST_FP8 1
+#define PLT_INST_NAME main_fp8_d128_n3r1
+#include "plt_main_bf16_inst.inl"

@@ -27,15 +27,16 @@ def to_torch(a: Optional[np.ndarray], dtype: str, device, pin: bool = False):
 class DeviceProblem:
     """Tensors of one decode step on a device (or, with device=None, in pinned host memory)."""
 
-    FIELDS = ("q", "k_cache", "v_cache", "seq_lens", "k_win", "v_win", "gate_logits", "page_table", "win_lens")
+    FIELDS = ("q", "k_cache", "v_cache", "seq_lens", "k_win", "v_win", "gate_logits", "page_table", "win_lens",
+              "k_scale", "v_scale")
 
     def __init__(self, p, device="cuda:0", pin: bool = False):
         self.problem = p
         self.device = device
         for f in self.FIELDS:
             a = getattr(p, f)
-            is_data = f in ("q", "k_cache", "v_cache", "k_win", "v_win")
-            setattr(self, f, to_torch(a, p.dtype if is_data else "", device, pin))
+            is_data = f == "q" or (f in ("k_cache", "v_cache", "k_win", "v_win") and p.kv_dtype != "e4m3")
+            setattr(self, f, to_torch(a, p.dtype if is_data else "", device, pin))   # E4M3 codes stay uint8
         tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
         if device is None:
             self.out = torch.empty((p.B, p.L, p.Hq, p.d), dtype=tdt)
@@ -50,7 +51,8 @@ class DeviceProblem:
             p.B, self.q, self.k_cache, self.v_cache, self.seq_lens, self.out if out is None else out,
             k_win=self.k_win if p.L > 1 else None, v_win=self.v_win if p.L > 1 else None,
             gate_logits=self.gate_logits if p.L > 1 else None, page_table=self.page_table,
-            max_pages=p.max_pages, num_pool_pages=p.num_pool_pages, win_lens=self.win_lens)
+            max_pages=p.max_pages, num_pool_pages=p.num_pool_pages, win_lens=self.win_lens,
+            k_scale=self.k_scale, v_scale=self.v_scale)
 
     def h2d_bytes(self) -> int:
         n = 0
@@ -71,7 +73,8 @@ class DecodeAttn:
         self.config = B.make_config(
             p.dtype, max_batch or max(p.B, 1), p.L, p.Hq, p.Hkv, p.d, p.max_seq_len, p.w, page_size=p.page_size,
             sm_scale=p.sm_scale, device=device_index,
-            loop_offset=None if p.loop_offset is None else [int(x) for x in p.loop_offset], **tuning)
+            loop_offset=None if p.loop_offset is None else [int(x) for x in p.loop_offset], kv_dtype=p.kv_dtype,
+            **tuning)
         self.handle = B.plt_decode_attn_create(self.config)
         self.info = B.plt_decode_attn_launch_info(self.handle)
 
