@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--cps", type=int, default=0)
     ap.add_argument("--loops", type=int, default=0, help="override the workload's number of loops L (for the traffic-vs-L sweep)")
     ap.add_argument("--path", type=int, default=0, help="kernel path: 0 automatic, 1 warp-level mma, 2 tcgen05")
+    ap.add_argument("--kv", default="", choices=["", "e4m3"],
+                    help="store the shared cache and the windows as E4M3 codes with per-KV-head scales (q and out stay bf16)")
     ap.add_argument("--prestep", action="store_true",
                     help="time plt_decode_attn_step: the pre-step kernel (cache append, window ring update, gate linear) "
                          "ahead of the attention, three launches per step")
@@ -146,7 +148,7 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def replica_spec(index: int, rank: int, loops: int = 0) -> dict:
+def replica_spec(index: int, rank: int, loops: int = 0, kv: str = "") -> dict:
     """Workload of one replica: every rank streams its own data (seed offset by rank), same shapes."""
     from paper_2510_24824_b200.inputs import workload
     spec = workload(index)
@@ -154,6 +156,9 @@ def replica_spec(index: int, rank: int, loops: int = 0) -> dict:
     if loops > 0:
         spec["L"] = loops
         spec["name"] = f"{spec['name']}_L{loops}"
+    if kv:
+        spec["kv_dtype"] = kv
+        spec["name"] = f"{spec['name']}_{kv}"
     return spec
 
 
@@ -276,7 +281,9 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    p = make_problem(replica_spec(args.workload, rank, args.loops))
+    p = make_problem(replica_spec(args.workload, rank, args.loops, args.kv))
+    if args.kv:
+        args.no_e2e = True   # the host-buffer entry point takes caches stored like q only
     dp = DeviceProblem(p, dev)
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
                   kernel_path=args.path)
@@ -411,7 +418,7 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": p.dtype, "data": "synthetic", "config": cfg,
+            "vs_baseline": None, "dtype": p.dtype + ("+e4m3 cache" if p.kv_dtype else ""), "data": "synthetic", "config": cfg,
             "loop_queries_per_s": value * p.B * p.L,
             "hbm_gbs_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9,
             "hbm_frac_of_8tbs": by["total"] / (ms_per_step * 1e-3) / 8e12,

@@ -20,9 +20,9 @@ def sample_rows(p, n, rng, forced=()):
     return np.array(sorted(rows), dtype=np.int32)
 
 
-@pytest.mark.parametrize("index", [1, 2, 3, 4])
-def test_full_size_sampled_rows(index):
-    p = make_problem(workload(index))
+@pytest.mark.parametrize("index,kv", [(1, ""), (2, ""), (3, ""), (4, ""), (1, "e4m3"), (4, "e4m3")])
+def test_full_size_sampled_rows(index, kv):
+    p = make_problem(dict(workload(index), kv_dtype=kv))
     dp = DeviceProblem(p, "cuda:0")
     dp.out.fill_(float("nan"))
     with DecodeAttn(p) as op:
@@ -35,7 +35,10 @@ def test_full_size_sampled_rows(index):
     got = dp.out.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     # convexity: every output lies within the range of the values it can mix
-    vmax = float(max(dp.v_cache.float().abs().max().item(), dp.v_win.float().abs().max().item()))
+    if kv:   # E4M3 codes: the largest finite code value is 448, times the largest V scale
+        vmax = 448.0 * float(p.v_scale.max())
+    else:
+        vmax = float(max(dp.v_cache.float().abs().max().item(), dp.v_win.float().abs().max().item()))
     assert np.abs(got).max() <= vmax * (1 + 2 ** -7)
     inactive = p.cuts() == 0
     assert np.all(got[inactive] == 0.0)
