@@ -4,7 +4,8 @@
 //   * each later loop's row replaces the oldest entry of its window, slot (cut_l - 1) mod w (a non-first loop keeps
 //     only its w newest entries, Sec. 2.2.2);
 //   * gate_logits[b, l, h] = <w_gate[h], Q[b, l, h]> + b_gate[h] for loops 2..L (one scalar per head).
-// One block per (sequence, loop): 16-byte copies of the two rows, then one warp per query head for the dot products.
+// One block per (sequence, loop): the dot products of the gate (a warp takes four heads at a time), then 16-byte
+// copies of the two rows.
 // One launch instead of three; the attention kernels follow in the same stream.
 #include <cuda_bf16.h>
 
@@ -16,7 +17,7 @@ namespace plt {
 
 namespace {
 
-constexpr int kPreThreads = 128;
+constexpr int kPreThreads = 256;
 
 template <bool BF16>
 __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_constant__ Params p, const void* k_new,
@@ -30,6 +31,36 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
     const int32_t n = seq_len_clamped(p, b, flags);
     int cut = n - p.delta[l];
     cut = cut > 0 ? cut : 0;
+
+    if (l > 0) {
+        // head-wise gate linear; written for every sequence and loop (the attention ignores it where cut = 0).
+        // A warp takes kGateHeads heads at a time with all their loads in flight together.
+        constexpr int kGateHeads = 4;
+        for (int h0 = wid * kGateHeads; h0 < p.Hq; h0 += (kPreThreads / 32) * kGateHeads) {
+            float acc[kGateHeads];
+#pragma unroll
+            for (int i = 0; i < kGateHeads; ++i) {
+                const int h = h0 + i;
+                acc[i] = 0.f;
+                if (h < p.Hq) {
+                    const T* q = (const T*)p.q + (((int64_t)b * p.L + l) * p.Hq + h) * p.d;
+                    for (int j = lane; j < p.d; j += 32) {
+                        float x;
+                        if constexpr (BF16) x = __bfloat162float(q[j]);
+                        else x = q[j];
+                        acc[i] = fmaf(w_gate[(int64_t)h * p.d + j], x, acc[i]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kGateHeads; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+                const int h = h0 + i;
+                if (lane == 0 && h < p.Hq) gate_out[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h] = acc[i] + b_gate[h];
+            }
+        }
+    }
 
     if (cut > 0) {
         // destination rows of this loop's K and V: [Hkv] rows of d elements, kd elements apart
@@ -66,22 +97,6 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
             const uint4 vv = *((const uint4*)((const T*)v_new + src + (int64_t)h * p.d) + c);
             *((uint4*)(kd + h * head_stride) + c) = kk;
             *((uint4*)(vd + h * head_stride) + c) = vv;
-        }
-    }
-    if (l > 0) {
-        // head-wise gate linear; written for every sequence and loop (the attention ignores it where cut = 0)
-        for (int h = wid; h < p.Hq; h += kPreThreads / 32) {
-            const T* q = (const T*)p.q + (((int64_t)b * p.L + l) * p.Hq + h) * p.d;
-            float acc = 0.f;
-            for (int j = lane; j < p.d; j += 32) {
-                float x;
-                if constexpr (BF16) x = __bfloat162float(q[j]);
-                else x = q[j];
-                acc = fmaf(w_gate[(int64_t)h * p.d + j], x, acc);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (lane == 0) gate_out[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h] = acc + b_gate[h];
         }
     }
     if (flags && tid == 0) atomicOr(p.status, flags);
