@@ -527,7 +527,7 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
             e = launch_main_umma(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox,
                                  c.loads_in_flight > 0 ? c.loads_in_flight : 2, stream);
         else
-            e = launch_main_bf16(h->var, h->maps, p, step != nullptr, stream);
+            e = launch_main_bf16(h->var, h->maps, p, /*overlap=*/true, stream);
     } else {
         if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
         e = launch_main_f32(p, h->var.grid, h->var.smem, stream);

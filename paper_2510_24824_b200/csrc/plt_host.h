@@ -25,8 +25,10 @@ size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages
 int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8 = false);
 // Sets the shared-memory attribute and reports how many blocks fit one SM.
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
-// after_prestep: the launch before it in the stream is the pre-step kernel; overlap this grid's set-up with it.
-cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, bool after_prestep,
+// overlap: launch with programmatic stream serialisation, so that this grid's set-up (which reads only what the caller
+// passed) runs while the kernel before it in the stream (the pre-step kernel, or the merge kernel of the step before)
+// finishes; the kernel waits for that kernel's completion before it reads or writes anything else.
+cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, bool overlap,
                              cudaStream_t stream);
 
 // fp32 SIMT main kernel (same plan, tile of kF32TileKeys keys, one KV head per block).

@@ -365,8 +365,10 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         mbar_fence_init();
     }
     build_prefix(p, s_prefix, flags, s_lens);  // contains __syncthreads
-    // Everything above reads only what the caller passed. If this grid was launched to overlap the pre-step kernel,
-    // the caches, windows and query rows may be read only from here on (a no-op for an ordinary launch).
+    // Everything above reads only what the caller passed (lengths) and writes only shared memory. This grid is launched
+    // to overlap the end of the kernel before it in the stream (the pre-step kernel, or the merge kernel of the step
+    // before, which still reads the partials): caches, windows and query rows are read, and the workspace is written,
+    // only from here on.
     grid_dependency_wait();
     // The merge kernel may be set up from now on (it reads the gate logits, which the pre-step may have written, before
     // its own wait, hence not earlier); it waits for this grid to complete before it reads the partials.

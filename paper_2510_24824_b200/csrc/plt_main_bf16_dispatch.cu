@@ -53,9 +53,9 @@ cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm) {
     return dispatch(1, v, nullptr, nullptr, nullptr, blocks_per_sm);
 }
 
-cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, bool after_prestep,
+cudaError_t launch_main_bf16(const MainVariant& v, const CUtensorMap maps[4], const Params& p, bool overlap,
                              cudaStream_t stream) {
-    return dispatch(after_prestep ? 5 : 2, v, maps, &p, stream, nullptr);
+    return dispatch(overlap ? 5 : 2, v, maps, &p, stream, nullptr);
 }
 
 }  // namespace plt

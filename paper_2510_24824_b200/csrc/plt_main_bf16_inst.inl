@@ -35,8 +35,8 @@ cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const 
         *out = (int)C::smem_bytes(v.stages, v.grid /* max_batch passed in grid for this query */);
         return cudaSuccess;
     }
-    // op 2: plain launch; op 5: launch with programmatic stream serialisation (the kernel before it in the stream is the
-    // pre-step kernel: this grid's blocks are set up while it runs and wait for its results in grid_dependency_wait()).
+    // op 2: plain launch; op 5: launch with programmatic stream serialisation (this grid's blocks are set up while the
+    // kernel before it in the stream finishes and wait for its completion in grid_dependency_wait()).
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)v.grid);
     cfg.blockDim = dim3(C::NTHREADS);

@@ -68,6 +68,9 @@ __device__ __forceinline__ float merge_item(const Params& p, int item, int hl, i
 
 template <int D, bool BF16>
 __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __grid_constant__ Params p, const int chunks) {
+    // The next kernel in the stream (the main kernel of the following step, or whatever the caller enqueued with
+    // programmatic serialisation) may be set up once every block of this grid has started.
+    grid_launch_dependents();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int HG = p.Hkv / p.hpc;
     const int chunk = (int)(blockIdx.x % chunks);
