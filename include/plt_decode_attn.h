@@ -153,6 +153,10 @@ plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_deco
  * arguments are validated first and nothing is launched on error.  Two kernels
  * are launched: the split-KV main kernel and the merge/gate kernel.
  * Calls on the same handle must be stream-ordered (they share the workspace).
+ * The main kernel is launched with programmatic stream serialisation: its set-up reads seq_lens and win_lens while
+ * the kernel before it in the stream finishes, everything else after that kernel has completed.  A kernel of yours
+ * that writes seq_lens or win_lens right before this call must therefore not release its programmatic dependents
+ * early (kernels that never call griddepcontrol.launch_dependents release them when they end: nothing to do).
  */
 plt_status plt_decode_attn_run(plt_decode_attn_t handle, const plt_decode_attn_args* args, void* cuda_stream);
 
