@@ -287,3 +287,28 @@ def test_host_buffer_entry_point(index):
         assert op.check() == 0
     assert torch.equal(out, out2)
     assert_parity(out.float().numpy().astype(np.float64), oracle.decode_attn(p), p.dtype, "run_host")
+
+
+def test_back_to_back_steps_on_one_handle_do_not_disturb_each_other():
+    """Consecutive launches overlap at their edges (the merge kernel's and the next main kernel's set-up start early):
+    two different batches alternated on one handle, 40 runs with no host synchronisation in between, must each
+    give exactly what they give alone."""
+    big = make_problem(custom(B=6, L=3, Hq=12, Hkv=2, w=40, lens=("list", [3000, 2500, 4000, 3500, 2000, 3900]), max_seq_len=4096))
+    small = make_problem(custom(B=2, L=3, Hq=12, Hkv=2, w=40, lens=("list", [70, 5]), max_seq_len=4096, seed=5))
+    dbig, dsmall = DeviceProblem(big, "cuda:0"), DeviceProblem(small, "cuda:0")
+    with DecodeAttn(big) as op:
+        op.run(dbig)
+        op.run(dsmall)
+        torch.cuda.synchronize()
+        alone_big, alone_small = dbig.out.clone(), dsmall.out.clone()
+        outs = []
+        for i in range(40):
+            dp = dbig if i % 2 == 0 else dsmall
+            o = torch.full_like(dp.out, float("nan"))
+            op.run(dp, out=o)
+            outs.append(o)
+        torch.cuda.synchronize()
+        assert op.check() == 0
+    for i, o in enumerate(outs):
+        assert torch.equal(o, alone_big if i % 2 == 0 else alone_small), f"run {i} differs"
+    assert_parity(alone_big.float().cpu().numpy().astype(np.float64), oracle.decode_attn(big), "bf16", "big")
