@@ -37,9 +37,6 @@ struct Params {
     int32_t* item_blocks;      // [items][2] first and last main-kernel block holding a piece of the item (written by
                                // the blocks that own the item's first / last tile; items without tiles are not written)
     uint32_t* status;          // device status word
-#ifdef PLT_TIMELINE
-    void* timeline;            // [grid][8] u64, instrumentation builds only
-#endif
     int64_t kv_stride_b, kv_stride_n, kv_stride_h;  // elements
     int32_t B, L, Hq, Hkv, G, R, d, w;
     int32_t max_seq_len, page_size, max_pages, num_pool_pages;
@@ -141,11 +138,6 @@ __device__ __forceinline__ int plan_ctas(int64_t T, int launched) { return T < l
 
 // Range of the tile line owned by block c of C: [c*T/C, (c+1)*T/C).
 __device__ __forceinline__ int64_t cta_begin(int64_t T, int c, int C) { return (T * c) / C; }
-
-// The block that owns tile position pos.
-__device__ __forceinline__ int cta_of(int64_t T, int64_t pos, int C) {
-    return (int)(((pos + 1) * C - 1) / T);
-}
 
 // Work item index: (sequence, head group, kind) with kind 0 = shared cache, 1 = windows.
 __device__ __forceinline__ int item_index(const Params& p, int b, int hg, int kind) {

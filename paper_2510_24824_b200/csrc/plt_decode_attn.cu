@@ -66,9 +66,6 @@ struct plt_decode_attn {
     // device staging for plt_decode_attn_run_host (grow-only)
     Staging st[10];
     cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // optional, caller-owned
-#ifdef PLT_TIMELINE
-    void* timeline = nullptr;
-#endif
     char err[512];
 };
 
@@ -388,10 +385,6 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
     e = cudaMemset(h->status, 0, 4);
     if (e != cudaSuccess) { cudaFree(ws); delete h; return cuda_fail(nullptr, "cudaMemset", e); }
-#ifdef PLT_TIMELINE
-    cudaMalloc(&h->timeline, (size_t)h->var.grid * 64);
-    cudaMemset(h->timeline, 0, (size_t)h->var.grid * 64);
-#endif
     *out_handle = h;
     return PLT_OK;
 }
@@ -475,9 +468,6 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
     p.v_scale = fp8 ? a->v_scale : nullptr;
     p.part_acc = h->part_acc; p.part_ml = h->part_ml; p.prefix = h->prefix; p.item_blocks = h->item_blocks;
     p.status = h->status;
-#ifdef PLT_TIMELINE
-    p.timeline = h->timeline;
-#endif
     p.kv_stride_b = sb; p.kv_stride_n = sn; p.kv_stride_h = sh;
     p.B = a->batch; p.L = c.L; p.Hq = c.Hq; p.Hkv = c.Hkv; p.G = h->G; p.R = h->R; p.d = c.d; p.w = c.w;
     p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
@@ -681,13 +671,6 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
 
 }  // extern "C"
 
-#ifdef PLT_TIMELINE
-extern "C" PLT_API int plt_debug_timeline(plt_decode_attn_t h, unsigned long long* host, int max_ctas) {
-    int n = h->var.grid < max_ctas ? h->var.grid : max_ctas;
-    cudaMemcpy(host, h->timeline, (size_t)n * 64, cudaMemcpyDeviceToHost);
-    return n;
-}
-#endif
 
 // ===================================================================================================
 // Allocation-free entry point.
