@@ -312,3 +312,10 @@ def test_back_to_back_steps_on_one_handle_do_not_disturb_each_other():
     for i, o in enumerate(outs):
         assert torch.equal(o, alone_big if i % 2 == 0 else alone_small), f"run {i} differs"
     assert_parity(alone_big.float().cpu().numpy().astype(np.float64), oracle.decode_attn(big), "bf16", "big")
+
+
+@pytest.mark.parametrize("kv", ["", "e4m3"])
+def test_maximum_batch_of_short_sequences(kv):
+    """4096 sequences (the largest batch a handle takes) of 0..70 tokens: thousands of items, most blocks hold dozens."""
+    p = make_problem(custom(B=4096, L=3, Hq=8, Hkv=2, w=24, lens=("uniform", 0, 70), kv_dtype=kv, seed=3))
+    assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", f"B=4096 {kv}")
