@@ -7,6 +7,9 @@ Prints ONE JSON line. Default workload: bf16 decode batch B=64, L=2, Hq=32, Hkv=
 (the configuration the headline metric is quoted on). Under torchrun (N > 1) every rank runs an
 independent replica of the workload on its own GPU (no collective in the data path; weak scaling).
 `--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+Other legs: `--kv e4m3` stores the caches as E4M3 codes, `--prestep` times plt_decode_attn_step (pre-step kernel +
+attention), `--ablation` adds the L loops as sequential single-loop calls, `--path` / `--loops` / `--hpc` / `--kw` /
+`--stages` / `--cps` select the kernel path, an overridden L and launch variants.
 """
 from __future__ import annotations
 
