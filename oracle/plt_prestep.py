@@ -11,6 +11,9 @@ to be where the attention reads them, and its gate needs the logits of f_gate:
 
 With the convention of the attention oracle (seq_lens counts the current token, loop l sees
 cut_l = max(0, N - delta_l) keys) the token loop l handles in this step has index cut_l - 1 in its stream.
+With caches of E4M3 codes (one fp32 scale per KV head) the new rows arrive in the type of the queries and are
+quantised on the way in: code = round-to-nearest-even of (x / scale) in float32, clamped to the largest finite
+magnitude 448 (the rounding itself is a library cast).
 Plain numpy and Python loops, copies of the inputs, nothing shared with the CUDA path.
 """
 from __future__ import annotations
@@ -25,6 +28,18 @@ def _to_f64(a: np.ndarray) -> np.ndarray:
     if a.dtype == np.uint16:
         return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     return a.astype(np.float64)
+
+
+def quantise_e4m3(x: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """E4M3 codes (uint8) of rows x[..., Hkv, d] (stored values) for per-KV-head scales: float32 division by the
+    scale, clamp to [-448, 448], round to nearest even (torch's float32 -> float8_e4m3fn cast)."""
+    import torch
+
+    xf = _to_f64(x).astype(np.float32)                       # stored values are exact in float32
+    y = xf / scale.astype(np.float32).reshape((1,) * (xf.ndim - 2) + (-1, 1))
+    y = np.clip(y, np.float32(-448.0), np.float32(448.0))
+    t = torch.from_numpy(np.ascontiguousarray(y)).to(torch.float8_e4m3fn)
+    return t.view(torch.uint8).numpy()
 
 
 def gate_logits(q: np.ndarray, w_gate: np.ndarray, b_gate: np.ndarray) -> np.ndarray:
@@ -46,8 +61,10 @@ def prestep(p, k_new: np.ndarray, v_new: np.ndarray, w_gate: np.ndarray, b_gate:
     """Returns (problem after the step's cache updates with the new gate logits stored as float32, logits in float64).
 
     p: the synthetic-input container with the caches as they were BEFORE this step and seq_lens already counting the
-    current token. k_new, v_new: [B, L, Hkv, d] in the storage type of the caches (row l = what loop l+1 produced).
+    current token. k_new, v_new: [B, L, Hkv, d] in the storage type of the queries (row l = what loop l+1 produced).
     """
+    if getattr(p, "kv_dtype", "") == "e4m3":               # rows are quantised with the head's scale on the way in
+        k_new, v_new = quantise_e4m3(k_new, p.k_scale), quantise_e4m3(v_new, p.v_scale)
     kc, vc = p.k_cache.copy(), p.v_cache.copy()
     kw, vw = p.k_win.copy(), p.v_win.copy()
     cuts = p.cuts()                                    # [B, L]

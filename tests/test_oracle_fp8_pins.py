@@ -84,3 +84,42 @@ def test_quantised_problem_stays_close_to_the_unquantised_one():
     assert np.all(q8.k_scale * 448.0 >= kmax * 0.999) and np.all((q8.k_cache & 0x7F) != 0x7F)
     a, b = oracle.decode_attn(raw), oracle.decode_attn(q8)
     assert np.abs(a - b).max() < 0.15 and np.abs(a - b).mean() < 0.02
+
+
+def test_quantisation_of_appended_rows():
+    """Facts of round-to-nearest-even onto the E4M3 grid, with power-of-two scales so that everything is exact."""
+    scale = np.array([0.5, 2.0], dtype=np.float32)
+
+    def q(vals):   # vals: per head a list -> [1, Hkv, d]
+        x = np.array(vals, dtype=np.float32)[None]
+        return oracle.quantise_e4m3(x, scale)[0]
+
+    # representable values come back as their own codes (head 0: x / 0.5; head 1: x / 2)
+    codes = q([[0.5, -0.5, 224.0, 0.0], [2.0, 3.5, -896.0, 2.0 ** -8]])
+    assert list(codes[0]) == [0x38, 0xB8, 0x7E, 0x00] and list(codes[1]) == [0x38, 0x3E, 0xFE, 0x01]
+    # ties go to the even mantissa: 1.0625 -> 1.0 (0x38), 1.1875 -> 1.25 (0x3A); halfway to the smallest subnormal -> 0
+    codes = q([[0.53125, 0.59375, 2.0 ** -11, 3 * 2.0 ** -11], [0, 0, 0, 0]])
+    assert list(codes[0]) == [0x38, 0x3A, 0x00, 0x02]
+    # beyond the largest finite value: clamped, never NaN
+    codes = q([[1e6, -1e6, 225.0, 240.0], [0, 0, 0, 0]])
+    assert list(codes[0]) == [0x7E, 0xFE, 0x7E, 0x7E]
+    # every code value, times the scale, maps back to its own code (negative zero keeps its sign bit)
+    vals = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    ok = np.isfinite(vals)
+    back = oracle.quantise_e4m3((vals[ok] * 0.5).reshape(1, 1, -1).repeat(2, axis=1), scale)[0, 0]
+    assert np.array_equal(back, np.arange(256, dtype=np.uint8)[ok])
+
+
+def test_prestep_on_e4m3_caches_appends_quantised_rows():
+    p = make_problem(spec(lens=("list", [9, 4, 1])))
+    rng = np.random.default_rng(2)
+    from paper_2510_24824_b200.inputs import f32_to_bf16_bits
+    k_new = f32_to_bf16_bits(rng.standard_normal((p.B, p.L, p.Hkv, p.d)).astype(np.float32))
+    v_new = f32_to_bf16_bits(rng.standard_normal((p.B, p.L, p.Hkv, p.d)).astype(np.float32))
+    after, _ = oracle.prestep(p, k_new, v_new, np.zeros((p.Hq, p.d)), np.zeros(p.Hq))
+    want = oracle.quantise_e4m3(k_new, p.k_scale)
+    assert np.array_equal(after.k_cache[0, 8], want[0, 0]) and np.array_equal(after.k_win[0, 0, (9 - 1 - 1) % p.w], want[0, 1])
+    # the stored code is the nearest grid point: dequantised error at most half a grid step of that magnitude
+    deq = torch.from_numpy(after.k_cache[0, 8]).view(torch.float8_e4m3fn).to(torch.float32).numpy() * p.k_scale[:, None]
+    x = bf16_bits_to_f32(k_new[0, 0])
+    assert np.all(np.abs(deq - x) <= np.maximum(np.abs(x) * 2.0 ** -4, p.k_scale[:, None] * 2.0 ** -10) * 1.0001)
