@@ -60,8 +60,8 @@ typedef enum {
                           fp32 scale per KV head for K and one for V: value = code value * scale.  The attention is the
                           same definition on those dequantised values (the paper's efficiency runs use FP8 attention,
                           Sec. 3.2).  Needs dtype = PLT_BF16 and d = 128; q and out stay bf16; softmax and
-                          accumulation stay fp32.  Served by the warp-level kernel; plt_decode_attn_run_host and
-                          plt_decode_attn_step refuse it. */
+                          accumulation stay fp32.  Served by the warp-level kernel; plt_decode_attn_run_host refuses
+                          it; plt_decode_attn_step quantises the rows it appends. */
 } plt_kv_dtype;
 
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
@@ -177,7 +177,9 @@ plt_status plt_decode_attn_run_host(plt_decode_attn_t handle, const plt_decode_a
  */
 typedef struct {
     uint32_t struct_size;
-    const void* k_new;        /* [B, L, Hkv, d], dtype of the caches: row l-1 = keys of the token loop l handles now */
+    const void* k_new;        /* [B, L, Hkv, d], dtype of q: row l-1 = keys of the token loop l handles now.  With
+                                 PLT_KV_E4M3 the rows are stored as round-to-nearest-even codes of x / scale[head]
+                                 (fp32 division, clamped to the largest finite magnitude 448) */
     const void* v_new;        /* [B, L, Hkv, d] */
     const float* w_gate;      /* [Hq, d] fp32 (ignored when L == 1) */
     const float* b_gate;      /* [Hq] fp32 */

@@ -439,7 +439,6 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
     const bool fp8 = h->cfg.kv_dtype == PLT_KV_E4M3;
     const int es = fp8 ? 1 : elem_size(h->bf16);   // element size of the caches and windows
     if (fp8 && (!a->k_scale || !a->v_scale)) return fail(h, PLT_ERR_INVALID_ARG, "k_scale and v_scale must not be NULL with E4M3 caches");
-    if (fp8 && step) return fail(h, PLT_ERR_UNSUPPORTED, "plt_decode_attn_step with E4M3 caches");
     int64_t sb = a->kv_stride_b, sn = a->kv_stride_n, sh = a->kv_stride_h;
     if (sb == 0 && sn == 0 && sh == 0) {
         sh = c.d;

@@ -19,7 +19,27 @@ namespace {
 
 constexpr int kPreThreads = 256;
 
-template <bool BF16>
+// FP8: the caches hold E4M3 codes; the new rows (bf16) are quantised on the way in: code = round to nearest even of
+// x / scale[head] in fp32, clamped to the largest finite magnitude.
+// Eight bf16 values -> eight E4M3 codes for one scale.
+__device__ __forceinline__ uint32_t e4m3x2_from(float lo, float hi) {
+    unsigned short r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint2 quantise8(uint4 v, float scale) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __fdiv_rn(__uint_as_float(w[i] << 16), scale);
+        const float hi = __fdiv_rn(__uint_as_float(w[i] & 0xffff0000u), scale);
+        c[i] = e4m3x2_from(lo, hi);
+    }
+    return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+}
+
+template <bool BF16, bool FP8>
 __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_constant__ Params p, const void* k_new,
                                                                   const void* v_new, const float* w_gate,
                                                                   const float* b_gate, float* gate_out) {
@@ -64,7 +84,8 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
 
     if (cut > 0) {
         // destination rows of this loop's K and V: [Hkv] rows of d elements, kd elements apart
-        T *kd, *vd;
+        using TD = typename std::conditional<FP8, uint8_t, T>::type;   // element of the caches and windows
+        TD *kd, *vd;
         int64_t head_stride;
         if (l == 0) {
             const int pos = cut - 1;
@@ -79,14 +100,14 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
             } else {
                 base = (int64_t)b * p.kv_stride_b + (int64_t)pos * p.kv_stride_n;
             }
-            kd = (T*)p.k_cache + base;
-            vd = (T*)p.v_cache + base;
+            kd = (TD*)p.k_cache + base;
+            vd = (TD*)p.v_cache + base;
             head_stride = p.kv_stride_h;
         } else {
             const int slot = (cut - 1) % p.w;
             const int64_t base = ((((int64_t)b * (p.L - 1) + (l - 1)) * p.w + slot) * p.Hkv) * p.d;
-            kd = (T*)p.k_win + base;
-            vd = (T*)p.v_win + base;
+            kd = (TD*)p.k_win + base;
+            vd = (TD*)p.v_win + base;
             head_stride = p.d;
         }
         const int64_t src = (((int64_t)b * p.L + l) * p.Hkv) * p.d;
@@ -95,8 +116,13 @@ __global__ void __launch_bounds__(kPreThreads) plt_decode_prestep(const __grid_c
             const int h = i / per_row, c = i - h * per_row;
             const uint4 kk = *((const uint4*)((const T*)k_new + src + (int64_t)h * p.d) + c);
             const uint4 vv = *((const uint4*)((const T*)v_new + src + (int64_t)h * p.d) + c);
-            *((uint4*)(kd + h * head_stride) + c) = kk;
-            *((uint4*)(vd + h * head_stride) + c) = vv;
+            if constexpr (FP8) {
+                *((uint2*)(kd + h * head_stride) + c) = quantise8(kk, p.k_scale[h]);
+                *((uint2*)(vd + h * head_stride) + c) = quantise8(vv, p.v_scale[h]);
+            } else {
+                *((uint4*)(kd + h * head_stride) + c) = kk;
+                *((uint4*)(vd + h * head_stride) + c) = vv;
+            }
         }
     }
     if (flags && tid == 0) atomicOr(p.status, flags);
@@ -108,8 +134,9 @@ cudaError_t launch_prestep(const Params& p, bool bf16, const void* k_new, const 
                            const float* b_gate, float* gate_out, cudaStream_t stream) {
     const unsigned grid = (unsigned)(p.B * p.L);
     if (grid == 0) return cudaSuccess;
-    if (bf16) plt_decode_prestep<true><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
-    else plt_decode_prestep<false><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
+    if (p.k_scale != nullptr) plt_decode_prestep<true, true><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
+    else if (bf16) plt_decode_prestep<true, false><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
+    else plt_decode_prestep<false, false><<<grid, kPreThreads, 0, stream>>>(p, k_new, v_new, w_gate, b_gate, gate_out);
     return cudaGetLastError();
 }
 

@@ -74,6 +74,27 @@ def test_one_step(spec):
     check_against_oracle(p, dp, got, *rows, what=spec.get("name", ""))
 
 
+@pytest.mark.parametrize("spec", [
+    custom(kv_dtype="e4m3"),
+    custom(kv_dtype="e4m3", B=6, lens=("list", [0, 1, 2, 3, 41, 80])),
+    custom(kv_dtype="e4m3", B=4, L=4, Hq=16, Hkv=4, w=16, lens=("list", [16, 17, 33, 500])),
+    custom(kv_dtype="e4m3", B=3, page_size=64, lens=("list", [63, 64, 300])),
+], ids=["plain", "short", "ring-edge", "paged"])
+def test_one_step_on_e4m3_caches(spec):
+    """The appended rows are quantised with the head's scale: the codes in the caches must match the oracle's bit for
+    bit (including values beyond the range the scales were made for, which saturate)."""
+    p = make_problem(spec)
+    k_new, v_new, w_gate, b_gate = new_rows(p, 9)
+    from paper_2510_24824_b200.inputs import bf16_bits_to_f32
+    big = bf16_bits_to_f32(k_new)
+    big[0, 0, 0, :4] = [1e4, -1e4, 0.0, 3e-6]          # saturation, zero, a value in the subnormal range of the grid
+    k_new = f32_to_bf16_bits(big)
+    dp = DeviceProblem(p, "cuda:0")
+    with DecodeAttn(p) as op:
+        got = run_step(p, op, dp, k_new, v_new, w_gate, b_gate)
+    check_against_oracle(p, dp, got, k_new, v_new, w_gate, b_gate, what=spec.get("name", ""))
+
+
 @pytest.mark.parametrize("page_size", [16, 64])
 def test_one_step_paged(page_size):
     p = make_problem(shrunk_workload(4, B=9, lens=("list", [1, 2, 3, 63, 64, 255, 700, 129, 16]), page_size=page_size, w=100))
