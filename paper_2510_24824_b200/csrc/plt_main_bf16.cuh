@@ -57,43 +57,13 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     return d;
 }
 
-// One consumer-warp step: this warp's 16 KS keys of a tile against its 8 NT packed rows.
-// Thread (grp = lane / 4, tq = lane % 4) holds of S^T, per 16-key slice ki, the keys grp and grp + 8 and, per 8-row
-// group nt, the rows 2 tq and 2 tq + 1: s[ki][nt][0..1] = key grp, s[ki][nt][2..3] = key grp + 8. lim[nt][j] (keys
-// visible to row 8 nt + 2 tq + j) and nvalid (keys that hold data) count from the first key of the tile and are used
-// only when MASKED. mref[nt][j] is the reference maximum (log2 units; kNoMax while the row has seen no key) the
-// accumulators of that row are scaled to; lacc[nt][j] the row's softmax denominator, accumulated on the tensor cores
-// from exactly the bf16-rounded weights that multiply V.
-template <int D, int NT, int KS, int HPC, int KW, int TKEYS, int BOXB, bool MASKED>
-__device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uint32_t (&qb)[D / 16][NT][2],
-                                             float (&acc)[D / 16][NT][4], float (&mref)[NT][2], float (&lacc)[NT][4],
-                                             const int (&lim)[NT][2], int nvalid, float scale_log2, int lane, int kw,
-                                             int h_local) {
-    const int grp = lane >> 2, tq = lane & 3;
-    const int kbase = kw * 16 * KS;   // first key of this warp in the tile
-    // ---- S^T = K Q^T ---------------------------------------------------------------------------------
-    // Shared-memory rows are 128 bytes (64 elements) with the 16-byte chunks XOR-swizzled by (row & 7); the two
-    // 64-element halves of a 128-wide head are BOXB bytes apart. Chunk (2 k + dhalf) ^ x of a row = base ^ (k << 5).
-    float s[KS][NT][4];
-#pragma unroll
-    for (int ki = 0; ki < KS; ++ki)
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) s[ki][nt][0] = s[ki][nt][1] = s[ki][nt][2] = s[ki][nt][3] = 0.f;
-    {
-        const int key = kbase + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const uint32_t base = sK + (uint32_t)((h_local * TKEYS + key) * 128 + (((lane >> 4) ^ (key & 7)) << 4));
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t addr = (base ^ (uint32_t)((ks & 3) << 5)) + (uint32_t)((ks >> 2) * BOXB);
-#pragma unroll
-            for (int ki = 0; ki < KS; ++ki) {
-                uint32_t a[4];
-                ldmatrix_x4(addr + (uint32_t)(ki * 16 * 128), a[0], a[1], a[2], a[3]);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(s[ki][nt], a, qb[ks][nt][0], qb[ks][nt][1]);
-            }
-        }
-    }
+// The softmax part of a consumer-warp step, shared by the bf16 and the E4M3 kernels: masks (boundary tiles only), the
+// lazily updated reference maxima with the rescale of the accumulators when a score outruns its reference by more than
+// kSlack powers of two, and the probabilities packed (bf16 or, F16, f16) and moved into B-operand layout.
+template <int D, int NT, int KS, bool MASKED, bool F16>
+__device__ __forceinline__ void softmax_slices(float (&s)[KS][NT][4], float (&acc)[D / 16][NT][4], float (&mref)[NT][2],
+                                               float (&lacc)[NT][4], const int (&lim)[NT][2], float scale_log2, int kbase,
+                                               int grp, uint32_t (&pb)[KS][NT][2]) {
     // ---- per-loop causal cutoff / window length (only on boundary tiles) ------------------------------
     if (MASKED) {
 #pragma unroll
@@ -141,7 +111,6 @@ __device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uin
             }
     }
     // ---- probabilities, transposed into the B operand of the second product --------------------------
-    uint32_t pb[KS][NT][2];
 #pragma unroll
     for (int ki = 0; ki < KS; ++ki)
 #pragma unroll
@@ -150,9 +119,50 @@ __device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uin
             const float p1 = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
             const float p2 = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
             const float p3 = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
-            pb[ki][nt][0] = movmatrix_trans(pack_bf16x2(p0, p1));   // keys 0-7 of the slice
-            pb[ki][nt][1] = movmatrix_trans(pack_bf16x2(p2, p3));   // keys 8-15
+            pb[ki][nt][0] = movmatrix_trans((F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1)));   // keys 0-7 of the slice
+            pb[ki][nt][1] = movmatrix_trans((F16 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3)));   // keys 8-15
         }
+}
+
+// One consumer-warp step: this warp's 16 KS keys of a tile against its 8 NT packed rows.
+// Thread (grp = lane / 4, tq = lane % 4) holds of S^T, per 16-key slice ki, the keys grp and grp + 8 and, per 8-row
+// group nt, the rows 2 tq and 2 tq + 1: s[ki][nt][0..1] = key grp, s[ki][nt][2..3] = key grp + 8. lim[nt][j] (keys
+// visible to row 8 nt + 2 tq + j) and nvalid (keys that hold data) count from the first key of the tile and are used
+// only when MASKED. mref[nt][j] is the reference maximum (log2 units; kNoMax while the row has seen no key) the
+// accumulators of that row are scaled to; lacc[nt][j] the row's softmax denominator, accumulated on the tensor cores
+// from exactly the bf16-rounded weights that multiply V.
+template <int D, int NT, int KS, int HPC, int KW, int TKEYS, int BOXB, bool MASKED>
+__device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uint32_t (&qb)[D / 16][NT][2],
+                                             float (&acc)[D / 16][NT][4], float (&mref)[NT][2], float (&lacc)[NT][4],
+                                             const int (&lim)[NT][2], int nvalid, float scale_log2, int lane, int kw,
+                                             int h_local) {
+    const int grp = lane >> 2, tq = lane & 3;
+    const int kbase = kw * 16 * KS;   // first key of this warp in the tile
+    // ---- S^T = K Q^T ---------------------------------------------------------------------------------
+    // Shared-memory rows are 128 bytes (64 elements) with the 16-byte chunks XOR-swizzled by (row & 7); the two
+    // 64-element halves of a 128-wide head are BOXB bytes apart. Chunk (2 k + dhalf) ^ x of a row = base ^ (k << 5).
+    float s[KS][NT][4];
+#pragma unroll
+    for (int ki = 0; ki < KS; ++ki)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) s[ki][nt][0] = s[ki][nt][1] = s[ki][nt][2] = s[ki][nt][3] = 0.f;
+    {
+        const int key = kbase + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const uint32_t base = sK + (uint32_t)((h_local * TKEYS + key) * 128 + (((lane >> 4) ^ (key & 7)) << 4));
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t addr = (base ^ (uint32_t)((ks & 3) << 5)) + (uint32_t)((ks >> 2) * BOXB);
+#pragma unroll
+            for (int ki = 0; ki < KS; ++ki) {
+                uint32_t a[4];
+                ldmatrix_x4(addr + (uint32_t)(ki * 16 * 128), a[0], a[1], a[2], a[3]);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(s[ki][nt], a, qb[ks][nt][0], qb[ks][nt][1]);
+            }
+        }
+    }
+    uint32_t pb[KS][NT][2];
+    softmax_slices<D, NT, KS, MASKED, false>(s, acc, mref, lacc, lim, scale_log2, kbase, grp, pb);
     // ---- O^T += V^T P^T, denominators += 1 P^T --------------------------------------------------------
     {
         const int key = kbase + (lane & 7) + (lane >> 4) * 8;
@@ -235,62 +245,8 @@ __device__ __forceinline__ void process_keys_fp8(uint32_t sK, uint32_t sV, const
             }
         }
     }
-    if (MASKED) {
-#pragma unroll
-        for (int ki = 0; ki < KS; ++ki)
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int kk = kbase + ki * 16 + grp + (e >= 2 ? 8 : 0);
-                    if (kk >= lim[nt][e & 1]) s[ki][nt][e] = -INFINITY;
-                }
-    }
-    bool grow = false;
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
-#pragma unroll
-            for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
-            grow = grow || (fmaf(mx, scale_log2, -mref[nt][j]) > kSlack);
-        }
-    if (__any_sync(0xffffffffu, grow)) {
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                float mx = fmaxf(s[0][nt][j], s[0][nt][2 + j]);
-#pragma unroll
-                for (int ki = 1; ki < KS; ++ki) mx = fmaxf(mx, fmaxf(s[ki][nt][j], s[ki][nt][2 + j]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-                const float m_new = fmaxf(mref[nt][j], mx * scale_log2);
-                const float alpha = fast_exp2(mref[nt][j] - m_new);
-                mref[nt][j] = m_new;
-                lacc[nt][j] *= alpha;
-                lacc[nt][2 + j] *= alpha;
-#pragma unroll
-                for (int mt = 0; mt < D / 16; ++mt) {
-                    acc[mt][nt][j] *= alpha;
-                    acc[mt][nt][2 + j] *= alpha;
-                }
-            }
-    }
     uint32_t pb[KS][NT][2];
-#pragma unroll
-    for (int ki = 0; ki < KS; ++ki)
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const float p0 = fast_exp2(fmaf(s[ki][nt][0], scale_log2, -mref[nt][0]));
-            const float p1 = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
-            const float p2 = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
-            const float p3 = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
-            pb[ki][nt][0] = movmatrix_trans(pack_f16x2(p0, p1));
-            pb[ki][nt][1] = movmatrix_trans(pack_f16x2(p2, p3));
-        }
+    softmax_slices<D, NT, KS, MASKED, true>(s, acc, mref, lacc, lim, scale_log2, kbase, grp, pb);
     {
         const int key = kbase + (lane & 7) + (lane >> 4) * 8;
         const uint32_t base = sV + (uint32_t)((h_local * TKEYS + key) * 128 + ((((lane >> 3) & 1) ^ (key & 7)) << 4));
