@@ -152,7 +152,9 @@ plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_deco
  * Asynchronous: no allocation and no host synchronisation.  Host-visible
  * arguments are validated first and nothing is launched on error.  Two kernels
  * are launched: the split-KV main kernel and the merge/gate kernel.
- * Calls on the same handle must be stream-ordered (they share the workspace).
+ * Calls on the same handle must be stream-ordered (they share the workspace).  Once a first call has seen the
+ * tensor addresses (it encodes the TMA descriptors on the host), calls with the same addresses do no host work
+ * besides the launches and can be captured in a CUDA graph.
  * The main kernel is launched with programmatic stream serialisation: its set-up reads seq_lens and win_lens while
  * the kernel before it in the stream finishes, everything else after that kernel has completed.  A kernel of yours
  * that writes seq_lens or win_lens right before this call must therefore not release its programmatic dependents

@@ -319,3 +319,27 @@ def test_maximum_batch_of_short_sequences(kv):
     """4096 sequences (the largest batch a handle takes) of 0..70 tokens: thousands of items, most blocks hold dozens."""
     p = make_problem(custom(B=4096, L=3, Hq=8, Hkv=2, w=24, lens=("uniform", 0, 70), kv_dtype=kv, seed=3))
     assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", f"B=4096 {kv}")
+
+
+def test_runs_can_be_captured_in_a_cuda_graph():
+    """plt_decode_attn_run allocates nothing and never synchronises: a stream capture records its two launches (with
+    their programmatic dependencies) and replays give the same bits."""
+    p = make_problem(custom(B=6, L=3, Hq=12, Hkv=2, w=40, lens=("list", [3000, 2500, 4000, 3500, 2000, 3900]), max_seq_len=4096))
+    dp = DeviceProblem(p, "cuda:0")
+    with DecodeAttn(p) as op:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            op.run(dp, stream=side.cuda_stream)       # first call encodes the tensor maps (host work, not captured)
+        torch.cuda.synchronize()
+        want = dp.out.clone()
+        dp.out.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(3):
+                op.run(dp, stream=torch.cuda.current_stream().cuda_stream)
+        for _ in range(4):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dp.out, want)
+        assert op.check() == 0
+    assert_parity(want.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "graph")
