@@ -343,3 +343,10 @@ def test_runs_can_be_captured_in_a_cuda_graph():
         assert torch.equal(dp.out, want)
         assert op.check() == 0
     assert_parity(want.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "graph")
+
+
+@pytest.mark.parametrize("kv", ["", "e4m3"])
+def test_one_very_long_sequence(kv):
+    """A single sequence of 131069 tokens: one item split over every block of the grid, merged from hundreds of pieces."""
+    p = make_problem(custom(B=1, L=2, Hq=8, Hkv=2, w=64, lens=("list", [131069]), kv_dtype=kv, seed=9))
+    assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", f"N=131069 {kv}")
