@@ -132,9 +132,15 @@ __device__ __forceinline__ int32_t seq_tiles(const Params& p, int b, uint32_t& f
     return (p.Hkv / p.hpc) * (line_len(p, s.gt) + line_len(p, s.lt));
 }
 
-// Blocks that take part in the plan: never more than there are tiles, so that every taking-part
-// block owns at least one tile and the blocks of one item are consecutive.
-__device__ __forceinline__ int plan_ctas(int64_t T, int launched) { return T < launched ? (int)T : launched; }
+// Blocks that take part in the plan: at least kMinLinePerBlock positions of the line each (so never more blocks than
+// tiles, every taking-part block owns work, and the blocks of one item are consecutive). On small batches fewer,
+// longer pieces are merged faster than many short ones: B=4, N=1024 measured 18.7 -> 13.7 us per step with 8.
+constexpr int kMinLinePerBlock = 8;
+__device__ __forceinline__ int plan_ctas(int64_t T, int launched) {
+    int64_t c = T / kMinLinePerBlock;
+    if (c < 1) c = 1;
+    return c < launched ? (int)c : launched;
+}
 
 // Range of the tile line owned by block c of C: [c*T/C, (c+1)*T/C).
 __device__ __forceinline__ int64_t cta_begin(int64_t T, int c, int C) { return (T * c) / C; }
