@@ -270,6 +270,15 @@ def main():
         run_reference(args, rank)
         return
 
+    from paper_2510_24824_b200 import build as lib_build
+    if not lib_build.LIB.exists():   # fresh checkout: the library is a build product (rank 0 compiles, the others wait)
+        if local_rank == 0:
+            lib_build.build()
+        else:
+            for _ in range(1800):
+                if lib_build.LIB.exists():
+                    break
+                time.sleep(1.0)
     import torch
     import torch.distributed as dist
     from paper_2510_24824_b200 import binding as B
