@@ -14,6 +14,9 @@ cut_l = max(0, N - delta_l) keys) the token loop l handles in this step has inde
 With caches of E4M3 codes (one fp32 scale per KV head) the new rows arrive in the type of the queries and are
 quantised on the way in: code = round-to-nearest-even of (x / scale) in float32, clamped to the largest finite
 magnitude 448 (the rounding itself is a library cast).
+The paper fixes WHICH entries a window keeps, not where they sit: the slot rule and the E4M3 scaling are conventions of
+this library (parity unpinned by the paper for them; pinned against the replay over plain token lists, which does not
+depend on the slot order, and against the format's facts).
 Plain numpy and Python loops, copies of the inputs, nothing shared with the CUDA path.
 """
 from __future__ import annotations
