@@ -345,6 +345,7 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tma_prefetch_desc(&tmKw);
                 tma_prefetch_desc(&tmVw);
             }
+            const uint64_t stream_once = l2_evict_first_policy();
             uint32_t it = 0;
             int stage = 0;
             uint32_t use = 0;  // how many times `stage` has been filled before
@@ -406,9 +407,9 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
 #pragma unroll
                         for (int hf = 0; hf < C::NH; ++hf) {
-                            tma_load_4d(dst + hf * C::BOX_BYTES, mk, &full_bar[stage], hf * 64, c1, head0, c3);
+                            tma_load_4d(dst + hf * C::BOX_BYTES, mk, &full_bar[stage], hf * 64, c1, head0, c3, stream_once);
                             tma_load_4d(dst + C::TENSOR_BYTES + hf * C::BOX_BYTES, mv, &full_bar[stage], hf * 64, c1,
-                                        head0, c3);
+                                        head0, c3, stream_once);
                         }
                     }
                     if (!ok) break;

@@ -470,7 +470,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf)
                         tma_load_4d(dst + hf * kHalfBytes + i * tc.box_keys * 128, map, &full[cur.slot], hf * 64, tc.c1[i],
-                                    tc.head, tc.c3[i]);
+                                    tc.head, tc.c3[i], l2_evict_first_policy());
                 cur.advance(ring);
             }
             s_ctl[is_v ? 3 : 2] = (int32_t)n;
