@@ -294,8 +294,6 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     p = make_problem(replica_spec(args.workload, rank, args.loops, args.kv))
-    if args.kv:
-        args.no_e2e = True   # the host-buffer entry point takes caches stored like q only
     dp = DeviceProblem(p, dev)
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
                   kernel_path=args.path)

@@ -60,8 +60,8 @@ typedef enum {
                           fp32 scale per KV head for K and one for V: value = code value * scale.  The attention is the
                           same definition on those dequantised values (the paper's efficiency runs use FP8 attention,
                           Sec. 3.2).  Needs dtype = PLT_BF16 and d = 128; q and out stay bf16; softmax and
-                          accumulation stay fp32.  Served by the warp-level kernel; plt_decode_attn_run_host refuses
-                          it; plt_decode_attn_step quantises the rows it appends. */
+                          accumulation stay fp32.  Served by the warp-level kernel;
+                          plt_decode_attn_step quantises the rows it appends. */
 } plt_kv_dtype;
 
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */

@@ -64,7 +64,7 @@ struct plt_decode_attn {
     MapKey keys[4];
     bool map_valid[4] = {false, false, false, false};
     // device staging for plt_decode_attn_run_host (grow-only)
-    Staging st[10];
+    Staging st[12];
     cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // optional, caller-owned
     char err[512];
 };
@@ -561,14 +561,15 @@ PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decod
     if (a->batch < 0) return fail(h, PLT_ERR_INVALID_ARG, "batch %d < 0", a->batch);
     if (a->batch > c.max_batch) return fail(h, PLT_ERR_CAPACITY, "batch %d > max_batch %d", a->batch, c.max_batch);
     if (a->batch == 0) return PLT_OK;
-    if (c.kv_dtype == PLT_KV_E4M3) return fail(h, PLT_ERR_UNSUPPORTED, "run_host with E4M3 caches");
     if (a->kv_stride_b || a->kv_stride_n || a->kv_stride_h)
         return fail(h, PLT_ERR_UNSUPPORTED, "run_host takes dense shared caches only (strides must be 0)");
     if (!a->q || !a->k_cache || !a->v_cache || !a->seq_lens || !a->out)
         return fail(h, PLT_ERR_INVALID_ARG, "q, k_cache, v_cache, seq_lens and out must not be NULL");
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const bool fp8 = c.kv_dtype == PLT_KV_E4M3;
+    if (fp8 && (!a->k_scale || !a->v_scale)) return fail(h, PLT_ERR_INVALID_ARG, "k_scale and v_scale must not be NULL with E4M3 caches");
     const size_t es = elem_size(h->bf16), B = (size_t)a->batch;
-    const size_t row = (size_t)c.Hkv * c.d * es;
+    const size_t row = (size_t)c.Hkv * c.d * (fp8 ? 1 : es);   // K (or V) of one token, all KV heads, as stored
     size_t kv_bytes;
     if (c.page_size > 0) {
         if (a->num_pool_pages < 1 || (size_t)a->num_pool_pages > (size_t)c.max_batch * (size_t)(a->max_pages > 0 ? a->max_pages : 0))
@@ -595,6 +596,8 @@ PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decod
     PLT_STAGE(6, v_win, win_bytes)
     PLT_STAGE(7, win_lens, c.L > 1 ? B * (c.L - 1) * 4 : 0)
     PLT_STAGE(8, gate_logits, c.L > 1 ? B * (c.L - 1) * c.Hq * 4 : 0)
+    PLT_STAGE(10, k_scale, fp8 ? (size_t)c.Hkv * 4 : 0)
+    PLT_STAGE(11, v_scale, fp8 ? (size_t)c.Hkv * 4 : 0)
 #undef PLT_STAGE
     Staging& so = h->st[9];
     if (so.bytes < qo_bytes) {

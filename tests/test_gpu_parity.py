@@ -277,9 +277,9 @@ def test_run_argument_errors():
     assert_parity(dp.out.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "after errors")
 
 
-@pytest.mark.parametrize("index", [0, 1, 4])
-def test_host_buffer_entry_point(index):
-    p = make_problem(shrunk_workload(index))
+@pytest.mark.parametrize("index,kv", [(0, ""), (1, ""), (4, ""), (1, "e4m3"), (4, "e4m3")])
+def test_host_buffer_entry_point(index, kv):
+    p = make_problem(shrunk_workload(index, kv_dtype=kv))
     hp = DeviceProblem(p, device=None, pin=True)
     with DecodeAttn(p) as op:
         out = op.run_host(hp)
