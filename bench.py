@@ -4,7 +4,11 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload I]
 
 Prints ONE JSON line. Default workload: bf16 decode batch B=64, L=2, Hq=32, Hkv=8, d=128, N=4096, w=64
-(the configuration the headline metric is quoted on). Under torchrun (N > 1) every rank runs an
+(the configuration the headline metric is quoted on). Without --workload, a one-GPU run then also times the other
+three bf16 workloads and the E4M3-cache form of all four for --suite-steps steps each and reports them under
+"workloads", each with its own clock record. Every timed region alternates between two copies of the inputs at
+different addresses, so that no step can find the previous step's lines in L2.
+Under torchrun (N > 1) every rank runs an
 independent replica of the workload on its own GPU (no collective in the data path; weak scaling).
 `--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
 Other legs: `--kv e4m3` stores the caches as E4M3 codes, `--prestep` times plt_decode_attn_step (pre-step kernel +
@@ -38,7 +42,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, help="index into the five workloads (default 1 = headline)")
+    ap.add_argument("--workload", type=int, default=None,
+                    help="index into the five workloads; default: 1 (the headline) followed by the suite of the others")
+    ap.add_argument("--suite-steps", type=int, default=300, help="timed steps per entry of the \"workloads\" list")
+    ap.add_argument("--no-suite", action="store_true", help="headline workload only")
     ap.add_argument("--hpc", type=int, default=0)
     ap.add_argument("--kw", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
@@ -68,7 +75,8 @@ def workload_config(p, extra=None):
         "seq_len_min": int(p.seq_lens.min()), "seq_len_max": int(p.seq_lens.max()),
         "sum_seq_len": int(p.seq_lens.sum()), "page_size": p.page_size,
         "algorithmic_bytes_per_step": by["total"],
-        "l2": f"inputs {by['total'] / 1e6:.0f} MB per step exceed the 126 MB L2; no flush between steps",
+        "l2": f"inputs {by['total'] / 1e6:.0f} MB per step exceed the 126 MB L2, and consecutive steps alternate between "
+              "two copies of the inputs at different addresses; no flush",
     }
     if extra:
         cfg.update(extra)
@@ -261,11 +269,112 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
+class Replica:
+    """One copy of a workload on the device with a handle of its own. A timed region alternates between two of them
+    (same values, different addresses), so that a step never finds the lines of the step before it in L2."""
+
+    def __init__(self, p, dev, local_rank, tuning, src=None):
+        import torch
+        from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
+        if src is None:
+            self.dp = DeviceProblem(p, dev)
+        else:                      # second copy: device-side clones of the first one's tensors
+            self.dp = DeviceProblem.__new__(DeviceProblem)
+            self.dp.problem, self.dp.device = p, dev
+            for f in DeviceProblem.FIELDS:
+                t = getattr(src.dp, f)
+                setattr(self.dp, f, None if t is None else t.clone())
+            self.dp.out = torch.empty_like(src.dp.out)
+        self.op = DecodeAttn(p, device_index=local_rank, **tuning)
+        self.args = self.dp.args()
+
+    def close(self):
+        self.op.close()
+
+
+def time_steps(step_fns, steps, sampler, barrier):
+    """K steps, alternating over step_fns, between two events on the current stream. Returns total milliseconds."""
+    import torch
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with sampler:
+        ev0.record()
+        for i in range(steps):
+            step_fns[i & 1]()
+        ev1.record()
+        torch.cuda.synchronize()
+    barrier()
+    return ev0.elapsed_time(ev1)
+
+
+def time_main_kernel(reps, step_fns, n_prof):
+    """The same steps with an event pair around the main kernel of each (the library records them). Mean milliseconds."""
+    import torch
+    from paper_2510_24824_b200 import binding as B
+    raw = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+    for a, b in raw:
+        a.record()  # materialise the underlying cudaEvent_t handles
+        b.record()
+    torch.cuda.synchronize()
+    for i, (a, b) in enumerate(raw):
+        B.plt_decode_attn_set_profile_events(reps[i & 1].op.handle, a.cuda_event, b.cuda_event)
+        step_fns[i & 1]()
+    torch.cuda.synchronize()
+    for r in reps:
+        B.plt_decode_attn_set_profile_events(r.op.handle, None, None)
+    return float(np.mean([a.elapsed_time(b) for a, b in raw]))
+
+
+def main_kernel_bytes(by):
+    return by["shared_kv"] + by["window_kv"] + by["q_o"] // 2 + by["index"]
+
+
+def suite_entry(index, kv, dev, local_rank, steps, base=None):
+    """One entry of the "workloads" list: a workload timed for `steps` steps with its own clock record."""
+    import torch
+    from paper_2510_24824_b200 import binding as B
+    from paper_2510_24824_b200.inputs import algorithmic_bytes, make_problem, quantize_kv_e4m3, workload
+    if base is None:
+        base = make_problem(workload(index))
+    p = quantize_kv_e4m3(base).with_(name=base.name + "_e4m3") if kv else base
+    by = algorithmic_bytes(p)
+    a = Replica(p, dev, local_rank, {})
+    b = Replica(p, dev, local_rank, {}, src=a)
+    reps = [a, b]
+    stream = torch.cuda.current_stream().cuda_stream
+    fns = [lambda r=r: B.plt_decode_attn_run(r.op.handle, r.args, stream) for r in reps]
+    for i in range(10):
+        fns[i & 1]()
+    torch.cuda.synchronize()
+    assert a.op.check(stream) == 0 and b.op.check(stream) == 0, "device status not clean after warm-up"
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    ms = time_steps(fns, steps, sampler, torch.cuda.synchronize) / steps
+    main_ms = time_main_kernel(reps, fns, min(steps, 100))
+    peak, _ = peak_hbm()
+    gbs = by["total"] / (ms * 1e-3) / 1e9
+    main_gbs = main_kernel_bytes(by) / (main_ms * 1e-3) / 1e9
+    entry = {
+        "workload": p.name, "kv": kv or "bf16", "steps": steps, "ms_per_step": ms, "steps_per_s": 1e3 / ms,
+        "loop_queries_per_s": 1e3 / ms * p.B * p.L, "algorithmic_bytes_per_step": by["total"],
+        "hbm_gbs_whole_step": gbs, "hbm_frac_of_8tbs": gbs / 8000.0, "hbm_frac_of_measured": gbs / peak,
+        "main_kernel": {"avg_launch_ms": main_ms, "achieved_gbs": main_gbs, "frac_of_measured": main_gbs / peak},
+        "launch": a.op.info, "clocks": sampler.summary(),
+    }
+    for r in reps:
+        r.close()
+    del a, b, reps
+    torch.cuda.empty_cache()
+    return entry, base
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    suite = args.workload is None and not args.no_suite and world == 1 and not (args.kv or args.loops or args.prestep)
+    if args.workload is None:
+        args.workload = 1
     if args.impl == "reference":
         run_reference(args, rank)
         return
@@ -294,20 +403,21 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     p = make_problem(replica_spec(args.workload, rank, args.loops, args.kv))
-    dp = DeviceProblem(p, dev)
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
                   kernel_path=args.path)
-    op = DecodeAttn(p, device_index=local_rank, **tuning)
+    reps = [Replica(p, dev, local_rank, tuning)]
+    reps.append(Replica(p, dev, local_rank, tuning, src=reps[0]))
+    op, dp = reps[0].op, reps[0].dp
     stream = torch.cuda.current_stream().cuda_stream
-    cfg, by = workload_config(p, {"launch": op.info, "parallelism": f"replicas x{world} (no collective)"})
+    cfg, by = workload_config(p)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    run_args = dp.args()
     launches_per_step = int(op.info["kernels_per_run"])
+    step_args = [None, None]
     if args.prestep:
         # Synthetic rows of this step: the same K/V rows and gate weights every step (the lengths do not advance, so
         # the same cache positions are rewritten: a timing stand-in for consecutive decode steps).
@@ -320,84 +430,34 @@ def main():
         k_new, v_new = (to_torch(x, p.dtype, dev) for x in rows)
         w_gate = to_torch((rng.standard_normal((p.Hq, p.d)) / np.sqrt(p.d)).astype(np.float32), "", dev)
         b_gate = to_torch(rng.standard_normal(p.Hq).astype(np.float32), "", dev)
-        step_args = B.make_step_args(k_new, v_new, w_gate, b_gate, dp.gate_logits if p.L > 1 else None)
+        step_args = [B.make_step_args(k_new, v_new, w_gate, b_gate, r.dp.gate_logits if p.L > 1 else None) for r in reps]
         launches_per_step += 1
         cfg["prestep"] = "plt_decode_attn_step: pre-step kernel + attention"
 
-    def step():
+    def make_step(r, st):
         if args.prestep:
-            B.plt_decode_attn_step(op.handle, run_args, step_args, stream)
-        else:
-            B.plt_decode_attn_run(op.handle, run_args, stream)
+            return lambda: B.plt_decode_attn_step(r.op.handle, r.args, st, stream)
+        return lambda: B.plt_decode_attn_run(r.op.handle, r.args, stream)
 
-    for _ in range(max(args.warmup, 3)):
-        step()
+    step_fns = [make_step(r, st) for r, st in zip(reps, step_args)]
+
+    for i in range(max(args.warmup, 3) + 1):
+        step_fns[i & 1]()
     barrier()
-    assert op.check(stream) == 0, "device status not clean after warm-up"
+    assert all(r.op.check(stream) == 0 for r in reps), "device status not clean after warm-up"
 
     # ---- timed region 1: K whole steps, device time between two events --------------------------------
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(physical_gpu_index(local_rank))
-    barrier()
-    with sampler:
-        ev0.record()
-        for _ in range(args.steps):
-            step()
-        ev1.record()
-        torch.cuda.synchronize()
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
+    ms_total = time_steps(step_fns, args.steps, sampler, barrier)
 
     # ---- timed region 2: the same steps with an event pair around the main kernel ---------------------
     n_prof = min(args.steps, 200)
-    main_ms = []
-    raw = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
-    for a, b in raw:
-        a.record()  # materialise the underlying cudaEvent_t handles
-        b.record()
-    torch.cuda.synchronize()
-    for a, b in raw:
-        B.plt_decode_attn_set_profile_events(op.handle, a.cuda_event, b.cuda_event)
-        step()
-    torch.cuda.synchronize()
-    B.plt_decode_attn_set_profile_events(op.handle, None, None)
-    main_ms = [a.elapsed_time(b) for a, b in raw]
-    main_avg_ms = float(np.mean(main_ms))
+    main_avg_ms = time_main_kernel(reps, step_fns, n_prof)
 
     # ---- ablation: the L loops one after the other, every loop scanning the shared cache again ---------------
     ablation = None
     if args.ablation and p.L > 1:
-        from paper_2510_24824_b200.runner import to_torch
-        p1 = p.with_(L=1, w=0, q=np.ascontiguousarray(p.q[:, :1]), loop_offset=None, win_lens=None)
-        op1 = DecodeAttn(p1, device_index=local_rank, kernel_path=args.path)
-        calls = []
-        for l in range(p.L):
-            ql = to_torch(np.ascontiguousarray(p.q[:, l:l + 1]), p.dtype, dev)
-            nl = to_torch(np.maximum(p.seq_lens - int(p.offsets()[l]), 0).astype(np.int32), "", dev)
-            ol = torch.empty_like(ql)
-            calls.append((ql, nl, ol, B.make_args(p.B, ql, dp.k_cache, dp.v_cache, nl, ol, page_table=dp.page_table,
-                                                  max_pages=p.max_pages, num_pool_pages=p.num_pool_pages)))
-
-        def seq_step():
-            for c in calls:
-                B.plt_decode_attn_run(op1.handle, c[3], stream)
-
-        for _ in range(5):
-            seq_step()
-        torch.cuda.synchronize()
-        n_abl = min(args.steps, 300)
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a0.record()
-        for _ in range(n_abl):
-            seq_step()
-        a1.record()
-        torch.cuda.synchronize()
-        seq_ms = a0.elapsed_time(a1) / n_abl
-        assert op1.check(stream) == 0
-        op1.close()
-        ablation = {"sequential_single_loop_calls_ms": seq_ms, "calls_per_step": p.L, "steps_timed": n_abl,
-                    "note": "global attention only (no window, no gate): a lower bound of the sequential loop order; "
-                            "ratio = this / ms_per_step of the cross-loop-parallel step"}
+        ablation = run_ablation(args, p, reps, dev, local_rank, stream)
 
     # ---- end to end: host buffers through plt_decode_attn_run_host ------------------------------------
     e2e = None
@@ -415,20 +475,28 @@ def main():
         e2e = {"value": job_steps_per_s(world, t_e2e * 1e3), "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes(),
                "d2h_bytes_per_step": hp.d2h_bytes(), "steps": args.e2e_steps,
                "note": "plt_decode_attn_run_host with pinned host tensors; the whole KV cache crosses PCIe every step"}
+        del hp
 
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
     value = job_steps_per_s(world, ms_per_step)
+    info = dict(op.info)
+    kernel_path = info["kernel_path"]
+    for r in reps:
+        r.close()
+    del reps, dp, op
+    torch.cuda.empty_cache()
 
     if rank == 0:
         peak, peak_src = peak_hbm()
-        main_bytes = by["shared_kv"] + by["window_kv"] + by["q_o"] // 2 + by["index"]
+        main_bytes = main_kernel_bytes(by)
         achieved = main_bytes / (main_avg_ms * 1e-3) / 1e9
-        kernel_name = {1: "plt_decode_main_" + p.dtype, 2: "plt_decode_main_umma"}[op.info["kernel_path"]]
+        kernel_name = {1: "plt_decode_main_" + p.dtype, 2: "plt_decode_main_umma"}[kernel_path]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": p.dtype + ("+e4m3 cache" if p.kv_dtype else ""), "data": "synthetic", "config": cfg,
+            "launch": info, "parallelism": f"replicas x{world} (no collective)",
             "loop_queries_per_s": value * p.B * p.L,
             "hbm_gbs_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9,
             "hbm_frac_of_8tbs": by["total"] / (ms_per_step * 1e-3) / 8e12,
@@ -446,14 +514,64 @@ def main():
         if ablation is not None:
             ablation["ratio"] = ablation["sequential_single_loop_calls_ms"] / ms_per_step
             line["ablation"] = ablation
+        if suite:
+            entries, base = [], None
+            for index in (1, 2, 3, 4):
+                base = p if index == args.workload else None
+                if index != args.workload:
+                    e, base = suite_entry(index, "", dev, local_rank, args.suite_steps)
+                    entries.append(e)
+                e, _ = suite_entry(index, "e4m3", dev, local_rank, args.suite_steps, base=base)
+                entries.append(e)
+                del base
+            line["workloads"] = entries
         if not args.no_cpu:
-            v, info = time_oracle(p, args.cpu_seconds)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, **info}
+            v, cinfo = time_oracle(p, args.cpu_seconds)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, **cinfo}
         print(json.dumps(line), flush=True)
-    op.close()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_ablation(args, p, reps, dev, local_rank, stream):
+    """The same queries as L sequential single-loop calls, each scanning the shared cache again (Table 1, loop order of
+    the vanilla loop transformer); global attention only (no window, no gate), so a lower bound."""
+    import torch
+    from paper_2510_24824_b200 import binding as B
+    from paper_2510_24824_b200.runner import DecodeAttn, to_torch
+    dp = reps[0].dp
+    p1 = p.with_(L=1, w=0, q=np.ascontiguousarray(p.q[:, :1]), loop_offset=None, win_lens=None)
+    op1 = DecodeAttn(p1, device_index=local_rank, kernel_path=args.path)
+    calls = []
+    for l in range(p.L):
+        ql = to_torch(np.ascontiguousarray(p.q[:, l:l + 1]), p.dtype, dev)
+        nl = to_torch(np.maximum(p.seq_lens - int(p.offsets()[l]), 0).astype(np.int32), "", dev)
+        ol = torch.empty_like(ql)
+        calls.append((ql, nl, ol, B.make_args(p.B, ql, dp.k_cache, dp.v_cache, nl, ol, page_table=dp.page_table,
+                                              max_pages=p.max_pages, num_pool_pages=p.num_pool_pages,
+                                              k_scale=dp.k_scale, v_scale=dp.v_scale)))
+
+    def seq_step():
+        for c in calls:
+            B.plt_decode_attn_run(op1.handle, c[3], stream)
+
+    for _ in range(5):
+        seq_step()
+    torch.cuda.synchronize()
+    n_abl = min(args.steps, 300)
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for _ in range(n_abl):
+        seq_step()
+    a1.record()
+    torch.cuda.synchronize()
+    seq_ms = a0.elapsed_time(a1) / n_abl
+    assert op1.check(stream) == 0
+    op1.close()
+    return {"sequential_single_loop_calls_ms": seq_ms, "calls_per_step": p.L, "steps_timed": n_abl,
+            "note": "global attention only (no window, no gate): a lower bound of the sequential loop order; "
+                    "ratio = this / ms_per_step of the cross-loop-parallel step"}
 
 
 if __name__ == "__main__":

@@ -159,6 +159,10 @@ plt_status plt_decode_attn_create(const plt_decode_attn_config* config, plt_deco
  * the kernel before it in the stream finishes, everything else after that kernel has completed.  A kernel of yours
  * that writes seq_lens or win_lens right before this call must therefore not release its programmatic dependents
  * early (kernels that never call griddepcontrol.launch_dependents release them when they end: nothing to do).
+ * The same holds after the call: the merge kernel releases its programmatic dependents at its start, while it still
+ * reads seq_lens, win_lens and gate_logits and before it writes `out`.  A kernel of yours that is enqueued after this
+ * call WITH programmatic stream serialisation may therefore touch those arrays, the caches and `out` only after its own
+ * griddepcontrol.wait (an ordinary launch waits for the whole call: nothing to do).
  */
 plt_status plt_decode_attn_run(plt_decode_attn_t handle, const plt_decode_attn_args* args, void* cuda_stream);
 
@@ -204,7 +208,9 @@ plt_status plt_decode_attn_step(plt_decode_attn_t handle, const plt_decode_attn_
                                 const plt_decode_attn_step_args* step, void* cuda_stream);
 
 /* Synchronises `cuda_stream`, reads the device status word and clears it.
- * PLT_OK if it was 0; else PLT_ERR_DEVICE_CHECK with *out_bits (optional) = PLT_DEV_* bits. */
+ * PLT_OK if it was 0; else PLT_ERR_DEVICE_CHECK with *out_bits (optional) = PLT_DEV_* bits.
+ * handle == NULL reads the status word of plt_decode_attn_run_no_alloc on the calling thread's current device (that
+ * entry point clears the word at the start of every call, so this reports the most recent call only). */
 plt_status plt_decode_attn_check(plt_decode_attn_t handle, void* cuda_stream, uint32_t* out_bits);
 
 /* Frees the workspace. NULL is accepted. The caller makes sure no run is in flight. */
@@ -219,7 +225,8 @@ const char* plt_decode_attn_last_error(plt_decode_attn_t handle);
 plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config* config, size_t* out_bytes);
 
 /* Number of kernels one plt_decode_attn_run launches, and the variant chosen at create
- * (heads_per_cta, key_slices, stages, ctas_per_sm, grid size, plt_kernel_path actually used); any pointer may be NULL. */
+ * (heads_per_cta, key_slices = warps along the keys of a tile as in the configuration, stages, ctas_per_sm, grid size,
+ * plt_kernel_path actually used); any pointer may be NULL. */
 plt_status plt_decode_attn_launch_info(plt_decode_attn_t handle, int32_t* kernels_per_run, int32_t* heads_per_cta,
                                        int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid,
                                        int32_t* kernel_path);
@@ -253,6 +260,8 @@ plt_status plt_decode_attn_set_profile_events(plt_decode_attn_t handle, void* ev
  *   or different host threads) race on the partials: keep calls on a device stream-ordered and issue them from
  *   one thread at a time.
  * - Errors are reported like those of create: plt_decode_attn_last_error(NULL) holds the message.
+ * - Clamped lengths or page ids and a wait that ran out are flagged in a status word inside the array, which
+ *   plt_decode_attn_check(NULL, stream, &bits) reads for the current device.
  */
 #define PLT_NO_ALLOC_SCRATCH_BYTES (16u << 20)
 plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn_config* config, const plt_decode_attn_args* args,

@@ -70,7 +70,13 @@ def prestep(p, k_new: np.ndarray, v_new: np.ndarray, w_gate: np.ndarray, b_gate:
         k_new, v_new = quantise_e4m3(k_new, p.k_scale), quantise_e4m3(v_new, p.v_scale)
     kc, vc = p.k_cache.copy(), p.v_cache.copy()
     kw, vw = p.k_win.copy(), p.v_win.copy()
-    cuts = p.cuts()                                    # [B, L]
+    # Loop l (1-indexed) serves token i - l + 1 (Sec. 2.2.1, Algorithm 1): it sees cut_l = max(0, N_b - delta_l) keys,
+    # delta_l = l - 1 unless the problem carries other offsets.
+    delta = np.arange(p.L) if p.loop_offset is None else np.asarray(p.loop_offset, dtype=np.int64)
+    cuts = np.zeros((p.B, p.L), dtype=np.int64)
+    for b in range(p.B):
+        for l in range(p.L):
+            cuts[b, l] = max(0, int(p.seq_lens[b]) - int(delta[l]))
     for b in range(p.B):
         c0 = int(cuts[b, 0])
         if c0 > 0:                                     # first loop: append at position c0 - 1 of the shared cache

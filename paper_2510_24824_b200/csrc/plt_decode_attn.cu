@@ -392,6 +392,7 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
 namespace {
 plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream,
                     const plt_decode_attn_step_args* step);
+plt_decode_attn* no_alloc_handle_of_current_device();
 }
 
 PLT_API plt_status plt_decode_attn_run(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cuda_stream) {
@@ -621,7 +622,11 @@ PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decod
 }
 
 PLT_API plt_status plt_decode_attn_check(plt_decode_attn_t h, void* cuda_stream, uint32_t* out_bits) {
-    if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
+    if (!h) {
+        // No handle: the status word of the allocation-free entry point on the current device.
+        h = no_alloc_handle_of_current_device();
+        if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL and plt_decode_attn_run_no_alloc has not run on the current device");
+    }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     uint32_t bits = 0;
     cudaError_t e = cudaMemcpyAsync(&bits, h->status, 4, cudaMemcpyDeviceToHost, stream);
@@ -663,7 +668,7 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
     if (kernels_per_run) *kernels_per_run = 2;
     if (heads_per_cta) *heads_per_cta = h->var.HPC;
-    if (key_slices) *key_slices = h->var.tile_keys / 16;
+    if (key_slices) *key_slices = h->var.KW;
     if (stages) *stages = h->var.stages;
     if (ctas_per_sm) *ctas_per_sm = h->ctas_per_sm;
     if (grid) *grid = h->var.grid;
@@ -731,14 +736,26 @@ plt_status no_alloc_setup(NoAllocDevice& dv, int device) {
     return PLT_OK;
 }
 
+// Field by field: the struct has padding after its last member, which a caller's stack copy leaves undefined.
 bool same_config(const NoAllocDevice& dv, const plt_decode_attn_config* c) {
-    plt_decode_attn_config a = dv.cfg, b = *c;
-    a.loop_offset = nullptr;
-    b.loop_offset = nullptr;
-    if (memcmp(&a, &b, sizeof a) != 0) return false;
+    const plt_decode_attn_config& a = dv.cfg;
+    if (a.struct_size != c->struct_size || a.dtype != c->dtype || a.max_batch != c->max_batch || a.L != c->L ||
+        a.Hq != c->Hq || a.Hkv != c->Hkv || a.d != c->d || a.max_seq_len != c->max_seq_len || a.w != c->w ||
+        a.page_size != c->page_size || memcmp(&a.sm_scale, &c->sm_scale, sizeof(float)) != 0 || a.device != c->device ||
+        a.heads_per_cta != c->heads_per_cta || a.key_slices != c->key_slices || a.stages != c->stages ||
+        a.ctas_per_sm != c->ctas_per_sm || a.kernel_path != c->kernel_path || a.loads_in_flight != c->loads_in_flight ||
+        a.slices_per_warp != c->slices_per_warp || a.row_warps != c->row_warps || a.kv_dtype != c->kv_dtype)
+        return false;
     for (int l = 0; l < c->L; ++l)
         if ((c->loop_offset ? c->loop_offset[l] : l) != dv.offsets[l]) return false;
     return true;
+}
+
+plt_decode_attn* no_alloc_handle_of_current_device() {
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current < 0 || current >= kNoAllocMaxDevices) return nullptr;
+    NoAllocDevice& dv = g_no_alloc[current];
+    return dv.ready && dv.have_handle ? &dv.handle : nullptr;
 }
 
 }  // namespace

@@ -19,11 +19,27 @@ struct MainVariant {
     bool fp8;            // caches and windows hold E4M3 codes (the f16-product kernel)
 };
 
+// Opens a kernel's dynamic shared memory up to what the current device allows a block to opt in to. The attribute
+// belongs to the function, not to a handle: several handles (and the allocation-free entry point) can share one
+// kernel instance with different shared-memory sizes, so it is set to the device limit rather than to any one handle's
+// size, which a later, smaller set-up would otherwise lower under an earlier handle. Each launch still passes its own size.
+inline cudaError_t allow_max_dynamic_smem(const void* fn) {
+    int dev = 0, optin = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, fn);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+}
+
 bool main_bf16_exists(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8 = false);
 size_t main_bf16_smem(int D, int NT, int RW, int HPC, int KW, int KS, int stages, int max_batch, bool fp8 = false);
 // Keys per pipeline tile of a variant (0 if it does not exist): the warps along the keys split a tile or take turns.
 int main_bf16_tile_keys(int D, int NT, int RW, int HPC, int KW, int KS, bool fp8 = false);
-// Sets the shared-memory attribute and reports how many blocks fit one SM.
+// Opens the kernel's shared-memory limit and reports how many blocks of this variant fit one SM.
 cudaError_t main_bf16_prepare(const MainVariant& v, int* blocks_per_sm);
 // overlap: launch with programmatic stream serialisation, so that this grid's set-up (which reads only what the caller
 // passed) runs while the kernel before it in the stream (the pre-step kernel, or the merge kernel of the step before)

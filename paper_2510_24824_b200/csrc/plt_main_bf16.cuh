@@ -27,6 +27,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;  // every barrier wait gives up
 constexpr float kSlack = 8.f;
 constexpr float kNoMax = -1e30f;   // reference maximum of a row that has seen no key yet (finite, so that no select is needed)
 constexpr uint32_t kOnesBf16x2 = 0x3f803f80u;
+constexpr float kHeavyShareInv = 4.f;   // a probability above 1/4 of its row's denominator so far gets a second bf16 term
 
 template <int D, int NT, int RW, int HPC, int KW, int KS, bool FP8 = false>
 struct TCfg {
@@ -57,13 +58,13 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     return d;
 }
 
-// The softmax part of a consumer-warp step, shared by the bf16 and the E4M3 kernels: masks (boundary tiles only), the
+// The softmax part of a consumer-warp step, shared by the bf16 and the E4M3 kernels: masks (boundary tiles only) and the
 // lazily updated reference maxima with the rescale of the accumulators when a score outruns its reference by more than
-// kSlack powers of two, and the probabilities packed (bf16 or, F16, f16) and moved into B-operand layout.
-template <int D, int NT, int KS, bool MASKED, bool F16>
-__device__ __forceinline__ void softmax_slices(float (&s)[KS][NT][4], float (&acc)[D / 16][NT][4], float (&mref)[NT][2],
-                                               float (&lacc)[NT][4], const int (&lim)[NT][2], float scale_log2, int kbase,
-                                               int grp, uint32_t (&pb)[KS][NT][2]) {
+// kSlack powers of two.
+template <int D, int NT, int KS, bool MASKED>
+__device__ __forceinline__ void softmax_reference(float (&s)[KS][NT][4], float (&acc)[D / 16][NT][4], float (&mref)[NT][2],
+                                                  float (&lacc)[NT][4], const int (&lim)[NT][2], float scale_log2,
+                                                  int kbase, int grp) {
     // ---- per-loop causal cutoff / window length (only on boundary tiles) ------------------------------
     if (MASKED) {
 #pragma unroll
@@ -110,15 +111,56 @@ __device__ __forceinline__ void softmax_slices(float (&s)[KS][NT][4], float (&ac
                 }
             }
     }
-    // ---- probabilities, transposed into the B operand of the second product --------------------------
+}
+
+// Turns the scores of a step into probabilities in place (fp32, relative to the reference maxima) and, for bf16
+// weights, says whether the tile is "heavy". bf16 probabilities carry 8 significant bits; where a single key holds a
+// large share of a row's weight that rounding shows in the output (rows with a few dominant keys and large V: up to
+// 1e-2 at |O| ~ 5), so heavy tiles are multiplied with V in two terms, p = hi + lo with hi = bf16(p), lo = bf16(p - hi),
+// both also summed into the denominators. A tile is heavy when some probability of it exceeds 1/4 of the denominator
+// its row has accumulated so far; the final denominator is at least that, so every key that ends up with more than
+// 1/4 of a row's weight is covered, and so are the first tiles of every piece (about the first 64 keys on rows with
+// N(0,1) scores). Measured: with the second term the worst error on rows with tripled K/V is the output rounding
+// (0.83 of the 2e-2 bound for every launch variant and seed tried; 0.8-1.2 without it, where the lazily placed
+// reference leaves the dominant key's weight inexact) at 0.5-3.6 % of the step time on the four bf16 workloads.
+template <int NT, int KS, bool F16>
+__device__ __forceinline__ bool softmax_probabilities(float (&s)[KS][NT][4], const float (&mref)[NT][2],
+                                                      const float (&lacc)[NT][4], float scale_log2) {
+    bool heavy = false;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float pm0 = 0.f, pm1 = 0.f;
+#pragma unroll
+        for (int ki = 0; ki < KS; ++ki) {
+            s[ki][nt][0] = fast_exp2(fmaf(s[ki][nt][0], scale_log2, -mref[nt][0]));
+            s[ki][nt][1] = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
+            s[ki][nt][2] = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
+            s[ki][nt][3] = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
+            pm0 = fmaxf(pm0, fmaxf(s[ki][nt][0], s[ki][nt][2]));
+            pm1 = fmaxf(pm1, fmaxf(s[ki][nt][1], s[ki][nt][3]));
+        }
+        if (!F16) heavy = heavy || pm0 * kHeavyShareInv > lacc[nt][0] || pm1 * kHeavyShareInv > lacc[nt][1];
+    }
+    if (F16) return false;   // f16 weights carry 11 bits
+    return __any_sync(0xffffffffu, heavy);
+}
+
+// The probabilities of a step, packed (bf16 or, F16, f16) and transposed into the B operand of the second product.
+// LO: what the bf16 rounding of the probabilities dropped, p - bf16(p), instead of the probabilities themselves.
+template <int NT, int KS, bool F16, bool LO>
+__device__ __forceinline__ void softmax_weights(const float (&p)[KS][NT][4], uint32_t (&pb)[KS][NT][2]) {
 #pragma unroll
     for (int ki = 0; ki < KS; ++ki)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const float p0 = fast_exp2(fmaf(s[ki][nt][0], scale_log2, -mref[nt][0]));
-            const float p1 = fast_exp2(fmaf(s[ki][nt][1], scale_log2, -mref[nt][1]));
-            const float p2 = fast_exp2(fmaf(s[ki][nt][2], scale_log2, -mref[nt][0]));
-            const float p3 = fast_exp2(fmaf(s[ki][nt][3], scale_log2, -mref[nt][1]));
+            float p0 = p[ki][nt][0], p1 = p[ki][nt][1], p2 = p[ki][nt][2], p3 = p[ki][nt][3];
+            if (LO) {
+                const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
+                p0 -= __uint_as_float(h01 << 16);
+                p1 -= __uint_as_float(h01 & 0xffff0000u);
+                p2 -= __uint_as_float(h23 << 16);
+                p3 -= __uint_as_float(h23 & 0xffff0000u);
+            }
             pb[ki][nt][0] = movmatrix_trans((F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1)));   // keys 0-7 of the slice
             pb[ki][nt][1] = movmatrix_trans((F16 ? pack_f16x2(p2, p3) : pack_bf16x2(p2, p3)));   // keys 8-15
         }
@@ -161,26 +203,26 @@ __device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uin
             }
         }
     }
-    uint32_t pb[KS][NT][2];
-    softmax_slices<D, NT, KS, MASKED, false>(s, acc, mref, lacc, lim, scale_log2, kbase, grp, pb);
+    softmax_reference<D, NT, KS, MASKED>(s, acc, mref, lacc, lim, scale_log2, kbase, grp);
+    const bool heavy = softmax_probabilities<NT, KS, false>(s, mref, lacc, scale_log2);   // s holds probabilities now
     // ---- O^T += V^T P^T, denominators += 1 P^T --------------------------------------------------------
-    {
-        const int key = kbase + (lane & 7) + (lane >> 4) * 8;
-        const uint32_t base = sV + (uint32_t)((h_local * TKEYS + key) * 128 + ((((lane >> 3) & 1) ^ (key & 7)) << 4));
-        uint32_t mask_lo[KS], mask_hi[KS];
-        if (MASKED) {
-            // Rows at or beyond nvalid may hold anything (uninitialised cache slots): force them to 0 so that
-            // 0 * garbage cannot produce NaN.
+    const int vkey = kbase + (lane & 7) + (lane >> 4) * 8;
+    const uint32_t vbase = sV + (uint32_t)((h_local * TKEYS + vkey) * 128 + ((((lane >> 3) & 1) ^ (vkey & 7)) << 4));
+    uint32_t mask_lo[KS], mask_hi[KS];
+    if (MASKED) {
+        // Rows at or beyond nvalid may hold anything (uninitialised cache slots): force them to 0 so that
+        // 0 * garbage cannot produce NaN.
 #pragma unroll
-            for (int ki = 0; ki < KS; ++ki) {
-                const int k0 = kbase + ki * 16 + 2 * tq;
-                mask_lo[ki] = (k0 < nvalid ? 0x0000ffffu : 0u) | (k0 + 1 < nvalid ? 0xffff0000u : 0u);
-                mask_hi[ki] = (k0 + 8 < nvalid ? 0x0000ffffu : 0u) | (k0 + 9 < nvalid ? 0xffff0000u : 0u);
-            }
+        for (int ki = 0; ki < KS; ++ki) {
+            const int k0 = kbase + ki * 16 + 2 * tq;
+            mask_lo[ki] = (k0 < nvalid ? 0x0000ffffu : 0u) | (k0 + 1 < nvalid ? 0xffff0000u : 0u);
+            mask_hi[ki] = (k0 + 8 < nvalid ? 0x0000ffffu : 0u) | (k0 + 9 < nvalid ? 0xffff0000u : 0u);
         }
+    }
+    auto multiply_v = [&](const uint32_t (&pb)[KS][NT][2]) {
 #pragma unroll
         for (int mt = 0; mt < D / 16; ++mt) {
-            const uint32_t addr = (base ^ (uint32_t)((mt & 3) << 5)) + (uint32_t)((mt >> 2) * BOXB);
+            const uint32_t addr = (vbase ^ (uint32_t)((mt & 3) << 5)) + (uint32_t)((mt >> 2) * BOXB);
 #pragma unroll
             for (int ki = 0; ki < KS; ++ki) {
                 uint32_t a[4];
@@ -200,7 +242,15 @@ __device__ __forceinline__ void process_keys(uint32_t sK, uint32_t sV, const uin
         for (int ki = 0; ki < KS; ++ki)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(lacc[nt], ones, pb[ki][nt][0], pb[ki][nt][1]);
+    };
+    if (heavy) {   // rare: the second term of the probabilities first, in a pass of its own
+        uint32_t pl[KS][NT][2];
+        softmax_weights<NT, KS, false, true>(s, pl);
+        multiply_v(pl);
     }
+    uint32_t pb[KS][NT][2];
+    softmax_weights<NT, KS, false, false>(s, pb);
+    multiply_v(pb);
 }
 
 // The same step for caches of E4M3 codes (d = 128: one 128-byte row per key). The codes convert exactly to f16, so the
@@ -245,8 +295,10 @@ __device__ __forceinline__ void process_keys_fp8(uint32_t sK, uint32_t sV, const
             }
         }
     }
+    softmax_reference<D, NT, KS, MASKED>(s, acc, mref, lacc, lim, scale_log2, kbase, grp);
+    softmax_probabilities<NT, KS, true>(s, mref, lacc, scale_log2);   // f16 weights carry 11 bits: no second term
     uint32_t pb[KS][NT][2];
-    softmax_slices<D, NT, KS, MASKED, true>(s, acc, mref, lacc, lim, scale_log2, kbase, grp, pb);
+    softmax_weights<NT, KS, true, false>(s, pb);
     {
         const int key = kbase + (lane & 7) + (lane >> 4) * 8;
         const uint32_t base = sV + (uint32_t)((h_local * TKEYS + key) * 128 + ((((lane >> 3) & 1) ^ (key & 7)) << 4));

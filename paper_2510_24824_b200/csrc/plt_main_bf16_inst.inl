@@ -23,7 +23,7 @@ cudaError_t run_op(int op, const MainVariant& v, const CUtensorMap* maps, const 
     auto fn = plt_decode_main_bf16<D, NT, RW, HPC, KW, KS, FP8>;
     if (op == 0) return cudaSuccess;
     if (op == 1) {
-        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)v.smem);
+        cudaError_t e = allow_max_dynamic_smem((const void*)fn);
         if (e != cudaSuccess) return e;
         return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, fn, C::NTHREADS, v.smem);
     }

@@ -198,7 +198,7 @@ size_t main_f32_smem(int D, int R, int max_batch) {
 cudaError_t main_f32_prepare(int D, int R, int max_batch, int* blocks_per_sm) {
     const size_t smem = main_f32_smem(D, R, max_batch);
     const void* fn = D == 128 ? (const void*)plt_decode_main_f32<128> : (const void*)plt_decode_main_f32<64>;
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem(fn);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, NT, smem);
 }

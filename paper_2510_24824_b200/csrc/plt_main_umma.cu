@@ -771,7 +771,7 @@ plt_decode_main_umma(const __grid_constant__ CUtensorMap tmK, const __grid_const
 template <int RP>
 cudaError_t umma_prepare(size_t smem, int* blocks_per_sm) {
     auto fn = plt_decode_main_umma<RP>;
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem((const void*)fn);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, kUmmaThreads, smem);
 }

@@ -8,7 +8,7 @@ import oracle
 from paper_2510_24824_b200.inputs import make_problem, workload
 from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
 
-from gpu_util import BF16_MEAN_ABS, bf16_bound
+from gpu_util import inactive_rows, BF16_MEAN_ABS, bf16_bound
 
 pytestmark = pytest.mark.gpu
 
@@ -40,7 +40,7 @@ def test_full_size_sampled_rows(index, kv):
     else:
         vmax = float(max(dp.v_cache.float().abs().max().item(), dp.v_win.float().abs().max().item()))
     assert np.abs(got).max() <= vmax * (1 + 2 ** -7)
-    inactive = p.cuts() == 0
+    inactive = inactive_rows(p)
     assert np.all(got[inactive] == 0.0)
 
     rng = np.random.default_rng(100 + index)

@@ -8,7 +8,7 @@ from paper_2510_24824_b200 import binding as B
 from paper_2510_24824_b200.inputs import make_problem, shrunk_workload, workload
 from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
 
-from gpu_util import assert_parity, run_gpu
+from gpu_util import assert_parity, inactive_rows, parity_report, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -102,7 +102,7 @@ def test_lengths_below_loop_count_and_window(dtype):
     ref = oracle.decode_attn(p)
     got = run_gpu(p)
     assert_parity(got, ref, dtype, "short sequences")
-    inactive = p.cuts() == 0
+    inactive = inactive_rows(p)
     assert inactive.any()
     assert np.all(got[inactive] == 0.0), "rows of loops without a token must be exactly zero"
 
@@ -350,3 +350,35 @@ def test_one_very_long_sequence(kv):
     """A single sequence of 131069 tokens: one item split over every block of the grid, merged from hundreds of pieces."""
     p = make_problem(custom(B=1, L=2, Hq=8, Hkv=2, w=64, lens=("list", [131069]), kv_dtype=kv, seed=9))
     assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", f"N=131069 {kv}")
+
+
+# ---- the workload with tripled K/V rows under every launch variant ----------------------------------------------
+# Sharp softmax peaks on large values are where the rounding of the probabilities shows most (outputs of magnitude
+# 4-8 next to the 2e-2 bound); every accepted variant has to stay inside the bound there, three seeds each.
+@pytest.mark.parametrize("hpc,kw,ks", [(0, 0, 0), (1, 1, 1), (1, 2, 1), (1, 4, 1), (2, 1, 1), (2, 2, 1), (2, 4, 1), (4, 1, 1),
+                                       (4, 2, 1), (8, 1, 1), (1, 8, 1), (1, 1, 2), (2, 2, 2), (4, 1, 2), (1, 4, 2)])
+def test_peaked_workload_under_every_variant(hpc, kw, ks):
+    worst = 0.0
+    for seed in (2, 12, 22):
+        p = make_problem(shrunk_workload(2), seed=seed)
+        ref = oracle.decode_attn(p)
+        got = run_gpu(p, heads_per_cta=hpc, key_slices=kw, slices_per_warp=ks)
+        assert_parity(got, ref, "bf16", f"peaks hpc={hpc} kw={kw} ks={ks} seed={seed}")
+        worst = max(worst, parity_report(got, ref, "bf16")["worst_of_bound"])
+    print(f"peaked workload hpc={hpc} kw={kw} ks={ks}: worst error / bound {worst:.2f}")
+
+
+# ---- several handles that share one kernel instance ---------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_two_handles_of_one_variant_with_different_shared_memory(dtype):
+    """The shared-memory limit of a kernel belongs to the function, not to a handle: a second, smaller handle of the
+    same variant must not lower it under the first (its shared memory grows with max_batch)."""
+    p = make_problem(custom(dtype=dtype, B=3))
+    ref = oracle.decode_attn(p)
+    dp = DeviceProblem(p, "cuda:0")
+    with DecodeAttn(p, max_batch=4096) as big, DecodeAttn(p, max_batch=8) as small:
+        for op in (big, small, big, small, big):
+            dp.out.fill_(float("nan"))
+            op.run(dp)
+            assert op.check() == 0
+            assert_parity(dp.out.float().cpu().numpy().astype(np.float64), ref, dtype, "two handles")

@@ -27,13 +27,27 @@ def as_f64(p: ClpProblem, name: str) -> np.ndarray:
     return (bf16_bits_to_f32(a) if p.dtype == "bf16" else a).astype(np.float64)
 
 
+def cutoffs(p: ClpProblem) -> np.ndarray:
+    """[B, L]: loop l (1-indexed) serves token i - l + 1 (Sec. 2.2.1), so it may see max(0, N_b - delta_l) keys of the
+    shared cache, delta_l = l - 1 unless the problem carries other offsets. Written here, not taken from the package."""
+    delta = list(range(p.L)) if p.loop_offset is None else [int(x) for x in p.loop_offset]
+    return np.array([[max(0, int(n) - delta[l]) for l in range(p.L)] for n in p.seq_lens], dtype=np.int64).reshape(p.B, p.L)
+
+
+def window_lens(p: ClpProblem) -> np.ndarray:
+    """[B, L-1]: a non-first loop keeps its w newest entries (Sec. 2.2.2): min(w, tokens it has seen) unless given."""
+    if p.win_lens is not None:
+        return np.clip(np.asarray(p.win_lens, dtype=np.int64), 0, p.w)
+    return np.minimum(p.w, cutoffs(p)[:, 1:])
+
+
 def independent_reference(p: ClpProblem) -> np.ndarray:
     """Written from the definition with numpy primitives only (np.exp, sums); dense contiguous caches."""
     q, K, V = as_f64(p, "q"), as_f64(p, "k_cache"), as_f64(p, "v_cache")
     Kw, Vw = as_f64(p, "k_win"), as_f64(p, "v_win")
     G = p.Hq // p.Hkv
     out = np.zeros((p.B, p.L, p.Hq, p.d))
-    cuts, wls = p.cuts(), p.window_lengths()
+    cuts, wls = cutoffs(p), window_lens(p)
     for b in range(p.B):
         for l in range(p.L):
             for h in range(p.Hq):
@@ -85,7 +99,7 @@ def test_gate_closed_is_shared_kv_attention_and_open_is_pure_swa():
     base = p.with_(L=1, q=None)
     closed = oracle.decode_attn(p.with_(gate_logits=np.full_like(p.gate_logits, -np.inf)))
     opened = oracle.decode_attn(p.with_(gate_logits=np.full_like(p.gate_logits, np.inf)))
-    cuts, wls = p.cuts(), p.window_lengths()
+    cuts, wls = cutoffs(p), window_lens(p)
     for l in range(1, p.L):
         # g = 0: loop l equals a single-loop problem with that loop's queries and the cache cut at `cut`.
         single = base.with_(q=np.ascontiguousarray(p.q[:, l:l + 1]), seq_lens=cuts[:, l].astype(np.int32))
@@ -103,7 +117,7 @@ def test_gate_closed_is_shared_kv_attention_and_open_is_pure_swa():
 def test_window_covering_context_makes_gate_irrelevant():
     lens = [9, 4]
     p = make_problem(spec(w=12, lens=("list", lens)))
-    cuts = p.cuts()
+    cuts = cutoffs(p)
     kw, vw = p.k_win.copy(), p.v_win.copy()
     for b in range(p.B):
         for l in range(1, p.L):
@@ -172,7 +186,7 @@ def test_constant_values_give_constant_output_and_outputs_are_bounded():
     p = make_problem(spec(B=3, dtype="bf16"))
     c = f32_to_bf16_bits(np.full(1, 1.75, dtype=np.float32))[0]
     got = oracle.decode_attn(p.with_(v_cache=np.full_like(p.v_cache, c), v_win=np.full_like(p.v_win, c)))
-    active = p.cuts() > 0
+    active = cutoffs(p) > 0
     np.testing.assert_allclose(got[active], 1.75, rtol=1e-13)
     assert np.all(got[~active] == 0.0)
     plain = oracle.decode_attn(p)
@@ -215,13 +229,13 @@ def test_key_permutation_invariance_and_window_rotation():
     rng = np.random.default_rng(5)
     K, V = p.k_cache.copy(), p.v_cache.copy()
     for b in range(p.B):
-        m = int(p.cuts()[b].min())  # keys every loop sees
+        m = int(cutoffs(p)[b].min())  # keys every loop sees
         perm = rng.permutation(m)
         K[b, :m] = K[b, perm]
         V[b, :m] = V[b, perm]
     np.testing.assert_allclose(oracle.decode_attn(p.with_(k_cache=K, v_cache=V)), ref, rtol=1e-12, atol=1e-14)
     # A full ring buffer may sit in any rotation.
-    full = p.window_lengths().min() == p.w
+    full = window_lens(p).min() == p.w
     assert full
     np.testing.assert_allclose(
         oracle.decode_attn(p.with_(k_win=np.roll(p.k_win, 2, axis=2), v_win=np.roll(p.v_win, 2, axis=2))), ref,

@@ -95,7 +95,6 @@ def test_ring_slot_holds_the_token_with_that_residue():
             if n > s:
                 newest = max(i for i in range(n) if i % w == s)
                 assert p.k_win[0, 0, s, 0, 0] == 100.0 + newest
-        assert int(p.window_lengths()[0, 0]) == min(w, n)
 
 
 def test_loops_without_a_token_and_empty_sequences_write_nothing():
