@@ -3,6 +3,9 @@
 This module only draws random numbers, lays them out and converts storage
 types.  It contains none of the attention arithmetic and is the one piece of
 code that both the tests' CPU oracle and the CUDA binding are fed from.
+The two length helpers of the container (``cuts``, ``window_lengths``) serve the
+byte model (``algorithmic_bytes``) and the generator's tail fill only: neither the
+kernels nor the oracle nor the oracle's pins take their cutoffs from here.
 
 Recipe: numpy ``default_rng(seed)``, draw order fixed: ``Q, lens, page permutation,
 Kwin, Vwin, gate``; the shared cache of sequence ``b`` comes from its own stream
@@ -31,6 +34,9 @@ __all__ = [
     "f32_to_bf16_bits",
     "bf16_bits_to_f32",
     "algorithmic_bytes",
+    "SeqProblem",
+    "make_seq_problem",
+    "seq_attn_flops",
 ]
 
 
@@ -321,3 +327,66 @@ def quantize_kv_e4m3(p: ClpProblem) -> ClpProblem:
     return replace(p, kv_dtype="e4m3", k_scale=k_scale.astype(np.float32), v_scale=v_scale.astype(np.float32),
                    k_cache=codes(p.k_cache, k_scale), v_cache=codes(p.v_cache, v_scale),
                    k_win=codes(p.k_win, k_scale), v_win=codes(p.v_win, v_scale))
+
+
+# ---- sequence-shaped problems (prefill / training-forward attention) --------------------------------------------
+@dataclass
+class SeqProblem:
+    """Inputs of the sequence-shaped PLT attention, host side: every decode step of a sequence at once. Arrays hold
+    bf16 bit patterns (uint16); T is the padded length, seq_lens the true ones."""
+
+    name: str
+    B: int
+    L: int
+    T: int
+    Hq: int
+    Hkv: int
+    d: int
+    w: int
+    q: np.ndarray            # [B, L, T, Hq, d]
+    k_share: np.ndarray      # [B, T, Hkv, d]  first-loop keys (shared by every loop)
+    v_share: np.ndarray
+    k_loc: np.ndarray        # [B, max(L-1,1), T, Hkv, d]  own keys of loops 2..L
+    v_loc: np.ndarray
+    gate_logits: np.ndarray  # [B, max(L-1,1), T, Hq] float32, pre-sigmoid
+    seq_lens: np.ndarray     # [B] int32
+    loop_offset: Optional[np.ndarray] = None
+    sm_scale: float = 0.0
+    dtype: str = "bf16"
+
+    def with_(self, **kw) -> "SeqProblem":
+        return replace(self, **kw)
+
+
+def make_seq_problem(B: int, L: int, T: int, Hq: int, Hkv: int, d: int, w: int, lens=None, seed: int = 0,
+                     gate_std: float = 1.0, loop_offset=None, name: str = "seq", sm_scale: float = 0.0) -> SeqProblem:
+    """Seeded N(0,1) values rounded to bf16; draw order q, k_share, v_share, k_loc, v_loc, gate. The shapes follow the
+    paper's serving recipe (prefill 5000, batch 4-64, GQA 32/8, d = 128, w = 64, L in {2, 3})."""
+    rng = np.random.default_rng([seed, 7])
+    Lm = max(L - 1, 1)
+    draw = lambda *shape: f32_to_bf16_bits(rng.standard_normal(shape, dtype=np.float32))
+    q = draw(B, L, T, Hq, d)
+    k_share, v_share = draw(B, T, Hkv, d), draw(B, T, Hkv, d)
+    k_loc, v_loc = draw(B, Lm, T, Hkv, d), draw(B, Lm, T, Hkv, d)
+    gate = (rng.standard_normal((B, Lm, T, Hq), dtype=np.float32) * np.float32(gate_std)).astype(np.float32)
+    seq_lens = np.full(B, T, dtype=np.int32) if lens is None else np.asarray(lens, dtype=np.int32)
+    assert seq_lens.shape == (B,) and int(seq_lens.max(initial=0)) <= T
+    return SeqProblem(name=name, B=B, L=L, T=T, Hq=Hq, Hkv=Hkv, d=d, w=w, q=q, k_share=k_share, v_share=v_share,
+                      k_loc=k_loc, v_loc=v_loc, gate_logits=gate, seq_lens=seq_lens,
+                      loop_offset=None if loop_offset is None else np.asarray(loop_offset, dtype=np.int32),
+                      sm_scale=sm_scale)
+
+
+def seq_attn_flops(p: SeqProblem) -> int:
+    """Multiply-adds x 2 of the two products over the key sets the definition names (masked-out keys not counted)."""
+    delta = np.arange(p.L) if p.loop_offset is None else np.asarray(p.loop_offset, dtype=np.int64)
+    total = 0
+    for n in p.seq_lens.astype(np.int64):
+        t = np.arange(int(n), dtype=np.int64)
+        for l in range(p.L):
+            cut = np.maximum(0, t + 1 - delta[l])
+            keys = int(cut.sum())
+            if l > 0:
+                keys += int(np.where(cut > 0, np.minimum(cut, p.w), 0).sum())
+            total += keys * p.Hq * p.d * 4
+    return int(total)
