@@ -25,6 +25,7 @@ EXPORTS = (
     "plt_decode_attn_destroy", "plt_decode_attn_last_error", "plt_decode_attn_workspace_bytes",
     "plt_decode_attn_launch_info", "plt_decode_attn_set_profile_events", "plt_decode_attn_run_no_alloc",
     "plt_decode_attn_step",
+    "plt_seq_attn_create", "plt_seq_attn_run", "plt_seq_attn_check", "plt_seq_attn_destroy", "plt_seq_attn_last_error",
 )
 PLT_NO_ALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -69,6 +70,23 @@ class StepArgs(ctypes.Structure):
     ]
 
 
+class SeqConfig(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("max_batch", ctypes.c_int32), ("L", ctypes.c_int32), ("Hq", ctypes.c_int32),
+        ("Hkv", ctypes.c_int32), ("d", ctypes.c_int32), ("max_seq_len", ctypes.c_int32), ("w", ctypes.c_int32),
+        ("sm_scale", ctypes.c_float), ("device", ctypes.c_int32), ("loop_offset", ctypes.POINTER(ctypes.c_int32)),
+    ]
+
+
+class SeqArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("batch", ctypes.c_int32), ("q", ctypes.c_void_p),
+        ("k_share", ctypes.c_void_p), ("v_share", ctypes.c_void_p), ("k_loc", ctypes.c_void_p),
+        ("v_loc", ctypes.c_void_p), ("gate_logits", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p),
+        ("out", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -93,8 +111,14 @@ def load_library() -> ctypes.CDLL:
         lib.plt_decode_attn_launch_info.argtypes = [h, i32p, i32p, i32p, i32p, i32p, i32p, i32p]
         lib.plt_decode_attn_set_profile_events.argtypes = [h, ctypes.c_void_p, ctypes.c_void_p]
         lib.plt_decode_attn_run_no_alloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Args), ctypes.c_void_p]
+        lib.plt_seq_attn_create.argtypes = [ctypes.POINTER(SeqConfig), ctypes.POINTER(h)]
+        lib.plt_seq_attn_run.argtypes = [h, ctypes.POINTER(SeqArgs), ctypes.c_void_p]
+        lib.plt_seq_attn_check.argtypes = [h, ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        lib.plt_seq_attn_destroy.argtypes = [h]
+        lib.plt_seq_attn_last_error.argtypes = [h]
+        lib.plt_seq_attn_last_error.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name != "plt_decode_attn_last_error":
+            if not name.endswith("_last_error"):
                 getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -235,3 +259,60 @@ def plt_decode_attn_run_no_alloc(config: Config, args: Args, stream: int = 0) ->
     st = load_library().plt_decode_attn_run_no_alloc(ctypes.byref(config), ctypes.byref(args), ctypes.c_void_p(stream))
     if st != PLT_OK:
         _raise(st, None)
+
+
+# ---- sequence-shaped attention (plt_seq_attn.h) -------------------------------------------------------------------
+def _raise_seq(status: int, handle) -> None:
+    msg = load_library().plt_seq_attn_last_error(handle)
+    raise PltError(status, msg.decode() if msg else "")
+
+
+def make_seq_config(max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_seq_len: int, w: int, sm_scale: float = 0.0,
+                    device: int = 0, loop_offset: Optional[Sequence[int]] = None) -> SeqConfig:
+    c = SeqConfig()
+    c.struct_size = ctypes.sizeof(SeqConfig)
+    c.max_batch, c.L, c.Hq, c.Hkv, c.d, c.max_seq_len, c.w = max_batch, L, Hq, Hkv, d, max_seq_len, w
+    c.sm_scale, c.device = sm_scale, device
+    if loop_offset is not None:
+        arr = (ctypes.c_int32 * len(loop_offset))(*[int(x) for x in loop_offset])
+        c._keep = arr
+        c.loop_offset = ctypes.cast(arr, ctypes.POINTER(ctypes.c_int32))
+    return c
+
+
+def make_seq_args(batch: int, q, k_share, v_share, seq_lens, out, k_loc=None, v_loc=None, gate_logits=None) -> SeqArgs:
+    """Tensors are anything with data_ptr() (device memory); None becomes NULL."""
+    a = SeqArgs()
+    a.struct_size = ctypes.sizeof(SeqArgs)
+    a.batch = batch
+    ptr = lambda t: None if t is None else t.data_ptr()
+    a.q, a.k_share, a.v_share, a.k_loc, a.v_loc = ptr(q), ptr(k_share), ptr(v_share), ptr(k_loc), ptr(v_loc)
+    a.gate_logits, a.seq_lens, a.out = ptr(gate_logits), ptr(seq_lens), ptr(out)
+    a._keep = (q, k_share, v_share, k_loc, v_loc, gate_logits, seq_lens, out)
+    return a
+
+
+def plt_seq_attn_create(config: SeqConfig):
+    handle = ctypes.c_void_p()
+    st = load_library().plt_seq_attn_create(ctypes.byref(config), ctypes.byref(handle))
+    if st != PLT_OK:
+        _raise_seq(st, None)
+    return handle
+
+
+def plt_seq_attn_run(handle, args: SeqArgs, stream: int = 0) -> None:
+    st = load_library().plt_seq_attn_run(handle, ctypes.byref(args), ctypes.c_void_p(stream))
+    if st != PLT_OK:
+        _raise_seq(st, handle)
+
+
+def plt_seq_attn_check(handle, stream: int = 0) -> int:
+    bits = ctypes.c_uint32()
+    st = load_library().plt_seq_attn_check(handle, ctypes.c_void_p(stream), ctypes.byref(bits))
+    if st not in (PLT_OK, PLT_ERR_DEVICE_CHECK):
+        _raise_seq(st, handle)
+    return int(bits.value)
+
+
+def plt_seq_attn_destroy(handle) -> None:
+    load_library().plt_seq_attn_destroy(handle)

@@ -120,3 +120,47 @@ class DecodeAttn:
             self.close()
         except Exception:
             pass
+
+
+class SeqAttn:
+    """One plt_seq_attn handle and the device tensors of a sequence problem (torch for memory and streams only)."""
+
+    FIELDS = ("q", "k_share", "v_share", "k_loc", "v_loc")
+
+    def __init__(self, p, device="cuda:0", device_index: int = 0):
+        self.problem = p
+        for f in self.FIELDS:
+            setattr(self, f, to_torch(getattr(p, f), "bf16", device))
+        self.gate_logits = to_torch(p.gate_logits, "", device)
+        self.seq_lens = to_torch(p.seq_lens, "", device)
+        self.out = torch.empty((p.B, p.L, p.T, p.Hq, p.d), dtype=torch.bfloat16, device=device)
+        self.config = B.make_seq_config(
+            max(p.B, 1), p.L, p.Hq, p.Hkv, p.d, p.T, p.w, sm_scale=p.sm_scale, device=device_index,
+            loop_offset=None if p.loop_offset is None else [int(x) for x in p.loop_offset])
+        self.handle = B.plt_seq_attn_create(self.config)
+        many = p.L > 1
+        self.args = B.make_seq_args(p.B, self.q, self.k_share, self.v_share, self.seq_lens, self.out,
+                                    k_loc=self.k_loc if many else None, v_loc=self.v_loc if many else None,
+                                    gate_logits=self.gate_logits if many else None)
+
+    def run(self, stream: Optional[int] = None):
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        B.plt_seq_attn_run(self.handle, self.args, stream)
+        return self.out
+
+    def check(self, stream: Optional[int] = None) -> int:
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        return B.plt_seq_attn_check(self.handle, stream)
+
+    def close(self):
+        if self.handle is not None:
+            B.plt_seq_attn_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()

@@ -18,14 +18,17 @@ def lib():
 
 
 def header_functions():
-    text = (ROOT / "include" / "plt_decode_attn.h").read_text()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(plt_decode_attn_\w+)\s*\(", text)))
+    names = set()
+    for header in sorted((ROOT / "include").glob("*.h")):
+        text = re.sub(r"/\*.*?\*/", "", header.read_text(), flags=re.S)
+        names |= set(re.findall(r"\b(plt_(?:decode|seq)_attn_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(lib):
     names = header_functions()
     assert "plt_decode_attn_create" in names and "plt_decode_attn_run" in names and "plt_decode_attn_destroy" in names
+    assert "plt_seq_attn_create" in names and "plt_seq_attn_run" in names and "plt_seq_attn_destroy" in names
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in the header but not exported"
     from paper_2510_24824_b200 import binding
@@ -36,21 +39,22 @@ def test_struct_layout_matches_c(tmp_path):
     """Compile a tiny C program against the header and compare sizeof/offsetof with the ctypes structs."""
     import subprocess
     from paper_2510_24824_b200 import binding
-    fields_c = [f for f, _ in binding.Config._fields_]
-    fields_a = [f for f, _ in binding.Args._fields_]
+    structs = [("plt_decode_attn_config", binding.Config), ("plt_decode_attn_args", binding.Args),
+               ("plt_decode_attn_step_args", binding.StepArgs), ("plt_seq_attn_config", binding.SeqConfig),
+               ("plt_seq_attn_args", binding.SeqArgs)]
     src = tmp_path / "layout.c"
-    lines = ['#include <stdio.h>', '#include <stddef.h>', f'#include "{ROOT}/include/plt_decode_attn.h"', 'int main(void){',
-             'printf("%zu\\n", sizeof(plt_decode_attn_config));']
-    lines += [f'printf("%zu\\n", offsetof(plt_decode_attn_config, {f}));' for f in fields_c]
-    lines += ['printf("%zu\\n", sizeof(plt_decode_attn_args));']
-    lines += [f'printf("%zu\\n", offsetof(plt_decode_attn_args, {f}));' for f in fields_a]
+    lines = ['#include <stdio.h>', '#include <stddef.h>', f'#include "{ROOT}/include/plt_seq_attn.h"', 'int main(void){']
+    for cname, st in structs:
+        lines += [f'printf("%zu\\n", sizeof({cname}));']
+        lines += [f'printf("%zu\\n", offsetof({cname}, {f}));' for f, _ in st._fields_]
     lines += ['return 0;}']
     src.write_text("\n".join(lines))
     exe = tmp_path / "layout"
     subprocess.run(["gcc", "-std=c11", "-o", str(exe), str(src)], check=True)
     vals = [int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
-    want = [ctypes.sizeof(binding.Config)] + [getattr(binding.Config, f).offset for f in fields_c]
-    want += [ctypes.sizeof(binding.Args)] + [getattr(binding.Args, f).offset for f in fields_a]
+    want = []
+    for _, st in structs:
+        want += [ctypes.sizeof(st)] + [getattr(st, f).offset for f, _ in st._fields_]
     assert vals == want
 
 
@@ -82,6 +86,15 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert e.value.status == B.PLT_ERR_INVALID_ARG
     assert B.plt_decode_attn_workspace_bytes(B.make_config(**ok)) > 0
     B.plt_decode_attn_destroy(None)  # NULL is accepted
+    # the sequence-shaped entry points validate before they touch a device too
+    for kw, code in [(dict(d=64), B.PLT_ERR_UNSUPPORTED), (dict(Hq=7), B.PLT_ERR_INVALID_ARG), (dict(L=9), B.PLT_ERR_UNSUPPORTED),
+                     (dict(w=0), B.PLT_ERR_INVALID_ARG), (dict(loop_offset=[0, -2]), B.PLT_ERR_INVALID_ARG)]:
+        base = dict(max_batch=2, L=2, Hq=8, Hkv=2, d=128, max_seq_len=512, w=64)
+        base.update(kw)
+        with pytest.raises(B.PltError) as e:
+            B.plt_seq_attn_create(B.make_seq_config(**base))
+        assert e.value.status == code, (kw, e.value)
+    B.plt_seq_attn_destroy(None)
 
 
 def test_create_without_a_device_fails_loudly(lib):
