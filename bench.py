@@ -60,6 +60,13 @@ def parse_args():
     ap.add_argument("--ablation", action="store_true",
                     help="also time the same queries as L sequential single-loop calls, each scanning the shared cache "
                          "again (the vanilla loop order of Table 1), and report the ratio")
+    ap.add_argument("--seq", action="store_true",
+                    help="time the sequence-shaped attention (plt_seq_attn_run: prefill / training-forward) instead and "
+                         "print its line: TFLOP/s over the key sets the definition names, against the measured bf16 peak")
+    ap.add_argument("--seq-batch", type=int, default=4)
+    ap.add_argument("--seq-len", type=int, default=5000)
+    ap.add_argument("--seq-loops", type=int, default=2)
+    ap.add_argument("--seq-steps", type=int, default=20)
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
@@ -329,6 +336,54 @@ def main_kernel_bytes(by):
     return by["shared_kv"] + by["window_kv"] + by["q_o"] // 2 + by["index"]
 
 
+def peak_tflops():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"
+        except Exception:
+            pass
+    return 1400.0, "fallback (1.4 PFLOP/s sustained, earlier measurement on this pool)"
+
+
+def seq_entry(batch, loops, n, dev, local_rank, steps, seed=0):
+    """The sequence-shaped attention on the paper's serving shapes (prefill n, GQA 32/8, d = 128, w = 64): TFLOP/s."""
+    import torch
+    from paper_2510_24824_b200.inputs import make_seq_problem, seq_attn_flops
+    from paper_2510_24824_b200.runner import SeqAttn
+    p = make_seq_problem(B=batch, L=loops, T=n, Hq=32, Hkv=8, d=128, w=64, seed=seed, name=f"seq_B{batch}_L{loops}_n{n}")
+    flops = seq_attn_flops(p)
+    op = SeqAttn(p, dev, local_rank)
+    for _ in range(3):
+        op.run()
+    torch.cuda.synchronize()
+    assert op.check() == 0, "device status not clean after warm-up"
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with sampler:
+        ev0.record()
+        for _ in range(steps):
+            op.run()
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    peak, src = peak_tflops()
+    tf = flops / (ms * 1e-3) / 1e12
+    entry = {
+        "workload": p.name, "B": batch, "L": loops, "n": n, "Hq": 32, "Hkv": 8, "d": 128, "w": 64, "steps": steps,
+        "ms_per_call": ms, "algorithmic_flops_per_call": flops, "tflops": tf, "tokens_per_s": batch * n / (ms * 1e-3),
+        "roofline": {"bound": "tensor", "kernel": "plt_seq_attn_kernel", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
+                     "frac": tf / peak, "peak_source": src,
+                     "note": "flops of the two products over visible keys only (masked halves of diagonal tiles not counted)"},
+        "inputs_bytes": int(sum(getattr(op, f).numel() * 2 for f in SeqAttn.FIELDS)),
+        "clocks": sampler.summary(),
+    }
+    op.close()
+    del op
+    torch.cuda.empty_cache()
+    return entry
+
+
 def suite_entry(index, kv, dev, local_rank, steps, base=None):
     """One entry of the "workloads" list: a workload timed for `steps` steps with its own clock record."""
     import torch
@@ -401,6 +456,19 @@ def main():
     dev = f"cuda:{local_rank}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    if args.seq:
+        if rank == 0:
+            e = seq_entry(args.seq_batch, args.seq_loops, args.seq_len, dev, local_rank, args.seq_steps)
+            line = {"metric": "plt_seq_attn_tflops", "value": e["tflops"], "unit": "TFLOP/s", "n_gpus": 1, "steps": args.seq_steps,
+                    "warmup": 3, "ms_per_step": e["ms_per_call"], "higher_is_better": True, "scaling": "weak",
+                    "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": {"workload": e["workload"]},
+                    "gpu_launches": args.seq_steps, **e}
+            print(json.dumps(line), flush=True)
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
 
     p = make_problem(replica_spec(args.workload, rank, args.loops, args.kv))
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
@@ -525,6 +593,8 @@ def main():
                 entries.append(e)
                 del base
             line["workloads"] = entries
+            # the compute-bound sibling: sequence-shaped attention at the paper's prefill length
+            line["seq_attn"] = [seq_entry(4, 2, 5000, dev, local_rank, 10), seq_entry(16, 3, 5000, dev, local_rank, 5)]
         if not args.no_cpu:
             v, cinfo = time_oracle(p, args.cpu_seconds)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, **cinfo}

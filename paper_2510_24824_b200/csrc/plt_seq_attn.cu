@@ -47,7 +47,7 @@ constexpr int kTileBytes = SK * SD * 2;    // one Q, K or V tile
 constexpr int kHalf = SK * 128;            // one 64-element half of a tile: [128 rows][128 bytes]
 constexpr int kRing = 5;                   // K/V ring slots
 constexpr int kSeqThreads = 384;
-constexpr float kSeqSlack = 8.f;
+constexpr float kSeqBig = 256.f;           // probabilities stay below 2^8 of their row's reference, else the slow path
 constexpr float kSeqNoMax = -1e30f;
 constexpr uint64_t kSeqWaitNs = 1000000000ull;
 constexpr int kSeqMaxLoops = 8;
@@ -74,11 +74,13 @@ struct SeqParams {
 };
 
 // The steps of one block: nG tiles of the shared K/V (tile A takes part in the first ntA of them), then for loops
-// 2..L the tiles [lX0, lX0 + nLX) of the loop's own K/V, scores only (kind 1) for A then B, then again with the
-// second product (kind 2) for A then B.
+// 2..L the tiles [l0, l0 + nL) of the loop's own K/V that the windows of the block's rows touch, scores only (kind 1),
+// then the same tiles again with the second product (kind 2). Tile A takes part in the own-K/V tiles [lA0, lA0 + nLA),
+// tile B in [lB0, lB0 + nLB); where both do, the step is shared like a step of the first phase.
 struct SeqPlan {
     int ntA, ntB, nG;
     int lA0, nLA, lB0, nLB;
+    int l0, nL;
     int total;
 };
 struct SeqStep {
@@ -95,9 +97,9 @@ __device__ __forceinline__ SeqStep seq_step_at(const SeqPlan& pl, int i) {
     }
     i -= pl.nG;
     s.kind = 1;
-    if (i >= pl.nLA + pl.nLB) { i -= pl.nLA + pl.nLB; s.kind = 2; }
-    if (i < pl.nLA) { s.jk = pl.lA0 + i; s.qmask = 1; }
-    else { s.jk = pl.lB0 + (i - pl.nLA); s.qmask = 2; }
+    if (i >= pl.nL) { i -= pl.nL; s.kind = 2; }
+    s.jk = pl.l0 + i;
+    s.qmask = ((s.jk >= pl.lA0 && s.jk < pl.lA0 + pl.nLA) ? 1 : 0) | ((s.jk >= pl.lB0 && s.jk < pl.lB0 + pl.nLB) ? 2 : 0);
     return s;
 }
 
@@ -185,32 +187,51 @@ struct RowCtx {
     bool live;        // t < n_b and cut > 0
 };
 
-// One pass over the 128 scores of this thread's row (tensor-memory lane) of a shared-K/V step: probabilities against
-// the reference mref, packed bf16 into pk[64], their sum (of the rounded values) and the largest exponent seen.
-// kbase: index of the tile's first key. full: no key of the tile is masked for any row of the block's tile.
-__device__ __forceinline__ void global_pass(uint32_t tS, const RowCtx& rc, int kbase, bool full, float scale, float mref,
-                                            uint32_t (&pk)[64], float& lsum, float& tmax) {
-    lsum = 0.f;
-    tmax = -INFINITY;
-    const int lim = rc.cut - kbase;   // keys [0, lim) of the tile are visible to this row
+// 32 scores of a row -> probabilities against the reference: packed bf16 into pk[16], summed (fp32, two lanes) and
+// their packed maximum tracked (bf16 bit patterns of non-negative numbers order like integers).
+template <bool FULL>
+__device__ __forceinline__ void global_chunk(const uint32_t (&r)[32], int c, int lim, float2 sc2, float2 nm2, uint32_t* pk,
+                                             float2& sum2, uint32_t& pmax) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tS + c * 32, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-            float t0 = fmaf(__uint_as_float(r[i]), scale, -mref), t1 = fmaf(__uint_as_float(r[i + 1]), scale, -mref);
-            if (!full) {
-                if (c * 32 + i >= lim) t0 = -INFINITY;
-                if (c * 32 + i + 1 >= lim) t1 = -INFINITY;
-            }
-            tmax = fmaxf(tmax, fmaxf(t0, t1));
-            const uint32_t h = pack_bf16x2(fast_exp2(t0), fast_exp2(t1));
-            pk[c * 16 + i / 2] = h;
-            lsum += __uint_as_float(h << 16) + __uint_as_float(h & 0xffff0000u);
+    for (int i = 0; i < 32; i += 2) {
+        float2 t = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
+        if (!FULL) {
+            if (c * 32 + i >= lim) t.x = -INFINITY;
+            if (c * 32 + i + 1 >= lim) t.y = -INFINITY;
         }
+        const float2 pr = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+        sum2 = __fadd2_rn(sum2, pr);
+        const uint32_t h = pack_bf16x2(pr.x, pr.y);
+        pk[i / 2] = h;
+        asm("max.u16x2 %0, %0, %1;" : "+r"(pmax) : "r"(h));
     }
+}
+
+// One pass over the 128 scores of this thread's row (tensor-memory lane) of a shared-K/V step: probabilities against
+// the reference mref, packed bf16 into pk[64], their sum and the largest probability. kbase: index of the tile's first
+// key. full: no key of the tile is masked for any row of the block's tile. The loads of a chunk are in flight while
+// the chunk before it is worked on.
+__device__ __forceinline__ void global_pass(uint32_t tS, const RowCtx& rc, int kbase, bool full, float scale, float mref,
+                                            uint32_t (&pk)[64], float& lsum, float& pbig) {
+    const int lim = rc.cut - kbase;   // keys [0, lim) of the tile are visible to this row
+    const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-mref, -mref);
+    float2 sum2 = make_float2(0.f, 0.f);
+    uint32_t pmax = 0;
+    uint32_t ra[32], rb[32];
+    tmem_ld32(tS, ra);
+    tmem_wait_ld();
+    tmem_ld32(tS + 32, rb);
+    if (full) global_chunk<true>(ra, 0, lim, sc2, nm2, &pk[0], sum2, pmax); else global_chunk<false>(ra, 0, lim, sc2, nm2, &pk[0], sum2, pmax);
+    tmem_wait_ld();
+    tmem_ld32(tS + 64, ra);
+    if (full) global_chunk<true>(rb, 1, lim, sc2, nm2, &pk[16], sum2, pmax); else global_chunk<false>(rb, 1, lim, sc2, nm2, &pk[16], sum2, pmax);
+    tmem_wait_ld();
+    tmem_ld32(tS + 96, rb);
+    if (full) global_chunk<true>(ra, 2, lim, sc2, nm2, &pk[32], sum2, pmax); else global_chunk<false>(ra, 2, lim, sc2, nm2, &pk[32], sum2, pmax);
+    tmem_wait_ld();
+    if (full) global_chunk<true>(rb, 3, lim, sc2, nm2, &pk[48], sum2, pmax); else global_chunk<false>(rb, 3, lim, sc2, nm2, &pk[48], sum2, pmax);
+    lsum = sum2.x + sum2.y;
+    pbig = fmaxf(__uint_as_float(pmax << 16), __uint_as_float(pmax & 0xffff0000u));
 }
 
 // Largest visible score of the row in the tile (slow path of the shared-K/V pass).
@@ -227,6 +248,71 @@ __device__ __forceinline__ float global_row_max(uint32_t tS, const RowCtx& rc, i
             if (c * 32 + i < lim) mx = fmaxf(mx, __uint_as_float(r[i]));
     }
     return mx;
+}
+
+// Scores-only pass over a tile of the loop's own keys: folds the visible columns [c_lo, c_hi] of this thread's row into
+// the window softmax's exact running maximum ml (log2 units) and denominator ll. Rows without a visible key keep
+// ml = -inf, ll = 0. Every lane runs every load (they are collective over the warp).
+__device__ __forceinline__ void window_stats_chunk(const uint32_t (&r)[32], int c, int c_lo, int c_hi, float scale, float& ml,
+                                                   float& ll) {
+    float t[32], cmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int col = c * 32 + i;
+        t[i] = (col >= c_lo && col <= c_hi) ? __uint_as_float(r[i]) * scale : -INFINITY;
+        cmax = fmaxf(cmax, t[i]);
+    }
+    const float m_new = fmaxf(ml, cmax);
+    const float m_use = m_new > -INFINITY ? m_new : 0.f;
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) sum += fast_exp2(t[i] - m_use);
+    ll = ll * fast_exp2(ml - m_use) + sum;   // ml = -inf: the old denominator is 0 and stays 0
+    ml = m_new;
+}
+__device__ __forceinline__ void window_stats(uint32_t tS, int c_lo, int c_hi, float scale, float& ml, float& ll) {
+    uint32_t ra[32], rb[32];
+    tmem_ld32(tS, ra);
+    tmem_wait_ld();
+    tmem_ld32(tS + 32, rb);
+    window_stats_chunk(ra, 0, c_lo, c_hi, scale, ml, ll);
+    tmem_wait_ld();
+    tmem_ld32(tS + 64, ra);
+    window_stats_chunk(rb, 1, c_lo, c_hi, scale, ml, ll);
+    tmem_wait_ld();
+    tmem_ld32(tS + 96, rb);
+    window_stats_chunk(ra, 2, c_lo, c_hi, scale, ml, ll);
+    tmem_wait_ld();
+    window_stats_chunk(rb, 3, c_lo, c_hi, scale, ml, ll);
+}
+
+// Second pass over the same tile: the weights 2^(s * scale + negm) of the visible columns (0 elsewhere), packed bf16.
+__device__ __forceinline__ void window_weights_chunk(const uint32_t (&r)[32], int c, int c_lo, int c_hi, float2 sc2, float2 nm2,
+                                                     uint32_t* pk) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const int col = c * 32 + i;
+        float2 t = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
+        if (!(col >= c_lo && col <= c_hi)) t.x = -INFINITY;
+        if (!(col + 1 >= c_lo && col + 1 <= c_hi)) t.y = -INFINITY;
+        pk[i / 2] = pack_bf16x2(fast_exp2(t.x), fast_exp2(t.y));
+    }
+}
+__device__ __forceinline__ void window_weights(uint32_t tS, int c_lo, int c_hi, float scale, float negm, uint32_t (&pk)[64]) {
+    const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(negm, negm);
+    uint32_t ra[32], rb[32];
+    tmem_ld32(tS, ra);
+    tmem_wait_ld();
+    tmem_ld32(tS + 32, rb);
+    window_weights_chunk(ra, 0, c_lo, c_hi, sc2, nm2, &pk[0]);
+    tmem_wait_ld();
+    tmem_ld32(tS + 64, ra);
+    window_weights_chunk(rb, 1, c_lo, c_hi, sc2, nm2, &pk[16]);
+    tmem_wait_ld();
+    tmem_ld32(tS + 96, rb);
+    window_weights_chunk(ra, 2, c_lo, c_hi, sc2, nm2, &pk[32]);
+    tmem_wait_ld();
+    window_weights_chunk(rb, 3, c_lo, c_hi, sc2, nm2, &pk[48]);
 }
 
 // Multiplies this thread's row of O (128 fp32 columns) by f.
@@ -300,7 +386,14 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             own(r0A, pl.ntA, pl.lA0, pl.nLA);
             own(r0B, pl.ntB, pl.lB0, pl.nLB);
         }
-        pl.total = pl.nG + 2 * (pl.nLA + pl.nLB);
+        pl.l0 = pl.nL = 0;
+        if (pl.nLA > 0 || pl.nLB > 0) {
+            const int a0 = pl.nLA > 0 ? pl.lA0 : pl.lB0, b0 = pl.nLB > 0 ? pl.lB0 : pl.lA0;
+            const int a1 = pl.nLA > 0 ? pl.lA0 + pl.nLA : 0, b1 = pl.nLB > 0 ? pl.lB0 + pl.nLB : 0;
+            pl.l0 = min(a0, b0);
+            pl.nL = max(a1, b1) - pl.l0;   // the two ranges overlap or touch: every tile in between belongs to one
+        }
+        pl.total = pl.nG + 2 * pl.nL;
     }
     const bool activeA = pl.ntA > 0, activeB = pl.ntB > 0;
 
@@ -374,12 +467,13 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             // ahead of PV products), so positions are recomputed from a running count.
             // slot_of(count) = count % kRing, parity = (count / kRing) & 1
             uint32_t s_issued[2] = {0, 0};    // per tile: S products issued (= steps of that tile started)
+            int s_mask_step[2] = {-1, -1}, s_mask[2] = {0, 0};   // tiles whose S of a step has been issued (two steps in flight at most)
             uint32_t p_parity[2] = {0, 0};    // parity of the next P_FULL wait per tile
             bool o_started[2] = {false, false};
             // tile count before step i: prefix over steps (1 or 2 tiles each)
             auto tiles_before = [&](int i) {
                 // steps [0, nG) and kind-2 steps have two tiles, kind-1 steps one
-                const int nl = pl.nLA + pl.nLB;
+                const int nl = pl.nL;
                 if (i <= pl.nG) return 2 * i;
                 if (i <= pl.nG + nl) return 2 * pl.nG + (i - pl.nG);
                 return 2 * pl.nG + nl + 2 * (i - pl.nG - nl);
@@ -400,8 +494,15 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         umma_bf16(tmem_base + x * 128, seq_smem_desc(qa + (kk >> 2) * kHalf + (kk & 3) * 32, 16, 1024),
                                   seq_smem_desc(ka + (kk >> 2) * kHalf + (kk & 3) * 32, 16, 1024), idesc_qk, kk == 0 ? 0u : 1u);
                     umma_commit(&bars[SB_SFULL + x]);
-                    if (x == ((st.qmask & 2) ? 1 : 0)) umma_commit(&bars[SB_EMPTY + slot]);   // last tile to read this K
                 }
+                // The K slot is free once every tile that takes part in the step has issued its S product; which of the
+                // two comes last depends on which of them ran ahead.
+                if (s_mask_step[i & 1] != i) {
+                    s_mask_step[i & 1] = i;
+                    s_mask[i & 1] = 0;
+                }
+                s_mask[i & 1] |= 1 << x;
+                if (s_mask[i & 1] == st.qmask && lane == 0) umma_commit(&bars[SB_EMPTY + slot]);
                 __syncwarp();
                 ++s_issued[x];
             };
@@ -489,7 +590,7 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const float scale = p.scale_log2;
         float mref = kSeqNoMax, lg = 0.f;       // shared-K/V softmax: reference maximum (log2 units) and denominator
         float ml = -INFINITY, ll = 0.f;          // window softmax: exact maximum (log2 units) and denominator
-        float gate = 0.f, beta = 0.f;
+        float gate = 0.f;
         bool ok = true, o_scaled = false;
         uint32_t s_parity = 0;
         int gsteps = 0;
@@ -511,9 +612,9 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     // ---- shared K/V: online softmax against the lazily updated reference ----------------
                     const bool full = kbase + SK <= r0 + 1 - delta && kbase + SK <= n;
                     uint32_t pk[64];
-                    float lsum, tmax;
-                    global_pass(tS, rc, kbase, full, scale, mref, pk, lsum, tmax);
-                    if (__any_sync(0xffffffffu, tmax > kSeqSlack)) {
+                    float lsum, pbig;
+                    global_pass(tS, rc, kbase, full, scale, mref, pk, lsum, pbig);
+                    if (__any_sync(0xffffffffu, rc.live && !(pbig <= kSeqBig))) {   // a probability of a live row beyond 2^8 of its reference
                         // slow path: true maximum, rescale of this row of O (every product into it has completed: the
                         // commit behind S_FULL covers them), probabilities again
                         const float mx = global_row_max(tS, rc, kbase);
@@ -522,7 +623,7 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         mref = m_new;
                         lg *= alpha;
                         if (gsteps > 0) scale_o_row(tO, alpha);
-                        global_pass(tS, rc, kbase, full, scale, mref, pk, lsum, tmax);
+                        global_pass(tS, rc, kbase, full, scale, mref, pk, lsum, pbig);
                     }
                     lg += lsum;
                     ++gsteps;
@@ -535,55 +636,16 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         o_scaled = true;
                         scale_o_row(tO, (rc.live && lg > 0.f) ? (1.f - gate) / lg : 0.f);
                     }
-                    // own keys lo .. t of the row
-                    const int c_lo = rc.lo - kbase, c_hi = rc.t - kbase;   // visible columns [c_lo, c_hi]
+                    // own keys lo .. t of the row: columns [c_lo, c_hi] of the tile
+                    const int c_lo = rc.lo - kbase, c_hi = rc.t - kbase;
                     if (st.kind == 1) {
-                        float mx = -INFINITY;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tS + c * 32, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; ++i2)
-                                if (c * 32 + i2 >= c_lo && c * 32 + i2 <= c_hi) mx = fmaxf(mx, __uint_as_float(r[i2]) * scale);
-                        }
-                        // (the loads are collective over the warp: every lane runs them, rows without a visible key
-                        // included; those keep ml = -inf, ll = 0)
-                        const float m_new = fmaxf(ml, mx);
-                        const float m_use = m_new > -INFINITY ? m_new : 0.f;
-                        float sum = 0.f;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tS + c * 32, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; ++i2)
-                                if (c * 32 + i2 >= c_lo && c * 32 + i2 <= c_hi)
-                                    sum += fast_exp2(fmaf(__uint_as_float(r[i2]), scale, -m_use));
-                        }
-                        if (m_new > -INFINITY) {
-                            ll = (ml > -INFINITY ? ll * fast_exp2(ml - m_new) : 0.f) + sum;
-                            ml = m_new;
-                        }
+                        window_stats(tS, c_lo, c_hi, scale, ml, ll);
                     } else {
-                        beta = (rc.live && ll > 0.f) ? gate / ll : 0.f;
+                        // probabilities already normalised and gated: g * 2^(s - m) / l = 2^(s - m + log2(g / l))
+                        const float beta = (rc.live && ll > 0.f) ? gate / ll : 0.f;
+                        const float negm = beta > 0.f ? fast_log2(beta) - ml : -INFINITY;
                         uint32_t pk[64];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tS + c * 32, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; i2 += 2) {
-                                const int c0 = c * 32 + i2;
-                                float p0 = 0.f, p1 = 0.f;
-                                if (c0 >= c_lo && c0 <= c_hi) p0 = beta * fast_exp2(fmaf(__uint_as_float(r[i2]), scale, -ml));
-                                if (c0 + 1 >= c_lo && c0 + 1 <= c_hi) p1 = beta * fast_exp2(fmaf(__uint_as_float(r[i2 + 1]), scale, -ml));
-                                pk[c * 16 + i2 / 2] = pack_bf16x2(p0, p1);
-                            }
-                        }
+                        window_weights(tS, c_lo, c_hi, scale, negm, pk);
 #pragma unroll
                         for (int c = 0; c < 2; ++c) tmem_st32(tS + c * 32, &pk[c * 32]);
                         tmem_wait_st();
