@@ -581,6 +581,7 @@ def main():
             line["e2e"] = e2e
         if ablation is not None:
             ablation["ratio"] = ablation["sequential_single_loop_calls_ms"] / ms_per_step
+            ablation["private_caches_ratio"] = ablation["private_caches_one_call_ms"] / ms_per_step
             line["ablation"] = ablation
         if suite:
             entries, base = [], None
@@ -605,43 +606,36 @@ def main():
 
 
 def run_ablation(args, p, reps, dev, local_rank, stream):
-    """The same queries as L sequential single-loop calls, each scanning the shared cache again (Table 1, loop order of
-    the vanilla loop transformer); global attention only (no window, no gate), so a lower bound."""
+    """The ablation rows of Table 1 at kernel level, beside the cross-loop-parallel step over one shared cache: the same
+    loop-queries as L sequential single-loop calls, each scanning the shared cache again (loop order of the vanilla
+    loop transformer), and as one cross-loop-parallel call over L private caches ("Loop+CLP" before KV sharing).
+    Global attention only (no window, no gate): a lower bound for both."""
     import torch
-    from paper_2510_24824_b200 import binding as B
-    from paper_2510_24824_b200.runner import DecodeAttn, to_torch
-    dp = reps[0].dp
-    p1 = p.with_(L=1, w=0, q=np.ascontiguousarray(p.q[:, :1]), loop_offset=None, win_lens=None)
-    op1 = DecodeAttn(p1, device_index=local_rank, kernel_path=args.path)
-    calls = []
-    for l in range(p.L):
-        ql = to_torch(np.ascontiguousarray(p.q[:, l:l + 1]), p.dtype, dev)
-        nl = to_torch(np.maximum(p.seq_lens - int(p.offsets()[l]), 0).astype(np.int32), "", dev)
-        ol = torch.empty_like(ql)
-        calls.append((ql, nl, ol, B.make_args(p.B, ql, dp.k_cache, dp.v_cache, nl, ol, page_table=dp.page_table,
-                                              max_pages=p.max_pages, num_pool_pages=p.num_pool_pages,
-                                              k_scale=dp.k_scale, v_scale=dp.v_scale)))
-
-    def seq_step():
-        for c in calls:
-            B.plt_decode_attn_run(op1.handle, c[3], stream)
-
-    for _ in range(5):
-        seq_step()
-    torch.cuda.synchronize()
+    from paper_2510_24824_b200.runner import LoopOrderAblation
+    abl = LoopOrderAblation(p, reps[0].dp, device_index=local_rank, kernel_path=args.path)
     n_abl = min(args.steps, 300)
-    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a0.record()
-    for _ in range(n_abl):
-        seq_step()
-    a1.record()
-    torch.cuda.synchronize()
-    seq_ms = a0.elapsed_time(a1) / n_abl
-    assert op1.check(stream) == 0
-    op1.close()
-    return {"sequential_single_loop_calls_ms": seq_ms, "calls_per_step": p.L, "steps_timed": n_abl,
-            "note": "global attention only (no window, no gate): a lower bound of the sequential loop order; "
-                    "ratio = this / ms_per_step of the cross-loop-parallel step"}
+
+    def timed(fn):
+        for _ in range(5):
+            fn(stream)
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(n_abl):
+            fn(stream)
+        a1.record()
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) / n_abl
+
+    seq_ms = timed(abl.run_sequential)
+    priv_ms = timed(abl.run_private)
+    assert abl.check(stream) == 0
+    abl.close()
+    return {"sequential_single_loop_calls_ms": seq_ms, "private_caches_one_call_ms": priv_ms, "calls_per_step": p.L,
+            "steps_timed": n_abl,
+            "note": "global attention only (no window, no gate): lower bounds of the sequential loop order (L launches, "
+                    "L scans of the shared cache) and of cross-loop parallelism over L private caches (one launch, L "
+                    "caches); ratios = these / ms_per_step of the step over one shared cache"}
 
 
 if __name__ == "__main__":

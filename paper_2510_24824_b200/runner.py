@@ -164,3 +164,78 @@ class SeqAttn:
 
     def __exit__(self, *exc):
         self.close()
+
+
+class LoopOrderAblation:
+    """The ablation rows of Table 1 at kernel level, on the tensors of a device problem: the same loop-queries served
+
+      * as L sequential single-loop calls, each scanning the shared cache again (the loop order of the vanilla loop
+        transformer: L launches, L scans), and
+      * as ONE cross-loop-parallel call over L private caches, one per loop ("Loop+CLP" before KV sharing: one launch,
+        L caches read once each; the private caches are device-side copies of the shared one at other addresses),
+
+    beside the library's own step (one launch, one shared cache). Global attention only (no window, no gate): what
+    the three have in common. torch is used for device memory only.
+    """
+
+    def __init__(self, p, dp: DeviceProblem, device_index: int = 0, kernel_path: int = 0, private: bool = True):
+        self.p, self.dp, self.L = p, dp, p.L
+        dev = dp.q.device
+        offs = [int(x) for x in p.offsets()]
+        lens = dp.seq_lens.to(torch.int64)
+        self.loop_lens = [torch.clamp(lens - o, min=0).to(torch.int32) for o in offs]
+        p1 = p.with_(L=1, w=0, q=np.ascontiguousarray(p.q[:, :1]), loop_offset=None, win_lens=None)
+        # ---- sequential single-loop calls over the shared cache ----
+        self.seq_op = DecodeAttn(p1, device_index=device_index, kernel_path=kernel_path)
+        self.seq_q = [dp.q[:, l:l + 1].contiguous() for l in range(p.L)]
+        self.seq_out = [torch.empty_like(q) for q in self.seq_q]
+        self.seq_args = [B.make_args(p.B, q, dp.k_cache, dp.v_cache, n, o, page_table=dp.page_table, max_pages=p.max_pages,
+                                     num_pool_pages=p.num_pool_pages, k_scale=dp.k_scale, v_scale=dp.v_scale)
+                         for q, n, o in zip(self.seq_q, self.loop_lens, self.seq_out)]
+        # ---- one call over L private caches: sequence b * L + l is loop l of sequence b with a cache of its own ----
+        self.priv_op = None
+        if private:
+            self.priv_op = DecodeAttn(p1, device_index=device_index, kernel_path=kernel_path, max_batch=p.B * p.L)
+            self.priv_q = dp.q.reshape(p.B * p.L, 1, p.Hq, p.d)
+            self.priv_out = torch.empty_like(self.priv_q)
+            self.priv_lens = torch.stack(self.loop_lens, dim=1).reshape(-1).contiguous()
+            if p.page_size:
+                P = p.num_pool_pages
+                self.priv_k = dp.k_cache.repeat(p.L, 1, 1, 1)
+                self.priv_v = dp.v_cache.repeat(p.L, 1, 1, 1)
+                shift = (torch.arange(p.L, device=dev, dtype=torch.int32) * P).view(1, p.L, 1)
+                self.priv_table = (dp.page_table.view(p.B, 1, -1) + shift).reshape(p.B * p.L, -1).contiguous()
+                pool = P * p.L
+            else:
+                self.priv_k = dp.k_cache.repeat_interleave(p.L, dim=0)
+                self.priv_v = dp.v_cache.repeat_interleave(p.L, dim=0)
+                self.priv_table, pool = None, 0
+            self.priv_args = B.make_args(p.B * p.L, self.priv_q, self.priv_k, self.priv_v, self.priv_lens, self.priv_out,
+                                         page_table=self.priv_table, max_pages=p.max_pages, num_pool_pages=pool,
+                                         k_scale=dp.k_scale, v_scale=dp.v_scale)
+
+    def run_sequential(self, stream: Optional[int] = None):
+        """L launches of the single-loop attention; returns the outputs stacked as [B, L, Hq, d]."""
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        for a in self.seq_args:
+            B.plt_decode_attn_run(self.seq_op.handle, a, stream)
+        return self.seq_out
+
+    def run_private(self, stream: Optional[int] = None):
+        """One launch over the L private caches; returns [B * L, 1, Hq, d] (row b * L + l)."""
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        B.plt_decode_attn_run(self.priv_op.handle, self.priv_args, stream)
+        return self.priv_out
+
+    def check(self, stream: Optional[int] = None) -> int:
+        bits = self.seq_op.check(stream)
+        if self.priv_op is not None:
+            bits |= self.priv_op.check(stream)
+        return bits
+
+    def close(self):
+        self.seq_op.close()
+        if self.priv_op is not None:
+            self.priv_op.close()
