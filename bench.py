@@ -13,7 +13,7 @@ independent replica of the workload on its own GPU (no collective in the data pa
 `--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
 Other legs: `--kv e4m3` stores the caches as E4M3 codes, `--prestep` times plt_decode_attn_step (pre-step kernel +
 attention), `--ablation` adds the L loops as sequential single-loop calls, `--path` / `--loops` / `--hpc` / `--kw` /
-`--stages` / `--cps` select the kernel path, an overridden L and launch variants.
+`--stages` / `--cps` / `--rw` / `--ks` select the kernel path, an overridden L and launch variants.
 """
 from __future__ import annotations
 
@@ -46,10 +46,15 @@ def parse_args():
                     help="index into the five workloads; default: 1 (the headline) followed by the suite of the others")
     ap.add_argument("--suite-steps", type=int, default=300, help="timed steps per entry of the \"workloads\" list")
     ap.add_argument("--no-suite", action="store_true", help="headline workload only")
+    ap.add_argument("--copies", type=int, default=2, choices=[1, 2],
+                    help="copies of the inputs the timed steps alternate between (1: for profiler captures, which "
+                         "save and restore device memory per pass and flush the caches themselves)")
     ap.add_argument("--hpc", type=int, default=0)
     ap.add_argument("--kw", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--cps", type=int, default=0)
+    ap.add_argument("--rw", type=int, default=0, help="warps that split the packed rows of a KV head (0 = automatic)")
+    ap.add_argument("--ks", type=int, default=0, help="16-key slices per warp and tile (0 = automatic)")
     ap.add_argument("--loops", type=int, default=0, help="override the workload's number of loops L (for the traffic-vs-L sweep)")
     ap.add_argument("--path", type=int, default=0, help="kernel path: 0 automatic, 1 warp-level mma, 2 tcgen05")
     ap.add_argument("--kv", default="", choices=["", "e4m3"],
@@ -327,7 +332,7 @@ def time_main_kernel(reps, step_fns, n_prof):
         B.plt_decode_attn_set_profile_events(reps[i & 1].op.handle, a.cuda_event, b.cuda_event)
         step_fns[i & 1]()
     torch.cuda.synchronize()
-    for r in reps:
+    for r in set(reps):
         B.plt_decode_attn_set_profile_events(r.op.handle, None, None)
     return float(np.mean([a.elapsed_time(b) for a, b in raw]))
 
@@ -472,12 +477,14 @@ def main():
 
     p = make_problem(replica_spec(args.workload, rank, args.loops, args.kv))
     tuning = dict(heads_per_cta=args.hpc, key_slices=args.kw, stages=args.stages, ctas_per_sm=args.cps,
-                  kernel_path=args.path)
+                  kernel_path=args.path, row_warps=args.rw, slices_per_warp=args.ks)
     reps = [Replica(p, dev, local_rank, tuning)]
-    reps.append(Replica(p, dev, local_rank, tuning, src=reps[0]))
+    reps.append(Replica(p, dev, local_rank, tuning, src=reps[0]) if args.copies == 2 else reps[0])
     op, dp = reps[0].op, reps[0].dp
     stream = torch.cuda.current_stream().cuda_stream
     cfg, by = workload_config(p)
+    if args.copies == 1:
+        cfg["l2"] = f"inputs {by['total'] / 1e6:.0f} MB per step exceed the 126 MB L2; one copy of the inputs, no flush"
 
     def barrier():
         if world > 1:
@@ -550,7 +557,7 @@ def main():
     value = job_steps_per_s(world, ms_per_step)
     info = dict(op.info)
     kernel_path = info["kernel_path"]
-    for r in reps:
+    for r in set(reps):
         r.close()
     del reps, dp, op
     torch.cuda.empty_cache()

@@ -34,6 +34,10 @@ __device__ __forceinline__ void load_vec(const float* src, Vec<D>& x) {
 }
 
 // Sum over the pieces held by blocks [c0, c1] of one item, rescaled to a common maximum. Returns the denominator.
+// An item of a small batch is spread over many blocks (one sequence of a batch of four over dozens), so the loads
+// must not wait for one another: the lanes of the warp read the (maximum, denominator) pairs of 32 pieces at a time,
+// the common maximum and the denominator come from warp reductions, and the partial vectors are read four pieces at a
+// time with the scale factors handed round by shuffles. The order of every sum is fixed by the piece index alone.
 template <int D>
 __device__ __forceinline__ float merge_item(const Params& p, int item, int hl, int r, int c0, int c1, int lane,
                                             Vec<D>& y) {
@@ -49,19 +53,41 @@ __device__ __forceinline__ float merge_item(const Params& p, int item, int hl, i
         load_vec<D>(p.part_acc + row0 * D + lane * Vec<D>::N, y);
         return ml.y;
     }
+    const int np = c1 - c0 + 1;
+    // common maximum: every lane takes the pieces lane, lane + 32, ...
     float mstar = -INFINITY;
-    for (int c = c0; c <= c1; ++c) mstar = fmaxf(mstar, p.part_ml[(row0 + (c - c0) * step) * 2]);
+    for (int j = lane; j < np; j += 32) mstar = fmaxf(mstar, p.part_ml[(row0 + j * step) * 2]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
     if (mstar == -INFINITY) return 0.f;  // no visible key anywhere
     float denom = 0.f;
-    for (int c = c0; c <= c1; ++c) {
-        const int64_t row = row0 + (c - c0) * step;
-        const float2 ml = *(const float2*)(p.part_ml + row * 2);
-        const float sc = exp2f(ml.x - mstar);  // exp2f(-inf) = 0 for pieces that saw nothing
-        denom = fmaf(ml.y, sc, denom);
-        Vec<D> a;
-        load_vec<D>(p.part_acc + row * D + lane * Vec<D>::N, a);
+    for (int j0 = 0; j0 < np; j0 += 32) {
+        // scale factor and weighted denominator of piece j0 + lane
+        float sc = 0.f, dl = 0.f;
+        if (j0 + lane < np) {
+            const float2 ml = *(const float2*)(p.part_ml + (row0 + (j0 + lane) * step) * 2);
+            sc = exp2f(ml.x - mstar);  // exp2f(-inf) = 0 for pieces that saw nothing
+            dl = ml.y * sc;
+        }
 #pragma unroll
-        for (int i = 0; i < Vec<D>::N; ++i) y.v[i] = fmaf(a.v[i], sc, y.v[i]);
+        for (int o = 16; o > 0; o >>= 1) dl += __shfl_xor_sync(0xffffffffu, dl, o);
+        denom += dl;
+        const int cnt = min(32, np - j0);
+        for (int j = 0; j < cnt; j += 4) {
+            Vec<D> a[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int jj = j + u < cnt ? j + u : cnt - 1;   // past the end: a load that is multiplied by 0
+                load_vec<D>(p.part_acc + (row0 + (j0 + jj) * step) * D + lane * Vec<D>::N, a[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float su = __shfl_sync(0xffffffffu, sc, (j + u) & 31);
+                if (j + u >= cnt) su = 0.f;
+#pragma unroll
+                for (int i = 0; i < Vec<D>::N; ++i) y.v[i] = fmaf(a[u].v[i], su, y.v[i]);
+            }
+        }
     }
     return denom;
 }
