@@ -132,3 +132,33 @@ def decode_attn_rows(p, rows) -> np.ndarray:
         raise RuntimeError(f"plt_oracle_decode_attn_rows failed with code {rc}")
     del keep
     return out
+
+
+def decode_attn_multi(p, q, gate_logits, q_len: int) -> np.ndarray:
+    """Multi-token decode step: O[B, L, q_len, Hq, d] in float64.
+
+    q: [B, L, q_len, Hq, d] stored values, gate_logits: [B, L-1, q_len, Hq]; p carries the caches, windows (in age
+    order, oldest entry in slot 0) and seq_lens AFTER all q_len tokens of the step were appended. The loops are
+    displaced by whole tokens (Sec. 2.2.1), so token j (oldest first) of every loop is served exactly as a single-token
+    step would have served it q_len-1-j tokens earlier: it sees that many fewer entries of the shared cache and that
+    many fewer (the newest) slots of its loop's window. Written as q_len calls of the single-token definition above,
+    each on the shortened lengths."""
+    from dataclasses import replace
+    B, L = p.B, p.L
+    delta = list(range(L)) if p.loop_offset is None else [int(x) for x in p.loop_offset]
+    out = np.zeros((B, L, q_len, p.Hq, p.d), dtype=np.float64)
+    for j in range(q_len):
+        newer = q_len - 1 - j
+        lens = np.maximum(p.seq_lens.astype(np.int64) - newer, 0).astype(np.int32)
+        win = None
+        if L > 1:
+            win = np.zeros((B, L - 1), dtype=np.int32)
+            for b in range(B):
+                for l in range(1, L):
+                    cut_loop = max(0, int(p.seq_lens[b]) - delta[l])          # keys the loop's newest token sees
+                    wl_loop = min(p.w, cut_loop) if p.win_lens is None else int(np.clip(p.win_lens[b, l - 1], 0, p.w))
+                    win[b, l - 1] = max(0, wl_loop - newer)
+        pj = replace(p, q=np.ascontiguousarray(q[:, :, j]), seq_lens=lens, win_lens=win,
+                     gate_logits=np.ascontiguousarray(gate_logits[:, :, j]) if L > 1 else p.gate_logits)
+        out[:, :, j] = decode_attn(pj)
+    return out
