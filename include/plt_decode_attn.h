@@ -81,8 +81,8 @@ typedef enum {
 
 /*
  * Fixed at create.  struct_size = sizeof(plt_decode_attn_config) (versioning).
- * Supported: d in {64, 128}; Hq % Hkv == 0; L * (Hq / Hkv) <= 64 packed query
- * rows per KV head; L <= 8; paged caches need page_size % 16 == 0.
+ * Supported: d in {64, 128}; Hq % Hkv == 0; L * q_len * (Hq / Hkv) <= 64 packed
+ * query rows per KV head; L <= 8; paged caches need page_size % 16 == 0.
  */
 typedef struct {
     uint32_t struct_size;
@@ -109,6 +109,15 @@ typedef struct {
     int32_t row_warps;     /* PLT_PATH_WARP_MMA: warps that split the L * Hq/Hkv packed rows of a KV head (1 or 2; each
                               takes at most 32 rows) */
     int32_t kv_dtype;      /* plt_kv_dtype of k_cache, v_cache, k_win, v_win; strides are then in bytes (= elements) */
+    int32_t q_len;         /* query tokens per loop in one step (multi-token / speculative decode); 0 or 1: one.
+                              With q_len = Qn > 1 (bf16, PLT_PATH_WARP_MMA only; L * Qn * Hq/Hkv <= 64): q and out are
+                              [B, L, Qn, Hq, d] and gate_logits [B, L-1, Qn, Hq], token j = 0..Qn-1 oldest first; the
+                              caller has appended all Qn tokens of the step (N_b counts them; each window holds its
+                              loop's newest entries IN AGE ORDER, oldest in slot 0). Token j of loop l is served as it
+                              would have been Qn-1-j steps earlier: it sees the first cut(b,l) - (Qn-1-j) entries of the
+                              shared cache and the first wl - (Qn-1-j) slots of its loop's window (the loops are
+                              displaced by whole tokens, Sec. 2.2.1, so the causal cutoff moves by one per token).
+                              plt_decode_attn_step and plt_decode_attn_run_host take q_len <= 1 only. */
 } plt_decode_attn_config;
 
 /*

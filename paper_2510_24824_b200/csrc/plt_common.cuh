@@ -8,7 +8,7 @@
 namespace plt {
 
 constexpr int kMaxLoops = 8;
-constexpr int kMaxRows = 64;     // packed query rows per KV head: L * (Hq / Hkv)
+constexpr int kMaxRows = 64;     // packed query rows per KV head: L * q_len * (Hq / Hkv)
 constexpr int kMaxBatch = 4096;
 
 // Device status bits (mirrors the PLT_DEV_* values of the public header).
@@ -39,6 +39,7 @@ struct Params {
     uint32_t* status;          // device status word
     int64_t kv_stride_b, kv_stride_n, kv_stride_h;  // elements
     int32_t B, L, Hq, Hkv, G, R, d, w;
+    int32_t Qn;                // query tokens per loop in this step (multi-token decode); packed row = (loop * Qn + token) * G + head in group
     int32_t max_seq_len, page_size, max_pages, num_pool_pages;
     int32_t hpc;               // KV heads per work item
     int32_t tile_keys;         // keys per plan tile

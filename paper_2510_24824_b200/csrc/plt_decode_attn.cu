@@ -42,7 +42,7 @@ struct Staging {
 struct plt_decode_attn {
     plt_decode_attn_config cfg;
     int32_t delta[kMaxLoops];
-    int G, R;
+    int G, R, Qn = 1;
     bool bf16;
     int sm_count;
     MainVariant var;      // bf16: full variant; fp32: only grid/smem used
@@ -87,7 +87,7 @@ plt_status cuda_fail(plt_decode_attn_t h, const char* what, cudaError_t e) {
 int elem_size(bool bf16) { return bf16 ? 2 : 4; }
 
 struct Geometry {
-    int G, R;
+    int G, R, Qn;
 };
 
 plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
@@ -111,10 +111,14 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
         if (c->kernel_path == PLT_PATH_TCGEN05)
             return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches are served by the warp-level kernel only");
     }
+    if (c->q_len < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "q_len %d < 0", c->q_len);
+    g->Qn = c->q_len > 1 ? c->q_len : 1;
+    if (g->Qn > 1 && (c->dtype != PLT_BF16 || c->kernel_path == PLT_PATH_TCGEN05))
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "q_len > 1 is served by the warp-level bf16 kernel only");
     g->G = c->Hq / c->Hkv;
-    g->R = c->L * g->G;
+    g->R = c->L * g->Qn * g->G;
     if (g->R > kMaxRows)
-        return fail(nullptr, PLT_ERR_UNSUPPORTED, "L * Hq/Hkv = %d packed rows > %d", g->R, kMaxRows);
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "L * q_len * Hq/Hkv = %d packed rows > %d", g->R, kMaxRows);
     if (c->page_size > 0 && c->page_size % 16 != 0)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "page_size %d is not a multiple of 16", c->page_size);
     if (c->loop_offset)
@@ -228,7 +232,7 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
-    if (c->kernel_path == PLT_PATH_WARP_MMA || c->kv_dtype == PLT_KV_E4M3) return false;
+    if (c->kernel_path == PLT_PATH_WARP_MMA || c->kv_dtype == PLT_KV_E4M3 || c->q_len > 1) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
@@ -360,6 +364,7 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     for (int l = 0; l < kMaxLoops; ++l) h->delta[l] = config->loop_offset && l < config->L ? config->loop_offset[l] : l;
     h->G = g.G;
     h->R = g.R;
+    h->Qn = g.Qn;
     h->bf16 = config->dtype == PLT_BF16;
     h->sm_count = prop.multiProcessorCount;
     const float scale = config->sm_scale > 0.f ? config->sm_scale : 1.0f / sqrtf((float)config->d);
@@ -414,6 +419,7 @@ PLT_API plt_status plt_decode_attn_step(plt_decode_attn_t h, const plt_decode_at
     if (h->cfg.L > 1 && (!step->w_gate || !step->b_gate || !step->gate_logits))
         return fail(h, PLT_ERR_INVALID_ARG, "w_gate, b_gate and gate_logits must not be NULL when L > 1");
     if (a->win_lens) return fail(h, PLT_ERR_INVALID_ARG, "win_lens must be NULL: the ring update fixes wl = min(w, cut)");
+    if (h->Qn > 1) return fail(h, PLT_ERR_UNSUPPORTED, "plt_decode_attn_step takes one query token per loop (q_len <= 1)");
     plt_decode_attn_args a2 = *a;
     a2.gate_logits = step->gate_logits;
     return run_impl(h, &a2, cuda_stream, step);
@@ -470,6 +476,7 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
     p.status = h->status;
     p.kv_stride_b = sb; p.kv_stride_n = sn; p.kv_stride_h = sh;
     p.B = a->batch; p.L = c.L; p.Hq = c.Hq; p.Hkv = c.Hkv; p.G = h->G; p.R = h->R; p.d = c.d; p.w = c.w;
+    p.Qn = h->Qn;
     p.max_seq_len = c.max_seq_len; p.page_size = c.page_size; p.max_pages = a->max_pages;
     p.num_pool_pages = a->num_pool_pages;
     p.hpc = h->var.HPC;
@@ -564,6 +571,7 @@ PLT_API plt_status plt_decode_attn_run_host(plt_decode_attn_t h, const plt_decod
     if (a->batch == 0) return PLT_OK;
     if (a->kv_stride_b || a->kv_stride_n || a->kv_stride_h)
         return fail(h, PLT_ERR_UNSUPPORTED, "run_host takes dense shared caches only (strides must be 0)");
+    if (h->Qn > 1) return fail(h, PLT_ERR_UNSUPPORTED, "run_host takes one query token per loop (q_len <= 1)");
     if (!a->q || !a->k_cache || !a->v_cache || !a->seq_lens || !a->out)
         return fail(h, PLT_ERR_INVALID_ARG, "q, k_cache, v_cache, seq_lens and out must not be NULL");
     cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -744,7 +752,8 @@ bool same_config(const NoAllocDevice& dv, const plt_decode_attn_config* c) {
         a.page_size != c->page_size || memcmp(&a.sm_scale, &c->sm_scale, sizeof(float)) != 0 || a.device != c->device ||
         a.heads_per_cta != c->heads_per_cta || a.key_slices != c->key_slices || a.stages != c->stages ||
         a.ctas_per_sm != c->ctas_per_sm || a.kernel_path != c->kernel_path || a.loads_in_flight != c->loads_in_flight ||
-        a.slices_per_warp != c->slices_per_warp || a.row_warps != c->row_warps || a.kv_dtype != c->kv_dtype)
+        a.slices_per_warp != c->slices_per_warp || a.row_warps != c->row_warps || a.kv_dtype != c->kv_dtype ||
+        a.q_len != c->q_len)
         return false;
     for (int l = 0; l < c->L; ++l)
         if ((c->loop_offset ? c->loop_offset[l] : l) != dv.offsets[l]) return false;
@@ -785,6 +794,7 @@ extern "C" PLT_API plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn
         for (int l = 0; l < kMaxLoops; ++l) h->delta[l] = config->loop_offset && l < config->L ? config->loop_offset[l] : l;
         h->G = g.G;
         h->R = g.R;
+        h->Qn = g.Qn;
         h->bf16 = config->dtype == PLT_BF16;
         h->sm_count = dv.sm_count;
         const float scale = config->sm_scale > 0.f ? config->sm_scale : 1.0f / sqrtf((float)config->d);

@@ -483,13 +483,17 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const int rb = rw * C::ROWS_W;              // first packed row of this warp
         const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
         // Rows as the accumulator fragments see them: column 2 tq + j of 8-row group nt.
-        int lc[NT][2];                               // loop (0-based) of the row, kMaxLoops for rows beyond R
+        // loop (0-based) of the row in the low byte, kMaxLoops for rows beyond R; above it how many of the step's
+        // tokens of that loop are NEWER than the row's (0 with one query token per loop): the row sees that many fewer
+        // keys of the shared cache and that many fewer slots of its (age-ordered) window
+        int lc[NT][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int r = rb + nt * 8 + 2 * tq + j;
-                lc[nt][j] = r < p.R ? r / p.G : kMaxLoops;
+                const int lq = r / p.G;               // loop * Qn + token
+                lc[nt][j] = r < p.R ? (lq / p.Qn) | ((p.Qn - 1 - lq % p.Qn) << 8) : kMaxLoops;
             }
 
         int stage = 0;
@@ -509,8 +513,8 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 for (int nt = 0; nt < NT; ++nt) {
                     const int r = rb + nt * 8 + grp;
                     const bool v = r < p.R;
-                    const int l = v ? r / p.G : 0;
-                    const int64_t qrow = (((int64_t)pc.b * p.L + l) * p.Hq + kvh * p.G + (r - l * p.G)) * D;
+                    const int lq = v ? r / p.G : 0;       // loop * Qn + token: q is [B, L, Qn, Hq, d]
+                    const int64_t qrow = (((int64_t)pc.b * p.L * p.Qn + lq) * p.Hq + kvh * p.G + (r - lq * p.G)) * D;
                     if constexpr (FP8) {
                         // contraction order of process_keys_fp8: k-step ks takes d = 16 ks + 4 tq .. + 3; bf16 -> f16
 #pragma unroll
@@ -537,11 +541,11 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int l = 0; l < kMaxLoops; ++l)
                 if (l < p.L) {
                     const int c = pc.sp.cut[l];
-                    cmin = min(cmin, c);
+                    cmin = min(cmin, max(c - (p.Qn - 1), 0));
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        if (lc[nt][0] == l) cutr[nt][0] = c;
-                        if (lc[nt][1] == l) cutr[nt][1] = c;
+                        if ((lc[nt][0] & 0xff) == l) cutr[nt][0] = max(c - (lc[nt][0] >> 8), 0);
+                        if ((lc[nt][1] & 0xff) == l) cutr[nt][1] = max(c - (lc[nt][1] >> 8), 0);
                     }
                 }
             float acc[D / 16][NT][4], mref[NT][2], lacc[NT][4];
@@ -597,14 +601,14 @@ plt_decode_main_bf16(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
                     for (int k = 1; k < kMaxLoops; ++k)
                         if (k == l) wl = pc.sp.wl[k];
-                    const int row_lo = l * p.G, row_hi = row_lo + p.G;
+                    const int row_lo = l * p.Qn * p.G, row_hi = row_lo + p.Qn * p.G;
                     const bool any = row_lo < rb + C::ROWS_W && row_hi > rb;
                     if (ok && any) {
                         const int n = wl - cur.key0;
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-                            lim[nt][0] = lc[nt][0] == l ? n : 0;
-                            lim[nt][1] = lc[nt][1] == l ? n : 0;
+                            lim[nt][0] = (lc[nt][0] & 0xff) == l ? n - (lc[nt][0] >> 8) : 0;
+                            lim[nt][1] = (lc[nt][1] & 0xff) == l ? n - (lc[nt][1] >> 8) : 0;
                         }
                         if constexpr (FP8)
                             process_keys_fp8<D, NT, KS, HPC, KW, C::TK, true>(sK, sV, qb, acc, mref, lacc, lim, n, sc2, lane, kw,

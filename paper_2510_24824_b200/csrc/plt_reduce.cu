@@ -105,24 +105,28 @@ __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __g
     const int row = chunk * kReduceWarps + wid;   // packed row of this head group: hl * R + r
     if (row >= p.hpc * p.R) return;
     const int hl = row / p.R, r = row - hl * p.R;
-    const int l = r / p.G, g = r - l * p.G;
+    const int lq = r / p.G, g = r - lq * p.G;        // lq = loop * Qn + token of the step
+    const int l = lq / p.Qn, newer = p.Qn - 1 - lq % p.Qn;   // tokens of this loop in the step that are newer than the row's
     const int h = (hg * p.hpc + hl) * p.G + g;
 
     // What the caller passed (length, window length, gate logit) is read while the main kernel still drains; this
     // row's loop alone decides what is merged: cut = keys of the shared cache it may see, wl = its window's valid slots.
     uint32_t flags = 0;
     const int32_t n = seq_len_clamped(p, b, flags);
-    int cut = n - p.delta[l];
+    int cut_loop = n - p.delta[l];                    // keys the loop's newest token sees
+    cut_loop = cut_loop > 0 ? cut_loop : 0;
+    int cut = cut_loop - newer;                       // keys this row sees
     cut = cut > 0 ? cut : 0;
     int wl = 0;
     float x = 0.f;
     if (l > 0) {
-        wl = cut < p.w ? cut : p.w;
-        if (p.win_lens != nullptr && cut > 0) {
+        wl = cut_loop < p.w ? cut_loop : p.w;
+        if (p.win_lens != nullptr && cut_loop > 0) {
             wl = p.win_lens[b * (p.L - 1) + (l - 1)];
             wl = wl < 0 ? 0 : (wl > p.w ? p.w : wl);
         }
-        x = p.gate_logits[((int64_t)b * (p.L - 1) + (l - 1)) * p.Hq + h];
+        // wl > 0 says that the loop's window item exists; a row that sees none of its slots finds an empty partial
+        x = p.gate_logits[(((int64_t)b * (p.L - 1) + (l - 1)) * p.Qn + (lq - l * p.Qn)) * p.Hq + h];
     }
     const int item_g = item_index(p, b, hg, 0), item_l = item_index(p, b, hg, 1);
 
@@ -174,7 +178,7 @@ __global__ void __launch_bounds__(kReduceWarps * 32) plt_decode_reduce(const __g
             for (int i = 0; i < Vec<D>::N; ++i) out[i] = gate * (yl.v[i] * il) + (1.f - gate) * (yg.v[i] * ig);
         }
     }
-    const int64_t o = (((int64_t)b * p.L + l) * p.Hq + h) * D + lane * Vec<D>::N;
+    const int64_t o = (((int64_t)b * p.L * p.Qn + lq) * p.Hq + h) * D + lane * Vec<D>::N;
     if (BF16) {
         __nv_bfloat16* dst = (__nv_bfloat16*)p.out + o;
         if constexpr (Vec<D>::N == 4) {
