@@ -1,8 +1,9 @@
 // Sequence-shaped PLT attention (prefill / training-forward; Algorithm 2 with the attention of Algorithm 3) on the
 // 5th-generation tensor cores: tcgen05.mma with the QUERIES as the M dimension and accumulators in tensor memory.
 //
-// One thread block owns 256 consecutive rows t of one (sequence, loop, query head): two 128-row query tiles A and B,
-// each with its own score tile S (128 lanes x 128 fp32 columns of tensor memory) and output tile O (128 x 128).
+// One thread block owns two 128-row query tiles A and B of one (sequence, loop): the same 128 rows t of two query heads
+// that share a KV head (any even GQA group), else 256 consecutive rows of one head. Each tile has its own score tile S
+// (128 lanes x 128 fp32 columns of tensor memory) and output tile O (128 x 128).
 //
 //   S_X [128 rows x 128 keys] = Q_X [128 x d] . K_tile^T [d x 128]     A = Q tile, B = K tile, both as TMA wrote them
 //                                                                      (K-major, 128-byte swizzle)
@@ -68,7 +69,8 @@ struct SeqParams {
     const int32_t* seq_lens;    // [B]
     __nv_bfloat16* out;         // [B, L, T, Hq, d]
     uint32_t* status;
-    int32_t B, L, T, Hq, Hkv, G, w, nqb;   // nqb: 256-row blocks per sequence
+    int32_t B, L, T, Hq, Hkv, G, w, nqb;   // nqb: row blocks per sequence (128 rows with paired heads, else 256)
+    int32_t pair_heads, heads_per_grid;      // tiles of a block = two heads of one KV group; grid entries per (row block, loop)
     float scale_log2;
     int32_t delta[kSeqMaxLoops];
 };
@@ -345,11 +347,16 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     // ---- which rows ------------------------------------------------------------------------------------
     // Blocks with the most key tiles (the last rows of a sequence) come first in the grid.
+    // The block's two tiles are, where two query heads share a KV head (an even GQA group), the SAME 128 rows of two
+    // neighbouring heads: both then walk exactly the same key tiles with the same masks, every K/V tile in shared memory
+    // serves two products and neither tile idles on a step. Otherwise they are two consecutive 128-row tiles of one head
+    // (the second then has one more key tile than the first).
     int item = blockIdx.x;
-    const int h = item % p.Hq; item /= p.Hq;
+    const int hh = item % p.heads_per_grid; item /= p.heads_per_grid;
     const int l = item % p.L; item /= p.L;
     const int b = item % p.B; item /= p.B;
     const int qb = p.nqb - 1 - item;
+    const int hA = p.pair_heads ? 2 * hh : hh, hB = p.pair_heads ? 2 * hh + 1 : hh;
     uint32_t flags = 0;
     int n = p.seq_lens[b];
     if (n < 0 || n > p.T) {
@@ -357,8 +364,8 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         n = n < 0 ? 0 : p.T;
     }
     const int delta = p.delta[l];
-    const int r0A = qb * 2 * SQ, r0B = r0A + SQ;
-    const int kvh = h / p.G;
+    const int r0A = p.pair_heads ? qb * SQ : qb * 2 * SQ, r0B = p.pair_heads ? r0A : r0A + SQ;
+    const int kvh = hA / p.G;
 
     SeqPlan pl;
     {
@@ -432,7 +439,7 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!(x == 0 ? activeA : activeB)) continue;
                 const int r0 = x == 0 ? r0A : r0B;
                 for (int hf = 0; hf < 2; ++hf)
-                    tma_load_4d(q_smem + x * kTileBytes + hf * kHalf, &tmQ, &bars[SB_QFULL], hf * 64, h, r0, b * p.L + l, keep);
+                    tma_load_4d(q_smem + x * kTileBytes + hf * kHalf, &tmQ, &bars[SB_QFULL], hf * 64, x == 0 ? hA : hB, r0, b * p.L + l, keep);
             }
             SeqRing rg;
             uint32_t issued = 0;
@@ -580,6 +587,7 @@ plt_seq_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int wq = wid & 3;                            // lane quarter of tensor memory this warp may touch
         const bool active = x == 0 ? activeA : activeB;
         const int r0 = x == 0 ? r0A : r0B;
+        const int h = x == 0 ? hA : hB;
         RowCtx rc;
         rc.t = r0 + wq * 32 + lane;
         rc.cut = max(0, min(rc.t, n - 1) + 1 - delta);
@@ -876,10 +884,12 @@ PLT_API plt_status plt_seq_attn_run(plt_seq_attn_t h, const plt_seq_attn_args* a
     p.out = (__nv_bfloat16*)a->out;
     p.status = h->status;
     p.B = a->batch; p.L = c.L; p.T = T; p.Hq = c.Hq; p.Hkv = c.Hkv; p.G = c.Hq / c.Hkv; p.w = c.w;
-    p.nqb = (T + 2 * SQ - 1) / (2 * SQ);
+    p.pair_heads = (p.G % 2 == 0) ? 1 : 0;
+    p.heads_per_grid = p.pair_heads ? p.Hq / 2 : p.Hq;
+    p.nqb = p.pair_heads ? (T + SQ - 1) / SQ : (T + 2 * SQ - 1) / (2 * SQ);
     p.scale_log2 = h->scale_log2;
     for (int l = 0; l < kSeqMaxLoops; ++l) p.delta[l] = h->delta[l];
-    const unsigned grid = (unsigned)((int64_t)p.nqb * p.B * p.L * p.Hq);
+    const unsigned grid = (unsigned)((int64_t)p.nqb * p.B * p.L * p.heads_per_grid);
     plt_seq_attn_kernel<<<grid, kSeqThreads, kSeqSmem, (cudaStream_t)cuda_stream>>>(h->maps[0], h->maps[1], h->maps[2],
                                                                                     h->maps[3], h->maps[4], p);
     cudaError_t e = cudaGetLastError();

@@ -31,6 +31,15 @@ def oracle_seq(p):
         return oracle.seq_attn(p)
 
 
+def oracle_seq_planes(p, planes):
+    with np.errstate(over="ignore"):
+        return oracle.seq_attn(p, planes)
+
+
+def oracle_f32(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32)
+
+
 # lengths around the tile sizes (128-key tiles, 256 rows per block), loop counts of the paper, window 64
 @pytest.mark.parametrize("L", [2, 3])
 @pytest.mark.parametrize("n", [1, 127, 128, 129, 255, 256, 257, 700])
@@ -124,3 +133,18 @@ def test_argument_errors_and_clamped_lengths():
         assert op.check() == B.PLT_DEV_SEQ_LEN_CLAMPED
         clamped = p.with_(seq_lens=np.array([200, 0], dtype=np.int32))
         assert_parity(op.out.float().cpu().numpy().astype(np.float64), oracle_seq(clamped), "bf16", "clamped")
+
+
+def test_bench_shape_sampled_planes():
+    """The shape bench.py times (B=4, L=2, n=5000, GQA 32/8, w=64), checked on sampled (sequence, loop, head) planes the
+    oracle computes one by one, plus properties that hold for every row."""
+    p = make_seq_problem(B=4, L=2, T=5000, Hq=32, Hkv=8, d=128, w=64, seed=0, name="seq_B4_L2_n5000")
+    got = run_seq(p)
+    assert np.isfinite(got).all()
+    vmax = float(max(np.abs(oracle_f32(p.v_share)).max(), np.abs(oracle_f32(p.v_loc)).max()))
+    assert np.abs(got).max() <= vmax * (1 + 2 ** -7)              # convex mixes of V rows
+    assert np.all(got[:, 1, 0] == 0.0)                            # loop 2 has no token at step 0 (delta = 1)
+    planes = [(0, 0, 0), (1, 1, 5), (2, 0, 31), (3, 1, 16), (0, 1, 30), (2, 1, 9)]
+    ref = oracle_seq_planes(p, planes)
+    for b, l, h in planes:
+        assert_parity(got[b, l, :, h], ref[b, l, :, h], "bf16", f"plane {(b, l, h)}")
