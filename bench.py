@@ -566,7 +566,7 @@ def main():
         peak, peak_src = peak_hbm()
         main_bytes = main_kernel_bytes(by)
         achieved = main_bytes / (main_avg_ms * 1e-3) / 1e9
-        kernel_name = {1: "plt_decode_main_" + p.dtype, 2: "plt_decode_main_umma"}[kernel_path]
+        kernel_name = {1: "plt_decode_main_" + p.dtype, 2: "plt_decode_main_umma" + ("_e4m3" if p.kv_dtype else "")}[kernel_path]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

@@ -46,7 +46,10 @@ struct plt_decode_attn {
     bool bf16;
     int sm_count;
     MainVariant var;      // bf16: full variant; fp32: only grid/smem used
-    bool umma = false;    // bf16 path on tcgen05 / tensor memory (var.HPC = 1, var.KW = 8, var.stages = ring slots)
+    bool umma = false;    // path on tcgen05 / tensor memory (var.HPC = 1, var.KW = 8, var.stages = ring slots)
+    bool umma_e4m3 = false;  // ... its kernel for E4M3 caches
+    uint8_t* qimg = nullptr;  // that kernel's query images and their scale factors (inside the workspace)
+    float* qinv = nullptr;
     int kbox = 0, wbox = 0;  // keys per TMA box of the shared cache / of a window on that path
     int ctas_per_sm;
     int piece_cost = 0;   // Params::piece_cost of the main kernel in use
@@ -108,8 +111,6 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
     if (c->kv_dtype == PLT_KV_E4M3) {
         if (c->dtype != PLT_BF16 || c->d != 128)
             return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches need bf16 queries and head dim 128");
-        if (c->kernel_path == PLT_PATH_TCGEN05)
-            return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches are served by the warp-level kernel only");
     }
     if (c->q_len < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "q_len %d < 0", c->q_len);
     g->Qn = c->q_len > 1 ? c->q_len : 1;
@@ -119,6 +120,8 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
     g->R = c->L * g->Qn * g->G;
     if (g->R > kMaxRows)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "L * q_len * Hq/Hkv = %d packed rows > %d", g->R, kMaxRows);
+    if (c->kv_dtype == PLT_KV_E4M3 && c->kernel_path == PLT_PATH_TCGEN05 && g->R > 32)
+        return fail(nullptr, PLT_ERR_UNSUPPORTED, "the tcgen05 path takes E4M3 caches up to 32 packed rows (%d here)", g->R);
     if (c->page_size > 0 && c->page_size % 16 != 0)
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "page_size %d is not a multiple of 16", c->page_size);
     if (c->loop_offset)
@@ -190,13 +193,40 @@ plt_status choose_variant(const plt_decode_attn_config* c, const Geometry& g, Ma
     return PLT_OK;
 }
 
-size_t workspace_bytes_for(const plt_decode_attn_config* c, const Geometry& g, int hpc, int grid, size_t* acc_floats,
-                           size_t* ml_floats) {
+// Workspace: split partials, first / last block of every item, tile prefix, status word; for the tcgen05 kernel on
+// E4M3 caches also one query image and one scale factor per (sequence, KV head), from a 256-byte boundary on.
+size_t workspace_base_bytes(const plt_decode_attn_config* c, int hpc, size_t acc_floats, size_t ml_floats) {
+    const size_t items = (size_t)c->max_batch * (c->Hkv / hpc) * 2;
+    return (acc_floats + ml_floats) * 4 + items * 8 + (size_t)(c->max_batch + 1) * 4 + 256;
+}
+
+size_t workspace_bytes_for(const plt_decode_attn_config* c, const Geometry& g, int hpc, int grid, bool e4m3_images,
+                           size_t* acc_floats, size_t* ml_floats) {
     const size_t slots = (size_t)c->max_batch * (c->Hkv / hpc) * 2 + (size_t)grid;
     *acc_floats = slots * hpc * g.R * c->d;
     *ml_floats = slots * hpc * g.R * 2;
-    const size_t items = (size_t)c->max_batch * (c->Hkv / hpc) * 2;
-    return (*acc_floats + *ml_floats) * 4 + items * 8 + (size_t)(c->max_batch + 1) * 4 + 256;
+    size_t bytes = workspace_base_bytes(c, hpc, *acc_floats, *ml_floats);
+    if (e4m3_images) {
+        const size_t n = (size_t)c->max_batch * c->Hkv;
+        bytes = ((bytes + 255) & ~(size_t)255) + n * main_umma_e4m3_image_bytes(g.R) + n * 4 + 256;
+    }
+    return bytes;
+}
+
+// Points the handle's workspace pointers into `ws` (256-byte aligned, workspace_bytes_for bytes).
+void place_workspace(plt_decode_attn* h, const plt_decode_attn_config* c, void* ws, size_t acc_floats, size_t ml_floats) {
+    h->part_acc = (float*)ws;
+    h->part_ml = h->part_acc + acc_floats;
+    h->item_blocks = (int32_t*)(h->part_ml + ml_floats);   // 16-byte aligned: both float counts are multiples of 4
+    h->prefix = h->item_blocks + (size_t)c->max_batch * (c->Hkv / h->var.HPC) * 4;
+    h->status = (uint32_t*)(h->prefix + c->max_batch + 1);
+    h->qimg = nullptr;
+    h->qinv = nullptr;
+    if (h->umma_e4m3) {
+        const size_t base = (workspace_base_bytes(c, h->var.HPC, acc_floats, ml_floats) + 255) & ~(size_t)255;
+        h->qimg = (uint8_t*)ws + base;
+        h->qinv = (float*)(h->qimg + (size_t)c->max_batch * c->Hkv * main_umma_e4m3_image_bytes(h->R));
+    }
 }
 
 plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, int D, int64_t d1, int64_t d2, int64_t d3,
@@ -219,7 +249,8 @@ plt_status encode_map(plt_decode_attn_t h, int idx, const void* base, int es, in
     return PLT_OK;
 }
 
-// Can the tcgen05 kernel take this configuration? (bf16, d = 128, pages that tile or are tiled by 128 keys)
+// Can a tcgen05 kernel take this configuration? (bf16, d = 128, pages that tile or are tiled by 128 keys; with E4M3
+// caches at most 32 packed rows, which check_config has already seen to)
 bool umma_eligible(const plt_decode_attn_config* c) {
     if (c->dtype != PLT_BF16 || c->d != 128) return false;
     if (c->page_size > 0 && c->page_size % 128 != 0 && 128 % c->page_size != 0) return false;
@@ -232,8 +263,9 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
-    if (c->kernel_path == PLT_PATH_WARP_MMA || c->kv_dtype == PLT_KV_E4M3 || c->q_len > 1) return false;
+    if (c->kernel_path == PLT_PATH_WARP_MMA || c->q_len > 1) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
+    if (c->kv_dtype == PLT_KV_E4M3) return false;
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
     return umma_eligible(c) && c->L * (c->Hq / c->Hkv) > 48 && c->max_seq_len >= 16384 &&
@@ -253,7 +285,28 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
     if (config->kernel_path == PLT_PATH_TCGEN05 && !umma_eligible(config))
         return fail(nullptr, PLT_ERR_UNSUPPORTED,
                     "the tcgen05 path needs bf16, d = 128 and a page size that divides or is a multiple of 128");
-    if (h->bf16 && want_umma(config)) {
+    h->umma_e4m3 = false;
+    if (h->bf16 && want_umma(config) && config->kv_dtype == PLT_KV_E4M3) {
+        // Ring slots of 32 KB (K and V tile of one head); 5 fit beside the probability and query buffers.
+        int nslot = config->stages;
+        if (nslot == 0) nslot = main_umma_e4m3_max_slots();
+        if (nslot < 2 || nslot > main_umma_e4m3_max_slots())
+            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path with E4M3 caches (supported: 2 to %d ring slots)",
+                        nslot, main_umma_e4m3_max_slots());
+        const size_t smem = main_umma_e4m3_smem(g.R, nslot, config->max_batch);
+        if (smem > 227 * 1024)
+            return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 path needs %zu bytes of shared memory (> 227 KB)", smem);
+        e = main_umma_e4m3_prepare(g.R, smem, &blocks);
+        if (e != cudaSuccess) return cuda_fail(nullptr, "preparing the tcgen05 main kernel for E4M3 caches", e);
+        if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
+        h->umma = true;
+        h->umma_e4m3 = true;
+        h->var = MainVariant{config->d, 0, 0, 1, 4, 1, 128, nslot, 0, smem, true};
+        h->ctas_per_sm = 1;
+        h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)
+                                        : (config->max_seq_len < 128 ? config->max_seq_len : 128);
+        h->wbox = config->w < 128 ? (config->w > 0 ? config->w : 1) : 128;
+    } else if (h->bf16 && want_umma(config)) {
         // Ring slots: an even number, so that a slot is always refilled by the stream (K or V) that used it before.
         int nslot = config->stages;
         if (nslot == 0) nslot = main_umma_smem(g.R, 6, config->max_batch) <= 227 * 1024 ? 6 : 4;
@@ -328,8 +381,10 @@ PLT_API plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config*
     if (cudaGetDeviceProperties(&prop, config->device) == cudaSuccess) sms = prop.multiProcessorCount;
     else (void)cudaGetLastError();
     int hpc = 1, cps = config->ctas_per_sm > 0 ? config->ctas_per_sm : 2;
+    bool images = false;
     if (config->dtype == PLT_BF16 && want_umma(config)) {
         cps = 1;
+        images = config->kv_dtype == PLT_KV_E4M3;
     } else if (config->dtype == PLT_BF16) {
         MainVariant v;
         s = choose_variant(config, g, &v, &cps);
@@ -337,7 +392,7 @@ PLT_API plt_status plt_decode_attn_workspace_bytes(const plt_decode_attn_config*
         hpc = v.HPC;
     }
     size_t a, m;
-    *out_bytes = workspace_bytes_for(config, g, hpc, sms * cps, &a, &m);
+    *out_bytes = workspace_bytes_for(config, g, hpc, sms * cps, images, &a, &m);
     return PLT_OK;
 }
 
@@ -375,7 +430,7 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
     if (s != PLT_OK) { delete h; return s; }
 
     size_t acc_floats, ml_floats;
-    h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
+    h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, h->umma_e4m3, &acc_floats, &ml_floats);
     void* ws = nullptr;
     e = cudaMalloc(&ws, h->ws_bytes);
     if (e != cudaSuccess) {
@@ -383,11 +438,7 @@ PLT_API plt_status plt_decode_attn_create(const plt_decode_attn_config* config, 
         delete h;
         return fail(nullptr, PLT_ERR_OUT_OF_MEMORY, "cudaMalloc of %zu workspace bytes failed", h->ws_bytes);
     }
-    h->part_acc = (float*)ws;
-    h->part_ml = h->part_acc + acc_floats;
-    h->item_blocks = (int32_t*)(h->part_ml + ml_floats);   // 16-byte aligned: both float counts are multiples of 4
-    h->prefix = h->item_blocks + (size_t)config->max_batch * (config->Hkv / h->var.HPC) * 4;
-    h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
+    place_workspace(h, config, ws, acc_floats, ml_floats);
     e = cudaMemset(h->status, 0, 4);
     if (e != cudaSuccess) { cudaFree(ws); delete h; return cuda_fail(nullptr, "cudaMemset", e); }
     *out_handle = h;
@@ -519,8 +570,15 @@ plt_status run_impl(plt_decode_attn_t h, const plt_decode_attn_args* a, void* cu
             h->maps[2] = h->maps[0];
             h->maps[3] = h->maps[1];
         }
+        if (h->umma_e4m3) {
+            e = launch_pack_q_e4m3(p, h->qimg, h->qinv, stream);
+            if (e != cudaSuccess) return cuda_fail(h, "launching the query pack kernel", e);
+        }
         if (h->ev_begin) cudaEventRecord(h->ev_begin, stream);
-        if (h->umma)
+        if (h->umma_e4m3)
+            e = launch_main_umma_e4m3(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox,
+                                      c.loads_in_flight > 0 ? c.loads_in_flight : 4, h->qimg, h->qinv, stream);
+        else if (h->umma)
             e = launch_main_umma(h->maps, p, h->var.grid, h->var.smem, h->var.stages, h->kbox, h->wbox,
                                  c.loads_in_flight > 0 ? c.loads_in_flight : 2, stream);
         else
@@ -674,7 +732,7 @@ PLT_API plt_status plt_decode_attn_launch_info(plt_decode_attn_t h, int32_t* ker
                                        int32_t* key_slices, int32_t* stages, int32_t* ctas_per_sm, int32_t* grid,
                                        int32_t* kernel_path) {
     if (!h) return fail(nullptr, PLT_ERR_INVALID_ARG, "handle is NULL");
-    if (kernels_per_run) *kernels_per_run = 2;
+    if (kernels_per_run) *kernels_per_run = h->umma_e4m3 ? 3 : 2;   // (query pack,) main, merge
     if (heads_per_cta) *heads_per_cta = h->var.HPC;
     if (key_slices) *key_slices = h->var.KW;
     if (stages) *stages = h->var.stages;
@@ -804,17 +862,13 @@ extern "C" PLT_API plt_status plt_decode_attn_run_no_alloc(const plt_decode_attn
         s = setup_kernels(h, config, g);
         if (s != PLT_OK) return s;
         size_t acc_floats, ml_floats;
-        h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, &acc_floats, &ml_floats);
+        h->ws_bytes = workspace_bytes_for(config, g, h->var.HPC, h->var.grid, h->umma_e4m3, &acc_floats, &ml_floats);
         if (h->ws_bytes > kNoAllocScratchBytes)
             return fail(nullptr, PLT_ERR_CAPACITY,
                         "this configuration needs %zu bytes of scratch but the built-in array holds %zu: lower max_batch "
                         "(scratch grows with max_batch * Hkv * L * Hq/Hkv * d) or use plt_decode_attn_create",
                         h->ws_bytes, kNoAllocScratchBytes);
-        h->part_acc = (float*)dv.scratch;
-        h->part_ml = h->part_acc + acc_floats;
-        h->item_blocks = (int32_t*)(h->part_ml + ml_floats);
-        h->prefix = h->item_blocks + (size_t)config->max_batch * (config->Hkv / h->var.HPC) * 4;
-        h->status = (uint32_t*)(h->prefix + config->max_batch + 1);
+        place_workspace(h, config, dv.scratch, acc_floats, ml_floats);
         dv.cfg = *config;
         for (int l = 0; l < kMaxLoops; ++l) dv.offsets[l] = h->delta[l];
         dv.have_handle = true;

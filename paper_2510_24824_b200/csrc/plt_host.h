@@ -62,6 +62,18 @@ cudaError_t main_umma_prepare(int R, size_t smem, int* blocks_per_sm);
 cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                              int wbox, int cap, cudaStream_t stream);
 
+// The same layout for E4M3 caches (tcgen05.mma kind::f8f6f4 on the codes, up to 32 packed rows; queries and
+// probabilities as sums of E4M3 terms). `qimg` / `qinv`: device scratch of max_batch * Hkv query images
+// (main_umma_e4m3_image_bytes each) and as many floats, written by a pack kernel launched first.
+int main_umma_e4m3_rows(int R);       // 16 or 32
+int main_umma_e4m3_max_slots();
+size_t main_umma_e4m3_smem(int R, int nslot, int max_batch);
+size_t main_umma_e4m3_image_bytes(int R);
+cudaError_t main_umma_e4m3_prepare(int R, size_t smem, int* blocks_per_sm);
+cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream);
+cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
+                                  int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream);
+
 // Pre-step of a decode step: shared-cache append, window ring update, gate linear (writes through p.k_cache,
 // p.v_cache, p.k_win, p.v_win, which the attention kernels only read).
 cudaError_t launch_prestep(const Params& p, bool bf16, const void* k_new, const void* v_new, const float* w_gate,

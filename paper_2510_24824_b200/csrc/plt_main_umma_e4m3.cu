@@ -1,0 +1,722 @@
+// Split-KV main kernel of the CLP decode attention for E4M3 caches on the 5th-generation tensor cores
+// (tcgen05.mma kind::f8f6f4 reading the codes from shared memory as TMA wrote them, accumulators in tensor
+// memory), head dimension 128, up to 32 packed query rows.
+//
+// y_global and y_local of Algorithm 3 for all L loops, same tile plan and split-partial format as the other main
+// kernels: one persistent block per SM walks its share of the line of 128-key tiles, one KV head per work item.
+// No code is converted on the way: both products take 8-bit operands, so the bf16 queries and the fp32
+// probabilities are each written as a SUM of E4M3 numbers and the terms are laid side by side along N:
+//
+//   S^T [128 keys x 2 RP]  = K_tile [128 x 128] . [Q_hi ; Q_lo]^T      A = K codes (K-major, 128-byte swizzle)
+//   O^T [128 dims x 3 RP] += V_tile^T [128 x 128] . [P_hi ; 2^10 P_mid ; 2^14 P_lo]^T   A = V codes (MN-major)
+//
+// A bf16 number times a power of two IS the sum of two E4M3 numbers (8 significant bits = 4 + 4) as long as its low
+// part stays above the E4M3 subnormal step, so the scores are those of the bf16 queries; a probability keeps 12
+// significant bits in three terms, the second and third scaled up by 2^10 and 2^14 so that probabilities far below
+// the E4M3 subnormal step (2^-9) still count: many keys of tiny weight next to one peak must not be dropped. The
+// softmax threads add the two score columns of a row, and the epilogue adds the three accumulator columns. One tcgen05.mma costs the same issue slot whatever N is, so the extra terms are
+// free on the tensor side: 8 instructions per 32 KB tile.
+//
+// Warp roles (192 threads): warps 0-3 softmax and epilogue (thread = key = tensor-memory lane); warp 4, one lane:
+// TMA producer of K and V tiles (one ring of 32 KB slots, K then V); warp 5, one lane: issues every product, copies
+// the packed query image of the next piece (cp.async.bulk) and owns the tensor-memory allocation.
+// The query image (codes in the core-matrix order the instruction reads, and the power of two they were scaled
+// by) is written per (sequence, KV head) by plt_decode_pack_q_e4m3, launched before this kernel.
+// Online softmax with a lazily updated reference maximum, as in the bf16 tcgen05 kernel. Every wait is bounded.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "plt_common.cuh"
+#include "plt_host.h"
+#include "plt_ptx.cuh"
+#include "plt_umma_util.cuh"
+
+namespace plt {
+
+namespace {
+
+constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 keys x 128 codes
+constexpr int kSlot8 = 2 * kTile8;     // a ring slot: the K tile, then the V tile
+constexpr int kMaxRing8 = 5;
+constexpr int kThreads8 = 192;
+// A probability may exceed the lazily updated reference by 3 powers of two at most (p <= 8), which fixes the powers of
+// two the second and third term are scaled by: |p - hi| <= 2^-2 and |p - hi - mid| <= 2^-7 times 2^10 and 2^14 stay
+// below 448. The third term then resolves 2^-23, the step of the f16 the probability is rounded to first.
+constexpr float kSlack8 = 3.f;
+constexpr uint32_t kMidScaleH2 = 0x64006400u;   // 2^10 as f16x2
+constexpr uint32_t kLoScaleH2 = 0x4c004c00u;    // 2^4 as f16x2 (on top of the 2^10)
+constexpr float kMidInv = 1.f / 1024.f, kLoInv = 1.f / 16384.f;
+
+// mbarrier indices
+constexpr int E_FULL = 0, E_EMPTY = 5, E_SFULL = 10 /* two */, E_SFREE = 12 /* two */, E_PFULL = 14 /* two */,
+              E_PFREE = 16 /* two */, E_OFULL = 18 /* two */, E_OFREE = 20 /* two */, E_QFULL = 22 /* two */,
+              E_DRAIN = 24, E_COUNT = 26;
+
+template <int RP>
+struct ECfg {
+    static constexpr int QLBO = 2 * RP * 16;   // bytes between the 16-code column chunks of the query image
+    static constexpr int QBUF = 8 * QLBO;      // [8 chunks][2 RP rows: hi then lo][16 codes]
+    static constexpr int PBUF = 3 * RP * UK;   // [3 RP / 16 row groups: hi, mid, lo][128 keys][16 codes]
+    // Tensor memory: two S^T buffers of 2 RP columns (tile parity), two O^T buffers of 3 RP columns (piece parity).
+    static constexpr int TMEM_COLS = RP == 16 ? 256 : 512;
+    __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
+        return 1024 + (size_t)nslot * kSlot8 + 2 * PBUF + 2 * QBUF + E_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 4) + 64 +
+               (size_t)(2 * max_batch + 4) * 4;
+    }
+};
+
+// ---- the query image ---------------------------------------------------------------------------------------
+// One block per (sequence, KV head), one thread per (packed row, 16-element chunk). q * 2^k = hi + lo with hi and lo
+// E4M3 numbers; 2^k puts the largest |q| of the block's rows into [128, 256).
+template <int RP>
+__global__ void __launch_bounds__(RP * 8) plt_decode_pack_q_e4m3(const Params p, uint8_t* qimg, float* qinv) {
+    using C = ECfg<RP>;
+    __shared__ float wmax[RP * 8 / 32];
+    const int b = blockIdx.x / p.Hkv, hg = blockIdx.x - b * p.Hkv;
+    const int r = threadIdx.x >> 3, c = threadIdx.x & 7;
+    float x[16];
+    float mx = 0.f;
+    if (r < p.R) {
+        const int l = r / p.G, g = r - l * p.G;
+        const __nv_bfloat16* src = (const __nv_bfloat16*)p.q + (((int64_t)b * p.L + l) * p.Hq + hg * p.G + g) * UD + c * 16;
+        uint4 raw[2] = {*(const uint4*)src, *(const uint4*)(src + 8)};
+        const __nv_bfloat162* h2 = (const __nv_bfloat162*)raw;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float2 f = __bfloat1622float2(h2[i]);
+            x[2 * i] = f.x;
+            x[2 * i + 1] = f.y;
+            mx = fmaxf(mx, fmaxf(fabsf(f.x), fabsf(f.y)));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = 0.f;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = wmax[0];
+#pragma unroll
+    for (int i = 1; i < RP * 8 / 32; ++i) mx = fmaxf(mx, wmax[i]);
+    // k = 7 - floor(log2 max), kept inside the normal range; 0 for an all-zero or non-finite block
+    int k = 0;
+    if (mx > 0.f && mx < INFINITY) {
+        k = 7 - ((int)((__float_as_uint(mx) >> 23) & 0xffu) - 127);
+        k = k > 120 ? 120 : k;
+    }
+    const float qs = __uint_as_float((uint32_t)(127 + k) << 23);
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float a0 = x[2 * i] * qs, a1 = x[2 * i + 1] * qs;
+        const uint32_t ch = f16x2_to_e4m3x2(pack_f16x2(a0, a1));   // a0, a1 are bf16 values below 2^8: exact in f16 above 2^-14
+        const uint32_t bh = e4m3x2_to_f16x2(ch);
+        const float2 back = __half22float2(*(const __half2*)&bh);
+        const uint32_t cl = f16x2_to_e4m3x2(pack_f16x2(a0 - back.x, a1 - back.y));
+        if (i & 1) {
+            hi[i >> 1] |= ch << 16;
+            lo[i >> 1] |= cl << 16;
+        } else {
+            hi[i >> 1] = ch;
+            lo[i >> 1] = cl;
+        }
+    }
+    uint8_t* img = qimg + ((size_t)b * p.Hkv + hg) * C::QBUF + c * C::QLBO;
+    *(uint4*)(img + r * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *(uint4*)(img + (RP + r) * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    if (threadIdx.x == 0) qinv[b * p.Hkv + hg] = __uint_as_float((uint32_t)(127 - k) << 23);
+}
+
+// ---- softmax side: per-block context and the work that is off the per-tile path -----------------------------
+struct ECtx {
+    float* negm;       // [RP] minus the reference maximum of each row (1e30 while the row has none)
+    float* mref;       // [RP] reference maximum, log2 units
+    float* alpha;      // [RP] rescale factors of the slow path
+    float* red;        // [4][RP] cross-warp reduction scratch
+    float* mfin;       // [2][RP] reference maxima of a finished piece, by O^T buffer
+    float* lfin;       // [2][RP] its denominators
+    int32_t* lim;      // [RP] keys visible to each row in the current segment
+    int32_t* rowloop;  // [RP] loop (0-based) of each packed row
+    uint64_t* bars;
+    volatile int* abort_flag;
+    uint32_t lane_off;  // this warp's lane quarter in a tensor-memory address
+    float scale;        // raw score -> log2 units, for the piece in hand (softmax scale, K scale, query scaling)
+    int tid, lane, wid;
+};
+
+// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima, and (unless
+// this is the first tile of the piece) the rescale of the three O^T column groups and of the denominators. All 128
+// softmax threads call it together. `done_bar` / `done_parity`: completion of the last product into O^T.
+template <int RP>
+__device__ __noinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, bool rescale, uint32_t tOb,
+                                         uint64_t* done_bar, uint32_t done_parity, bool failed) {
+    {
+        float v[RP];
+#pragma unroll
+        for (int r = 0; r < RP; ++r) v[r] = s[r] * cx.scale;
+        warp_reduce_rows<RP, true>(v, cx.lane, cx.red + cx.wid * RP);
+    }
+    named_barrier_sync(1, kSmThreads);
+    if (cx.tid < RP) {
+        const int t = cx.tid;
+        const float mo = cx.mref[t];
+        const float mn = fmaxf(fmaxf(mo, fmaxf(cx.red[t], cx.red[RP + t])), fmaxf(cx.red[2 * RP + t], cx.red[3 * RP + t]));
+        cx.alpha[t] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
+        cx.mref[t] = mn;
+        cx.negm[t] = (mn == -INFINITY) ? 1e30f : -mn;
+    }
+    named_barrier_sync(1, kSmThreads);
+    if (rescale) {
+        failed = sm_wait(done_bar, done_parity, cx.abort_flag, failed);
+        if (!failed) {
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 3 * RP / 16; ++c) {
+                uint32_t o[16];
+                tmem_ld16(tOb + cx.lane_off + c * 16, o);
+                tmem_wait_ld();
+                const int r0 = (c * 16) % RP;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[r0 + j]);
+                tmem_st16(tOb + cx.lane_off + c * 16, o);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+        }
+#pragma unroll
+        for (int r = 0; r < RP; ++r) lsum[r] *= cx.alpha[r];
+    }
+    return failed;
+}
+
+// Epilogue of a finished piece: the three column groups of O^T summed, times the V scale of the head, and the
+// denominators, out of tensor memory into the split partial.
+template <int RP>
+__device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
+                                        float vscale, bool failed) {
+    failed = sm_wait(&cx.bars[E_OFULL + ob], parity, cx.abort_flag, failed);
+#pragma unroll 1
+    for (int c = 0; c < RP / 16; ++c) {
+        uint32_t o0[16], o1[16], o2[16];
+        if (!failed) {
+            tc_fence_after_sync();
+            tmem_ld16(tOb + cx.lane_off + c * 16, o0);
+            tmem_ld16(tOb + cx.lane_off + RP + c * 16, o1);
+            tmem_ld16(tOb + cx.lane_off + 2 * RP + c * 16, o2);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (c * 16 + j < p.R)
+                    p.part_acc[(prow + c * 16 + j) * UD + cx.tid] =
+                        (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
+        }
+    }
+    tc_fence_before_sync();
+    mbar_arrive(&cx.bars[E_OFREE + ob]);
+    if (!failed && cx.tid < p.R)
+        *(float2*)(p.part_ml + (prow + cx.tid) * 2) = make_float2(cx.mfin[ob * RP + cx.tid], cx.lfin[ob * RP + cx.tid]);
+    return failed;
+}
+
+// V rows of a boundary tile that hold no data may contain anything (NaN codes too): zero them so that 0 * garbage
+// stays 0. `vtile`: the V half of the slot.
+__device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t* full_bar, uint32_t parity, const ECtx& cx,
+                                           bool failed) {
+    failed = sm_wait(full_bar, parity, cx.abort_flag, failed);
+    if (!failed && cx.tid >= nvalid) {
+        uint8_t* row = vtile + cx.tid * 128;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) *(uint4*)(row + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    return failed;
+}
+
+// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of each row.
+__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, const Piece& pc, int RP, int win_loop, int wl,
+                                          bool new_piece) {
+    // Threads still forming the probabilities of the tile before read negm and lim: nobody rewrites them earlier.
+    named_barrier_sync(1, kSmThreads);
+    if (cx.tid < RP) {
+        const int t = cx.tid;
+        if (new_piece) {
+            cx.mref[t] = -INFINITY;
+            cx.negm[t] = 1e30f;
+        }
+        int lim = 0;
+        if (t < p.R) {
+            if (pc.kind == 0) {
+#pragma unroll
+                for (int l = 0; l < kMaxLoops; ++l)
+                    if (l == cx.rowloop[t]) lim = pc.sp.cut[l];
+            } else if (cx.rowloop[t] == win_loop) {
+                lim = wl;
+            }
+        }
+        cx.lim[t] = lim;
+    }
+    named_barrier_sync(1, kSmThreads);
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kThreads8, 1)
+plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                          const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
+                          const __grid_constant__ Params p, const UmmaGeom geo, const uint8_t* __restrict__ qimg,
+                          const float* __restrict__ qinv) {
+    using C = ECfg<RP>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int ring = geo.ring;
+    uint8_t* slots = smem;                                  // ring of [K tile][V tile]
+    uint8_t* pbuf = smem + (size_t)ring * kSlot8;           // two buffers of PBUF (tile parity)
+    uint8_t* qbuf = pbuf + 2 * C::PBUF;                     // two buffers of QBUF (piece parity)
+    uint64_t* bars = (uint64_t*)(qbuf + 2 * C::QBUF);
+    float* s_negm = (float*)(bars + E_COUNT);
+    float* s_mref = s_negm + RP;
+    float* s_alpha = s_mref + RP;
+    float* s_red = s_alpha + RP;                            // [4][RP]
+    int32_t* s_lim = (int32_t*)(s_red + 4 * RP);
+    int32_t* s_rowloop = s_lim + RP;
+    float* s_mfin = (float*)(s_rowloop + RP);               // [2][RP]
+    float* s_lfin = s_mfin + 2 * RP;                        // [2][RP]
+    int32_t* s_ctl = (int32_t*)(s_lfin + 2 * RP);           // [0] abort flag, [1] tensor-memory base, [2] tiles issued by the producer
+    int32_t* s_prefix = s_ctl + 16;                         // [B + 1] tile prefix
+    int32_t* s_len = s_prefix + p.B + 1;                    // [B] clamped sequence lengths
+    volatile int* abort_flag = (volatile int*)&s_ctl[0];
+
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    uint32_t flags = 0;
+
+    if (tid == 0) {
+        s_ctl[0] = 0;
+        s_ctl[2] = 0;
+        for (int s = 0; s < kMaxRing8; ++s) {
+            mbar_init(&bars[E_FULL + s], 1);
+            mbar_init(&bars[E_EMPTY + s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars[E_SFULL + i], 1);
+            mbar_init(&bars[E_SFREE + i], kSmThreads);
+            mbar_init(&bars[E_PFULL + i], kSmThreads);
+            mbar_init(&bars[E_PFREE + i], 1);
+            mbar_init(&bars[E_OFULL + i], 1);
+            mbar_init(&bars[E_OFREE + i], kSmThreads);
+            mbar_init(&bars[E_QFULL + i], 1);
+        }
+        mbar_init(&bars[E_DRAIN], 1);
+        mbar_fence_init();
+    }
+    if (tid < RP) s_rowloop[tid] = tid / p.G;
+    if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
+    grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
+    build_prefix(p, s_prefix, flags, s_len, /*small=*/true);  // contains __syncthreads
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = (uint32_t)s_ctl[1];
+    // S^T of tile parity g at tS + 2 RP g; O^T of piece parity b at tO + 3 RP b
+    const uint32_t tS = tmem_base, tO = tmem_base + 4 * RP;
+
+    const int64_t T64 = s_prefix[p.B];
+    const int cta = blockIdx.x, nctas = plan_ctas(T64, (int)gridDim.x);
+    if (cta == 0)
+        for (int b = tid; b <= p.B; b += kThreads8) p.prefix[b] = s_prefix[b];
+    const bool in_plan = cta < nctas;
+    const int64_t lo = in_plan ? cta_begin(T64, cta, nctas) : 0, hi = in_plan ? cta_begin(T64, cta + 1, nctas) : 0;
+    const uint32_t T = (uint32_t)(hi - lo);   // tiles this block streams
+    bool q_pending[2] = {false, false};       // issuer only: a query image was asked for and not yet waited for
+    uint32_t q_parity[2] = {0u, 0u};          // and the phase of its barrier that ends when it has landed
+
+    if (wid == 4) {
+        // ================================ TMA producer of K and V tiles ================================
+        // At most `cap` tiles in flight (issued, not landed): more outstanding requests make the memory system
+        // slower, not faster. cap <= ring, so the slot of the tile issued `cap` tiles ago has not been refilled.
+        if (lane == 0 && T > 0) {
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+            if (p.L > 1) {
+                tma_prefetch_desc(&tmKw);
+                tma_prefetch_desc(&tmVw);
+            }
+            bool ok = true;
+            uint32_t n = 0;
+            Ring cur, old;   // slot of tile n, slot of tile n - cap
+            TileSource src(p, s_prefix, lo, hi, s_len);
+            TileCoords tc;
+            for (; n < T && ok; ++n) {
+                src.next(p, geo, tc, flags);
+                if (n >= (uint32_t)geo.cap) {
+                    ok = wait_or_abort(&bars[E_FULL + old.slot], old.parity, abort_flag);
+                    old.advance(ring);
+                }
+                if (ok && n >= (uint32_t)ring) ok = wait_or_abort(&bars[E_EMPTY + cur.slot], cur.parity ^ 1u, abort_flag);
+                if (!ok) break;
+                uint8_t* dst = slots + (size_t)cur.slot * kSlot8;
+                uint64_t* full = &bars[E_FULL + cur.slot];
+                mbar_expect_tx(full, (uint32_t)(tc.nbox * tc.box_keys * 256));
+                for (int i = 0; i < tc.nbox; ++i) {
+                    tma_load_4d(dst + i * tc.box_keys * 128, tc.window ? &tmKw : &tmK, full, 0, tc.c1[i], tc.head, tc.c3[i],
+                                l2_evict_first_policy());
+                    tma_load_4d(dst + kTile8 + i * tc.box_keys * 128, tc.window ? &tmVw : &tmV, full, 0, tc.c1[i], tc.head,
+                                tc.c3[i], l2_evict_first_policy());
+                }
+                cur.advance(ring);
+            }
+            s_ctl[2] = (int32_t)n;
+        }
+    } else if (wid == 5) {
+        // ===================== issuer of both products (one lane); owner of tensor memory ======================
+        // Order on the tensor pipe: S^T of tile g + 1 ahead of the O^T product of tile g, so that the scores of the
+        // next tile are ready while the softmax threads still form the probabilities of this one.
+        if (lane == 0 && T > 0) {
+            constexpr uint32_t idesc_qk = instr_desc_e4m3(UK, 2 * RP, 0, 0);
+            constexpr uint32_t idesc_pv = instr_desc_e4m3(UD, 3 * RP, 1, 1);
+            const uint32_t slots_a = smem_u32(slots), pbuf_a = smem_u32(pbuf), qbuf_a = smem_u32(qbuf);
+            bool ok = true;
+            auto fetch_q = [&](const Piece& q_pc, uint32_t piece) {
+                const int buf = (int)(piece & 1);
+                mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)C::QBUF);
+                bulk_load(qbuf + buf * C::QBUF, qimg + ((size_t)q_pc.b * p.Hkv + q_pc.hg) * C::QBUF, (uint32_t)C::QBUF,
+                          &bars[E_QFULL + buf]);
+                q_pending[buf] = true;
+                q_parity[buf] = (piece >> 1) & 1;
+            };
+            // cursor of the S^T products (runs one tile ahead) ...
+            PieceWalk walk_s(p, s_prefix, lo, hi, s_len);
+            Piece pcs, npcs;
+            walk_next(walk_s, pcs, flags);
+            fetch_q(pcs, 0);
+            int ts = pcs.t0;
+            uint32_t gs = 0, pis = 0;
+            Ring krs;
+            auto issue_s = [&]() {
+                const int sb = (int)(gs & 1);
+                const bool first = ts == pcs.t0;
+                if (first) {
+                    ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
+                    if (ok) q_pending[pis & 1] = false;
+                }
+                if (ok && gs >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
+                    ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_FULL + krs.slot], krs.parity, abort_flag);
+                if (ok) {
+                    tc_fence_after_sync();
+                    const uint32_t k_a = slots_a + (uint32_t)krs.slot * kSlot8;
+                    const uint32_t q_a = qbuf_a + (pis & 1) * C::QBUF;
+#pragma unroll
+                    for (int kk = 0; kk < UD / 32; ++kk)
+                        umma_f8(tS + sb * 2 * RP, smem_desc(k_a + kk * 32, 16, 1024, 2),
+                                smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
+                    umma_commit(&bars[E_SFULL + sb]);
+                }
+                krs.advance(ring);
+                if (first && ok) {
+                    // The other image buffer was last read by the S^T products of the piece before; the last of them
+                    // (tile gs - 1) must have completed before the next piece's image is copied into it.
+                    if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
+                    if (ok && walk_next(walk_s, npcs, flags)) fetch_q(npcs, pis + 1);
+                }
+                ++gs;
+                if (++ts == pcs.t1 && gs < T) {
+                    pcs = npcs;
+                    ts = pcs.t0;
+                    ++pis;
+                }
+            };
+            // ... and of the O^T products
+            PieceWalk walk_o(p, s_prefix, lo, hi, s_len);
+            Piece pco;
+            walk_next(walk_o, pco, flags);
+            int to = pco.t0;
+            uint32_t pio = 0;
+            Ring vro;
+            issue_s();
+            for (uint32_t g = 0; g < T && ok; ++g) {
+                if (g + 1 < T) issue_s();
+                if (!ok) break;
+                const int pb = (int)(g & 1);
+                const bool first = to == pco.t0, last = to == pco.t1 - 1;
+                const int ob = (int)(pio & 1);
+                if (first && pio >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
+                    ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t v_a = slots_a + (uint32_t)vro.slot * kSlot8 + kTile8;
+                const uint32_t tOb = tO + ob * 3 * RP;
+#pragma unroll
+                for (int ks = 0; ks < UK / 32; ++ks)
+                    umma_f8(tOb, smem_desc(v_a + ks * 4096, kTile8, 1024, 2), smem_desc(pbuf_a + pb * C::PBUF + ks * 512, 128, 2048, 0),
+                            idesc_pv, (first && ks == 0) ? 0u : 1u);
+                umma_commit(&bars[E_PFREE + pb]);
+                umma_commit(&bars[E_EMPTY + vro.slot]);
+                if (last) umma_commit(&bars[E_OFULL + ob]);
+                vro.advance(ring);
+                if (++to == pco.t1 && g + 1 < T) {
+                    walk_next(walk_o, pco, flags);
+                    to = pco.t0;
+                    ++pio;
+                }
+            }
+        }
+    } else {
+        // ================================ softmax and epilogue (warps 0-3) ================================
+        // Thread tid owns key tid of every tile (tensor-memory lane tid of S^T) and, in the epilogue, output
+        // dimension tid (lane tid of O^T).
+        ECtx cx;
+        cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lfin = s_lfin; cx.lim = s_lim;
+        cx.rowloop = s_rowloop; cx.bars = bars; cx.abort_flag = abort_flag;
+        cx.lane_off = (uint32_t)(wid * 32) << 16;
+        cx.scale = 0.f;
+        cx.tid = tid; cx.lane = lane; cx.wid = wid;
+        bool failed = false;    // a wait of this warp ran out; it stops touching data but keeps the common control flow
+        bool aborted = false;   // agreed by all 128 threads
+
+        // The epilogue of a piece runs one piece late, while the next piece is already streaming.
+        bool ep_pending = false;
+        uint32_t ep_pi = 0;
+        int64_t ep_prow = 0;
+        float ep_vscale = 1.f;
+
+        uint32_t gt = 0, pi = 0;
+        Ring vr;   // slot of tile gt (only boundary tiles look at it)
+        PieceWalk walk(p, s_prefix, lo, hi, s_len);
+        Piece pc;
+        bool have = walk_next(walk, pc, flags);
+        while (have && !aborted) {
+            const uint32_t tOb = tO + (pi & 1) * 3 * RP;   // O^T of this piece
+            const float scale = p.scale_log2 * p.k_scale[pc.hg] * qinv[pc.b * p.Hkv + pc.hg];
+            cx.scale = scale;
+            int cmin = 0x7fffffff;
+#pragma unroll
+            for (int l = 0; l < kMaxLoops; ++l)
+                if (l < p.L) cmin = min(cmin, pc.sp.cut[l]);
+            WinCursor cur;
+            cur.l = 0;
+            cur.key0 = 0;
+            int seg_l = -1, wl = 0;
+            if (pc.kind == 1) {
+                cur.seek(p, pc.sp, pc.t0);
+                seg_l = cur.l;
+#pragma unroll
+                for (int k = 1; k < kMaxLoops; ++k)
+                    if (k == cur.l) wl = pc.sp.wl[k];
+            }
+            e_set_limits(p, cx, pc, RP, seg_l, wl, true);
+            float lsum[RP];   // this key's share of the denominators
+#pragma unroll
+            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
+
+            for (int t = pc.t0; t < pc.t1; ++t, ++gt) {
+                int kbase, nvalid;
+                bool masked;
+                if (pc.kind == 0) {
+                    kbase = t * UK;
+                    nvalid = pc.sp.cmax - kbase;
+                    masked = kbase + UK > cmin;
+                } else {
+                    if (cur.l != seg_l) {   // a new window: only the rows of its loop see it
+                        seg_l = cur.l;
+#pragma unroll
+                        for (int k = 1; k < kMaxLoops; ++k)
+                            if (k == cur.l) wl = pc.sp.wl[k];
+                        e_set_limits(p, cx, pc, RP, seg_l, wl, false);
+                    }
+                    kbase = cur.key0;
+                    nvalid = wl - kbase;
+                    masked = true;
+                }
+                // ---- scores of this thread's key: the two terms of the queries added ----
+                const int sb = (int)(gt & 1);
+                failed = sm_wait(&bars[E_SFULL + sb], (gt >> 1) & 1, abort_flag, failed);
+                float s[RP];
+                if (!failed) {
+                    uint32_t sv[2 * RP];
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < 2 * RP / 16; ++c) tmem_ld16(tS + sb * 2 * RP + cx.lane_off + c * 16, sv + c * 16);
+                    tmem_wait_ld();
+                    tc_fence_before_sync();
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) s[r] = __uint_as_float(sv[r]) + __uint_as_float(sv[RP + r]);
+                } else {
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) s[r] = -INFINITY;
+                }
+                mbar_arrive(&bars[E_SFREE + sb]);
+                if (masked) {
+                    const int key = kbase + tid;
+#pragma unroll
+                    for (int r = 0; r < RP; ++r)
+                        if (key >= s_lim[r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
+                }
+                float over = -INFINITY;
+#pragma unroll
+                for (int r = 0; r < RP; ++r)
+                    if (r < p.R) over = fmaxf(over, fmaf(s[r], scale, s_negm[r]));
+                const bool trouble = failed || (*abort_flag != 0);
+                if (named_barrier_or(1, kSmThreads, over > kSlack8 || trouble)) {
+                    if (named_barrier_or(1, kSmThreads, trouble)) {
+                        aborted = true;
+                        break;
+                    }
+                    // Copies, so that the arrays of the per-tile path stay in registers (the out-of-line call takes
+                    // the addresses of its arguments).
+                    float s_c[RP], ls_c[RP];
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) {
+                        s_c[r] = s[r];
+                        ls_c[r] = lsum[r];
+                    }
+                    failed = e_slow_path<RP>(s_c, ls_c, cx, t != pc.t0, tOb, &bars[E_PFREE + ((gt - 1) & 1)], ((gt - 1) >> 1) & 1,
+                                             failed);
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
+                }
+                // ---- probabilities as three E4M3 terms into shared memory ----
+                const int pb = (int)(gt & 1);
+                if (gt >= 2) failed = sm_wait(&bars[E_PFREE + pb], ((gt >> 1) & 1) ^ 1u, abort_flag, failed);
+                uint8_t* pdst = pbuf + pb * C::PBUF + tid * 16;
+#pragma unroll
+                for (int j = 0; j < RP / 16; ++j) {
+                    uint32_t c_hi[4], c_mid[4], c_lo[4];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int r0 = j * 16 + 2 * q;
+                        const float p0 = fast_exp2(fmaf(s[r0], scale, s_negm[r0]));
+                        const float p1 = fast_exp2(fmaf(s[r0 + 1], scale, s_negm[r0 + 1]));
+                        lsum[r0] += p0;
+                        lsum[r0 + 1] += p1;
+                        const uint32_t h2 = pack_f16x2(p0, p1);
+                        const uint32_t c0 = f16x2_to_e4m3x2(h2);
+                        const uint32_t r1 = mul_f16x2(sub_f16x2(h2, e4m3x2_to_f16x2(c0)), kMidScaleH2);   // exact
+                        const uint32_t c1 = f16x2_to_e4m3x2(r1);
+                        const uint32_t r2 = mul_f16x2(sub_f16x2(r1, e4m3x2_to_f16x2(c1)), kLoScaleH2);    // exact
+                        const uint32_t c2 = f16x2_to_e4m3x2(r2);
+                        if (q & 1) {
+                            c_hi[q >> 1] |= c0 << 16;
+                            c_mid[q >> 1] |= c1 << 16;
+                            c_lo[q >> 1] |= c2 << 16;
+                        } else {
+                            c_hi[q >> 1] = c0;
+                            c_mid[q >> 1] = c1;
+                            c_lo[q >> 1] = c2;
+                        }
+                    }
+                    if (!failed) {
+                        *(uint4*)(pdst + (j) * 2048) = make_uint4(c_hi[0], c_hi[1], c_hi[2], c_hi[3]);
+                        *(uint4*)(pdst + (RP / 16 + j) * 2048) = make_uint4(c_mid[0], c_mid[1], c_mid[2], c_mid[3]);
+                        *(uint4*)(pdst + (2 * RP / 16 + j) * 2048) = make_uint4(c_lo[0], c_lo[1], c_lo[2], c_lo[3]);
+                    }
+                }
+                if (masked && nvalid < UK)
+                    failed = e_zero_v_rows(slots + (size_t)vr.slot * kSlot8 + kTile8, nvalid, &bars[E_FULL + vr.slot], vr.parity, cx,
+                                           failed);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[E_PFULL + pb]);
+                vr.advance(ring);
+                if (pc.kind == 1) cur.advance(p, pc.sp);
+                if (t == pc.t0 && ep_pending) {
+                    // put off so that the pipeline restarts first: the partial of the piece before
+                    failed = e_epilogue<RP>(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale,
+                                            failed);
+                    ep_pending = false;
+                }
+            }
+            if (aborted) break;
+
+            // ---- end of piece: denominators across the 128 keys, parked with the reference maxima; the epilogue
+            //      proper runs one piece late ----
+            warp_reduce_rows<RP, false>(lsum, lane, s_red + wid * RP);
+            named_barrier_sync(1, kSmThreads);
+            if (tid < RP) {
+                s_lfin[(pi & 1) * RP + tid] = (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]);
+                s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
+            }
+            ep_pending = true;
+            ep_pi = pi;
+            ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // one KV head per item on this path
+            ep_vscale = p.v_scale[pc.hg];
+            if (tid == 0) note_piece(p, pc, cta);
+            have = walk_next(walk, pc, flags);
+            ++pi;
+        }
+        if (ep_pending && !aborted) {
+            named_barrier_sync(1, kSmThreads);   // s_mfin of the last piece visible to all
+            failed = e_epilogue<RP>(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
+        }
+    }
+
+    // ---- common exit: nothing of this block may still be in flight when tensor memory is freed ----
+    __syncthreads();
+    const bool gave_up = *abort_flag != 0;
+    if (wid == 5 && lane == 0) {
+        umma_commit(&bars[E_DRAIN]);   // arrives once every product issued by this thread has completed
+        mbar_wait_bounded(&bars[E_DRAIN], 0, kUmmaWaitNs);
+        // a query image that was asked for and never waited for gets a bounded chance to land
+        for (int i = 0; i < 2; ++i)
+            if (q_pending[i]) mbar_wait_bounded(&bars[E_QFULL + i], q_parity[i], kUmmaWaitNs);
+    }
+    if (wid == 4 && lane == 0 && gave_up) {
+        // give every copy that was issued a bounded chance to land
+        const uint32_t issued = (uint32_t)s_ctl[2];
+        for (uint32_t m = issued > (uint32_t)ring ? issued - (uint32_t)ring : 0; m < issued; ++m)
+            mbar_wait_bounded(&bars[E_FULL + (int)(m % (uint32_t)ring)], (m / (uint32_t)ring) & 1, kUmmaWaitNs);
+    }
+    if (gave_up) flags |= kDevWaitTimeout;
+    if (flags) atomicOr(p.status, flags);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (wid == 5) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+template <int RP>
+cudaError_t e4m3_prepare(size_t smem, int* blocks_per_sm) {
+    auto fn = plt_decode_main_umma_e4m3<RP>;
+    cudaError_t e = allow_max_dynamic_smem((const void*)fn);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, kThreads8, smem);
+}
+
+template <int RP>
+cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, const UmmaGeom& geo,
+                        const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
+    plt_decode_main_umma_e4m3<RP><<<grid, kThreads8, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int main_umma_e4m3_rows(int R) { return R <= 16 ? 16 : 32; }
+
+int main_umma_e4m3_max_slots() { return kMaxRing8; }
+
+size_t main_umma_e4m3_smem(int R, int nslot, int max_batch) {
+    return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::smem_bytes(nslot, max_batch) : ECfg<32>::smem_bytes(nslot, max_batch);
+}
+
+// Bytes of the query image of one (sequence, KV head).
+size_t main_umma_e4m3_image_bytes(int R) { return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::QBUF : ECfg<32>::QBUF; }
+
+cudaError_t main_umma_e4m3_prepare(int R, size_t smem, int* blocks_per_sm) {
+    return main_umma_e4m3_rows(R) == 16 ? e4m3_prepare<16>(smem, blocks_per_sm) : e4m3_prepare<32>(smem, blocks_per_sm);
+}
+
+cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream) {
+    if (main_umma_e4m3_rows(p.R) == 16) plt_decode_pack_q_e4m3<16><<<p.B * p.Hkv, 128, 0, stream>>>(p, qimg, qinv);
+    else plt_decode_pack_q_e4m3<32><<<p.B * p.Hkv, 256, 0, stream>>>(p, qimg, qinv);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
+                                  int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
+    const UmmaGeom geo{nslot, kbox, wbox, cap < 1 ? 1 : (cap > nslot ? nslot : cap)};
+    return main_umma_e4m3_rows(p.R) == 16 ? e4m3_launch<16>(maps, p, grid, smem, geo, qimg, qinv, stream)
+                                          : e4m3_launch<32>(maps, p, grid, smem, geo, qimg, qinv, stream);
+}
+
+}  // namespace plt

@@ -87,9 +87,10 @@ def test_unsupported_combinations_are_refused():
     for bad in (custom(d=64), custom(dtype="f32"), custom(page_size=16)):
         with pytest.raises((B.PltError, Exception)):
             DecodeAttn(make_problem(bad))
-    p = make_problem(custom())
+    p = make_problem(custom(B=2, L=4, Hq=32, Hkv=2, w=33, lens=("list", [400, 5])))   # 64 packed rows
     with pytest.raises(B.PltError):
         DecodeAttn(p, kernel_path=B.PLT_PATH_TCGEN05)
+    p = make_problem(custom())
     dp = DeviceProblem(p, "cuda:0")
     with DecodeAttn(p) as op:
         a = dp.args()
