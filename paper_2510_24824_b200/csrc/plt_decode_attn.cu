@@ -290,8 +290,9 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         // Ring slots of 32 KB (K and V tile of one head); 5 fit beside the probability and query buffers.
         int nslot = config->stages;
         if (nslot == 0) nslot = main_umma_e4m3_max_slots();
-        if (nslot < 2 || nslot > main_umma_e4m3_max_slots())
-            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path with E4M3 caches (supported: 2 to %d ring slots)",
+        // at least 3: the scores run two tiles ahead of the product that frees a slot
+        if (nslot < 3 || nslot > main_umma_e4m3_max_slots())
+            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path with E4M3 caches (supported: 3 to %d ring slots)",
                         nslot, main_umma_e4m3_max_slots());
         const size_t smem = main_umma_e4m3_smem(g.R, nslot, config->max_batch);
         if (smem > 227 * 1024)

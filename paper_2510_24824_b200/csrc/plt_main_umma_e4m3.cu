@@ -17,9 +17,10 @@
 // softmax threads add the two score columns of a row, and the epilogue adds the three accumulator columns. One tcgen05.mma costs the same issue slot whatever N is, so the extra terms are
 // free on the tensor side: 8 instructions per 32 KB tile.
 //
-// Warp roles (192 threads): warps 0-3 softmax and epilogue (thread = key = tensor-memory lane); warp 4, one lane:
-// TMA producer of K and V tiles (one ring of 32 KB slots, K then V); warp 5, one lane: issues every product, copies
-// the packed query image of the next piece (cp.async.bulk) and owns the tensor-memory allocation.
+// Warp roles: four softmax-and-epilogue warps per 8 packed rows (thread = key = tensor-memory lane, 8 scores of it;
+// four such groups at 32 rows, so four softmax warps per scheduler); then one warp, one lane: TMA producer of K and
+// V tiles (one ring of 32 KB slots, K then V); then one warp, one lane: issues every product, copies the packed query
+// image of the next piece (cp.async.bulk) and owns the tensor-memory allocation.
 // The query image (codes in the core-matrix order the instruction reads, and the power of two they were scaled
 // by) is written per (sequence, KV head) by plt_decode_pack_q_e4m3, launched before this kernel.
 // Online softmax with a lazily updated reference maximum, as in the bf16 tcgen05 kernel. Every wait is bounded.
@@ -38,7 +39,8 @@ namespace {
 constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 keys x 128 codes
 constexpr int kSlot8 = 2 * kTile8;     // a ring slot: the K tile, then the V tile
 constexpr int kMaxRing8 = 5;
-constexpr int kThreads8 = 192;
+// Threads of a block: 128 softmax threads per group of 8 packed rows, the producer warp, the issuer warp.
+__host__ __device__ constexpr int threads8(int RP) { return (RP / 8) * 128 + 64; }
 // A probability may exceed the lazily updated reference by 3 powers of two at most (p <= 8), which fixes the powers of
 // two the second and third term are scaled by: |p - hi| <= 2^-2 and |p - hi - mid| <= 2^-7 times 2^10 and 2^14 stay
 // below 448. The third term then resolves 2^-23, the step of the f16 the probability is rounded to first.
@@ -128,7 +130,121 @@ __global__ void __launch_bounds__(RP * 8) plt_decode_pack_q_e4m3(const Params p,
     if (threadIdx.x == 0) qinv[b * p.Hkv + hg] = __uint_as_float((uint32_t)(127 - k) << 23);
 }
 
-// ---- softmax side: per-block context and the work that is off the per-tile path -----------------------------
+// ---- the tile plan, walked with scalars only --------------------------------------------------------------
+// The same plan as PieceWalk / SeqPlan (plt_common.cuh) yields, recomputed from the clamped sequence length with no
+// per-loop arrays, so that every role keeps its position in registers: with 200+ KB of shared memory the L1 that
+// would back a stack frame is a few KB, and a role that spills its plan there runs at a fraction of its speed.
+__device__ __forceinline__ int e_cut(const Params& p, int n, int l) {
+    const int c = n - p.delta[l];
+    return c > 0 ? c : 0;
+}
+// Valid window slots of loop l (1 .. L-1) of sequence b.
+__device__ __forceinline__ int e_wl(const Params& p, int b, int n, int l, uint32_t& flags) {
+    const int c = e_cut(p, n, l);
+    int wl = c < p.w ? c : p.w;
+    if (p.win_lens != nullptr && c > 0) {
+        wl = p.win_lens[b * (p.L - 1) + (l - 1)];
+        if (wl < 0 || wl > p.w) {
+            flags |= kDevWinLenClamped;
+            wl = wl < 0 ? 0 : p.w;
+        }
+    }
+    return wl;
+}
+// Largest cutoff over the loops, tiles of the shared cache and of all windows of sequence b.
+__device__ __forceinline__ void e_counts(const Params& p, int b, int n, uint32_t& flags, int& cmax, int& gt, int& lt) {
+    cmax = 0;
+    lt = 0;
+#pragma unroll 1
+    for (int l = 0; l < p.L; ++l) {
+        const int c = e_cut(p, n, l);
+        cmax = c > cmax ? c : cmax;
+        if (l >= 1) lt += ceil_div(e_wl(p, b, n, l, flags), UK);
+    }
+    gt = ceil_div(cmax, UK);
+}
+
+// One piece: tiles [t0, t1) of item (b, hg, kind); n = clamped length of b, cmax / total = what e_counts gave
+// (total = tiles of the whole item).
+struct EPiece {
+    int b, hg, kind, t0, t1, n, cmax, total;
+};
+
+// The step to the next piece is out of line and shared by the three roles (it runs once per piece); the per-tile
+// loops copy what they need of the piece into registers and stay small enough for the instruction cache.
+struct EWalk {
+    int pos, hi, b;
+    __device__ __forceinline__ EWalk(const Params& p, const int32_t* sp, int lo_, int hi_) : pos(lo_), hi(hi_), b(0) {
+        if (pos < hi) b = find_seq(sp, p.B, pos);
+    }
+    __device__ __noinline__ bool next(const Params& p, const int32_t* sp, const int32_t* lens, EPiece& pc, uint32_t& flags) {
+        for (;;) {
+            if (pos >= hi) return false;
+            while (sp[b + 1] <= pos) ++b;
+            const int n = lens[b];
+            int cmax, gt, lt;
+            e_counts(p, b, n, flags, cmax, gt, lt);
+            const int vg = line_len(p, gt), per = vg + line_len(p, lt);
+            const int o = pos - sp[b];
+            pc.b = b;
+            pc.n = n;
+            pc.cmax = cmax;
+            pc.hg = o / per;
+            const int o2 = o - pc.hg * per;
+            int v0, item_end;
+            if (o2 < vg) {
+                pc.kind = 0;
+                pc.total = gt;
+                v0 = o2;
+                item_end = pos + (vg - o2);
+            } else {
+                pc.kind = 1;
+                pc.total = lt;
+                v0 = o2 - vg;
+                item_end = pos + (per - o2);
+            }
+            const int end = item_end < hi ? item_end : hi;
+            const int v1 = v0 + (end - pos);
+            pos = end;
+            pc.t0 = v0 > p.piece_cost ? v0 - p.piece_cost : 0;
+            pc.t1 = v1 > p.piece_cost ? v1 - p.piece_cost : 0;
+            if (pc.t1 > pc.t0) return true;   // else: only the item's lead-in positions fell to this block
+        }
+    }
+};
+
+// Window tile cursor of a windows item: loop (1 .. L-1), first key of the tile inside that loop's window, and the
+// window's length.
+struct EWin {
+    int l, key0, wl;
+    __device__ __noinline__ void seek(const Params& p, int b, int n, int t, uint32_t& flags) {
+        l = 1;
+        wl = e_wl(p, b, n, 1, flags);
+        while (l < p.L - 1) {
+            const int nt = ceil_div(wl, UK);
+            if (t < nt) break;
+            t -= nt;
+            ++l;
+            wl = e_wl(p, b, n, l, flags);
+        }
+        key0 = t * UK;
+    }
+    __device__ __noinline__ void advance(const Params& p, int b, int n, uint32_t& flags) {
+        key0 += UK;
+        while (key0 >= wl && l < p.L - 1) {
+            ++l;
+            key0 = 0;
+            wl = e_wl(p, b, n, l, flags);
+        }
+    }
+};
+
+// ---- softmax side: per-group context and the work that is off the per-tile path -----------------------------
+// The packed rows are split into groups of 8: softmax warps 4 g .. 4 g + 3 own rows 8 g .. 8 g + 7 of every tile
+// (thread = key, 8 scores), with their own reference maxima, vote and rescale. Four groups (32 packed rows) put four
+// softmax warps on each scheduler: the per-tile chain of a warp is latency-bound, and this is what hides it.
+constexpr int RT = 8;    // rows per softmax thread
+
 struct ECtx {
     float* negm;       // [RP] minus the reference maximum of each row (1e30 while the row has none)
     float* mref;       // [RP] reference maximum, log2 units
@@ -142,124 +258,124 @@ struct ECtx {
     volatile int* abort_flag;
     uint32_t lane_off;  // this warp's lane quarter in a tensor-memory address
     float scale;        // raw score -> log2 units, for the piece in hand (softmax scale, K scale, query scaling)
-    int tid, lane, wid;
+    int RP;             // packed rows rounded up to 16 or 32
+    int R;              // packed rows
+    int row0;           // first row of this thread's group
+    int bar_id;         // named barrier of the group's 128 threads
+    int ltid, lane, wq; // thread in the group (= key = output dimension), lane, warp in the group
 };
 
-// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima, and (unless
-// this is the first tile of the piece) the rescale of the three O^T column groups and of the denominators. All 128
-// softmax threads call it together. `done_bar` / `done_parity`: completion of the last product into O^T.
-template <int RP>
-__device__ __noinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, bool rescale, uint32_t tOb,
+// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima of the group's
+// rows, and (unless this is the first tile of the piece) the rescale of their three O^T column groups and of the
+// denominators. The 128 threads of a group call it together. `done_bar` / `done_parity`: completion of the last
+// product into O^T.
+__device__ __noinline__ bool e_slow_path(const float (&s)[RT], float (&lsum)[RT], const ECtx& cx, bool rescale, uint32_t tOb,
                                          uint64_t* done_bar, uint32_t done_parity, bool failed) {
+    const int RP = cx.RP;
     {
-        float v[RP];
+        float v[RT];
 #pragma unroll
-        for (int r = 0; r < RP; ++r) v[r] = s[r] * cx.scale;
-        warp_reduce_rows<RP, true>(v, cx.lane, cx.red + cx.wid * RP);
+        for (int r = 0; r < RT; ++r) v[r] = s[r] * cx.scale;
+        warp_reduce_rows<RT, true>(v, cx.lane, cx.red + cx.wq * RP + cx.row0);
     }
-    named_barrier_sync(1, kSmThreads);
-    if (cx.tid < RP) {
-        const int t = cx.tid;
+    named_barrier_sync(cx.bar_id, kSmThreads);
+    if (cx.ltid < RT) {
+        const int t = cx.row0 + cx.ltid;
         const float mo = cx.mref[t];
         const float mn = fmaxf(fmaxf(mo, fmaxf(cx.red[t], cx.red[RP + t])), fmaxf(cx.red[2 * RP + t], cx.red[3 * RP + t]));
         cx.alpha[t] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
         cx.mref[t] = mn;
-        cx.negm[t] = (mn == -INFINITY) ? 1e30f : -mn;
+        // rows beyond R (padding of the instruction's N) keep a reference that makes every probability 0
+        cx.negm[t] = t >= cx.R ? -1e30f : ((mn == -INFINITY) ? 1e30f : -mn);
     }
-    named_barrier_sync(1, kSmThreads);
+    named_barrier_sync(cx.bar_id, kSmThreads);
     if (rescale) {
         failed = sm_wait(done_bar, done_parity, cx.abort_flag, failed);
         if (!failed) {
             tc_fence_after_sync();
 #pragma unroll 1
-            for (int c = 0; c < 3 * RP / 16; ++c) {
-                uint32_t o[16];
-                tmem_ld16(tOb + cx.lane_off + c * 16, o);
+            for (int term = 0; term < 3; ++term) {
+                uint32_t o[RT];
+                const uint32_t addr = tOb + cx.lane_off + term * RP + cx.row0;
+                tmem_ld8(addr, o);
                 tmem_wait_ld();
-                const int r0 = (c * 16) % RP;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[r0 + j]);
-                tmem_st16(tOb + cx.lane_off + c * 16, o);
+                for (int j = 0; j < RT; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[cx.row0 + j]);
+                tmem_st8(addr, o);
             }
             tmem_wait_st();
             tc_fence_before_sync();
         }
 #pragma unroll
-        for (int r = 0; r < RP; ++r) lsum[r] *= cx.alpha[r];
+        for (int r = 0; r < RT; ++r) lsum[r] *= cx.alpha[cx.row0 + r];
     }
     return failed;
 }
 
-// Epilogue of a finished piece: the three column groups of O^T summed, times the V scale of the head, and the
-// denominators, out of tensor memory into the split partial.
-template <int RP>
+// Epilogue of a finished piece for the group's rows: the three column groups of O^T summed (the second and third
+// scaled back), times the V scale of the head, and the denominators, out of tensor memory into the split partial.
 __device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
                                         float vscale, bool failed) {
     failed = sm_wait(&cx.bars[E_OFULL + ob], parity, cx.abort_flag, failed);
-#pragma unroll 1
-    for (int c = 0; c < RP / 16; ++c) {
-        uint32_t o0[16], o1[16], o2[16];
-        if (!failed) {
-            tc_fence_after_sync();
-            tmem_ld16(tOb + cx.lane_off + c * 16, o0);
-            tmem_ld16(tOb + cx.lane_off + RP + c * 16, o1);
-            tmem_ld16(tOb + cx.lane_off + 2 * RP + c * 16, o2);
-            tmem_wait_ld();
+    if (!failed) {
+        uint32_t o0[RT], o1[RT], o2[RT];
+        tc_fence_after_sync();
+        tmem_ld8(tOb + cx.lane_off + cx.row0, o0);
+        tmem_ld8(tOb + cx.lane_off + cx.RP + cx.row0, o1);
+        tmem_ld8(tOb + cx.lane_off + 2 * cx.RP + cx.row0, o2);
+        tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (c * 16 + j < p.R)
-                    p.part_acc[(prow + c * 16 + j) * UD + cx.tid] =
-                        (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
-        }
+        for (int j = 0; j < RT; ++j)
+            if (cx.row0 + j < p.R)
+                p.part_acc[(prow + cx.row0 + j) * UD + cx.ltid] =
+                    (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
     }
     tc_fence_before_sync();
-    mbar_arrive(&cx.bars[E_OFREE + ob]);
-    if (!failed && cx.tid < p.R)
-        *(float2*)(p.part_ml + (prow + cx.tid) * 2) = make_float2(cx.mfin[ob * RP + cx.tid], cx.lfin[ob * RP + cx.tid]);
+    __syncwarp();
+    if (cx.lane == 0) mbar_arrive(&cx.bars[E_OFREE + ob]);
+    if (!failed && cx.ltid < RT && cx.row0 + cx.ltid < p.R) {
+        const int t = cx.row0 + cx.ltid;
+        *(float2*)(p.part_ml + (prow + t) * 2) = make_float2(cx.mfin[ob * cx.RP + t], cx.lfin[ob * cx.RP + t]);
+    }
     return failed;
 }
 
 // V rows of a boundary tile that hold no data may contain anything (NaN codes too): zero them so that 0 * garbage
-// stays 0. `vtile`: the V half of the slot.
+// stays 0. `vtile`: the V half of the slot. Called by the threads of group 0.
 __device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t* full_bar, uint32_t parity, const ECtx& cx,
                                            bool failed) {
     failed = sm_wait(full_bar, parity, cx.abort_flag, failed);
-    if (!failed && cx.tid >= nvalid) {
-        uint8_t* row = vtile + cx.tid * 128;
+    if (!failed && cx.ltid >= nvalid) {
+        uint8_t* row = vtile + cx.ltid * 128;
 #pragma unroll
         for (int i = 0; i < 8; ++i) *(uint4*)(row + i * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
     return failed;
 }
 
-// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of each row.
-__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, const Piece& pc, int RP, int win_loop, int wl,
-                                          bool new_piece) {
-    // Threads still forming the probabilities of the tile before read negm and lim: nobody rewrites them earlier.
-    named_barrier_sync(1, kSmThreads);
-    if (cx.tid < RP) {
-        const int t = cx.tid;
+// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of the group's rows.
+// n: clamped length of the sequence.
+__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int kind, int n, int win_loop, int wl, bool new_piece) {
+    // Threads still forming the probabilities of the tile before read lim: nobody rewrites it earlier.
+    named_barrier_sync(cx.bar_id, kSmThreads);
+    if (cx.ltid < RT) {
+        const int t = cx.row0 + cx.ltid;
         if (new_piece) {
             cx.mref[t] = -INFINITY;
-            cx.negm[t] = 1e30f;
+            cx.negm[t] = t >= cx.R ? -1e30f : 1e30f;
         }
         int lim = 0;
-        if (t < p.R) {
-            if (pc.kind == 0) {
-#pragma unroll
-                for (int l = 0; l < kMaxLoops; ++l)
-                    if (l == cx.rowloop[t]) lim = pc.sp.cut[l];
-            } else if (cx.rowloop[t] == win_loop) {
-                lim = wl;
-            }
+        if (t < cx.R) {
+            if (kind == 0) lim = e_cut(p, n, cx.rowloop[t]);
+            else if (cx.rowloop[t] == win_loop) lim = wl;
         }
         cx.lim[t] = lim;
     }
-    named_barrier_sync(1, kSmThreads);
+    named_barrier_sync(cx.bar_id, kSmThreads);
 }
 
 template <int RP>
-__global__ void __launch_bounds__(kThreads8, 1)
+__global__ void __launch_bounds__(threads8(RP), 1)
 plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                           const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
                           const __grid_constant__ Params p, const UmmaGeom geo, const uint8_t* __restrict__ qimg,
@@ -285,6 +401,10 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     int32_t* s_len = s_prefix + p.B + 1;                    // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
 
+    constexpr int NG = RP / RT;            // row groups = softmax warp quartets
+    constexpr int kSmWarps = NG * 4;       // softmax warps: one lane of each arrives on the barriers they feed (a
+                                           // block-wide count would put hundreds of arrivals on one shared-memory word per tile)
+    constexpr int kProducerWarp = 4 * NG, kIssuerWarp = 4 * NG + 1;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
 
@@ -297,18 +417,18 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars[E_SFULL + i], 1);
-            mbar_init(&bars[E_SFREE + i], kSmThreads);
-            mbar_init(&bars[E_PFULL + i], kSmThreads);
+            mbar_init(&bars[E_SFREE + i], kSmWarps);
+            mbar_init(&bars[E_PFULL + i], kSmWarps);
             mbar_init(&bars[E_PFREE + i], 1);
             mbar_init(&bars[E_OFULL + i], 1);
-            mbar_init(&bars[E_OFREE + i], kSmThreads);
+            mbar_init(&bars[E_OFREE + i], kSmWarps);
             mbar_init(&bars[E_QFULL + i], 1);
         }
         mbar_init(&bars[E_DRAIN], 1);
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
-    if (wid == 5) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
+    if (wid == kIssuerWarp) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags, s_len, /*small=*/true);  // contains __syncthreads
     tc_fence_before_sync();
@@ -321,14 +441,16 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     const int64_t T64 = s_prefix[p.B];
     const int cta = blockIdx.x, nctas = plan_ctas(T64, (int)gridDim.x);
     if (cta == 0)
-        for (int b = tid; b <= p.B; b += kThreads8) p.prefix[b] = s_prefix[b];
+        for (int b = tid; b <= p.B; b += threads8(RP)) p.prefix[b] = s_prefix[b];
     const bool in_plan = cta < nctas;
-    const int64_t lo = in_plan ? cta_begin(T64, cta, nctas) : 0, hi = in_plan ? cta_begin(T64, cta + 1, nctas) : 0;
-    const uint32_t T = (uint32_t)(hi - lo);   // tiles this block streams
+    const int lo = in_plan ? (int)cta_begin(T64, cta, nctas) : 0, hi = in_plan ? (int)cta_begin(T64, cta + 1, nctas) : 0;
+    // Tiles this block streams: the positions of its range minus the lead-in positions of its pieces (none on this
+    // path: piece_cost is 0, so every position is a tile).
+    const uint32_t T = (uint32_t)(hi - lo);
     bool q_pending[2] = {false, false};       // issuer only: a query image was asked for and not yet waited for
     uint32_t q_parity[2] = {0u, 0u};          // and the phase of its barrier that ends when it has landed
 
-    if (wid == 4) {
+    if (wid == kProducerWarp) {
         // ================================ TMA producer of K and V tiles ================================
         // At most `cap` tiles in flight (issued, not landed): more outstanding requests make the memory system
         // slower, not faster. cap <= ring, so the slot of the tile issued `cap` tiles ago has not been refilled.
@@ -339,13 +461,21 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 tma_prefetch_desc(&tmKw);
                 tma_prefetch_desc(&tmVw);
             }
+            const uint64_t pol = l2_evict_first_policy();
             bool ok = true;
             uint32_t n = 0;
             Ring cur, old;   // slot of tile n, slot of tile n - cap
-            TileSource src(p, s_prefix, lo, hi, s_len);
-            TileCoords tc;
+            EWalk walk(p, s_prefix, lo, hi);
+            EPiece pc;
+            EWin win;
+            pc.t0 = pc.t1 = 0;
+            int t = 0;
             for (; n < T && ok; ++n) {
-                src.next(p, geo, tc, flags);
+                if (t == pc.t1) {
+                    walk.next(p, s_prefix, s_len, pc, flags);
+                    t = pc.t0;
+                    if (pc.kind == 1) win.seek(p, pc.b, pc.n, t, flags);
+                }
                 if (n >= (uint32_t)geo.cap) {
                     ok = wait_or_abort(&bars[E_FULL + old.slot], old.parity, abort_flag);
                     old.advance(ring);
@@ -354,124 +484,163 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 if (!ok) break;
                 uint8_t* dst = slots + (size_t)cur.slot * kSlot8;
                 uint64_t* full = &bars[E_FULL + cur.slot];
-                mbar_expect_tx(full, (uint32_t)(tc.nbox * tc.box_keys * 256));
-                for (int i = 0; i < tc.nbox; ++i) {
-                    tma_load_4d(dst + i * tc.box_keys * 128, tc.window ? &tmKw : &tmK, full, 0, tc.c1[i], tc.head, tc.c3[i],
-                                l2_evict_first_policy());
-                    tma_load_4d(dst + kTile8 + i * tc.box_keys * 128, tc.window ? &tmVw : &tmV, full, 0, tc.c1[i], tc.head,
-                                tc.c3[i], l2_evict_first_policy());
+                if (pc.kind == 0 && p.page_size > 0) {
+                    const int key0 = t * UK;
+                    const int rem = pc.cmax - key0;   // keys that hold data from key0 on (>= 1)
+                    const int nbox = (min(rem, UK) + geo.kbox - 1) / geo.kbox;
+                    mbar_expect_tx(full, (uint32_t)(nbox * geo.kbox * 256));
+                    for (int i = 0; i < nbox; ++i) {
+                        const int key = key0 + i * geo.kbox;
+                        int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
+                        if (page < 0 || page >= p.num_pool_pages) {
+                            flags |= kDevPageIdClamped;
+                            page = page < 0 ? 0 : p.num_pool_pages - 1;
+                        }
+                        tma_load_4d(dst + i * geo.kbox * 128, &tmK, full, 0, key % p.page_size, pc.hg, page, pol);
+                        tma_load_4d(dst + kTile8 + i * geo.kbox * 128, &tmV, full, 0, key % p.page_size, pc.hg, page, pol);
+                    }
+                } else if (pc.kind == 0) {
+                    mbar_expect_tx(full, (uint32_t)(geo.kbox * 256));
+                    tma_load_4d(dst, &tmK, full, 0, t * UK, pc.hg, pc.b, pol);
+                    tma_load_4d(dst + kTile8, &tmV, full, 0, t * UK, pc.hg, pc.b, pol);
+                } else {
+                    const int outer = pc.b * (p.L - 1) + (win.l - 1);
+                    mbar_expect_tx(full, (uint32_t)(geo.wbox * 256));
+                    tma_load_4d(dst, &tmKw, full, 0, win.key0, pc.hg, outer, pol);
+                    tma_load_4d(dst + kTile8, &tmVw, full, 0, win.key0, pc.hg, outer, pol);
+                    win.advance(p, pc.b, pc.n, flags);
                 }
                 cur.advance(ring);
+                ++t;
             }
             s_ctl[2] = (int32_t)n;
         }
-    } else if (wid == 5) {
+    } else if (wid == kIssuerWarp) {
         // ===================== issuer of both products (one lane); owner of tensor memory ======================
-        // Order on the tensor pipe: S^T of tile g + 1 ahead of the O^T product of tile g, so that the scores of the
-        // next tile are ready while the softmax threads still form the probabilities of this one.
+        // All of its plan state is scalars: tiles left in the piece each cursor is in, the image index of the next piece.
         if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_qk = instr_desc_e4m3(UK, 2 * RP, 0, 0);
             constexpr uint32_t idesc_pv = instr_desc_e4m3(UD, 3 * RP, 1, 1);
-            const uint32_t slots_a = smem_u32(slots), pbuf_a = smem_u32(pbuf), qbuf_a = smem_u32(qbuf);
+            const uint32_t slots_a = smem_u32(slots);
+            // descriptors of slot 0 / buffer 0; the others differ in the start-address field (16-byte units) only
+            const uint64_t kdesc0 = smem_desc(slots_a, 16, 1024, 2), vdesc0 = smem_desc(slots_a + kTile8, kTile8, 1024, 2);
+            const uint64_t qdesc0 = smem_desc(smem_u32(qbuf), C::QLBO, 128, 0), pdesc0 = smem_desc(smem_u32(pbuf), 128, 2048, 0);
             bool ok = true;
-            auto fetch_q = [&](const Piece& q_pc, uint32_t piece) {
-                const int buf = (int)(piece & 1);
-                mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)C::QBUF);
-                bulk_load(qbuf + buf * C::QBUF, qimg + ((size_t)q_pc.b * p.Hkv + q_pc.hg) * C::QBUF, (uint32_t)C::QBUF,
-                          &bars[E_QFULL + buf]);
-                q_pending[buf] = true;
-                q_parity[buf] = (piece >> 1) & 1;
-            };
-            // cursor of the S^T products (runs one tile ahead) ...
-            PieceWalk walk_s(p, s_prefix, lo, hi, s_len);
-            Piece pcs, npcs;
-            walk_next(walk_s, pcs, flags);
-            fetch_q(pcs, 0);
-            int ts = pcs.t0;
-            uint32_t gs = 0, pis = 0;
+            EWalk walk_s(p, s_prefix, lo, hi), walk_o(p, s_prefix, lo, hi);
+            EPiece pc;
+            // cursor of the S^T products (runs one tile ahead): tiles left in its piece, first-tile flag, piece index
+            walk_s.next(p, s_prefix, s_len, pc, flags);
+            int s_left = pc.t1 - pc.t0, next_left = 0, next_image = pc.b * p.Hkv + pc.hg;
+            bool s_first = true, want_q = true;   // want_q: the image of piece q_piece is to be copied
+            uint32_t gs = 0, pis = 0, q_piece = 0;
             Ring krs;
-            auto issue_s = [&]() {
-                const int sb = (int)(gs & 1);
-                const bool first = ts == pcs.t0;
-                if (first) {
-                    ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
-                    if (ok) q_pending[pis & 1] = false;
-                }
-                if (ok && gs >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
-                    ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
-                if (ok) ok = wait_or_abort(&bars[E_FULL + krs.slot], krs.parity, abort_flag);
-                if (ok) {
-                    tc_fence_after_sync();
-                    const uint32_t k_a = slots_a + (uint32_t)krs.slot * kSlot8;
-                    const uint32_t q_a = qbuf_a + (pis & 1) * C::QBUF;
-#pragma unroll
-                    for (int kk = 0; kk < UD / 32; ++kk)
-                        umma_f8(tS + sb * 2 * RP, smem_desc(k_a + kk * 32, 16, 1024, 2),
-                                smem_desc(q_a + kk * 2 * C::QLBO, C::QLBO, 128, 0), idesc_qk, kk == 0 ? 0u : 1u);
-                    umma_commit(&bars[E_SFULL + sb]);
-                }
-                krs.advance(ring);
-                if (first && ok) {
-                    // The other image buffer was last read by the S^T products of the piece before; the last of them
-                    // (tile gs - 1) must have completed before the next piece's image is copied into it.
-                    if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
-                    if (ok && walk_next(walk_s, npcs, flags)) fetch_q(npcs, pis + 1);
-                }
-                ++gs;
-                if (++ts == pcs.t1 && gs < T) {
-                    pcs = npcs;
-                    ts = pcs.t0;
-                    ++pis;
-                }
-            };
             // ... and of the O^T products
-            PieceWalk walk_o(p, s_prefix, lo, hi, s_len);
-            Piece pco;
-            walk_next(walk_o, pco, flags);
-            int to = pco.t0;
+            walk_o.next(p, s_prefix, s_len, pc, flags);
+            int o_left = pc.t1 - pc.t0;
+            bool o_first = true;
             uint32_t pio = 0;
             Ring vro;
-            issue_s();
-            for (uint32_t g = 0; g < T && ok; ++g) {
-                if (g + 1 < T) issue_s();
-                if (!ok) break;
-                const int pb = (int)(g & 1);
-                const bool first = to == pco.t0, last = to == pco.t1 - 1;
-                const int ob = (int)(pio & 1);
-                if (first && pio >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
-                    ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
-                if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+            // Step i issues S^T of tile i (i < T) and the O^T product of tile i - 2 (i >= 2), one instruction of each in
+            // turn: the four instructions of a product accumulate into one another and so run one after the other at
+            // the latency of the tensor pipe, while two independent chains overlap. S^T thus runs two tiles ahead of
+            // the probabilities (its buffer is free as soon as the scores of tile i - 2 have been read).
+            for (uint32_t i = 0; i < T + 2 && ok; ++i) {
+                if (want_q) {
+                    const uint32_t buf = q_piece & 1;
+                    mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)C::QBUF);
+                    bulk_load(qbuf + buf * C::QBUF, qimg + (size_t)next_image * C::QBUF, (uint32_t)C::QBUF, &bars[E_QFULL + buf]);
+                    q_pending[buf] = true;
+                    q_parity[buf] = (q_piece >> 1) & 1;
+                    want_q = false;
+                }
+                const bool do_s = i < T, do_pv = i >= 2;
+                const uint32_t g = i - 2, pb = g & 1, ob = pio & 1, sb = gs & 1;
+                if (do_pv) {
+                    if (o_first && pio >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
+                        ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
+                    if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+                }
+                if (do_s && ok) {
+                    if (s_first) {
+                        ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
+                        if (ok) q_pending[pis & 1] = false;
+                    }
+                    if (ok && gs >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
+                        ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
+                    if (ok) ok = wait_or_abort(&bars[E_FULL + krs.slot], krs.parity, abort_flag);
+                }
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t v_a = slots_a + (uint32_t)vro.slot * kSlot8 + kTile8;
+                const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)krs.slot * (kSlot8 >> 4));
+                const uint64_t qd = qdesc0 + (uint64_t)((pis & 1) * (C::QBUF >> 4));
+                const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)vro.slot * (kSlot8 >> 4));
+                const uint64_t pd = pdesc0 + (uint64_t)(pb * (C::PBUF >> 4));
                 const uint32_t tOb = tO + ob * 3 * RP;
 #pragma unroll
-                for (int ks = 0; ks < UK / 32; ++ks)
-                    umma_f8(tOb, smem_desc(v_a + ks * 4096, kTile8, 1024, 2), smem_desc(pbuf_a + pb * C::PBUF + ks * 512, 128, 2048, 0),
-                            idesc_pv, (first && ks == 0) ? 0u : 1u);
-                umma_commit(&bars[E_PFREE + pb]);
-                umma_commit(&bars[E_EMPTY + vro.slot]);
-                if (last) umma_commit(&bars[E_OFULL + ob]);
-                vro.advance(ring);
-                if (++to == pco.t1 && g + 1 < T) {
-                    walk_next(walk_o, pco, flags);
-                    to = pco.t0;
-                    ++pio;
+                for (int k = 0; k < 4; ++k) {
+                    if (do_s)
+                        umma_f8(tS + sb * 2 * RP, kd + (uint64_t)(k * 2), qd + (uint64_t)(k * 2 * (C::QLBO >> 4)), idesc_qk,
+                                k == 0 ? 0u : 1u);
+                    if (do_pv)
+                        umma_f8(tOb, vd + (uint64_t)(k * (4096 >> 4)), pd + (uint64_t)(k * (512 >> 4)), idesc_pv,
+                                (o_first && k == 0) ? 0u : 1u);
+                }
+                if (do_s) {
+                    umma_commit(&bars[E_SFULL + sb]);
+                    krs.advance(ring);
+                    if (s_first) {
+                        // The other image buffer was last read by the S^T products of the piece before; the last of
+                        // them (tile gs - 1) must have completed before the next piece's image is copied into it.
+                        if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
+                        next_left = 0;
+                        if (ok && walk_s.next(p, s_prefix, s_len, pc, flags)) {
+                            next_left = pc.t1 - pc.t0;
+                            next_image = pc.b * p.Hkv + pc.hg;
+                            q_piece = pis + 1;
+                            want_q = true;   // copied at the top of the next step
+                        }
+                        s_first = false;
+                    }
+                    ++gs;
+                    if (--s_left == 0) {
+                        s_left = next_left;
+                        s_first = true;
+                        ++pis;
+                    }
+                }
+                if (do_pv) {
+                    umma_commit(&bars[E_PFREE + pb]);
+                    umma_commit(&bars[E_EMPTY + vro.slot]);
+                    vro.advance(ring);
+                    o_first = false;
+                    if (--o_left == 0) {
+                        umma_commit(&bars[E_OFULL + ob]);
+                        if (g + 1 < T) {
+                            walk_o.next(p, s_prefix, s_len, pc, flags);
+                            o_left = pc.t1 - pc.t0;
+                            o_first = true;
+                            ++pio;
+                        }
+                    }
                 }
             }
         }
     } else {
-        // ================================ softmax and epilogue (warps 0-3) ================================
-        // Thread tid owns key tid of every tile (tensor-memory lane tid of S^T) and, in the epilogue, output
-        // dimension tid (lane tid of O^T).
+        // ============================ softmax and epilogue (warps 0 .. 4 NG - 1) ============================
+        // Thread ltid of group grp owns key ltid of every tile (tensor-memory lane ltid of S^T), rows 8 grp .. + 7
+        // of it, and in the epilogue output dimension ltid (lane ltid of O^T) of the same rows.
         ECtx cx;
         cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lfin = s_lfin; cx.lim = s_lim;
         cx.rowloop = s_rowloop; cx.bars = bars; cx.abort_flag = abort_flag;
-        cx.lane_off = (uint32_t)(wid * 32) << 16;
+        cx.lane_off = (uint32_t)((wid & 3) * 32) << 16;
         cx.scale = 0.f;
-        cx.tid = tid; cx.lane = lane; cx.wid = wid;
+        cx.RP = RP;
+        cx.R = p.R;
+        const int grp = wid >> 2, row0 = grp * RT, ltid = tid & (kSmThreads - 1);
+        cx.row0 = row0; cx.bar_id = 1 + grp; cx.ltid = ltid; cx.lane = lane; cx.wq = wid & 3;
+        const uint32_t lane_off = cx.lane_off;
         bool failed = false;    // a wait of this warp ran out; it stops touching data but keeps the common control flow
-        bool aborted = false;   // agreed by all 128 threads
+        bool aborted = false;   // agreed by the 128 threads of the group
 
         // The epilogue of a piece runs one piece late, while the next piece is already streaming.
         bool ep_pending = false;
@@ -481,146 +650,145 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
 
         uint32_t gt = 0, pi = 0;
         Ring vr;   // slot of tile gt (only boundary tiles look at it)
-        PieceWalk walk(p, s_prefix, lo, hi, s_len);
-        Piece pc;
-        bool have = walk_next(walk, pc, flags);
+        EWalk walk(p, s_prefix, lo, hi);
+        EPiece pc;
+        EWin win;
+        bool have = walk.next(p, s_prefix, s_len, pc, flags);
         while (have && !aborted) {
             const uint32_t tOb = tO + (pi & 1) * 3 * RP;   // O^T of this piece
             const float scale = p.scale_log2 * p.k_scale[pc.hg] * qinv[pc.b * p.Hkv + pc.hg];
             cx.scale = scale;
+            const int kind = pc.kind, t0 = pc.t0, t1 = pc.t1, cmax = pc.cmax, pn = pc.n, pb_ = pc.b;
             int cmin = 0x7fffffff;
-#pragma unroll
-            for (int l = 0; l < kMaxLoops; ++l)
-                if (l < p.L) cmin = min(cmin, pc.sp.cut[l]);
-            WinCursor cur;
-            cur.l = 0;
-            cur.key0 = 0;
-            int seg_l = -1, wl = 0;
-            if (pc.kind == 1) {
-                cur.seek(p, pc.sp, pc.t0);
-                seg_l = cur.l;
-#pragma unroll
-                for (int k = 1; k < kMaxLoops; ++k)
-                    if (k == cur.l) wl = pc.sp.wl[k];
+#pragma unroll 1
+            for (int l = 0; l < p.L; ++l) cmin = min(cmin, e_cut(p, pn, l));
+            int seg_l = -1;
+            if (kind == 1) {
+                win.seek(p, pb_, pn, t0, flags);
+                seg_l = win.l;
             }
-            e_set_limits(p, cx, pc, RP, seg_l, wl, true);
-            float lsum[RP];   // this key's share of the denominators
+            e_set_limits(p, cx, kind, pn, seg_l, kind == 1 ? win.wl : 0, true);
+            float lsum[RT];    // this key's share of the denominators of the group's rows
+            float negm[RT];    // minus the reference maxima, kept in registers between the slow paths
 #pragma unroll
-            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
+            for (int r = 0; r < RT; ++r) {
+                lsum[r] = 0.f;
+                negm[r] = s_negm[row0 + r];
+            }
 
-            for (int t = pc.t0; t < pc.t1; ++t, ++gt) {
+            for (int t = t0; t < t1; ++t, ++gt) {
                 int kbase, nvalid;
                 bool masked;
-                if (pc.kind == 0) {
+                if (kind == 0) {
                     kbase = t * UK;
-                    nvalid = pc.sp.cmax - kbase;
+                    nvalid = cmax - kbase;
                     masked = kbase + UK > cmin;
                 } else {
-                    if (cur.l != seg_l) {   // a new window: only the rows of its loop see it
-                        seg_l = cur.l;
-#pragma unroll
-                        for (int k = 1; k < kMaxLoops; ++k)
-                            if (k == cur.l) wl = pc.sp.wl[k];
-                        e_set_limits(p, cx, pc, RP, seg_l, wl, false);
+                    if (win.l != seg_l) {   // a new window: only the rows of its loop see it
+                        seg_l = win.l;
+                        e_set_limits(p, cx, kind, pn, seg_l, win.wl, false);
                     }
-                    kbase = cur.key0;
-                    nvalid = wl - kbase;
+                    kbase = win.key0;
+                    nvalid = win.wl - kbase;
                     masked = true;
                 }
                 // ---- scores of this thread's key: the two terms of the queries added ----
-                const int sb = (int)(gt & 1);
+                const uint32_t sb = gt & 1;
                 failed = sm_wait(&bars[E_SFULL + sb], (gt >> 1) & 1, abort_flag, failed);
-                float s[RP];
+                float s[RT];
                 if (!failed) {
-                    uint32_t sv[2 * RP];
+                    uint32_t sv[2 * RT];
                     tc_fence_after_sync();
-#pragma unroll
-                    for (int c = 0; c < 2 * RP / 16; ++c) tmem_ld16(tS + sb * 2 * RP + cx.lane_off + c * 16, sv + c * 16);
+                    tmem_ld8(tS + sb * 2 * RP + lane_off + row0, sv);
+                    tmem_ld8(tS + sb * 2 * RP + lane_off + RP + row0, sv + RT);
                     tmem_wait_ld();
                     tc_fence_before_sync();
 #pragma unroll
-                    for (int r = 0; r < RP; ++r) s[r] = __uint_as_float(sv[r]) + __uint_as_float(sv[RP + r]);
+                    for (int r = 0; r < RT; ++r) s[r] = __uint_as_float(sv[r]) + __uint_as_float(sv[RT + r]);
                 } else {
 #pragma unroll
-                    for (int r = 0; r < RP; ++r) s[r] = -INFINITY;
+                    for (int r = 0; r < RT; ++r) s[r] = -INFINITY;
                 }
-                mbar_arrive(&bars[E_SFREE + sb]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[E_SFREE + sb]);
                 if (masked) {
-                    const int key = kbase + tid;
+                    const int key = kbase + ltid;
 #pragma unroll
-                    for (int r = 0; r < RP; ++r)
-                        if (key >= s_lim[r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
+                    for (int r = 0; r < RT; ++r)
+                        if (key >= s_lim[row0 + r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
                 }
+                float x[RT];   // exponents against the reference maxima (rows beyond R: -1e30, never the largest)
                 float over = -INFINITY;
 #pragma unroll
-                for (int r = 0; r < RP; ++r)
-                    if (r < p.R) over = fmaxf(over, fmaf(s[r], scale, s_negm[r]));
+                for (int r = 0; r < RT; ++r) {
+                    x[r] = fmaf(s[r], scale, negm[r]);
+                    over = fmaxf(over, x[r]);
+                }
                 const bool trouble = failed || (*abort_flag != 0);
-                if (named_barrier_or(1, kSmThreads, over > kSlack8 || trouble)) {
-                    if (named_barrier_or(1, kSmThreads, trouble)) {
+                if (named_barrier_or(cx.bar_id, kSmThreads, over > kSlack8 || trouble)) {
+                    if (named_barrier_or(cx.bar_id, kSmThreads, trouble)) {
                         aborted = true;
                         break;
                     }
                     // Copies, so that the arrays of the per-tile path stay in registers (the out-of-line call takes
                     // the addresses of its arguments).
-                    float s_c[RP], ls_c[RP];
+                    float s_c[RT], ls_c[RT];
 #pragma unroll
-                    for (int r = 0; r < RP; ++r) {
+                    for (int r = 0; r < RT; ++r) {
                         s_c[r] = s[r];
                         ls_c[r] = lsum[r];
                     }
-                    failed = e_slow_path<RP>(s_c, ls_c, cx, t != pc.t0, tOb, &bars[E_PFREE + ((gt - 1) & 1)], ((gt - 1) >> 1) & 1,
-                                             failed);
+                    failed = e_slow_path(s_c, ls_c, cx, t != t0, tOb, &bars[E_PFREE + ((gt - 1) & 1)], ((gt - 1) >> 1) & 1, failed);
 #pragma unroll
-                    for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
+                    for (int r = 0; r < RT; ++r) {
+                        lsum[r] = ls_c[r];
+                        negm[r] = s_negm[row0 + r];
+                        x[r] = fmaf(s[r], scale, negm[r]);
+                    }
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
-                const int pb = (int)(gt & 1);
+                const uint32_t pb = gt & 1;
                 if (gt >= 2) failed = sm_wait(&bars[E_PFREE + pb], ((gt >> 1) & 1) ^ 1u, abort_flag, failed);
-                uint8_t* pdst = pbuf + pb * C::PBUF + tid * 16;
+                uint32_t c_hi[RT / 4], c_mid[RT / 4], c_lo[RT / 4];
 #pragma unroll
-                for (int j = 0; j < RP / 16; ++j) {
-                    uint32_t c_hi[4], c_mid[4], c_lo[4];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const int r0 = j * 16 + 2 * q;
-                        const float p0 = fast_exp2(fmaf(s[r0], scale, s_negm[r0]));
-                        const float p1 = fast_exp2(fmaf(s[r0 + 1], scale, s_negm[r0 + 1]));
-                        lsum[r0] += p0;
-                        lsum[r0 + 1] += p1;
-                        const uint32_t h2 = pack_f16x2(p0, p1);
-                        const uint32_t c0 = f16x2_to_e4m3x2(h2);
-                        const uint32_t r1 = mul_f16x2(sub_f16x2(h2, e4m3x2_to_f16x2(c0)), kMidScaleH2);   // exact
-                        const uint32_t c1 = f16x2_to_e4m3x2(r1);
-                        const uint32_t r2 = mul_f16x2(sub_f16x2(r1, e4m3x2_to_f16x2(c1)), kLoScaleH2);    // exact
-                        const uint32_t c2 = f16x2_to_e4m3x2(r2);
-                        if (q & 1) {
-                            c_hi[q >> 1] |= c0 << 16;
-                            c_mid[q >> 1] |= c1 << 16;
-                            c_lo[q >> 1] |= c2 << 16;
-                        } else {
-                            c_hi[q >> 1] = c0;
-                            c_mid[q >> 1] = c1;
-                            c_lo[q >> 1] = c2;
-                        }
-                    }
-                    if (!failed) {
-                        *(uint4*)(pdst + (j) * 2048) = make_uint4(c_hi[0], c_hi[1], c_hi[2], c_hi[3]);
-                        *(uint4*)(pdst + (RP / 16 + j) * 2048) = make_uint4(c_mid[0], c_mid[1], c_mid[2], c_mid[3]);
-                        *(uint4*)(pdst + (2 * RP / 16 + j) * 2048) = make_uint4(c_lo[0], c_lo[1], c_lo[2], c_lo[3]);
+                for (int q = 0; q < RT / 2; ++q) {
+                    const float p0 = fast_exp2(x[2 * q]), p1 = fast_exp2(x[2 * q + 1]);
+                    lsum[2 * q] += p0;
+                    lsum[2 * q + 1] += p1;
+                    const uint32_t h2 = pack_f16x2(p0, p1);
+                    const uint32_t c0 = f16x2_to_e4m3x2(h2);
+                    const uint32_t r1 = mul_f16x2(sub_f16x2(h2, e4m3x2_to_f16x2(c0)), kMidScaleH2);   // exact
+                    const uint32_t c1 = f16x2_to_e4m3x2(r1);
+                    const uint32_t r2 = mul_f16x2(sub_f16x2(r1, e4m3x2_to_f16x2(c1)), kLoScaleH2);    // exact
+                    const uint32_t c2 = f16x2_to_e4m3x2(r2);
+                    if (q & 1) {
+                        c_hi[q >> 1] = byte_perm(c_hi[q >> 1], c0, 0x5410);
+                        c_mid[q >> 1] = byte_perm(c_mid[q >> 1], c1, 0x5410);
+                        c_lo[q >> 1] = byte_perm(c_lo[q >> 1], c2, 0x5410);
+                    } else {
+                        c_hi[q >> 1] = c0;
+                        c_mid[q >> 1] = c1;
+                        c_lo[q >> 1] = c2;
                     }
                 }
-                if (masked && nvalid < UK)
+                if (!failed) {
+                    // this group's half of a 16-row chunk of each term: [chunk][key][16 codes]
+                    uint8_t* pdst = pbuf + pb * C::PBUF + (row0 >> 4) * 2048 + ltid * 16 + (row0 & 15);
+                    *(uint2*)(pdst) = make_uint2(c_hi[0], c_hi[1]);
+                    *(uint2*)(pdst + (RP / 16) * 2048) = make_uint2(c_mid[0], c_mid[1]);
+                    *(uint2*)(pdst + 2 * (RP / 16) * 2048) = make_uint2(c_lo[0], c_lo[1]);
+                }
+                if (grp == 0 && masked && nvalid < UK)
                     failed = e_zero_v_rows(slots + (size_t)vr.slot * kSlot8 + kTile8, nvalid, &bars[E_FULL + vr.slot], vr.parity, cx,
                                            failed);
-                fence_proxy_async_smem();
-                mbar_arrive(&bars[E_PFULL + pb]);
+                fence_proxy_async_smem();   // by every thread that wrote, then one arrival per warp
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[E_PFULL + pb]);
                 vr.advance(ring);
-                if (pc.kind == 1) cur.advance(p, pc.sp);
-                if (t == pc.t0 && ep_pending) {
+                if (kind == 1) win.advance(p, pb_, pn, flags);
+                if (t == t0 && ep_pending) {
                     // put off so that the pipeline restarts first: the partial of the piece before
-                    failed = e_epilogue<RP>(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale,
-                                            failed);
+                    failed = e_epilogue(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
                     ep_pending = false;
                 }
             }
@@ -628,37 +796,42 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
 
             // ---- end of piece: denominators across the 128 keys, parked with the reference maxima; the epilogue
             //      proper runs one piece late ----
-            warp_reduce_rows<RP, false>(lsum, lane, s_red + wid * RP);
-            named_barrier_sync(1, kSmThreads);
-            if (tid < RP) {
-                s_lfin[(pi & 1) * RP + tid] = (s_red[tid] + s_red[RP + tid]) + (s_red[2 * RP + tid] + s_red[3 * RP + tid]);
-                s_mfin[(pi & 1) * RP + tid] = s_mref[tid];
+            warp_reduce_rows<RT, false>(lsum, lane, s_red + cx.wq * RP + row0);
+            named_barrier_sync(cx.bar_id, kSmThreads);
+            if (ltid < RT) {
+                const int tr = row0 + ltid;
+                s_lfin[(pi & 1) * RP + tr] = (s_red[tr] + s_red[RP + tr]) + (s_red[2 * RP + tr] + s_red[3 * RP + tr]);
+                s_mfin[(pi & 1) * RP + tr] = s_mref[tr];
             }
+            const int item = item_index(p, pb_, pc.hg, kind);
             ep_pending = true;
             ep_pi = pi;
-            ep_prow = slot_of(item_index(p, pc.b, pc.hg, pc.kind), cta) * p.R;   // one KV head per item on this path
+            ep_prow = slot_of(item, cta) * p.R;   // one KV head per item on this path
             ep_vscale = p.v_scale[pc.hg];
-            if (tid == 0) note_piece(p, pc, cta);
-            have = walk_next(walk, pc, flags);
+            if (tid == 0) {   // first and last block of the item, for the merge kernel
+                if (t0 == 0) p.item_blocks[2 * item] = cta;
+                if (t1 == pc.total) p.item_blocks[2 * item + 1] = cta;
+            }
+            have = walk.next(p, s_prefix, s_len, pc, flags);
             ++pi;
         }
         if (ep_pending && !aborted) {
-            named_barrier_sync(1, kSmThreads);   // s_mfin of the last piece visible to all
-            failed = e_epilogue<RP>(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
+            named_barrier_sync(cx.bar_id, kSmThreads);   // s_mfin of the last piece visible to the group
+            failed = e_epilogue(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
         }
     }
 
     // ---- common exit: nothing of this block may still be in flight when tensor memory is freed ----
     __syncthreads();
     const bool gave_up = *abort_flag != 0;
-    if (wid == 5 && lane == 0) {
+    if (wid == kIssuerWarp && lane == 0) {
         umma_commit(&bars[E_DRAIN]);   // arrives once every product issued by this thread has completed
         mbar_wait_bounded(&bars[E_DRAIN], 0, kUmmaWaitNs);
         // a query image that was asked for and never waited for gets a bounded chance to land
         for (int i = 0; i < 2; ++i)
             if (q_pending[i]) mbar_wait_bounded(&bars[E_QFULL + i], q_parity[i], kUmmaWaitNs);
     }
-    if (wid == 4 && lane == 0 && gave_up) {
+    if (wid == kProducerWarp && lane == 0 && gave_up) {
         // give every copy that was issued a bounded chance to land
         const uint32_t issued = (uint32_t)s_ctl[2];
         for (uint32_t m = issued > (uint32_t)ring ? issued - (uint32_t)ring : 0; m < issued; ++m)
@@ -668,7 +841,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     if (flags) atomicOr(p.status, flags);
     tc_fence_before_sync();
     __syncthreads();
-    if (wid == 5) {
+    if (wid == kIssuerWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
@@ -679,13 +852,13 @@ cudaError_t e4m3_prepare(size_t smem, int* blocks_per_sm) {
     auto fn = plt_decode_main_umma_e4m3<RP>;
     cudaError_t e = allow_max_dynamic_smem((const void*)fn);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, kThreads8, smem);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads8(RP), smem);
 }
 
 template <int RP>
 cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, const UmmaGeom& geo,
                         const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
-    plt_decode_main_umma_e4m3<RP><<<grid, kThreads8, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
+    plt_decode_main_umma_e4m3<RP><<<grid, threads8(RP), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
     return cudaGetLastError();
 }
 

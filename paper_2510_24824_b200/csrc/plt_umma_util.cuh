@@ -74,7 +74,7 @@ struct Ring {
 // dst[r] (shared memory).
 template <int N, bool MAX>
 __device__ __forceinline__ void warp_reduce_rows(float (&v)[N], int lane, float* dst) {
-    static_assert(N == 16 || N == 32 || N == 64, "rows per warp reduction");
+    static_assert(N == 8 || N == 16 || N == 32 || N == 64, "rows per warp reduction");
     if constexpr (N == 64) {
         float a[32], b[32];
 #pragma unroll
@@ -105,9 +105,10 @@ __device__ __forceinline__ void warp_reduce_rows(float (&v)[N], int lane, float*
                 v[0] = MAX ? fmaxf(v[0], got) : v[0] + got;
             }
         }
-        // N = 32: lane l holds row l. N = 16: lanes 2r and 2r + 1 both hold row r.
+        // N = 32: lane l holds row l. N = 16: lanes 2r and 2r + 1 both hold row r. N = 8: lanes 4r .. 4r + 3.
         if (N == 32) dst[lane] = v[0];
-        else if ((lane & 1) == 0) dst[lane >> 1] = v[0];
+        else if (N == 16) { if ((lane & 1) == 0) dst[lane >> 1] = v[0]; }
+        else if ((lane & 3) == 0) dst[lane >> 2] = v[0];
     }
 }
 

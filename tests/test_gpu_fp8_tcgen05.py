@@ -59,7 +59,7 @@ def test_shapes_and_edges(spec):
     assert np.all(got[inactive_rows(p)] == 0.0), "rows of loops without a token must be exactly zero"
 
 
-@pytest.mark.parametrize("stages,inflight", [(2, 1), (3, 2), (5, 5)])
+@pytest.mark.parametrize("stages,inflight", [(3, 1), (4, 2), (5, 5)])
 def test_ring_depths(stages, inflight):
     p = make_problem(custom(B=3, L=3, Hq=24, Hkv=4, w=50, lens=("list", [1700, 65, 3])))
     got = run_gpu(p, stages=stages, loads_in_flight=inflight, **T5)
