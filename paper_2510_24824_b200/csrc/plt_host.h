@@ -63,13 +63,13 @@ cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int gri
                              int wbox, int cap, cudaStream_t stream);
 
 // The same layout for E4M3 caches (tcgen05.mma kind::f8f6f4 on the codes, up to 32 packed rows; queries and
-// probabilities as sums of E4M3 terms). `qimg` / `qinv`: device scratch of max_batch * Hkv query images
+// probabilities as sums of E4M3 terms; hpc = 1 or 2 KV heads per work item, Params::hpc at launch). `qimg` / `qinv`: device scratch of max_batch * Hkv query images
 // (main_umma_e4m3_image_bytes each) and as many floats, written by a pack kernel launched first.
 int main_umma_e4m3_rows(int R);       // 16 or 32
 int main_umma_e4m3_max_slots();
-size_t main_umma_e4m3_smem(int R, int nslot, int max_batch);
+size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch);
 size_t main_umma_e4m3_image_bytes(int R);
-cudaError_t main_umma_e4m3_prepare(int R, size_t smem, int* blocks_per_sm);
+cudaError_t main_umma_e4m3_prepare(int R, int hpc, size_t smem, int* blocks_per_sm);
 cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream);
 cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                                   int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream);

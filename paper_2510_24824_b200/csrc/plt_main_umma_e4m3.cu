@@ -17,10 +17,13 @@
 // softmax threads add the two score columns of a row, and the epilogue adds the three accumulator columns. One tcgen05.mma costs the same issue slot whatever N is, so the extra terms are
 // free on the tensor side: 8 instructions per 32 KB tile.
 //
-// Warp roles: four softmax-and-epilogue warps per 8 packed rows (thread = key = tensor-memory lane, 8 scores of it;
-// four such groups at 32 rows, so four softmax warps per scheduler); then one warp, one lane: TMA producer of K and
-// V tiles (one ring of 32 KB slots, K then V); then one warp, one lane: issues every product, copies the packed query
-// image of the next piece (cp.async.bulk) and owns the tensor-memory allocation.
+// A work item is one or two KV heads of a sequence, and its steps alternate between them tile by tile: the codes of
+// a key of all heads lie side by side in memory, and neighbouring heads fetched within a short time of each other
+// stream at 6.4 TB/s where one head's 128 bytes per key alone stream at 4.5 (measured on B200).
+// Warp roles: one team of four softmax-and-epilogue warps per head of the item (thread = key = tensor-memory lane,
+// all RP scores of it); then one warp, one lane: TMA producer of K and V tiles (one ring of 32 KB slots, K then V);
+// then one warp, one lane: issues every product, copies the packed query images of the next piece (cp.async.bulk)
+// and owns the tensor-memory allocation.
 // The query image (codes in the core-matrix order the instruction reads, and the power of two they were scaled
 // by) is written per (sequence, KV head) by plt_decode_pack_q_e4m3, launched before this kernel.
 // Online softmax with a lazily updated reference maximum, as in the bf16 tcgen05 kernel. Every wait is bounded.
@@ -39,8 +42,8 @@ namespace {
 constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 keys x 128 codes
 constexpr int kSlot8 = 2 * kTile8;     // a ring slot: the K tile, then the V tile
 constexpr int kMaxRing8 = 5;
-// Threads of a block: 128 softmax threads per group of 8 packed rows, the producer warp, the issuer warp.
-__host__ __device__ constexpr int threads8(int RP) { return (RP / 8) * 128 + 64; }
+// Threads of a block: one team of 128 softmax threads per KV head of the item, the producer warp, the issuer warp.
+__host__ __device__ constexpr int threads8(int hpc) { return hpc * 128 + 64; }
 // A probability may exceed the lazily updated reference by 3 powers of two at most (p <= 8), which fixes the powers of
 // two the second and third term are scaled by: |p - hi| <= 2^-2 and |p - hi - mid| <= 2^-7 times 2^10 and 2^14 stay
 // below 448. The third term then resolves 2^-23, the step of the f16 the probability is rounded to first.
@@ -59,11 +62,13 @@ struct ECfg {
     static constexpr int QLBO = 2 * RP * 16;   // bytes between the 16-code column chunks of the query image
     static constexpr int QBUF = 8 * QLBO;      // [8 chunks][2 RP rows: hi then lo][16 codes]
     static constexpr int PBUF = 3 * RP * UK;   // [3 RP / 16 row groups: hi, mid, lo][128 keys][16 codes]
-    // Tensor memory: two S^T buffers of 2 RP columns (tile parity), two O^T buffers of 3 RP columns (piece parity).
+    // Tensor memory: two S^T buffers of 2 RP columns (step parity), then O^T buffers of 3 RP columns, one per piece
+    // parity and head of the item (two heads: 4 RP + 12 RP = 16 RP columns, all 512 at 32 rows).
     static constexpr int TMEM_COLS = RP == 16 ? 256 : 512;
-    __host__ __device__ static constexpr size_t smem_bytes(int nslot, int max_batch) {
-        return 1024 + (size_t)nslot * kSlot8 + 2 * PBUF + 2 * QBUF + E_COUNT * 8 + (size_t)RP * 4 * (3 + 4 + 2 + 4) + 64 +
-               (size_t)(2 * max_batch + 4) * 4;
+    // hpc: KV heads per work item (their tiles take turns; each has its own query image, reference maxima and O^T)
+    __host__ __device__ static constexpr size_t smem_bytes(int nslot, int hpc, int max_batch) {
+        return 1024 + (size_t)nslot * kSlot8 + 2 * PBUF + (size_t)2 * hpc * QBUF + E_COUNT * 8 +
+               (size_t)RP * 4 * (12 * hpc + 1) + 64 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
 
@@ -239,48 +244,46 @@ struct EWin {
     }
 };
 
-// ---- softmax side: per-group context and the work that is off the per-tile path -----------------------------
-// The packed rows are split into groups of 8: softmax warps 4 g .. 4 g + 3 own rows 8 g .. 8 g + 7 of every tile
-// (thread = key, 8 scores), with their own reference maxima, vote and rescale. Four groups (32 packed rows) put four
-// softmax warps on each scheduler: the per-tile chain of a warp is latency-bound, and this is what hides it.
-constexpr int RT = 8;    // rows per softmax thread
-
+// ---- softmax side: per-team context and the work that is off the per-step path -------------------------------
+// One team of four softmax warps per KV head of the item (thread = key, all RP scores of it). The steps of an item
+// alternate between its heads, so with two heads a team takes every other step and has two step times for each:
+// heads share nothing (own reference maxima, denominators, accumulator, score and probability buffer), so the two
+// teams never wait for one another.
 struct ECtx {
-    float* negm;       // [RP] minus the reference maximum of each row (1e30 while the row has none)
+    float* negm;       // [RP] of this team's head: minus the reference maximum of each row (1e30 while the row has none)
     float* mref;       // [RP] reference maximum, log2 units
     float* alpha;      // [RP] rescale factors of the slow path
     float* red;        // [4][RP] cross-warp reduction scratch
-    float* mfin;       // [2][RP] reference maxima of a finished piece, by O^T buffer
+    float* mfin;       // [2][RP] reference maxima of a finished piece, by piece parity
     float* lfin;       // [2][RP] its denominators
     int32_t* lim;      // [RP] keys visible to each row in the current segment
-    int32_t* rowloop;  // [RP] loop (0-based) of each packed row
+    int32_t* rowloop;  // [RP] loop (0-based) of each packed row (shared by the teams, read-only)
     uint64_t* bars;
     volatile int* abort_flag;
     uint32_t lane_off;  // this warp's lane quarter in a tensor-memory address
-    float scale;        // raw score -> log2 units, for the piece in hand (softmax scale, K scale, query scaling)
-    int RP;             // packed rows rounded up to 16 or 32
     int R;              // packed rows
-    int row0;           // first row of this thread's group
-    int bar_id;         // named barrier of the group's 128 threads
-    int ltid, lane, wq; // thread in the group (= key = output dimension), lane, warp in the group
+    int HPC;            // KV heads per work item = teams
+    int hh;             // this team's head within the item
+    int bar_id;         // named barrier of the team's 128 threads
+    int ltid, lane, wq; // thread in the team (= key = output dimension), lane, warp in the team
 };
 
-// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima of the group's
-// rows, and (unless this is the first tile of the piece) the rescale of their three O^T column groups and of the
-// denominators. The 128 threads of a group call it together. `done_bar` / `done_parity`: completion of the last
-// product into O^T.
-__device__ __noinline__ bool e_slow_path(const float (&s)[RT], float (&lsum)[RT], const ECtx& cx, bool rescale, uint32_t tOb,
-                                         uint64_t* done_bar, uint32_t done_parity, bool failed) {
-    const int RP = cx.RP;
+// Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima, and (unless this
+// is the head's first tile of the piece) the rescale of the three O^T column groups and of the denominators. The 128
+// threads of a team call it together. `scale`: raw score -> log2 units; `done_bar` / `done_parity`: completion of
+// the last product into this O^T.
+template <int RP>
+__device__ __noinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, float scale, bool rescale,
+                                         uint32_t tOb, uint64_t* done_bar, uint32_t done_parity, bool failed) {
     {
-        float v[RT];
+        float v[RP];
 #pragma unroll
-        for (int r = 0; r < RT; ++r) v[r] = s[r] * cx.scale;
-        warp_reduce_rows<RT, true>(v, cx.lane, cx.red + cx.wq * RP + cx.row0);
+        for (int r = 0; r < RP; ++r) v[r] = s[r] * scale;
+        warp_reduce_rows<RP, true>(v, cx.lane, cx.red + cx.wq * RP);
     }
     named_barrier_sync(cx.bar_id, kSmThreads);
-    if (cx.ltid < RT) {
-        const int t = cx.row0 + cx.ltid;
+    if (cx.ltid < RP) {
+        const int t = cx.ltid;
         const float mo = cx.mref[t];
         const float mn = fmaxf(fmaxf(mo, fmaxf(cx.red[t], cx.red[RP + t])), fmaxf(cx.red[2 * RP + t], cx.red[3 * RP + t]));
         cx.alpha[t] = (mo == -INFINITY) ? 1.f : exp2f(mo - mn);
@@ -294,54 +297,57 @@ __device__ __noinline__ bool e_slow_path(const float (&s)[RT], float (&lsum)[RT]
         if (!failed) {
             tc_fence_after_sync();
 #pragma unroll 1
-            for (int term = 0; term < 3; ++term) {
-                uint32_t o[RT];
-                const uint32_t addr = tOb + cx.lane_off + term * RP + cx.row0;
-                tmem_ld8(addr, o);
+            for (int c = 0; c < 3 * RP / 16; ++c) {
+                uint32_t o[16];
+                tmem_ld16(tOb + cx.lane_off + c * 16, o);
                 tmem_wait_ld();
+                const int r0 = (c * 16) % RP;
 #pragma unroll
-                for (int j = 0; j < RT; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[cx.row0 + j]);
-                tmem_st8(addr, o);
+                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * cx.alpha[r0 + j]);
+                tmem_st16(tOb + cx.lane_off + c * 16, o);
             }
             tmem_wait_st();
             tc_fence_before_sync();
         }
 #pragma unroll
-        for (int r = 0; r < RT; ++r) lsum[r] *= cx.alpha[cx.row0 + r];
+        for (int r = 0; r < RP; ++r) lsum[r] *= cx.alpha[r];
     }
     return failed;
 }
 
-// Epilogue of a finished piece for the group's rows: the three column groups of O^T summed (the second and third
+// Epilogue of a finished piece for this team's head: the three column groups of O^T summed (the second and third
 // scaled back), times the V scale of the head, and the denominators, out of tensor memory into the split partial.
+// tOb: O^T of the head in the piece; ob: piece parity; prow: first row of the head's partial.
+template <int RP>
 __device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
                                         float vscale, bool failed) {
     failed = sm_wait(&cx.bars[E_OFULL + ob], parity, cx.abort_flag, failed);
-    if (!failed) {
-        uint32_t o0[RT], o1[RT], o2[RT];
-        tc_fence_after_sync();
-        tmem_ld8(tOb + cx.lane_off + cx.row0, o0);
-        tmem_ld8(tOb + cx.lane_off + cx.RP + cx.row0, o1);
-        tmem_ld8(tOb + cx.lane_off + 2 * cx.RP + cx.row0, o2);
-        tmem_wait_ld();
+#pragma unroll 1
+    for (int c = 0; c < RP / 16; ++c) {
+        if (!failed) {
+            uint32_t o0[16], o1[16], o2[16];
+            tc_fence_after_sync();
+            tmem_ld16(tOb + cx.lane_off + c * 16, o0);
+            tmem_ld16(tOb + cx.lane_off + RP + c * 16, o1);
+            tmem_ld16(tOb + cx.lane_off + 2 * RP + c * 16, o2);
+            tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < RT; ++j)
-            if (cx.row0 + j < p.R)
-                p.part_acc[(prow + cx.row0 + j) * UD + cx.ltid] =
-                    (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
+            for (int j = 0; j < 16; ++j)
+                if (c * 16 + j < p.R)
+                    p.part_acc[(prow + c * 16 + j) * UD + cx.ltid] =
+                        (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
+        }
     }
     tc_fence_before_sync();
     __syncwarp();
     if (cx.lane == 0) mbar_arrive(&cx.bars[E_OFREE + ob]);
-    if (!failed && cx.ltid < RT && cx.row0 + cx.ltid < p.R) {
-        const int t = cx.row0 + cx.ltid;
-        *(float2*)(p.part_ml + (prow + t) * 2) = make_float2(cx.mfin[ob * cx.RP + t], cx.lfin[ob * cx.RP + t]);
-    }
+    if (!failed && cx.ltid < p.R)
+        *(float2*)(p.part_ml + (prow + cx.ltid) * 2) = make_float2(cx.mfin[ob * RP + cx.ltid], cx.lfin[ob * RP + cx.ltid]);
     return failed;
 }
 
 // V rows of a boundary tile that hold no data may contain anything (NaN codes too): zero them so that 0 * garbage
-// stays 0. `vtile`: the V half of the slot. Called by the threads of group 0.
+// stays 0. `vtile`: the V half of the slot. Called by the team that owns the step.
 __device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t* full_bar, uint32_t parity, const ECtx& cx,
                                            bool failed) {
     failed = sm_wait(full_bar, parity, cx.abort_flag, failed);
@@ -353,13 +359,14 @@ __device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t*
     return failed;
 }
 
-// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of the group's rows.
-// n: clamped length of the sequence.
-__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int kind, int n, int win_loop, int wl, bool new_piece) {
+// Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of each row; at the
+// start of a piece also the reference maxima. n: clamped length of the sequence.
+__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int RP, int kind, int n, int win_loop, int wl,
+                                          bool new_piece) {
     // Threads still forming the probabilities of the tile before read lim: nobody rewrites it earlier.
     named_barrier_sync(cx.bar_id, kSmThreads);
-    if (cx.ltid < RT) {
-        const int t = cx.row0 + cx.ltid;
+    if (cx.ltid < RP) {
+        const int t = cx.ltid;
         if (new_piece) {
             cx.mref[t] = -INFINITY;
             cx.negm[t] = t >= cx.R ? -1e30f : 1e30f;
@@ -374,8 +381,8 @@ __device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int k
     named_barrier_sync(cx.bar_id, kSmThreads);
 }
 
-template <int RP>
-__global__ void __launch_bounds__(threads8(RP), 1)
+template <int RP, int HPC>
+__global__ void __launch_bounds__(threads8(HPC), 1)
 plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                           const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
                           const __grid_constant__ Params p, const UmmaGeom geo, const uint8_t* __restrict__ qimg,
@@ -384,27 +391,22 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int ring = geo.ring;
-    uint8_t* slots = smem;                                  // ring of [K tile][V tile]
-    uint8_t* pbuf = smem + (size_t)ring * kSlot8;           // two buffers of PBUF (tile parity)
-    uint8_t* qbuf = pbuf + 2 * C::PBUF;                     // two buffers of QBUF (piece parity)
-    uint64_t* bars = (uint64_t*)(qbuf + 2 * C::QBUF);
-    float* s_negm = (float*)(bars + E_COUNT);
-    float* s_mref = s_negm + RP;
-    float* s_alpha = s_mref + RP;
-    float* s_red = s_alpha + RP;                            // [4][RP]
-    int32_t* s_lim = (int32_t*)(s_red + 4 * RP);
-    int32_t* s_rowloop = s_lim + RP;
-    float* s_mfin = (float*)(s_rowloop + RP);               // [2][RP]
-    float* s_lfin = s_mfin + 2 * RP;                        // [2][RP]
-    int32_t* s_ctl = (int32_t*)(s_lfin + 2 * RP);           // [0] abort flag, [1] tensor-memory base, [2] tiles issued by the producer
+    uint8_t* slots = smem;                                  // ring of [K tile][V tile] of one head
+    uint8_t* pbuf = smem + (size_t)ring * kSlot8;           // two buffers of PBUF (step parity)
+    uint8_t* qbuf = pbuf + 2 * C::PBUF;                     // two buffers (piece parity) of HPC query images
+    uint64_t* bars = (uint64_t*)(qbuf + 2 * HPC * C::QBUF);
+    // per team (= head of the item), kTeamFloats each: negm, mref, alpha [RP]; red [4][RP]; lim [RP]; mfin, lfin [2][RP]
+    constexpr int kTeamFloats = 12 * RP;
+    float* s_team = (float*)(bars + E_COUNT);
+    int32_t* s_rowloop = (int32_t*)(s_team + HPC * kTeamFloats);
+    int32_t* s_ctl = s_rowloop + RP;                        // [0] abort flag, [1] tensor-memory base, [2] steps issued by the producer
     int32_t* s_prefix = s_ctl + 16;                         // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                    // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
 
-    constexpr int NG = RP / RT;            // row groups = softmax warp quartets
-    constexpr int kSmWarps = NG * 4;       // softmax warps: one lane of each arrives on the barriers they feed (a
-                                           // block-wide count would put hundreds of arrivals on one shared-memory word per tile)
-    constexpr int kProducerWarp = 4 * NG, kIssuerWarp = 4 * NG + 1;
+    // One lane of each softmax warp arrives on the barriers they feed (a thread-wide count would put hundreds of
+    // arrivals on one shared-memory word per step). With two heads a score / probability buffer belongs to one team.
+    constexpr int kProducerWarp = 4 * HPC, kIssuerWarp = 4 * HPC + 1;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
 
@@ -417,11 +419,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars[E_SFULL + i], 1);
-            mbar_init(&bars[E_SFREE + i], kSmWarps);
-            mbar_init(&bars[E_PFULL + i], kSmWarps);
+            mbar_init(&bars[E_SFREE + i], 4);
+            mbar_init(&bars[E_PFULL + i], 4);
             mbar_init(&bars[E_PFREE + i], 1);
             mbar_init(&bars[E_OFULL + i], 1);
-            mbar_init(&bars[E_OFREE + i], kSmWarps);
+            mbar_init(&bars[E_OFREE + i], 4 * HPC);
             mbar_init(&bars[E_QFULL + i], 1);
         }
         mbar_init(&bars[E_DRAIN], 1);
@@ -435,26 +437,28 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = (uint32_t)s_ctl[1];
-    // S^T of tile parity g at tS + 2 RP g; O^T of piece parity b at tO + 3 RP b
+    // S^T of step parity g at tS + 2 RP g; O^T of piece parity b, head hh at tO + 3 RP (HPC b + hh)
     const uint32_t tS = tmem_base, tO = tmem_base + 4 * RP;
 
     const int64_t T64 = s_prefix[p.B];
     const int cta = blockIdx.x, nctas = plan_ctas(T64, (int)gridDim.x);
     if (cta == 0)
-        for (int b = tid; b <= p.B; b += threads8(RP)) p.prefix[b] = s_prefix[b];
+        for (int b = tid; b <= p.B; b += threads8(HPC)) p.prefix[b] = s_prefix[b];
     const bool in_plan = cta < nctas;
     const int lo = in_plan ? (int)cta_begin(T64, cta, nctas) : 0, hi = in_plan ? (int)cta_begin(T64, cta + 1, nctas) : 0;
-    // Tiles this block streams: the positions of its range minus the lead-in positions of its pieces (none on this
-    // path: piece_cost is 0, so every position is a tile).
-    const uint32_t T = (uint32_t)(hi - lo);
-    bool q_pending[2] = {false, false};       // issuer only: a query image was asked for and not yet waited for
-    uint32_t q_parity[2] = {0u, 0u};          // and the phase of its barrier that ends when it has landed
+    // Steps this block takes: one per (tile, head of the item). piece_cost is 0 on this path, so every position of
+    // the block's range of the line is a tile. The heads of a tile follow one another: a key's codes of all heads lie
+    // side by side in memory, and fetched within a short time of each other they come at 6.4 TB/s where one head's 128
+    // bytes per key alone come at 4.5 (measured on B200, 8 heads of 128 codes per key).
+    const uint32_t U = (uint32_t)(hi - lo) * HPC;
+    bool q_pending[2] = {false, false};       // issuer only: query images were asked for and not yet waited for
+    uint32_t q_parity[2] = {0u, 0u};          // and the phase of their barrier that ends when they have landed
 
     if (wid == kProducerWarp) {
         // ================================ TMA producer of K and V tiles ================================
-        // At most `cap` tiles in flight (issued, not landed): more outstanding requests make the memory system
-        // slower, not faster. cap <= ring, so the slot of the tile issued `cap` tiles ago has not been refilled.
-        if (lane == 0 && T > 0) {
+        // At most `cap` steps in flight (issued, not landed): more outstanding requests make the memory system
+        // slower, not faster. cap <= ring, so the slot of the step issued `cap` steps ago has not been refilled.
+        if (lane == 0 && U > 0) {
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmV);
             if (p.L > 1) {
@@ -464,14 +468,14 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             const uint64_t pol = l2_evict_first_policy();
             bool ok = true;
             uint32_t n = 0;
-            Ring cur, old;   // slot of tile n, slot of tile n - cap
+            Ring cur, old;   // slot of step n, slot of step n - cap
             EWalk walk(p, s_prefix, lo, hi);
             EPiece pc;
             EWin win;
             pc.t0 = pc.t1 = 0;
-            int t = 0;
-            for (; n < T && ok; ++n) {
-                if (t == pc.t1) {
+            int t = 0, hh = 0;
+            for (; n < U && ok; ++n) {
+                if (hh == 0 && t == pc.t1) {
                     walk.next(p, s_prefix, s_len, pc, flags);
                     t = pc.t0;
                     if (pc.kind == 1) win.seek(p, pc.b, pc.n, t, flags);
@@ -484,6 +488,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 if (!ok) break;
                 uint8_t* dst = slots + (size_t)cur.slot * kSlot8;
                 uint64_t* full = &bars[E_FULL + cur.slot];
+                const int head = pc.hg * HPC + hh;
                 if (pc.kind == 0 && p.page_size > 0) {
                     const int key0 = t * UK;
                     const int rem = pc.cmax - key0;   // keys that hold data from key0 on (>= 1)
@@ -496,29 +501,32 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                             flags |= kDevPageIdClamped;
                             page = page < 0 ? 0 : p.num_pool_pages - 1;
                         }
-                        tma_load_4d(dst + i * geo.kbox * 128, &tmK, full, 0, key % p.page_size, pc.hg, page, pol);
-                        tma_load_4d(dst + kTile8 + i * geo.kbox * 128, &tmV, full, 0, key % p.page_size, pc.hg, page, pol);
+                        tma_load_4d(dst + i * geo.kbox * 128, &tmK, full, 0, key % p.page_size, head, page, pol);
+                        tma_load_4d(dst + kTile8 + i * geo.kbox * 128, &tmV, full, 0, key % p.page_size, head, page, pol);
                     }
                 } else if (pc.kind == 0) {
                     mbar_expect_tx(full, (uint32_t)(geo.kbox * 256));
-                    tma_load_4d(dst, &tmK, full, 0, t * UK, pc.hg, pc.b, pol);
-                    tma_load_4d(dst + kTile8, &tmV, full, 0, t * UK, pc.hg, pc.b, pol);
+                    tma_load_4d(dst, &tmK, full, 0, t * UK, head, pc.b, pol);
+                    tma_load_4d(dst + kTile8, &tmV, full, 0, t * UK, head, pc.b, pol);
                 } else {
                     const int outer = pc.b * (p.L - 1) + (win.l - 1);
                     mbar_expect_tx(full, (uint32_t)(geo.wbox * 256));
-                    tma_load_4d(dst, &tmKw, full, 0, win.key0, pc.hg, outer, pol);
-                    tma_load_4d(dst + kTile8, &tmVw, full, 0, win.key0, pc.hg, outer, pol);
-                    win.advance(p, pc.b, pc.n, flags);
+                    tma_load_4d(dst, &tmKw, full, 0, win.key0, head, outer, pol);
+                    tma_load_4d(dst + kTile8, &tmVw, full, 0, win.key0, head, outer, pol);
                 }
                 cur.advance(ring);
-                ++t;
+                if (++hh == HPC) {
+                    hh = 0;
+                    if (pc.kind == 1) win.advance(p, pc.b, pc.n, flags);
+                    ++t;
+                }
             }
             s_ctl[2] = (int32_t)n;
         }
     } else if (wid == kIssuerWarp) {
         // ===================== issuer of both products (one lane); owner of tensor memory ======================
-        // All of its plan state is scalars: tiles left in the piece each cursor is in, the image index of the next piece.
-        if (lane == 0 && T > 0) {
+        // All of its plan state is scalars: steps left in the piece each cursor is in, the image index of the next piece.
+        if (lane == 0 && U > 0) {
             constexpr uint32_t idesc_qk = instr_desc_e4m3(UK, 2 * RP, 0, 0);
             constexpr uint32_t idesc_pv = instr_desc_e4m3(UD, 3 * RP, 1, 1);
             const uint32_t slots_a = smem_u32(slots);
@@ -528,35 +536,36 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             bool ok = true;
             EWalk walk_s(p, s_prefix, lo, hi), walk_o(p, s_prefix, lo, hi);
             EPiece pc;
-            // cursor of the S^T products (runs one tile ahead): tiles left in its piece, first-tile flag, piece index
+            // cursor of the S^T products (two steps ahead): steps left in its piece, steps done in it, piece index
             walk_s.next(p, s_prefix, s_len, pc, flags);
-            int s_left = pc.t1 - pc.t0, next_left = 0, next_image = pc.b * p.Hkv + pc.hg;
-            bool s_first = true, want_q = true;   // want_q: the image of piece q_piece is to be copied
-            uint32_t gs = 0, pis = 0, q_piece = 0;
+            int s_left = (pc.t1 - pc.t0) * HPC, next_left = 0, next_image = pc.b * p.Hkv + pc.hg * HPC;
+            bool s_first = true, want_q = true;   // want_q: the images of piece q_piece are to be copied
+            uint32_t gs = 0, pis = 0, q_piece = 0, s_head = 0;
             Ring krs;
             // ... and of the O^T products
             walk_o.next(p, s_prefix, s_len, pc, flags);
-            int o_left = pc.t1 - pc.t0;
-            bool o_first = true;
-            uint32_t pio = 0;
+            int o_left = (pc.t1 - pc.t0) * HPC;
+            uint32_t pio = 0, o_done = 0;   // o_done: steps of the piece done (the first HPC start an accumulator each)
             Ring vro;
-            // Step i issues S^T of tile i (i < T) and the O^T product of tile i - 2 (i >= 2), one instruction of each in
+            // Step i issues S^T of step i (i < U) and the O^T product of step i - 2 (i >= 2), one instruction of each in
             // turn: the four instructions of a product accumulate into one another and so run one after the other at
-            // the latency of the tensor pipe, while two independent chains overlap. S^T thus runs two tiles ahead of
-            // the probabilities (its buffer is free as soon as the scores of tile i - 2 have been read).
-            for (uint32_t i = 0; i < T + 2 && ok; ++i) {
+            // the latency of the tensor pipe, while two independent chains overlap. S^T thus runs two steps ahead of
+            // the probabilities (its buffer is free as soon as the scores of step i - 2 have been read).
+            for (uint32_t i = 0; i < U + 2 && ok; ++i) {
                 if (want_q) {
                     const uint32_t buf = q_piece & 1;
-                    mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)C::QBUF);
-                    bulk_load(qbuf + buf * C::QBUF, qimg + (size_t)next_image * C::QBUF, (uint32_t)C::QBUF, &bars[E_QFULL + buf]);
+                    mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)(HPC * C::QBUF));
+                    bulk_load(qbuf + buf * HPC * C::QBUF, qimg + (size_t)next_image * C::QBUF, (uint32_t)(HPC * C::QBUF),
+                              &bars[E_QFULL + buf]);   // the images of an item's heads are consecutive
                     q_pending[buf] = true;
                     q_parity[buf] = (q_piece >> 1) & 1;
                     want_q = false;
                 }
-                const bool do_s = i < T, do_pv = i >= 2;
+                const bool do_s = i < U, do_pv = i >= 2;
                 const uint32_t g = i - 2, pb = g & 1, ob = pio & 1, sb = gs & 1;
+                const uint32_t o_head = o_done < (uint32_t)HPC ? o_done : (o_done % HPC);
                 if (do_pv) {
-                    if (o_first && pio >= 2)   // the epilogue of the piece that used this O^T buffer before has read it
+                    if (o_done == 0 && pio >= 2)   // the epilogue of the piece that used these O^T buffers before has read them
                         ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
                     if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
                 }
@@ -565,17 +574,18 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                         ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
                         if (ok) q_pending[pis & 1] = false;
                     }
-                    if (ok && gs >= 2)   // the scores that were in this buffer (two tiles ago) have been read out
+                    if (ok && gs >= 2)   // the scores that were in this buffer (two steps ago) have been read out
                         ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
                     if (ok) ok = wait_or_abort(&bars[E_FULL + krs.slot], krs.parity, abort_flag);
                 }
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)krs.slot * (kSlot8 >> 4));
-                const uint64_t qd = qdesc0 + (uint64_t)((pis & 1) * (C::QBUF >> 4));
+                const uint64_t qd = qdesc0 + (uint64_t)(((pis & 1) * HPC + s_head) * (C::QBUF >> 4));
                 const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)vro.slot * (kSlot8 >> 4));
                 const uint64_t pd = pdesc0 + (uint64_t)(pb * (C::PBUF >> 4));
-                const uint32_t tOb = tO + ob * 3 * RP;
+                const uint32_t tOb = tO + (ob * HPC + o_head) * 3 * RP;
+                const bool o_start = o_done < (uint32_t)HPC;   // this head's first product of the piece
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if (do_s)
@@ -583,25 +593,26 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                                 k == 0 ? 0u : 1u);
                     if (do_pv)
                         umma_f8(tOb, vd + (uint64_t)(k * (4096 >> 4)), pd + (uint64_t)(k * (512 >> 4)), idesc_pv,
-                                (o_first && k == 0) ? 0u : 1u);
+                                (o_start && k == 0) ? 0u : 1u);
                 }
                 if (do_s) {
                     umma_commit(&bars[E_SFULL + sb]);
                     krs.advance(ring);
                     if (s_first) {
                         // The other image buffer was last read by the S^T products of the piece before; the last of
-                        // them (tile gs - 1) must have completed before the next piece's image is copied into it.
+                        // them (step gs - 1) must have completed before the next piece's images are copied into it.
                         if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
                         next_left = 0;
                         if (ok && walk_s.next(p, s_prefix, s_len, pc, flags)) {
-                            next_left = pc.t1 - pc.t0;
-                            next_image = pc.b * p.Hkv + pc.hg;
+                            next_left = (pc.t1 - pc.t0) * HPC;
+                            next_image = pc.b * p.Hkv + pc.hg * HPC;
                             q_piece = pis + 1;
                             want_q = true;   // copied at the top of the next step
                         }
                         s_first = false;
                     }
                     ++gs;
+                    if (++s_head == HPC) s_head = 0;
                     if (--s_left == 0) {
                         s_left = next_left;
                         s_first = true;
@@ -612,13 +623,13 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     umma_commit(&bars[E_PFREE + pb]);
                     umma_commit(&bars[E_EMPTY + vro.slot]);
                     vro.advance(ring);
-                    o_first = false;
+                    ++o_done;
                     if (--o_left == 0) {
                         umma_commit(&bars[E_OFULL + ob]);
-                        if (g + 1 < T) {
+                        if (g + 1 < U) {
                             walk_o.next(p, s_prefix, s_len, pc, flags);
-                            o_left = pc.t1 - pc.t0;
-                            o_first = true;
+                            o_left = (pc.t1 - pc.t0) * HPC;
+                            o_done = 0;
                             ++pio;
                         }
                     }
@@ -626,21 +637,26 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             }
         }
     } else {
-        // ============================ softmax and epilogue (warps 0 .. 4 NG - 1) ============================
-        // Thread ltid of group grp owns key ltid of every tile (tensor-memory lane ltid of S^T), rows 8 grp .. + 7
-        // of it, and in the epilogue output dimension ltid (lane ltid of O^T) of the same rows.
+        // ============================ softmax and epilogue (warps 0 .. 4 HPC - 1) ============================
+        // Team hh = warps 4 hh .. 4 hh + 3 takes the steps of head hh of every item. Thread ltid owns key ltid of
+        // its tiles (tensor-memory lane ltid of S^T) and, in the epilogue, output dimension ltid (lane of O^T).
+        const int hh = wid >> 2, ltid = tid & (kSmThreads - 1);
+        float* tf = s_team + hh * kTeamFloats;
+        float* s_negm = tf;
+        int32_t* s_lim = (int32_t*)(tf + 7 * RP);
+        float* s_red = tf + 3 * RP;
+        float* s_mfin = tf + 8 * RP;
+        float* s_lfin = tf + 10 * RP;
         ECtx cx;
-        cx.negm = s_negm; cx.mref = s_mref; cx.alpha = s_alpha; cx.red = s_red; cx.mfin = s_mfin; cx.lfin = s_lfin; cx.lim = s_lim;
+        cx.negm = s_negm; cx.mref = tf + RP; cx.alpha = tf + 2 * RP; cx.red = s_red; cx.mfin = s_mfin; cx.lfin = s_lfin; cx.lim = s_lim;
         cx.rowloop = s_rowloop; cx.bars = bars; cx.abort_flag = abort_flag;
         cx.lane_off = (uint32_t)((wid & 3) * 32) << 16;
-        cx.scale = 0.f;
-        cx.RP = RP;
         cx.R = p.R;
-        const int grp = wid >> 2, row0 = grp * RT, ltid = tid & (kSmThreads - 1);
-        cx.row0 = row0; cx.bar_id = 1 + grp; cx.ltid = ltid; cx.lane = lane; cx.wq = wid & 3;
+        cx.HPC = HPC;
+        cx.hh = hh; cx.bar_id = 1 + hh; cx.ltid = ltid; cx.lane = lane; cx.wq = wid & 3;
         const uint32_t lane_off = cx.lane_off;
         bool failed = false;    // a wait of this warp ran out; it stops touching data but keeps the common control flow
-        bool aborted = false;   // agreed by the 128 threads of the group
+        bool aborted = false;   // agreed by the 128 threads of the team
 
         // The epilogue of a piece runs one piece late, while the next piece is already streaming.
         bool ep_pending = false;
@@ -648,17 +664,18 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         int64_t ep_prow = 0;
         float ep_vscale = 1.f;
 
-        uint32_t gt = 0, pi = 0;
-        Ring vr;   // slot of tile gt (only boundary tiles look at it)
+        uint32_t g = (uint32_t)hh, pi = 0;   // this team's next step (all heads counted), pieces done
+        Ring vr;                             // slot of step g (only boundary tiles look at it)
+        for (int i = 0; i < hh; ++i) vr.advance(ring);
         EWalk walk(p, s_prefix, lo, hi);
         EPiece pc;
         EWin win;
         bool have = walk.next(p, s_prefix, s_len, pc, flags);
         while (have && !aborted) {
-            const uint32_t tOb = tO + (pi & 1) * 3 * RP;   // O^T of this piece
-            const float scale = p.scale_log2 * p.k_scale[pc.hg] * qinv[pc.b * p.Hkv + pc.hg];
-            cx.scale = scale;
-            const int kind = pc.kind, t0 = pc.t0, t1 = pc.t1, cmax = pc.cmax, pn = pc.n, pb_ = pc.b;
+            const uint32_t tOb = tO + ((pi & 1) * HPC + hh) * 3 * RP;   // O^T of this head in this piece
+            const int kind = pc.kind, t0 = pc.t0, t1 = pc.t1, cmax = pc.cmax, pn = pc.n, pb_ = pc.b, head = pc.hg * HPC + hh;
+            // raw score -> log2 units: softmax scale, K scale of the head, scaling of its query image
+            const float scale = p.scale_log2 * p.k_scale[head] * qinv[pb_ * p.Hkv + head];
             int cmin = 0x7fffffff;
 #pragma unroll 1
             for (int l = 0; l < p.L; ++l) cmin = min(cmin, e_cut(p, pn, l));
@@ -667,16 +684,12 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 win.seek(p, pb_, pn, t0, flags);
                 seg_l = win.l;
             }
-            e_set_limits(p, cx, kind, pn, seg_l, kind == 1 ? win.wl : 0, true);
-            float lsum[RT];    // this key's share of the denominators of the group's rows
-            float negm[RT];    // minus the reference maxima, kept in registers between the slow paths
+            e_set_limits(p, cx, RP, kind, pn, seg_l, kind == 1 ? win.wl : 0, true);
+            float lsum[RP];    // this key's share of the denominators
 #pragma unroll
-            for (int r = 0; r < RT; ++r) {
-                lsum[r] = 0.f;
-                negm[r] = s_negm[row0 + r];
-            }
+            for (int r = 0; r < RP; ++r) lsum[r] = 0.f;
 
-            for (int t = t0; t < t1; ++t, ++gt) {
+            for (int t = t0; t < t1; ++t, g += HPC) {
                 int kbase, nvalid;
                 bool masked;
                 if (kind == 0) {
@@ -686,109 +699,111 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 } else {
                     if (win.l != seg_l) {   // a new window: only the rows of its loop see it
                         seg_l = win.l;
-                        e_set_limits(p, cx, kind, pn, seg_l, win.wl, false);
+                        e_set_limits(p, cx, RP, kind, pn, seg_l, win.wl, false);
                     }
                     kbase = win.key0;
                     nvalid = win.wl - kbase;
                     masked = true;
                 }
                 // ---- scores of this thread's key: the two terms of the queries added ----
-                const uint32_t sb = gt & 1;
-                failed = sm_wait(&bars[E_SFULL + sb], (gt >> 1) & 1, abort_flag, failed);
-                float s[RT];
+                const uint32_t sb = g & 1;
+                failed = sm_wait(&bars[E_SFULL + sb], (g >> 1) & 1, abort_flag, failed);
+                float s[RP];
                 if (!failed) {
-                    uint32_t sv[2 * RT];
                     tc_fence_after_sync();
-                    tmem_ld8(tS + sb * 2 * RP + lane_off + row0, sv);
-                    tmem_ld8(tS + sb * 2 * RP + lane_off + RP + row0, sv + RT);
-                    tmem_wait_ld();
-                    tc_fence_before_sync();
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) s[r] = __uint_as_float(sv[r]) + __uint_as_float(sv[RT + r]);
+                    for (int c = 0; c < RP / 16; ++c) {
+                        uint32_t a[16], b[16];
+                        tmem_ld16(tS + sb * 2 * RP + lane_off + c * 16, a);
+                        tmem_ld16(tS + sb * 2 * RP + lane_off + RP + c * 16, b);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) s[c * 16 + j] = __uint_as_float(a[j]) + __uint_as_float(b[j]);
+                    }
+                    tc_fence_before_sync();
                 } else {
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) s[r] = -INFINITY;
+                    for (int r = 0; r < RP; ++r) s[r] = -INFINITY;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[E_SFREE + sb]);
                 if (masked) {
                     const int key = kbase + ltid;
 #pragma unroll
-                    for (int r = 0; r < RT; ++r)
-                        if (key >= s_lim[row0 + r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
+                    for (int r = 0; r < RP; ++r)
+                        if (key >= s_lim[r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
                 }
-                float x[RT];   // exponents against the reference maxima (rows beyond R: -1e30, never the largest)
+                // exponents against the reference maxima (rows beyond R: -1e30, never the largest), in place
                 float over = -INFINITY;
 #pragma unroll
-                for (int r = 0; r < RT; ++r) {
-                    x[r] = fmaf(s[r], scale, negm[r]);
-                    over = fmaxf(over, x[r]);
-                }
+                for (int r = 0; r < RP; ++r) over = fmaxf(over, fmaf(s[r], scale, s_negm[r]));
                 const bool trouble = failed || (*abort_flag != 0);
                 if (named_barrier_or(cx.bar_id, kSmThreads, over > kSlack8 || trouble)) {
                     if (named_barrier_or(cx.bar_id, kSmThreads, trouble)) {
                         aborted = true;
                         break;
                     }
-                    // Copies, so that the arrays of the per-tile path stay in registers (the out-of-line call takes
-                    // the addresses of its arguments).
-                    float s_c[RT], ls_c[RT];
+                    // Copies, so that the arrays of the per-step path stay in registers (the out-of-line call takes
+                    // the addresses of its arguments). The product before into this head's O^T was that of step g - HPC.
+                    float s_c[RP], ls_c[RP];
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) {
+                    for (int r = 0; r < RP; ++r) {
                         s_c[r] = s[r];
                         ls_c[r] = lsum[r];
                     }
-                    failed = e_slow_path(s_c, ls_c, cx, t != t0, tOb, &bars[E_PFREE + ((gt - 1) & 1)], ((gt - 1) >> 1) & 1, failed);
+                    failed = e_slow_path<RP>(s_c, ls_c, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) & 1)], ((g - HPC) >> 1) & 1, failed);
 #pragma unroll
-                    for (int r = 0; r < RT; ++r) {
-                        lsum[r] = ls_c[r];
-                        negm[r] = s_negm[row0 + r];
-                        x[r] = fmaf(s[r], scale, negm[r]);
-                    }
+                    for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
-                const uint32_t pb = gt & 1;
-                if (gt >= 2) failed = sm_wait(&bars[E_PFREE + pb], ((gt >> 1) & 1) ^ 1u, abort_flag, failed);
-                uint32_t c_hi[RT / 4], c_mid[RT / 4], c_lo[RT / 4];
+                const uint32_t pb = g & 1;
+                if (g >= 2) failed = sm_wait(&bars[E_PFREE + pb], ((g >> 1) & 1) ^ 1u, abort_flag, failed);
+                uint8_t* pdst = pbuf + pb * C::PBUF + ltid * 16;   // [3 RP / 16 chunks][key][16 codes]
 #pragma unroll
-                for (int q = 0; q < RT / 2; ++q) {
-                    const float p0 = fast_exp2(x[2 * q]), p1 = fast_exp2(x[2 * q + 1]);
-                    lsum[2 * q] += p0;
-                    lsum[2 * q + 1] += p1;
-                    const uint32_t h2 = pack_f16x2(p0, p1);
-                    const uint32_t c0 = f16x2_to_e4m3x2(h2);
-                    const uint32_t r1 = mul_f16x2(sub_f16x2(h2, e4m3x2_to_f16x2(c0)), kMidScaleH2);   // exact
-                    const uint32_t c1 = f16x2_to_e4m3x2(r1);
-                    const uint32_t r2 = mul_f16x2(sub_f16x2(r1, e4m3x2_to_f16x2(c1)), kLoScaleH2);    // exact
-                    const uint32_t c2 = f16x2_to_e4m3x2(r2);
-                    if (q & 1) {
-                        c_hi[q >> 1] = byte_perm(c_hi[q >> 1], c0, 0x5410);
-                        c_mid[q >> 1] = byte_perm(c_mid[q >> 1], c1, 0x5410);
-                        c_lo[q >> 1] = byte_perm(c_lo[q >> 1], c2, 0x5410);
-                    } else {
-                        c_hi[q >> 1] = c0;
-                        c_mid[q >> 1] = c1;
-                        c_lo[q >> 1] = c2;
+                for (int j = 0; j < RP / 16; ++j) {
+                    uint32_t c_hi[4], c_mid[4], c_lo[4];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int r0 = j * 16 + 2 * q;
+                        const float p0 = fast_exp2(fmaf(s[r0], scale, s_negm[r0]));
+                        const float p1 = fast_exp2(fmaf(s[r0 + 1], scale, s_negm[r0 + 1]));
+                        lsum[r0] += p0;
+                        lsum[r0 + 1] += p1;
+                        const uint32_t h2 = pack_f16x2(p0, p1);
+                        const uint32_t c0 = f16x2_to_e4m3x2(h2);
+                        const uint32_t r1 = mul_f16x2(sub_f16x2(h2, e4m3x2_to_f16x2(c0)), kMidScaleH2);   // exact
+                        const uint32_t c1 = f16x2_to_e4m3x2(r1);
+                        const uint32_t r2 = mul_f16x2(sub_f16x2(r1, e4m3x2_to_f16x2(c1)), kLoScaleH2);    // exact
+                        const uint32_t c2 = f16x2_to_e4m3x2(r2);
+                        if (q & 1) {
+                            c_hi[q >> 1] = byte_perm(c_hi[q >> 1], c0, 0x5410);
+                            c_mid[q >> 1] = byte_perm(c_mid[q >> 1], c1, 0x5410);
+                            c_lo[q >> 1] = byte_perm(c_lo[q >> 1], c2, 0x5410);
+                        } else {
+                            c_hi[q >> 1] = c0;
+                            c_mid[q >> 1] = c1;
+                            c_lo[q >> 1] = c2;
+                        }
+                    }
+                    if (!failed) {
+                        *(uint4*)(pdst + j * 2048) = make_uint4(c_hi[0], c_hi[1], c_hi[2], c_hi[3]);
+                        *(uint4*)(pdst + (RP / 16 + j) * 2048) = make_uint4(c_mid[0], c_mid[1], c_mid[2], c_mid[3]);
+                        *(uint4*)(pdst + (2 * RP / 16 + j) * 2048) = make_uint4(c_lo[0], c_lo[1], c_lo[2], c_lo[3]);
                     }
                 }
-                if (!failed) {
-                    // this group's half of a 16-row chunk of each term: [chunk][key][16 codes]
-                    uint8_t* pdst = pbuf + pb * C::PBUF + (row0 >> 4) * 2048 + ltid * 16 + (row0 & 15);
-                    *(uint2*)(pdst) = make_uint2(c_hi[0], c_hi[1]);
-                    *(uint2*)(pdst + (RP / 16) * 2048) = make_uint2(c_mid[0], c_mid[1]);
-                    *(uint2*)(pdst + 2 * (RP / 16) * 2048) = make_uint2(c_lo[0], c_lo[1]);
-                }
-                if (grp == 0 && masked && nvalid < UK)
+                if (masked && nvalid < UK)
                     failed = e_zero_v_rows(slots + (size_t)vr.slot * kSlot8 + kTile8, nvalid, &bars[E_FULL + vr.slot], vr.parity, cx,
                                            failed);
                 fence_proxy_async_smem();   // by every thread that wrote, then one arrival per warp
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[E_PFULL + pb]);
-                vr.advance(ring);
+#pragma unroll
+                for (int i = 0; i < HPC; ++i) vr.advance(ring);
                 if (kind == 1) win.advance(p, pb_, pn, flags);
                 if (t == t0 && ep_pending) {
                     // put off so that the pipeline restarts first: the partial of the piece before
-                    failed = e_epilogue(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
+                    failed = e_epilogue<RP>(p, cx, tO + ((ep_pi & 1) * HPC + hh) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow,
+                                            ep_vscale, failed);
                     ep_pending = false;
                 }
             }
@@ -796,18 +811,17 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
 
             // ---- end of piece: denominators across the 128 keys, parked with the reference maxima; the epilogue
             //      proper runs one piece late ----
-            warp_reduce_rows<RT, false>(lsum, lane, s_red + cx.wq * RP + row0);
+            warp_reduce_rows<RP, false>(lsum, lane, s_red + cx.wq * RP);
             named_barrier_sync(cx.bar_id, kSmThreads);
-            if (ltid < RT) {
-                const int tr = row0 + ltid;
-                s_lfin[(pi & 1) * RP + tr] = (s_red[tr] + s_red[RP + tr]) + (s_red[2 * RP + tr] + s_red[3 * RP + tr]);
-                s_mfin[(pi & 1) * RP + tr] = s_mref[tr];
+            if (ltid < RP) {
+                s_lfin[(pi & 1) * RP + ltid] = (s_red[ltid] + s_red[RP + ltid]) + (s_red[2 * RP + ltid] + s_red[3 * RP + ltid]);
+                s_mfin[(pi & 1) * RP + ltid] = cx.mref[ltid];
             }
             const int item = item_index(p, pb_, pc.hg, kind);
             ep_pending = true;
             ep_pi = pi;
-            ep_prow = slot_of(item, cta) * p.R;   // one KV head per item on this path
-            ep_vscale = p.v_scale[pc.hg];
+            ep_prow = (slot_of(item, cta) * HPC + hh) * p.R;
+            ep_vscale = p.v_scale[head];
             if (tid == 0) {   // first and last block of the item, for the merge kernel
                 if (t0 == 0) p.item_blocks[2 * item] = cta;
                 if (t1 == pc.total) p.item_blocks[2 * item + 1] = cta;
@@ -816,8 +830,9 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             ++pi;
         }
         if (ep_pending && !aborted) {
-            named_barrier_sync(cx.bar_id, kSmThreads);   // s_mfin of the last piece visible to the group
-            failed = e_epilogue(p, cx, tO + (ep_pi & 1) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale, failed);
+            named_barrier_sync(cx.bar_id, kSmThreads);   // s_mfin of the last piece visible to the team
+            failed = e_epilogue<RP>(p, cx, tO + ((ep_pi & 1) * HPC + hh) * 3 * RP, (int)(ep_pi & 1), (ep_pi >> 1) & 1, ep_prow, ep_vscale,
+                                    failed);
         }
     }
 
@@ -827,7 +842,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     if (wid == kIssuerWarp && lane == 0) {
         umma_commit(&bars[E_DRAIN]);   // arrives once every product issued by this thread has completed
         mbar_wait_bounded(&bars[E_DRAIN], 0, kUmmaWaitNs);
-        // a query image that was asked for and never waited for gets a bounded chance to land
+        // query images that were asked for and never waited for get a bounded chance to land
         for (int i = 0; i < 2; ++i)
             if (q_pending[i]) mbar_wait_bounded(&bars[E_QFULL + i], q_parity[i], kUmmaWaitNs);
     }
@@ -847,18 +862,18 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     }
 }
 
-template <int RP>
+template <int RP, int HPC>
 cudaError_t e4m3_prepare(size_t smem, int* blocks_per_sm) {
-    auto fn = plt_decode_main_umma_e4m3<RP>;
+    auto fn = plt_decode_main_umma_e4m3<RP, HPC>;
     cudaError_t e = allow_max_dynamic_smem((const void*)fn);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads8(RP), smem);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads8(HPC), smem);
 }
 
-template <int RP>
+template <int RP, int HPC>
 cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, const UmmaGeom& geo,
                         const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
-    plt_decode_main_umma_e4m3<RP><<<grid, threads8(RP), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
+    plt_decode_main_umma_e4m3<RP, HPC><<<grid, threads8(HPC), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
     return cudaGetLastError();
 }
 
@@ -868,15 +883,17 @@ int main_umma_e4m3_rows(int R) { return R <= 16 ? 16 : 32; }
 
 int main_umma_e4m3_max_slots() { return kMaxRing8; }
 
-size_t main_umma_e4m3_smem(int R, int nslot, int max_batch) {
-    return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::smem_bytes(nslot, max_batch) : ECfg<32>::smem_bytes(nslot, max_batch);
+size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch) {
+    return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::smem_bytes(nslot, hpc, max_batch) : ECfg<32>::smem_bytes(nslot, hpc, max_batch);
 }
 
 // Bytes of the query image of one (sequence, KV head).
 size_t main_umma_e4m3_image_bytes(int R) { return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::QBUF : ECfg<32>::QBUF; }
 
-cudaError_t main_umma_e4m3_prepare(int R, size_t smem, int* blocks_per_sm) {
-    return main_umma_e4m3_rows(R) == 16 ? e4m3_prepare<16>(smem, blocks_per_sm) : e4m3_prepare<32>(smem, blocks_per_sm);
+cudaError_t main_umma_e4m3_prepare(int R, int hpc, size_t smem, int* blocks_per_sm) {
+    if (main_umma_e4m3_rows(R) == 16)
+        return hpc == 2 ? e4m3_prepare<16, 2>(smem, blocks_per_sm) : e4m3_prepare<16, 1>(smem, blocks_per_sm);
+    return hpc == 2 ? e4m3_prepare<32, 2>(smem, blocks_per_sm) : e4m3_prepare<32, 1>(smem, blocks_per_sm);
 }
 
 cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream) {
@@ -888,8 +905,11 @@ cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cuda
 cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                                   int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
     const UmmaGeom geo{nslot, kbox, wbox, cap < 1 ? 1 : (cap > nslot ? nslot : cap)};
-    return main_umma_e4m3_rows(p.R) == 16 ? e4m3_launch<16>(maps, p, grid, smem, geo, qimg, qinv, stream)
-                                          : e4m3_launch<32>(maps, p, grid, smem, geo, qimg, qinv, stream);
+    if (main_umma_e4m3_rows(p.R) == 16)
+        return p.hpc == 2 ? e4m3_launch<16, 2>(maps, p, grid, smem, geo, qimg, qinv, stream)
+                          : e4m3_launch<16, 1>(maps, p, grid, smem, geo, qimg, qinv, stream);
+    return p.hpc == 2 ? e4m3_launch<32, 2>(maps, p, grid, smem, geo, qimg, qinv, stream)
+                      : e4m3_launch<32, 1>(maps, p, grid, smem, geo, qimg, qinv, stream);
 }
 
 }  // namespace plt

@@ -59,6 +59,29 @@ def test_shapes_and_edges(spec):
     assert np.all(got[inactive_rows(p)] == 0.0), "rows of loops without a token must be exactly zero"
 
 
+@pytest.mark.parametrize("hpc", [1, 2])
+@pytest.mark.parametrize("spec", [
+    custom(B=3, L=3, Hq=32, Hkv=4, w=50, lens=("list", [700, 65, 3])),                       # 24 packed rows
+    custom(B=2, L=3, Hq=8, Hkv=2, w=300, lens=("list", [2000, 290])),                        # windows of several tiles
+    custom(B=9, L=4, Hq=32, Hkv=4, w=100, page_size=64, lens=("list", [1, 2, 3, 63, 64, 255, 700, 129, 16])),
+], ids=["R24", "wide-window", "paged"])
+def test_heads_per_item(spec, hpc):
+    """One or two KV heads per work item (two: their tiles of the same keys take turns in one block)."""
+    p = make_problem(spec)
+    with DecodeAttn(p, heads_per_cta=hpc, **T5) as op:
+        assert op.info["heads_per_cta"] == hpc
+    assert_parity(run_gpu(p, heads_per_cta=hpc, **T5), oracle.decode_attn(p), "bf16", f"hpc={hpc}")
+
+
+def test_odd_number_of_kv_heads_takes_one_head_per_item():
+    p = make_problem(custom(B=3, L=2, Hq=12, Hkv=3, lens=("list", [700, 65, 3])))
+    with DecodeAttn(p, **T5) as op:
+        assert op.info["heads_per_cta"] == 1
+    with pytest.raises(B.PltError):
+        DecodeAttn(p, heads_per_cta=2, **T5)
+    assert_parity(run_gpu(p, **T5), oracle.decode_attn(p), "bf16", "Hkv=3")
+
+
 @pytest.mark.parametrize("stages,inflight", [(3, 1), (4, 2), (5, 5)])
 def test_ring_depths(stages, inflight):
     p = make_problem(custom(B=3, L=3, Hq=24, Hkv=4, w=50, lens=("list", [1700, 65, 3])))
