@@ -293,16 +293,16 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (hpc == 0) hpc = config->Hkv % 2 == 0 ? 2 : 1;
         if ((hpc != 1 && hpc != 2) || config->Hkv % hpc != 0)
             return fail(nullptr, PLT_ERR_INVALID_ARG, "heads_per_cta %d on the tcgen05 path with E4M3 caches (supported: 1, or 2 when Hkv is even)", hpc);
-        // Ring slots of 32 KB (K and V tile of one head): as many as fit beside the probability and query buffers,
-        // at least 3 (the scores run two steps ahead of the product that frees a slot).
+        // Ring slots of 16 KB (a K or a V tile of one head; 4 hold K tiles, the rest V tiles): as many as fit beside
+        // the probability and query buffers.
         int nslot = config->stages;
         if (nslot == 0) {
             nslot = main_umma_e4m3_max_slots();
-            while (nslot > 3 && main_umma_e4m3_smem(g.R, hpc, nslot, config->max_batch) > 227 * 1024) --nslot;
+            while (nslot > main_umma_e4m3_min_slots() && main_umma_e4m3_smem(g.R, hpc, nslot, config->max_batch) > 227 * 1024) --nslot;
         }
-        if (nslot < 3 || nslot > main_umma_e4m3_max_slots())
-            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path with E4M3 caches (supported: 3 to %d ring slots)",
-                        nslot, main_umma_e4m3_max_slots());
+        if (nslot < main_umma_e4m3_min_slots() || nslot > main_umma_e4m3_max_slots())
+            return fail(nullptr, PLT_ERR_INVALID_ARG, "stages %d on the tcgen05 path with E4M3 caches (supported: %d to %d ring slots)",
+                        nslot, main_umma_e4m3_min_slots(), main_umma_e4m3_max_slots());
         const size_t smem = main_umma_e4m3_smem(g.R, hpc, nslot, config->max_batch);
         if (smem > 227 * 1024)
             return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 path needs %zu bytes of shared memory (> 227 KB)", smem);

@@ -66,7 +66,8 @@ cudaError_t launch_main_umma(const CUtensorMap maps[4], const Params& p, int gri
 // probabilities as sums of E4M3 terms; hpc = 1 or 2 KV heads per work item, Params::hpc at launch). `qimg` / `qinv`: device scratch of max_batch * Hkv query images
 // (main_umma_e4m3_image_bytes each) and as many floats, written by a pack kernel launched first.
 int main_umma_e4m3_rows(int R);       // 16 or 32
-int main_umma_e4m3_max_slots();
+int main_umma_e4m3_max_slots();     // ring slots of 16 KB: 4 for K tiles, the rest (3 to 6) for V tiles
+int main_umma_e4m3_min_slots();
 size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch);
 size_t main_umma_e4m3_image_bytes(int R);
 cudaError_t main_umma_e4m3_prepare(int R, int hpc, size_t smem, int* blocks_per_sm);

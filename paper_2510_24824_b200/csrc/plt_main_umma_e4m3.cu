@@ -21,9 +21,9 @@
 // a key of all heads lie side by side in memory, and neighbouring heads fetched within a short time of each other
 // stream at 6.4 TB/s where one head's 128 bytes per key alone stream at 4.5 (measured on B200).
 // Warp roles: one team of four softmax-and-epilogue warps per head of the item (thread = key = tensor-memory lane,
-// all RP scores of it); then one warp, one lane: TMA producer of K and V tiles (one ring of 32 KB slots, K then V);
-// then one warp, one lane: issues every product, copies the packed query images of the next piece (cp.async.bulk)
-// and owns the tensor-memory allocation.
+// all RP scores of it); then four warps with one working lane each: the TMA producer of the K tiles and that of the
+// V tiles (a ring of 16 KB slots each), the issuer of the S^T products (which also copies the packed query images of
+// the next piece with cp.async.bulk and owns the tensor-memory allocation) and the issuer of the O^T products.
 // The query image (codes in the core-matrix order the instruction reads, and the power of two they were scaled
 // by) is written per (sequence, KV head) by plt_decode_pack_q_e4m3, launched before this kernel.
 // Online softmax with a lazily updated reference maximum, as in the bf16 tcgen05 kernel. Every wait is bounded.
@@ -39,11 +39,14 @@ namespace plt {
 
 namespace {
 
-constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 keys x 128 codes
-constexpr int kSlot8 = 2 * kTile8;     // a ring slot: the K tile, then the V tile
-constexpr int kMaxRing8 = 5;
-// Threads of a block: one team of 128 softmax threads per KV head of the item, the producer warp, the issuer warp.
-__host__ __device__ constexpr int threads8(int hpc) { return hpc * 128 + 64; }
+constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 keys x 128 codes = a ring slot
+// K tiles and V tiles have a ring each: a K tile is done with as soon as its scores are formed (two steps ahead of
+// the probabilities), a V tile only after the product that ends its step, so that one ring of K + V slots would
+// keep most of its slots waiting for that product and leave two loads in flight (measured: 4.7 TB/s at best).
+constexpr int kKRing8 = 4;             // K slots
+constexpr int kMaxVRing8 = 6;          // V slots at most
+// Threads of a block: one team of 128 softmax threads per KV head of the item, two producer warps, two issuer warps.
+__host__ __device__ constexpr int threads8(int hpc) { return hpc * 128 + 128; }
 // A probability may exceed the lazily updated reference by 3 powers of two at most (p <= 8), which fixes the powers of
 // two the second and third term are scaled by: |p - hi| <= 2^-2 and |p - hi - mid| <= 2^-7 times 2^10 and 2^14 stay
 // below 448. The third term then resolves 2^-23, the step of the f16 the probability is rounded to first.
@@ -53,9 +56,9 @@ constexpr uint32_t kLoScaleH2 = 0x4c004c00u;    // 2^4 as f16x2 (on top of the 2
 constexpr float kMidInv = 1.f / 1024.f, kLoInv = 1.f / 16384.f;
 
 // mbarrier indices
-constexpr int E_FULL = 0, E_EMPTY = 5, E_SFULL = 10 /* two */, E_SFREE = 12 /* two */, E_PFULL = 14 /* two */,
-              E_PFREE = 16 /* two */, E_OFULL = 18 /* two */, E_OFREE = 20 /* two */, E_QFULL = 22 /* two */,
-              E_DRAIN = 24, E_COUNT = 26;
+constexpr int E_KFULL = 0, E_KEMPTY = 4, E_VFULL = 8, E_VEMPTY = 14, E_SFULL = 20 /* two */, E_SFREE = 22 /* two */,
+              E_PFULL = 24 /* two */, E_PFREE = 26 /* two */, E_OFULL = 28 /* two */, E_OFREE = 30 /* two */,
+              E_QFULL = 32 /* two */, E_DRAIN = 34 /* two */, E_COUNT = 36;
 
 template <int RP>
 struct ECfg {
@@ -67,7 +70,7 @@ struct ECfg {
     static constexpr int TMEM_COLS = RP == 16 ? 256 : 512;
     // hpc: KV heads per work item (their tiles take turns; each has its own query image, reference maxima and O^T)
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int hpc, int max_batch) {
-        return 1024 + (size_t)nslot * kSlot8 + 2 * PBUF + (size_t)2 * hpc * QBUF + E_COUNT * 8 +
+        return 1024 + (size_t)nslot * kTile8 + 2 * PBUF + (size_t)2 * hpc * QBUF + E_COUNT * 8 +
                (size_t)RP * 4 * (12 * hpc + 1) + 64 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
@@ -381,6 +384,64 @@ __device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int R
     named_barrier_sync(cx.bar_id, kSmThreads);
 }
 
+// ---- the four single-lane roles: what happens once per piece, or on tiles that are not plain shared-cache tiles, is
+// out of line, so that the per-step loops of the producers and issuers are a few dozen instructions each. (Instruction
+// fetch decides the speed of this kernel: six loops run side by side on one SM.) ----
+struct ProdState {
+    EWalk walk;
+    EPiece pc;
+    EWin win;
+    int t;   // tile of the piece the next step belongs to
+    __device__ ProdState(const Params& p, const int32_t* sp, int lo, int hi) : walk(p, sp, lo, hi), t(0) { pc.t0 = pc.t1 = 0; }
+};
+
+// Next piece of a producer. Returns the steps it has (tiles x heads); `plain`: shared-cache tiles of a contiguous cache.
+__device__ __noinline__ int prod_next_piece(const Params& p, const int32_t* sp, const int32_t* lens, ProdState& st, int hpc, bool& plain,
+                                            uint32_t& flags) {
+    st.walk.next(p, sp, lens, st.pc, flags);
+    st.t = st.pc.t0;
+    if (st.pc.kind == 1) st.win.seek(p, st.pc.b, st.pc.n, st.t, flags);
+    plain = st.pc.kind == 0 && p.page_size == 0;
+    return (st.pc.t1 - st.pc.t0) * hpc;
+}
+
+// Loads of a tile of a paged cache or of a window (head `hh` of the item; after the item's last head the window
+// cursor moves on). `map`: the K or the V map of the tensor the tile belongs to.
+__device__ __noinline__ void prod_issue_special(const Params& p, const UmmaGeom& geo, ProdState& st, int hh, int hpc, uint8_t* dst,
+                                                uint64_t* full, const CUtensorMap* map, const CUtensorMap* wmap, uint64_t pol,
+                                                uint32_t& flags) {
+    const EPiece& pc = st.pc;
+    const int head = pc.hg * hpc + hh;
+    if (pc.kind == 0) {
+        const int key0 = st.t * UK;
+        const int rem = pc.cmax - key0;   // keys that hold data from key0 on (>= 1)
+        const int nbox = (min(rem, UK) + geo.kbox - 1) / geo.kbox;
+        mbar_expect_tx(full, (uint32_t)(nbox * geo.kbox * 128));
+        for (int i = 0; i < nbox; ++i) {
+            const int key = key0 + i * geo.kbox;
+            int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
+            if (page < 0 || page >= p.num_pool_pages) {
+                flags |= kDevPageIdClamped;
+                page = page < 0 ? 0 : p.num_pool_pages - 1;
+            }
+            tma_load_4d(dst + i * geo.kbox * 128, map, full, 0, key % p.page_size, head, page, pol);
+        }
+    } else {
+        mbar_expect_tx(full, (uint32_t)(geo.wbox * 128));
+        tma_load_4d(dst, wmap, full, 0, st.win.key0, head, pc.b * (p.L - 1) + (st.win.l - 1), pol);
+        if (hh == hpc - 1) st.win.advance(p, pc.b, pc.n, flags);
+    }
+}
+
+// Next piece of an issuer: its steps (0: none left) and the index of its first query image.
+__device__ __noinline__ int issuer_next_piece(const Params& p, const int32_t* sp, const int32_t* lens, EWalk& walk, int hpc, int& image,
+                                              uint32_t& flags) {
+    EPiece pc;
+    if (!walk.next(p, sp, lens, pc, flags)) return 0;
+    image = pc.b * p.Hkv + pc.hg * hpc;
+    return (pc.t1 - pc.t0) * hpc;
+}
+
 template <int RP, int HPC>
 __global__ void __launch_bounds__(threads8(HPC), 1)
 plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -390,32 +451,38 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     using C = ECfg<RP>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int ring = geo.ring;
-    uint8_t* slots = smem;                                  // ring of [K tile][V tile] of one head
-    uint8_t* pbuf = smem + (size_t)ring * kSlot8;           // two buffers of PBUF (step parity)
+    const int vring = geo.ring - kKRing8;                   // V slots (geo.ring counts all slots)
+    uint8_t* kslots = smem;                                 // ring of K tiles, then ring of V tiles
+    uint8_t* vslots = smem + (size_t)kKRing8 * kTile8;
+    uint8_t* pbuf = smem + (size_t)geo.ring * kTile8;       // two buffers of PBUF (step parity)
     uint8_t* qbuf = pbuf + 2 * C::PBUF;                     // two buffers (piece parity) of HPC query images
     uint64_t* bars = (uint64_t*)(qbuf + 2 * HPC * C::QBUF);
     // per team (= head of the item), kTeamFloats each: negm, mref, alpha [RP]; red [4][RP]; lim [RP]; mfin, lfin [2][RP]
     constexpr int kTeamFloats = 12 * RP;
     float* s_team = (float*)(bars + E_COUNT);
     int32_t* s_rowloop = (int32_t*)(s_team + HPC * kTeamFloats);
-    int32_t* s_ctl = s_rowloop + RP;                        // [0] abort flag, [1] tensor-memory base, [2] steps issued by the producer
+    int32_t* s_ctl = s_rowloop + RP;                        // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued
     int32_t* s_prefix = s_ctl + 16;                         // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                    // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
 
     // One lane of each softmax warp arrives on the barriers they feed (a thread-wide count would put hundreds of
     // arrivals on one shared-memory word per step). With two heads a score / probability buffer belongs to one team.
-    constexpr int kProducerWarp = 4 * HPC, kIssuerWarp = 4 * HPC + 1;
+    constexpr int kKProducerWarp = 4 * HPC, kVProducerWarp = 4 * HPC + 1, kSIssuerWarp = 4 * HPC + 2, kOIssuerWarp = 4 * HPC + 3;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     uint32_t flags = 0;
 
     if (tid == 0) {
         s_ctl[0] = 0;
         s_ctl[2] = 0;
-        for (int s = 0; s < kMaxRing8; ++s) {
-            mbar_init(&bars[E_FULL + s], 1);
-            mbar_init(&bars[E_EMPTY + s], 1);
+        s_ctl[3] = 0;
+        for (int s = 0; s < kKRing8; ++s) {
+            mbar_init(&bars[E_KFULL + s], 1);
+            mbar_init(&bars[E_KEMPTY + s], 1);
+        }
+        for (int s = 0; s < kMaxVRing8; ++s) {
+            mbar_init(&bars[E_VFULL + s], 1);
+            mbar_init(&bars[E_VEMPTY + s], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars[E_SFULL + i], 1);
@@ -427,10 +494,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             mbar_init(&bars[E_QFULL + i], 1);
         }
         mbar_init(&bars[E_DRAIN], 1);
+        mbar_init(&bars[E_DRAIN + 1], 1);
         mbar_fence_init();
     }
     if (tid < RP) s_rowloop[tid] = tid / p.G;
-    if (wid == kIssuerWarp) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
+    if (wid == kSIssuerWarp) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags, s_len, /*small=*/true);  // contains __syncthreads
     tc_fence_before_sync();
@@ -454,104 +522,77 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     bool q_pending[2] = {false, false};       // issuer only: query images were asked for and not yet waited for
     uint32_t q_parity[2] = {0u, 0u};          // and the phase of their barrier that ends when they have landed
 
-    if (wid == kProducerWarp) {
-        // ================================ TMA producer of K and V tiles ================================
-        // At most `cap` steps in flight (issued, not landed): more outstanding requests make the memory system
-        // slower, not faster. cap <= ring, so the slot of the step issued `cap` steps ago has not been refilled.
+    if (wid == kKProducerWarp || wid == kVProducerWarp) {
+        // ===================== TMA producers: one warp streams the K tiles, one the V tiles =====================
+        // Each keeps at most `cap` of its tiles in flight (issued, not landed): more outstanding requests make the
+        // memory system slower, not faster. cap <= ring, so the slot of the tile issued `cap` tiles ago has not been
+        // refilled and its phase parity is unambiguous.
         if (lane == 0 && U > 0) {
-            tma_prefetch_desc(&tmK);
-            tma_prefetch_desc(&tmV);
-            if (p.L > 1) {
-                tma_prefetch_desc(&tmKw);
-                tma_prefetch_desc(&tmVw);
-            }
+            const bool is_v = wid == kVProducerWarp;
+            const int ring = is_v ? vring : kKRing8, cap = geo.cap < ring ? geo.cap : ring;
+            uint8_t* slots = is_v ? vslots : kslots;
+            uint64_t* fullb = &bars[is_v ? E_VFULL : E_KFULL];
+            uint64_t* emptyb = &bars[is_v ? E_VEMPTY : E_KEMPTY];
+            const CUtensorMap* map = is_v ? &tmV : &tmK;
+            const CUtensorMap* wmap = is_v ? &tmVw : &tmKw;
+            tma_prefetch_desc(map);
+            if (p.L > 1) tma_prefetch_desc(wmap);
             const uint64_t pol = l2_evict_first_policy();
-            bool ok = true;
+            bool ok = true, plain = false;
+            Ring cur, old;   // slot of tile n, slot of tile n - cap
+            ProdState st(p, s_prefix, lo, hi);
+            int left = 0, hh = 0, key0 = 0, head0 = 0, outer = 0;   // of a plain piece: next tile's first key, first head, sequence
             uint32_t n = 0;
-            Ring cur, old;   // slot of step n, slot of step n - cap
-            EWalk walk(p, s_prefix, lo, hi);
-            EPiece pc;
-            EWin win;
-            pc.t0 = pc.t1 = 0;
-            int t = 0, hh = 0;
             for (; n < U && ok; ++n) {
-                if (hh == 0 && t == pc.t1) {
-                    walk.next(p, s_prefix, s_len, pc, flags);
-                    t = pc.t0;
-                    if (pc.kind == 1) win.seek(p, pc.b, pc.n, t, flags);
+                if (left == 0) {
+                    left = prod_next_piece(p, s_prefix, s_len, st, HPC, plain, flags);
+                    key0 = st.t * UK;
+                    head0 = st.pc.hg * HPC;
+                    outer = st.pc.b;
                 }
-                if (n >= (uint32_t)geo.cap) {
-                    ok = wait_or_abort(&bars[E_FULL + old.slot], old.parity, abort_flag);
+                if (n >= (uint32_t)cap) {
+                    ok = wait_or_abort(&fullb[old.slot], old.parity, abort_flag);
                     old.advance(ring);
                 }
-                if (ok && n >= (uint32_t)ring) ok = wait_or_abort(&bars[E_EMPTY + cur.slot], cur.parity ^ 1u, abort_flag);
+                if (ok && n >= (uint32_t)ring) ok = wait_or_abort(&emptyb[cur.slot], cur.parity ^ 1u, abort_flag);
                 if (!ok) break;
-                uint8_t* dst = slots + (size_t)cur.slot * kSlot8;
-                uint64_t* full = &bars[E_FULL + cur.slot];
-                const int head = pc.hg * HPC + hh;
-                if (pc.kind == 0 && p.page_size > 0) {
-                    const int key0 = t * UK;
-                    const int rem = pc.cmax - key0;   // keys that hold data from key0 on (>= 1)
-                    const int nbox = (min(rem, UK) + geo.kbox - 1) / geo.kbox;
-                    mbar_expect_tx(full, (uint32_t)(nbox * geo.kbox * 256));
-                    for (int i = 0; i < nbox; ++i) {
-                        const int key = key0 + i * geo.kbox;
-                        int page = p.page_table[(int64_t)pc.b * p.max_pages + key / p.page_size];
-                        if (page < 0 || page >= p.num_pool_pages) {
-                            flags |= kDevPageIdClamped;
-                            page = page < 0 ? 0 : p.num_pool_pages - 1;
-                        }
-                        tma_load_4d(dst + i * geo.kbox * 128, &tmK, full, 0, key % p.page_size, head, page, pol);
-                        tma_load_4d(dst + kTile8 + i * geo.kbox * 128, &tmV, full, 0, key % p.page_size, head, page, pol);
-                    }
-                } else if (pc.kind == 0) {
-                    mbar_expect_tx(full, (uint32_t)(geo.kbox * 256));
-                    tma_load_4d(dst, &tmK, full, 0, t * UK, head, pc.b, pol);
-                    tma_load_4d(dst + kTile8, &tmV, full, 0, t * UK, head, pc.b, pol);
+                uint8_t* dst = slots + (size_t)cur.slot * kTile8;
+                uint64_t* full = &fullb[cur.slot];
+                if (plain) {
+                    mbar_expect_tx(full, (uint32_t)(geo.kbox * 128));
+                    tma_load_4d(dst, map, full, 0, key0, head0 + hh, outer, pol);
                 } else {
-                    const int outer = pc.b * (p.L - 1) + (win.l - 1);
-                    mbar_expect_tx(full, (uint32_t)(geo.wbox * 256));
-                    tma_load_4d(dst, &tmKw, full, 0, win.key0, head, outer, pol);
-                    tma_load_4d(dst + kTile8, &tmVw, full, 0, win.key0, head, outer, pol);
+                    prod_issue_special(p, geo, st, hh, HPC, dst, full, map, wmap, pol, flags);
                 }
                 cur.advance(ring);
+                --left;
                 if (++hh == HPC) {
                     hh = 0;
-                    if (pc.kind == 1) win.advance(p, pc.b, pc.n, flags);
-                    ++t;
+                    key0 += UK;
+                    ++st.t;
                 }
             }
-            s_ctl[2] = (int32_t)n;
+            s_ctl[is_v ? 3 : 2] = (int32_t)n;
         }
-    } else if (wid == kIssuerWarp) {
-        // ===================== issuer of both products (one lane); owner of tensor memory ======================
-        // All of its plan state is scalars: steps left in the piece each cursor is in, the image index of the next piece.
+    } else if (wid == kSIssuerWarp) {
+        // ============ S^T = K [Q_hi ; Q_lo]^T issuer (one lane); owner of tensor memory and of the query images ============
+        // A score buffer is refilled as soon as the team that owns it has read the scores of its step before, so the
+        // scores of a team's next step are ready long before it has formed the probabilities of this one. The O^T
+        // products have an issuer of their own: each waits for its own conditions only.
         if (lane == 0 && U > 0) {
             constexpr uint32_t idesc_qk = instr_desc_e4m3(UK, 2 * RP, 0, 0);
-            constexpr uint32_t idesc_pv = instr_desc_e4m3(UD, 3 * RP, 1, 1);
-            const uint32_t slots_a = smem_u32(slots);
             // descriptors of slot 0 / buffer 0; the others differ in the start-address field (16-byte units) only
-            const uint64_t kdesc0 = smem_desc(slots_a, 16, 1024, 2), vdesc0 = smem_desc(slots_a + kTile8, kTile8, 1024, 2);
-            const uint64_t qdesc0 = smem_desc(smem_u32(qbuf), C::QLBO, 128, 0), pdesc0 = smem_desc(smem_u32(pbuf), 128, 2048, 0);
+            const uint64_t kdesc0 = smem_desc(smem_u32(kslots), 16, 1024, 2);
+            const uint64_t qdesc0 = smem_desc(smem_u32(qbuf), C::QLBO, 128, 0);
             bool ok = true;
-            EWalk walk_s(p, s_prefix, lo, hi), walk_o(p, s_prefix, lo, hi);
-            EPiece pc;
-            // cursor of the S^T products (two steps ahead): steps left in its piece, steps done in it, piece index
-            walk_s.next(p, s_prefix, s_len, pc, flags);
-            int s_left = (pc.t1 - pc.t0) * HPC, next_left = 0, next_image = pc.b * p.Hkv + pc.hg * HPC;
+            EWalk walk(p, s_prefix, lo, hi);
+            // steps left in the piece, and the piece after it (0 steps: none) with the index of its first image
+            int next_image = 0, next_left = 0;
+            int s_left = issuer_next_piece(p, s_prefix, s_len, walk, HPC, next_image, flags);
             bool s_first = true, want_q = true;   // want_q: the images of piece q_piece are to be copied
-            uint32_t gs = 0, pis = 0, q_piece = 0, s_head = 0;
+            uint32_t pis = 0, q_piece = 0, s_head = 0;
             Ring krs;
-            // ... and of the O^T products
-            walk_o.next(p, s_prefix, s_len, pc, flags);
-            int o_left = (pc.t1 - pc.t0) * HPC;
-            uint32_t pio = 0, o_done = 0;   // o_done: steps of the piece done (the first HPC start an accumulator each)
-            Ring vro;
-            // Step i issues S^T of step i (i < U) and the O^T product of step i - 2 (i >= 2), one instruction of each in
-            // turn: the four instructions of a product accumulate into one another and so run one after the other at
-            // the latency of the tensor pipe, while two independent chains overlap. S^T thus runs two steps ahead of
-            // the probabilities (its buffer is free as soon as the scores of step i - 2 have been read).
-            for (uint32_t i = 0; i < U + 2 && ok; ++i) {
+            for (uint32_t gs = 0; gs < U && ok; ++gs) {
                 if (want_q) {
                     const uint32_t buf = q_piece & 1;
                     mbar_expect_tx(&bars[E_QFULL + buf], (uint32_t)(HPC * C::QBUF));
@@ -561,77 +602,80 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     q_parity[buf] = (q_piece >> 1) & 1;
                     want_q = false;
                 }
-                const bool do_s = i < U, do_pv = i >= 2;
-                const uint32_t g = i - 2, pb = g & 1, ob = pio & 1, sb = gs & 1;
-                const uint32_t o_head = o_done < (uint32_t)HPC ? o_done : (o_done % HPC);
-                if (do_pv) {
-                    if (o_done == 0 && pio >= 2)   // the epilogue of the piece that used these O^T buffers before has read them
-                        ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
-                    if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+                const uint32_t sb = gs & 1;
+                if (s_first) {
+                    ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
+                    if (ok) q_pending[pis & 1] = false;
                 }
-                if (do_s && ok) {
-                    if (s_first) {
-                        ok = wait_or_abort(&bars[E_QFULL + (pis & 1)], (pis >> 1) & 1, abort_flag);
-                        if (ok) q_pending[pis & 1] = false;
-                    }
-                    if (ok && gs >= 2)   // the scores that were in this buffer (two steps ago) have been read out
-                        ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
-                    if (ok) ok = wait_or_abort(&bars[E_FULL + krs.slot], krs.parity, abort_flag);
-                }
+                if (ok && gs >= 2)   // the scores that were in this buffer (two steps ago) have been read out
+                    ok = wait_or_abort(&bars[E_SFREE + sb], ((gs >> 1) & 1) ^ 1u, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_KFULL + krs.slot], krs.parity, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)krs.slot * (kSlot8 >> 4));
+                const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)krs.slot * (kTile8 >> 4));
                 const uint64_t qd = qdesc0 + (uint64_t)(((pis & 1) * HPC + s_head) * (C::QBUF >> 4));
-                const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)vro.slot * (kSlot8 >> 4));
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    umma_f8(tS + sb * 2 * RP, kd + (uint64_t)(k * 2), qd + (uint64_t)(k * 2 * (C::QLBO >> 4)), idesc_qk, k == 0 ? 0u : 1u);
+                umma_commit(&bars[E_SFULL + sb]);
+                umma_commit(&bars[E_KEMPTY + krs.slot]);
+                krs.advance(kKRing8);
+                if (s_first) {
+                    // The other image buffer was last read by the products of the piece before; the last of them
+                    // (step gs - 1) must have completed before the next piece's images are copied into it.
+                    if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
+                    next_left = ok ? issuer_next_piece(p, s_prefix, s_len, walk, HPC, next_image, flags) : 0;
+                    if (next_left > 0) {
+                        q_piece = pis + 1;
+                        want_q = true;   // copied at the top of the next step
+                    }
+                    s_first = false;
+                }
+                if (++s_head == HPC) s_head = 0;
+                if (--s_left == 0) {
+                    s_left = next_left;
+                    s_first = true;
+                    ++pis;
+                }
+            }
+        }
+    } else if (wid == kOIssuerWarp) {
+        // ===================== O^T += V^T [P_hi ; P_mid ; P_lo]^T issuer (one lane) =====================
+        if (lane == 0 && U > 0) {
+            constexpr uint32_t idesc_pv = instr_desc_e4m3(UD, 3 * RP, 1, 1);
+            const uint64_t vdesc0 = smem_desc(smem_u32(vslots), kTile8, 1024, 2);
+            const uint64_t pdesc0 = smem_desc(smem_u32(pbuf), 128, 2048, 0);
+            bool ok = true;
+            EWalk walk(p, s_prefix, lo, hi);
+            int image_unused = 0;
+            int o_left = issuer_next_piece(p, s_prefix, s_len, walk, HPC, image_unused, flags);
+            uint32_t pio = 0, o_done = 0;   // o_done: steps of the piece done (the first HPC start an accumulator each)
+            Ring vro;
+            for (uint32_t g = 0; g < U && ok; ++g) {
+                const uint32_t pb = g & 1, ob = pio & 1, o_head = o_done % HPC;
+                if (o_done == 0 && pio >= 2)   // the epilogue of the piece that used these O^T buffers before has read them
+                    ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_VFULL + vro.slot], vro.parity, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)vro.slot * (kTile8 >> 4));
                 const uint64_t pd = pdesc0 + (uint64_t)(pb * (C::PBUF >> 4));
                 const uint32_t tOb = tO + (ob * HPC + o_head) * 3 * RP;
                 const bool o_start = o_done < (uint32_t)HPC;   // this head's first product of the piece
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (do_s)
-                        umma_f8(tS + sb * 2 * RP, kd + (uint64_t)(k * 2), qd + (uint64_t)(k * 2 * (C::QLBO >> 4)), idesc_qk,
-                                k == 0 ? 0u : 1u);
-                    if (do_pv)
-                        umma_f8(tOb, vd + (uint64_t)(k * (4096 >> 4)), pd + (uint64_t)(k * (512 >> 4)), idesc_pv,
-                                (o_start && k == 0) ? 0u : 1u);
-                }
-                if (do_s) {
-                    umma_commit(&bars[E_SFULL + sb]);
-                    krs.advance(ring);
-                    if (s_first) {
-                        // The other image buffer was last read by the S^T products of the piece before; the last of
-                        // them (step gs - 1) must have completed before the next piece's images are copied into it.
-                        if (gs > 0) ok = wait_or_abort(&bars[E_SFULL + (sb ^ 1)], ((gs - 1) >> 1) & 1, abort_flag);
-                        next_left = 0;
-                        if (ok && walk_s.next(p, s_prefix, s_len, pc, flags)) {
-                            next_left = (pc.t1 - pc.t0) * HPC;
-                            next_image = pc.b * p.Hkv + pc.hg * HPC;
-                            q_piece = pis + 1;
-                            want_q = true;   // copied at the top of the next step
-                        }
-                        s_first = false;
-                    }
-                    ++gs;
-                    if (++s_head == HPC) s_head = 0;
-                    if (--s_left == 0) {
-                        s_left = next_left;
-                        s_first = true;
-                        ++pis;
-                    }
-                }
-                if (do_pv) {
-                    umma_commit(&bars[E_PFREE + pb]);
-                    umma_commit(&bars[E_EMPTY + vro.slot]);
-                    vro.advance(ring);
-                    ++o_done;
-                    if (--o_left == 0) {
-                        umma_commit(&bars[E_OFULL + ob]);
-                        if (g + 1 < U) {
-                            walk_o.next(p, s_prefix, s_len, pc, flags);
-                            o_left = (pc.t1 - pc.t0) * HPC;
-                            o_done = 0;
-                            ++pio;
-                        }
+                for (int k = 0; k < 4; ++k)
+                    umma_f8(tOb, vd + (uint64_t)(k * (4096 >> 4)), pd + (uint64_t)(k * (512 >> 4)), idesc_pv, (o_start && k == 0) ? 0u : 1u);
+                umma_commit(&bars[E_PFREE + pb]);
+                umma_commit(&bars[E_VEMPTY + vro.slot]);
+                vro.advance(vring);
+                ++o_done;
+                if (--o_left == 0) {
+                    umma_commit(&bars[E_OFULL + ob]);
+                    if (g + 1 < U) {
+                        o_left = issuer_next_piece(p, s_prefix, s_len, walk, HPC, image_unused, flags);
+                        o_done = 0;
+                        ++pio;
                     }
                 }
             }
@@ -665,8 +709,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         float ep_vscale = 1.f;
 
         uint32_t g = (uint32_t)hh, pi = 0;   // this team's next step (all heads counted), pieces done
-        Ring vr;                             // slot of step g (only boundary tiles look at it)
-        for (int i = 0; i < hh; ++i) vr.advance(ring);
+        Ring vr;                             // V slot of step g (only boundary tiles look at it)
+        for (int i = 0; i < hh; ++i) vr.advance(vring);
         EWalk walk(p, s_prefix, lo, hi);
         EPiece pc;
         EWin win;
@@ -792,13 +836,12 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     }
                 }
                 if (masked && nvalid < UK)
-                    failed = e_zero_v_rows(slots + (size_t)vr.slot * kSlot8 + kTile8, nvalid, &bars[E_FULL + vr.slot], vr.parity, cx,
-                                           failed);
+                    failed = e_zero_v_rows(vslots + (size_t)vr.slot * kTile8, nvalid, &bars[E_VFULL + vr.slot], vr.parity, cx, failed);
                 fence_proxy_async_smem();   // by every thread that wrote, then one arrival per warp
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[E_PFULL + pb]);
 #pragma unroll
-                for (int i = 0; i < HPC; ++i) vr.advance(ring);
+                for (int i = 0; i < HPC; ++i) vr.advance(vring);
                 if (kind == 1) win.advance(p, pb_, pn, flags);
                 if (t == t0 && ep_pending) {
                     // put off so that the pipeline restarts first: the partial of the piece before
@@ -839,24 +882,28 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     // ---- common exit: nothing of this block may still be in flight when tensor memory is freed ----
     __syncthreads();
     const bool gave_up = *abort_flag != 0;
-    if (wid == kIssuerWarp && lane == 0) {
-        umma_commit(&bars[E_DRAIN]);   // arrives once every product issued by this thread has completed
-        mbar_wait_bounded(&bars[E_DRAIN], 0, kUmmaWaitNs);
+    if ((wid == kSIssuerWarp || wid == kOIssuerWarp) && lane == 0) {
+        uint64_t* drain = &bars[wid == kSIssuerWarp ? E_DRAIN : E_DRAIN + 1];
+        umma_commit(drain);   // arrives once every product issued by this thread has completed
+        mbar_wait_bounded(drain, 0, kUmmaWaitNs);
+    }
+    if (wid == kSIssuerWarp && lane == 0) {
         // query images that were asked for and never waited for get a bounded chance to land
         for (int i = 0; i < 2; ++i)
             if (q_pending[i]) mbar_wait_bounded(&bars[E_QFULL + i], q_parity[i], kUmmaWaitNs);
     }
-    if (wid == kProducerWarp && lane == 0 && gave_up) {
+    if ((wid == kKProducerWarp || wid == kVProducerWarp) && lane == 0 && gave_up) {
         // give every copy that was issued a bounded chance to land
-        const uint32_t issued = (uint32_t)s_ctl[2];
-        for (uint32_t m = issued > (uint32_t)ring ? issued - (uint32_t)ring : 0; m < issued; ++m)
-            mbar_wait_bounded(&bars[E_FULL + (int)(m % (uint32_t)ring)], (m / (uint32_t)ring) & 1, kUmmaWaitNs);
+        const bool is_v = wid == kVProducerWarp;
+        const uint32_t ring = (uint32_t)(is_v ? vring : kKRing8), issued = (uint32_t)s_ctl[is_v ? 3 : 2];
+        for (uint32_t m = issued > ring ? issued - ring : 0; m < issued; ++m)
+            mbar_wait_bounded(&bars[(is_v ? E_VFULL : E_KFULL) + (int)(m % ring)], (m / ring) & 1, kUmmaWaitNs);
     }
     if (gave_up) flags |= kDevWaitTimeout;
     if (flags) atomicOr(p.status, flags);
     tc_fence_before_sync();
     __syncthreads();
-    if (wid == kIssuerWarp) {
+    if (wid == kSIssuerWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
@@ -881,7 +928,9 @@ cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, si
 
 int main_umma_e4m3_rows(int R) { return R <= 16 ? 16 : 32; }
 
-int main_umma_e4m3_max_slots() { return kMaxRing8; }
+int main_umma_e4m3_max_slots() { return kKRing8 + kMaxVRing8; }
+
+int main_umma_e4m3_min_slots() { return kKRing8 + 3; }
 
 size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch) {
     return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::smem_bytes(nslot, hpc, max_batch) : ECfg<32>::smem_bytes(nslot, hpc, max_batch);
