@@ -60,17 +60,21 @@ typedef enum {
                           fp32 scale per KV head for K and one for V: value = code value * scale.  The attention is the
                           same definition on those dequantised values (the paper's efficiency runs use FP8 attention,
                           Sec. 3.2).  Needs dtype = PLT_BF16 and d = 128; q and out stay bf16; softmax and
-                          accumulation stay fp32.  Served by the warp-level kernel;
+                          accumulation stay fp32.  Served by the warp-level kernel (codes converted to f16
+                          in registers) or, up to 32 packed rows, by a tcgen05 kernel whose products take the
+                          codes as they are (queries and probabilities split into sums of E4M3 terms);
                           plt_decode_attn_step quantises the rows it appends. */
 } plt_kv_dtype;
 
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
 typedef enum {
     PLT_PATH_AUTO = 0,      /* the library chooses: tcgen05 above 48 packed rows (L * Hq / Hkv) when max_seq_len >= 16384
-                               and it applies, else the warp-level kernel */
+                               (bf16 caches), or at 25 to 32 packed rows on unpaged E4M3 caches when max_seq_len >=
+                               32768, and it applies; else the warp-level kernel */
     PLT_PATH_WARP_MMA = 1,  /* warp-level tensor-core products (mma.sync); fp32 inputs always use SIMT fp32 */
-    PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16, d = 128, pages that divide
-                               or are a multiple of 128 tokens; anything else is refused with PLT_ERR_UNSUPPORTED */
+    PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16 queries, d = 128, pages that divide
+                               or are a multiple of 128 tokens, q_len <= 1, with E4M3 caches at most 32 packed rows;
+                               anything else is refused with PLT_ERR_UNSUPPORTED */
 } plt_kernel_path;
 
 /* Bits of the device status word reported by plt_decode_attn_check. */
@@ -102,8 +106,12 @@ typedef struct {
     int32_t stages;        /* depth of the shared-memory pipeline (bf16 path) */
     int32_t ctas_per_sm;   /* persistent thread blocks per SM */
     int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (4 or 6) and
-                              heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block) */
-    int32_t loads_in_flight; /* PLT_PATH_TCGEN05: K tiles (and likewise V tiles) kept in flight at most, clamped to stages / 2; 0 = automatic */
+                              heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block).
+                              With E4M3 caches on that path: `stages` counts 16 KB slots (7 to 10: 4 for K tiles, the
+                              rest for V tiles) and heads_per_cta is 1 or 2 (KV heads of one work item, whose tiles of
+                              the same keys take turns; 2 needs an even Hkv and is the default then) */
+    int32_t loads_in_flight; /* PLT_PATH_TCGEN05: K tiles (and likewise V tiles) kept in flight at most, clamped to the
+                              ring of each; 0 = automatic */
     int32_t slices_per_warp; /* PLT_PATH_WARP_MMA: 16-key slices each of those warps takes per tile (1 or 2); a tile holds
                               16 * key_slices * slices_per_warp keys */
     int32_t row_warps;     /* PLT_PATH_WARP_MMA: warps that split the L * Hq/Hkv packed rows of a KV head (1 or 2; each

@@ -257,19 +257,25 @@ bool umma_eligible(const plt_decode_attn_config* c) {
     return true;
 }
 
-// Automatic choice: the warp-level kernel, except above 48 packed rows on long-context configurations, where the
-// tcgen05 kernel measured 8 % faster (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches
-// of short sequences at any row count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one.
+// Automatic choice: the warp-level kernel, except
+//  - bf16 caches above 48 packed rows on long-context configurations, where the tcgen05 kernel measured 8 % faster
+//    (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches of short sequences at any row
+//    count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one;
+//  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 32768 keys: the tcgen05 kernel for E4M3
+//    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays about 45 us more per
+//    launch for its pieces' starts and ends (measured at 32 rows: 259 vs 292 us at B = 16, N = 32768; 244 vs 279 us
+//    at B = 4, N = 131072; 176 vs 169 us at B = 16, N = 16384; at 24 rows 242 vs 226 us at N = 32768).
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
     if (c->kernel_path == PLT_PATH_WARP_MMA || c->q_len > 1) return false;
     if (c->kernel_path == PLT_PATH_TCGEN05) return true;
-    if (c->kv_dtype == PLT_KV_E4M3) return false;
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
-    return umma_eligible(c) && c->L * (c->Hq / c->Hkv) > 48 && c->max_seq_len >= 16384 &&
-           (c->stages == 0 || c->stages == 4 || c->stages == 6);
+    const int rows = c->L * (c->Hq / c->Hkv);
+    if (c->kv_dtype == PLT_KV_E4M3)
+        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size == 0 && c->max_seq_len >= 32768 && c->stages == 0;
+    return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
 // Chooses the kernel path and variant, prepares the kernels (shared-memory attribute, occupancy) and fills
