@@ -325,19 +325,22 @@ template <int RP>
 __device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
                                         float vscale, bool failed) {
     failed = sm_wait(&cx.bars[E_OFULL + ob], parity, cx.abort_flag, failed);
+    float* dst = p.part_acc + prow * UD + cx.ltid;
+    // Eight rows at a time in a loop that is not unrolled: this code is cold every time it runs (the per-step loops of
+    // six roles evict it) and a cold instruction line costs hundreds of cycles to fetch, so it is kept to a few lines.
 #pragma unroll 1
-    for (int c = 0; c < RP / 16; ++c) {
+    for (int c = 0; c < RP / 8; ++c) {
         if (!failed) {
-            uint32_t o0[16], o1[16], o2[16];
+            uint32_t o0[8], o1[8], o2[8];
             tc_fence_after_sync();
-            tmem_ld16(tOb + cx.lane_off + c * 16, o0);
-            tmem_ld16(tOb + cx.lane_off + RP + c * 16, o1);
-            tmem_ld16(tOb + cx.lane_off + 2 * RP + c * 16, o2);
+            tmem_ld8(tOb + cx.lane_off + c * 8, o0);
+            tmem_ld8(tOb + cx.lane_off + RP + c * 8, o1);
+            tmem_ld8(tOb + cx.lane_off + 2 * RP + c * 8, o2);
             tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (c * 16 + j < p.R)
-                    p.part_acc[(prow + c * 16 + j) * UD + cx.ltid] =
+            for (int j = 0; j < 8; ++j)
+                if (c * 8 + j < p.R)
+                    dst[(c * 8 + j) * UD] =
                         (__uint_as_float(o0[j]) + (__uint_as_float(o1[j]) * kMidInv + __uint_as_float(o2[j]) * kLoInv)) * vscale;
         }
     }
