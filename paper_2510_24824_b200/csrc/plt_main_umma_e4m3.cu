@@ -82,6 +82,8 @@ template <int RP>
 __global__ void __launch_bounds__(RP * 8) plt_decode_pack_q_e4m3(const Params p, uint8_t* qimg, float* qinv) {
     using C = ECfg<RP>;
     __shared__ float wmax[RP * 8 / 32];
+    grid_launch_dependents();   // the main kernel sets up and starts its cache loads meanwhile; it waits for this grid
+                                // to complete before it touches a query image
     const int b = blockIdx.x / p.Hkv, hg = blockIdx.x - b * p.Hkv;
     const int r = threadIdx.x >> 3, c = threadIdx.x & 7;
     float x[16];
@@ -588,6 +590,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             const uint64_t kdesc0 = smem_desc(smem_u32(kslots), 16, 1024, 2);
             const uint64_t qdesc0 = smem_desc(smem_u32(qbuf), C::QLBO, 128, 0);
             bool ok = true;
+            grid_dependency_wait();   // the query images are complete (the pack kernel ran just before this one)
             EWalk walk(p, s_prefix, lo, hi);
             // steps left in the piece, and the piece after it (0 steps: none) with the index of its first image
             int next_image = 0, next_left = 0;
@@ -718,6 +721,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         EPiece pc;
         EWin win;
         bool have = walk.next(p, s_prefix, s_len, pc, flags);
+        grid_dependency_wait();   // the scale factors of the query images are complete
         while (have && !aborted) {
             const uint32_t tOb = tO + ((pi & 1) * HPC + hh) * 3 * RP;   // O^T of this head in this piece
             const int kind = pc.kind, t0 = pc.t0, t1 = pc.t1, cmax = pc.cmax, pn = pc.n, pb_ = pc.b, head = pc.hg * HPC + hh;
@@ -923,8 +927,21 @@ cudaError_t e4m3_prepare(size_t smem, int* blocks_per_sm) {
 template <int RP, int HPC>
 cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, const UmmaGeom& geo,
                         const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
-    plt_decode_main_umma_e4m3<RP, HPC><<<grid, threads8(HPC), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
-    return cudaGetLastError();
+    // Programmatic stream serialisation: the blocks set up and the producers start streaming the caches (which the
+    // kernel before, the query pack kernel, does not touch) while that kernel still runs; whoever reads what it wrote
+    // waits for it first. The partials this kernel writes were last read by the merge kernel of the step before,
+    // which had completed before the pack kernel started.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads8(HPC));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, plt_decode_main_umma_e4m3<RP, HPC>, maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
 }
 
 }  // namespace
