@@ -197,3 +197,25 @@ def test_batch_smaller_than_capacity_and_reuse():
             got = op.run(dp).float().cpu().numpy().astype(np.float64)
             assert_parity(got, oracle.decode_attn(prob), "bf16", f"B={prob.B}")
         assert op.check() == 0
+
+
+def test_allocation_free_entry_point_with_this_kernel():
+    """plt_decode_attn_run_no_alloc places the query images and their scale factors in the built-in scratch array too."""
+    torch.cuda.set_device(0)
+    p = make_problem(custom(B=3, L=3, Hq=24, Hkv=4, w=50, lens=("list", [1700, 65, 3])))
+    dp = DeviceProblem(p, "cuda:0")
+    stream = torch.cuda.current_stream().cuda_stream
+    with DecodeAttn(p, **T5) as op:
+        want = op.run(dp).clone()
+        assert op.check() == 0
+    cfg = B.make_config(p.dtype, p.B, p.L, p.Hq, p.Hkv, p.d, p.max_seq_len, p.w, page_size=p.page_size, sm_scale=p.sm_scale,
+                        device=0, kv_dtype=p.kv_dtype, **T5)
+    assert B.plt_decode_attn_workspace_bytes(cfg) <= B.PLT_NO_ALLOC_SCRATCH_BYTES
+    out = torch.empty_like(dp.out)
+    for call in range(2):
+        out.fill_(float("nan"))
+        B.plt_decode_attn_run_no_alloc(cfg, dp.args(out), stream)
+        torch.cuda.synchronize()
+        assert B.plt_decode_attn_check(None, stream) == 0
+        assert torch.equal(out, want), f"call {call}: differs from the handle path"
+    assert_parity(out.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "no-alloc")
