@@ -264,7 +264,8 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 32768 keys: the tcgen05 kernel for E4M3
 //    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays about 45 us more per
 //    launch for its pieces' starts and ends (measured at 32 rows: 259 vs 292 us at B = 16, N = 32768; 244 vs 279 us
-//    at B = 4, N = 131072; 176 vs 169 us at B = 16, N = 16384; at 24 rows 242 vs 226 us at N = 32768).
+//    at B = 4, N = 131072; 176 vs 169 us at B = 16, N = 16384; at 24 rows 242 vs 226 us at N = 32768; with pages of
+//    128 or 256 tokens 359 vs 293 us: the producers fetch a page id per tile).
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
