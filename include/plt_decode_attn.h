@@ -107,7 +107,7 @@ typedef struct {
     int32_t ctas_per_sm;   /* persistent thread blocks per SM */
     int32_t kernel_path;   /* plt_kernel_path. On PLT_PATH_TCGEN05, `stages` counts 32 KB ring slots (4 or 6) and
                               heads_per_cta, key_slices and ctas_per_sm are ignored (1 head, 128-key tiles, 1 block).
-                              With E4M3 caches on that path: `stages` counts 16 KB slots (7 to 10: 4 for K tiles, the
+                              With E4M3 caches on that path: `stages` counts 16 KB slots (7 or 8: 4 for K tiles, the
                               rest for V tiles) and heads_per_cta is 1 or 2 (KV heads of one work item, whose tiles of
                               the same keys take turns; 2 needs an even Hkv and is the default then) */
     int32_t loads_in_flight; /* PLT_PATH_TCGEN05: K tiles (and likewise V tiles) kept in flight at most, clamped to the

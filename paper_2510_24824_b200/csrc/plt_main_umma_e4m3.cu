@@ -44,7 +44,7 @@ constexpr int kTile8 = UK * UD;        // one K (or V) tile of one KV head: 128 
 // the probabilities), a V tile only after the product that ends its step, so that one ring of K + V slots would
 // keep most of its slots waiting for that product and leave two loads in flight (measured: 4.7 TB/s at best).
 constexpr int kKRing8 = 4;             // K slots
-constexpr int kMaxVRing8 = 6;          // V slots at most
+constexpr int kMaxVRing8 = 4;          // V slots at most
 // Threads of a block: one team of 128 softmax threads per KV head of the item, two producer warps, two issuer warps.
 __host__ __device__ constexpr int threads8(int hpc) { return hpc * 128 + 128; }
 // A probability may exceed the lazily updated reference by 3 powers of two at most (p <= 8), which fixes the powers of
@@ -57,8 +57,12 @@ constexpr float kMidInv = 1.f / 1024.f, kLoInv = 1.f / 16384.f;
 
 // mbarrier indices
 constexpr int E_KFULL = 0, E_KEMPTY = 4, E_VFULL = 8, E_VEMPTY = 14, E_SFULL = 20 /* two */, E_SFREE = 22 /* two */,
-              E_PFULL = 24 /* two */, E_PFREE = 26 /* two */, E_OFULL = 28 /* two */, E_OFREE = 30 /* two */,
-              E_QFULL = 32 /* two */, E_DRAIN = 34 /* two */, E_COUNT = 36;
+              E_PFULL = 24 /* four */, E_PFREE = 28 /* four */, E_OFULL = 32 /* two */, E_OFREE = 34 /* two */,
+              E_QFULL = 36 /* two */, E_DRAIN = 38 /* two */, E_COUNT = 40;
+// Probability buffers: four, used in turn by the steps, so that a team (every other step with two heads) writes the
+// probabilities of a step without waiting for the O^T product of its step before, which is still queued behind the
+// S^T products of later steps on the tensor pipe (measured: 480 of a team's 3400 cycles per step).
+constexpr int kPBufs = 4;
 
 template <int RP>
 struct ECfg {
@@ -70,7 +74,7 @@ struct ECfg {
     static constexpr int TMEM_COLS = RP == 16 ? 256 : 512;
     // hpc: KV heads per work item (their tiles take turns; each has its own query image, reference maxima and O^T)
     __host__ __device__ static constexpr size_t smem_bytes(int nslot, int hpc, int max_batch) {
-        return 1024 + (size_t)nslot * kTile8 + 2 * PBUF + (size_t)2 * hpc * QBUF + E_COUNT * 8 +
+        return 1024 + (size_t)nslot * kTile8 + kPBufs * PBUF + (size_t)2 * hpc * QBUF + E_COUNT * 8 +
                (size_t)RP * 4 * (12 * hpc + 1) + 64 + (size_t)(2 * max_batch + 4) * 4;
     }
 };
@@ -459,8 +463,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     const int vring = geo.ring - kKRing8;                   // V slots (geo.ring counts all slots)
     uint8_t* kslots = smem;                                 // ring of K tiles, then ring of V tiles
     uint8_t* vslots = smem + (size_t)kKRing8 * kTile8;
-    uint8_t* pbuf = smem + (size_t)geo.ring * kTile8;       // two buffers of PBUF (step parity)
-    uint8_t* qbuf = pbuf + 2 * C::PBUF;                     // two buffers (piece parity) of HPC query images
+    uint8_t* pbuf = smem + (size_t)geo.ring * kTile8;       // kPBufs buffers of PBUF (step modulo kPBufs)
+    uint8_t* qbuf = pbuf + kPBufs * C::PBUF;                // two buffers (piece parity) of HPC query images
     uint64_t* bars = (uint64_t*)(qbuf + 2 * HPC * C::QBUF);
     // per team (= head of the item), kTeamFloats each: negm, mref, alpha [RP]; red [4][RP]; lim [RP]; mfin, lfin [2][RP]
     constexpr int kTeamFloats = 12 * RP;
@@ -492,11 +496,13 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars[E_SFULL + i], 1);
             mbar_init(&bars[E_SFREE + i], 4);
-            mbar_init(&bars[E_PFULL + i], 4);
-            mbar_init(&bars[E_PFREE + i], 1);
             mbar_init(&bars[E_OFULL + i], 1);
             mbar_init(&bars[E_OFREE + i], 4 * HPC);
             mbar_init(&bars[E_QFULL + i], 1);
+        }
+        for (int i = 0; i < kPBufs; ++i) {
+            mbar_init(&bars[E_PFULL + i], 4);
+            mbar_init(&bars[E_PFREE + i], 1);
         }
         mbar_init(&bars[E_DRAIN], 1);
         mbar_init(&bars[E_DRAIN + 1], 1);
@@ -658,11 +664,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             uint32_t pio = 0, o_done = 0;   // o_done: steps of the piece done (the first HPC start an accumulator each)
             Ring vro;
             for (uint32_t g = 0; g < U && ok; ++g) {
-                const uint32_t pb = g & 1, ob = pio & 1, o_head = o_done % HPC;
+                const uint32_t pb = g % kPBufs, ob = pio & 1, o_head = o_done % HPC;
                 if (o_done == 0 && pio >= 2)   // the epilogue of the piece that used these O^T buffers before has read them
                     ok = wait_or_abort(&bars[E_OFREE + ob], ((pio >> 1) & 1) ^ 1u, abort_flag);
                 if (ok) ok = wait_or_abort(&bars[E_VFULL + vro.slot], vro.parity, abort_flag);
-                if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g >> 1) & 1, abort_flag);
+                if (ok) ok = wait_or_abort(&bars[E_PFULL + pb], (g / kPBufs) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)vro.slot * (kTile8 >> 4));
@@ -802,13 +808,13 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                         s_c[r] = s[r];
                         ls_c[r] = lsum[r];
                     }
-                    failed = e_slow_path<RP>(s_c, ls_c, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) & 1)], ((g - HPC) >> 1) & 1, failed);
+                    failed = e_slow_path<RP>(s_c, ls_c, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
 #pragma unroll
                     for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
-                const uint32_t pb = g & 1;
-                if (g >= 2) failed = sm_wait(&bars[E_PFREE + pb], ((g >> 1) & 1) ^ 1u, abort_flag, failed);
+                const uint32_t pb = g % kPBufs;   // last used by step g - kPBufs
+                if (g >= (uint32_t)kPBufs) failed = sm_wait(&bars[E_PFREE + pb], ((g / kPBufs) & 1) ^ 1u, abort_flag, failed);
                 uint8_t* pdst = pbuf + pb * C::PBUF + ltid * 16;   // [3 RP / 16 chunks][key][16 codes]
 #pragma unroll
                 for (int j = 0; j < RP / 16; ++j) {

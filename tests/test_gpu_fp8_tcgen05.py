@@ -96,7 +96,7 @@ def test_odd_number_of_kv_heads_takes_one_head_per_item():
     assert_parity(run_gpu(p, **T5), oracle.decode_attn(p), "bf16", "Hkv=3")
 
 
-@pytest.mark.parametrize("stages,inflight", [(7, 1), (8, 2), (10, 6)])
+@pytest.mark.parametrize("stages,inflight", [(7, 1), (8, 2), (8, 4)])
 def test_ring_depths(stages, inflight):
     p = make_problem(custom(B=3, L=3, Hq=24, Hkv=4, w=50, lens=("list", [1700, 65, 3])))
     got = run_gpu(p, stages=stages, loads_in_flight=inflight, **T5)
