@@ -261,11 +261,12 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //  - bf16 caches above 48 packed rows on long-context configurations, where the tcgen05 kernel measured 8 % faster
 //    (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches of short sequences at any row
 //    count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one;
-//  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 32768 keys: the tcgen05 kernel for E4M3
-//    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays about 45 us more per
-//    launch for its pieces' starts and ends (measured at 32 rows: 259 vs 292 us at B = 16, N = 32768; 244 vs 279 us
-//    at B = 4, N = 131072; 176 vs 169 us at B = 16, N = 16384; at 24 rows 242 vs 226 us at N = 32768; with pages of
-//    128 or 256 tokens 359 vs 293 us: the producers fetch a page id per tile).
+//  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 16384 keys: the tcgen05 kernel for E4M3
+//    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays more per launch
+//    for its pieces' starts and ends (measured at 32 rows: 237 vs 292 us at B = 16, N = 32768; 216 vs 279 us at
+//    B = 4, N = 131072; 157 vs 169 us at B = 16, N = 16384; 331 vs 347 us at B = 64, N = 8192; but 131 vs 107 us at
+//    B = 16, N = 8192; at 24 rows 242 vs 226 us at N = 32768 before the plan's lead-in; with pages of 128 or 256 tokens
+//    359 vs 293 us: the producers fetch a page id per tile).
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
@@ -275,7 +276,7 @@ bool want_umma(const plt_decode_attn_config* c) {
         return false;
     const int rows = c->L * (c->Hq / c->Hkv);
     if (c->kv_dtype == PLT_KV_E4M3)
-        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size == 0 && c->max_seq_len >= 32768 && c->stages == 0;
+        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size == 0 && c->max_seq_len >= 16384 && c->stages == 0;
     return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
@@ -318,6 +319,14 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
         h->umma = true;
         h->umma_e4m3 = true;
+        // Starting and finishing a piece costs this kernel as long as 4-5 tiles take it (7.6 us measured: plan step,
+        // limits, first-tile maxima, end-of-piece reduction, epilogue), and the tiles of a windows item (all masked, a
+        // limits update per window) cost more than shared-cache tiles. The plan charges every item a lead-in, so that
+        // blocks with more item starts get fewer tiles; with equal tile counts the blocks of workload 4 finished
+        // between 176 and 244 us. Measured per-step times for a lead-in of 0 / 8 / 14 / 20 tiles: 260.8 / 241.3 / 237 /
+        // 240 us at B = 16, N = 32768; 174.5 / 160.4 / 156.6 / 159.5 us at N = 16384; 244.3 / 230.7 / 216.0 / 219.0 us at
+        // B = 4, N = 131072; 337.4 / 332.6 / 331.3 / 337.7 us at B = 64, N = 8192.
+        h->piece_cost = 14;
         h->var = MainVariant{config->d, 0, 0, hpc, 4, 1, 128, nslot, 0, smem, true};
         h->ctas_per_sm = 1;
         h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)

@@ -442,6 +442,16 @@ __device__ __noinline__ void prod_issue_special(const Params& p, const UmmaGeom&
     }
 }
 
+// Steps a block takes: one per tile and head of every piece in its range of the line (the positions of the range that
+// are lead-ins of items are not tiles).
+__device__ __noinline__ int count_steps(const Params& p, const int32_t* sp, const int32_t* lens, int lo, int hi, int hpc, uint32_t& flags) {
+    EWalk walk(p, sp, lo, hi);
+    EPiece pc;
+    int steps = 0;
+    while (walk.next(p, sp, lens, pc, flags)) steps += (pc.t1 - pc.t0) * hpc;
+    return steps;
+}
+
 // Next piece of an issuer: its steps (0: none left) and the index of its first query image.
 __device__ __noinline__ int issuer_next_piece(const Params& p, const int32_t* sp, const int32_t* lens, EWalk& walk, int hpc, int& image,
                                               uint32_t& flags) {
@@ -470,7 +480,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     constexpr int kTeamFloats = 12 * RP;
     float* s_team = (float*)(bars + E_COUNT);
     int32_t* s_rowloop = (int32_t*)(s_team + HPC * kTeamFloats);
-    int32_t* s_ctl = s_rowloop + RP;                        // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued
+    int32_t* s_ctl = s_rowloop + RP;                        // [0] abort flag, [1] tensor-memory base, [2] K / [3] V tiles issued, [4] steps
     int32_t* s_prefix = s_ctl + 16;                         // [B + 1] tile prefix
     int32_t* s_len = s_prefix + p.B + 1;                    // [B] clamped sequence lengths
     volatile int* abort_flag = (volatile int*)&s_ctl[0];
@@ -512,6 +522,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     if (wid == kSIssuerWarp) tmem_alloc((uint32_t*)&s_ctl[1], C::TMEM_COLS);
     grid_launch_dependents();  // the merge kernel may be set up meanwhile; it waits for this grid to complete
     build_prefix(p, s_prefix, flags, s_len, /*small=*/true);  // contains __syncthreads
+    if (tid == 0) {
+        const int64_t t64 = s_prefix[p.B];
+        const int c = blockIdx.x, nc = plan_ctas(t64, (int)gridDim.x);
+        s_ctl[4] = c < nc ? count_steps(p, s_prefix, s_len, (int)cta_begin(t64, c, nc), (int)cta_begin(t64, c + 1, nc), HPC, flags) : 0;
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -525,11 +540,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
         for (int b = tid; b <= p.B; b += threads8(HPC)) p.prefix[b] = s_prefix[b];
     const bool in_plan = cta < nctas;
     const int lo = in_plan ? (int)cta_begin(T64, cta, nctas) : 0, hi = in_plan ? (int)cta_begin(T64, cta + 1, nctas) : 0;
-    // Steps this block takes: one per (tile, head of the item). piece_cost is 0 on this path, so every position of
-    // the block's range of the line is a tile. The heads of a tile follow one another: a key's codes of all heads lie
-    // side by side in memory, and fetched within a short time of each other they come at 6.4 TB/s where one head's 128
-    // bytes per key alone come at 4.5 (measured on B200, 8 heads of 128 codes per key).
-    const uint32_t U = (uint32_t)(hi - lo) * HPC;
+    // Steps this block takes: one per (tile, head of the item) of the pieces in its range of the line. The heads of a
+    // tile follow one another: a key's codes of all heads lie side by side in memory, and fetched within a short time
+    // of each other they come at 6.4 TB/s where one head's 128 bytes per key alone come at 4.5 (measured on B200, 8
+    // heads of 128 codes per key).
+    const uint32_t U = (uint32_t)s_ctl[4];
     bool q_pending[2] = {false, false};       // issuer only: query images were asked for and not yet waited for
     uint32_t q_parity[2] = {0u, 0u};          // and the phase of their barrier that ends when they have landed
 
