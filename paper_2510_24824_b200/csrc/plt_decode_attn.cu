@@ -264,8 +264,8 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 16384 keys: the tcgen05 kernel for E4M3
 //    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays more per launch
 //    for its pieces' starts and ends (measured at 32 rows: 237 vs 292 us at B = 16, N = 32768; 216 vs 279 us at
-//    B = 4, N = 131072; 157 vs 169 us at B = 16, N = 16384; 331 vs 347 us at B = 64, N = 8192; but 131 vs 107 us at
-//    B = 16, N = 8192; at 24 rows 242 vs 226 us at N = 32768 before the plan's lead-in; with pages of 128 or 256 tokens
+//    B = 4, N = 131072; 157 vs 169 us at B = 16, N = 16384; 331 vs 347 us at B = 64, N = 8192; but 113 vs 107 us at
+//    B = 16, N = 8192; at 24 rows 224 vs 226 us at N = 32768 and 142 vs 129 us at N = 16384; with pages of 128 or 256 tokens
 //    359 vs 293 us: the producers fetch a page id per tile).
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
