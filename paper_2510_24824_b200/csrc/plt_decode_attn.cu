@@ -261,12 +261,14 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //  - bf16 caches above 48 packed rows on long-context configurations, where the tcgen05 kernel measured 8 % faster
 //    (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches of short sequences at any row
 //    count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one;
-//  - E4M3 caches, unpaged, at 25 to 32 packed rows when sequences can reach 16384 keys: the tcgen05 kernel for E4M3
+//  - E4M3 caches, contiguous or in pages of a multiple of 128 tokens, at 25 to 32 packed rows when sequences can
+//    reach 16384 keys: the tcgen05 kernel for E4M3
 //    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays more per launch
 //    for its pieces' starts and ends (measured at 32 rows: 237 vs 292 us at B = 16, N = 32768; 216 vs 279 us at
 //    B = 4, N = 131072; 157 vs 169 us at B = 16, N = 16384; 331 vs 347 us at B = 64, N = 8192; but 113 vs 107 us at
-//    B = 16, N = 8192; at 24 rows 224 vs 226 us at N = 32768 and 142 vs 129 us at N = 16384; with pages of 128 or 256 tokens
-//    359 vs 293 us: the producers fetch a page id per tile).
+//    B = 16, N = 8192; at 24 rows 224 vs 226 us at N = 32768 and 142 vs 129 us at N = 16384; with pages of 128 or 256
+//    tokens 232-236 vs 293 us, the page id of a tile being fetched one tile ahead; with pages of 64 tokens, two loads
+//    per tile through the producers' out-of-line path, 424 vs 293 us).
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
@@ -276,7 +278,7 @@ bool want_umma(const plt_decode_attn_config* c) {
         return false;
     const int rows = c->L * (c->Hq / c->Hkv);
     if (c->kv_dtype == PLT_KV_E4M3)
-        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size == 0 && c->max_seq_len >= 16384 && c->stages == 0;
+        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size % 128 == 0 && c->max_seq_len >= 16384 && c->stages == 0;
     return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 

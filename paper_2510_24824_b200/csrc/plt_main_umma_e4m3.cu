@@ -3,7 +3,7 @@
 // memory), head dimension 128, up to 32 packed query rows.
 //
 // y_global and y_local of Algorithm 3 for all L loops, same tile plan and split-partial format as the other main
-// kernels: one persistent block per SM walks its share of the line of 128-key tiles, one KV head per work item.
+// kernels: one persistent block per SM walks its share of the line of 128-key tiles.
 // No code is converted on the way: both products take 8-bit operands, so the bf16 queries and the fp32
 // probabilities are each written as a SUM of E4M3 numbers and the terms are laid side by side along N:
 //
@@ -14,8 +14,9 @@
 // part stays above the E4M3 subnormal step, so the scores are those of the bf16 queries; a probability keeps 12
 // significant bits in three terms, the second and third scaled up by 2^10 and 2^14 so that probabilities far below
 // the E4M3 subnormal step (2^-9) still count: many keys of tiny weight next to one peak must not be dropped. The
-// softmax threads add the two score columns of a row, and the epilogue adds the three accumulator columns. One tcgen05.mma costs the same issue slot whatever N is, so the extra terms are
-// free on the tensor side: 8 instructions per 32 KB tile.
+// softmax threads add the two score columns of a row, and the epilogue adds the three accumulator columns. One
+// tcgen05.mma costs the same issue slot whatever N is, so the extra terms are free on the tensor side: 8
+// instructions per 32 KB step.
 //
 // A work item is one or two KV heads of a sequence, and its steps alternate between them tile by tile: the codes of
 // a key of all heads lie side by side in memory, and neighbouring heads fetched within a short time of each other
@@ -404,13 +405,14 @@ struct ProdState {
     __device__ ProdState(const Params& p, const int32_t* sp, int lo, int hi) : walk(p, sp, lo, hi), t(0) { pc.t0 = pc.t1 = 0; }
 };
 
-// Next piece of a producer. Returns the steps it has (tiles x heads); `plain`: shared-cache tiles of a contiguous cache.
+// Next piece of a producer. Returns the steps it has (tiles x heads); `plain`: shared-cache tiles that are one TMA box
+// each (a contiguous cache, or pages that hold whole 128-key tiles).
 __device__ __noinline__ int prod_next_piece(const Params& p, const int32_t* sp, const int32_t* lens, ProdState& st, int hpc, bool& plain,
                                             uint32_t& flags) {
     st.walk.next(p, sp, lens, st.pc, flags);
     st.t = st.pc.t0;
     if (st.pc.kind == 1) st.win.seek(p, st.pc.b, st.pc.n, st.t, flags);
-    plain = st.pc.kind == 0 && p.page_size == 0;
+    plain = st.pc.kind == 0 && (p.page_size == 0 || p.page_size % UK == 0);
     return (st.pc.t1 - st.pc.t0) * hpc;
 }
 
@@ -568,6 +570,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             Ring cur, old;   // slot of tile n, slot of tile n - cap
             ProdState st(p, s_prefix, lo, hi);
             int left = 0, hh = 0, key0 = 0, head0 = 0, outer = 0;   // of a plain piece: next tile's first key, first head, sequence
+            // ... and with pages: the tile's offset in its page, the page's index in the sequence's table, its id, and
+            // the id of the next tile's page, fetched one tile ahead so that the load is never waited for
+            const bool paged = p.page_size > 0;
+            int poff = 0, pidx = 0, page_cur = 0, page_next = 0;
+            const int32_t* table = p.page_table;
             uint32_t n = 0;
             for (; n < U && ok; ++n) {
                 if (left == 0) {
@@ -575,6 +582,12 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     key0 = st.t * UK;
                     head0 = st.pc.hg * HPC;
                     outer = st.pc.b;
+                    if (plain && paged) {
+                        pidx = key0 / p.page_size;
+                        poff = key0 - pidx * p.page_size;
+                        table = p.page_table + (int64_t)outer * p.max_pages;
+                        page_cur = table[pidx];
+                    }
                 }
                 if (n >= (uint32_t)cap) {
                     ok = wait_or_abort(&fullb[old.slot], old.parity, abort_flag);
@@ -585,8 +598,20 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 uint8_t* dst = slots + (size_t)cur.slot * kTile8;
                 uint64_t* full = &fullb[cur.slot];
                 if (plain) {
+                    int c1 = key0, c3 = outer;
+                    if (paged) {
+                        if (hh == 0 && left > HPC)   // the piece has a next tile: its page id, if it starts a new page
+                            page_next = poff + UK == p.page_size ? table[pidx + 1] : page_cur;
+                        int page = page_cur;
+                        if (page < 0 || page >= p.num_pool_pages) {
+                            flags |= kDevPageIdClamped;
+                            page = page < 0 ? 0 : p.num_pool_pages - 1;
+                        }
+                        c1 = poff;
+                        c3 = page;
+                    }
                     mbar_expect_tx(full, (uint32_t)(geo.kbox * 128));
-                    tma_load_4d(dst, map, full, 0, key0, head0 + hh, outer, pol);
+                    tma_load_4d(dst, map, full, 0, c1, head0 + hh, c3, pol);
                 } else {
                     prod_issue_special(p, geo, st, hh, HPC, dst, full, map, wmap, pol, flags);
                 }
@@ -596,6 +621,14 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     hh = 0;
                     key0 += UK;
                     ++st.t;
+                    if (paged) {
+                        poff += UK;
+                        if (poff == p.page_size) {
+                            poff = 0;
+                            ++pidx;
+                        }
+                        page_cur = page_next;
+                    }
                 }
             }
             s_ctl[is_v ? 3 : 2] = (int32_t)n;

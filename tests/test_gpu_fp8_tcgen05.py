@@ -32,15 +32,20 @@ def test_path_is_reported():
 
 
 def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
-    """25 to 32 packed rows, unpaged E4M3 caches that can reach 16384 keys: the library picks this kernel by itself."""
+    """25 to 32 packed rows, E4M3 caches (contiguous or in pages that hold whole tiles) that can reach 16384 keys: the
+    library picks this kernel by itself."""
     spec = custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768)
     p = make_problem(spec)
     with DecodeAttn(p) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05 and op.info["heads_per_cta"] == 2
     assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", "automatic")
+    paged = make_problem(dict(spec, page_size=256))
+    with DecodeAttn(paged) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
+    assert_parity(run_gpu(paged), oracle.decode_attn(paged), "bf16", "automatic, paged")
     for other in (custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768),     # 24 rows
                   custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=8192),      # shorter caches
-                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=128)):
+                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=64)):
         with DecodeAttn(make_problem(other)) as op:
             assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
 
