@@ -224,3 +224,73 @@ def test_allocation_free_entry_point_with_this_kernel():
         assert B.plt_decode_attn_check(None, stream) == 0
         assert torch.equal(out, want), f"call {call}: differs from the handle path"
     assert_parity(out.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "no-alloc")
+
+
+def test_explicit_window_lengths():
+    p = make_problem(custom(B=4, L=3, Hq=12, Hkv=2, w=40, lens=("list", [300, 77, 5, 50])))
+    wl = np.array([[40, 0], [1, 17], [3, 0], [16, 33]], dtype=np.int32)
+    q = p.with_(win_lens=wl)
+    assert_parity(run_gpu(q, **T5), oracle.decode_attn(q), "bf16", "win_lens")
+
+
+def test_out_of_range_device_values_are_clamped_and_flagged():
+    p = make_problem(custom(B=3, lens=("list", [300, 77, 1]), max_seq_len=320))
+    bad = p.with_(seq_lens=np.array([300, 100000, -5], dtype=np.int32))
+    dp = DeviceProblem(bad, "cuda:0")
+    with DecodeAttn(bad, **T5) as op:
+        op.run(dp)
+        bits = op.check()
+        assert bits & B.PLT_DEV_SEQ_LEN_CLAMPED and not bits & B.PLT_DEV_WAIT_TIMEOUT
+        assert op.check() == 0  # cleared
+    clamped = p.with_(seq_lens=np.array([300, 320, 0], dtype=np.int32))
+    assert_parity(dp.out.float().cpu().numpy().astype(np.float64), oracle.decode_attn(clamped), "bf16", "clamped")
+    # page ids outside the pool: clamped and flagged, on pages that hold whole tiles and on smaller ones
+    for page_size in (128, 64):
+        pp = make_problem(custom(B=2, L=2, Hq=8, Hkv=2, lens=("list", [700, 130]), page_size=page_size))
+        table = pp.page_table.copy()
+        table[0, 1] = 10 ** 6
+        table[1, 0] = -3
+        dq = DeviceProblem(pp.with_(page_table=table), "cuda:0")
+        with DecodeAttn(pp, **T5) as op:
+            op.run(dq)
+            bits = op.check()
+            assert bits & B.PLT_DEV_PAGE_ID_CLAMPED and not bits & B.PLT_DEV_WAIT_TIMEOUT
+        assert np.isfinite(dq.out.float().cpu().numpy()).all()
+
+
+def test_runs_can_be_captured_in_a_cuda_graph():
+    """Three launches per run on this path (query pack, main with its programmatic dependency, merge): a stream
+    capture records them and replays give the same bits."""
+    p = make_problem(custom(B=6, L=4, Hq=16, Hkv=2, w=40, lens=("list", [3000, 2500, 4000, 3500, 2000, 3900]), max_seq_len=4096))
+    dp = DeviceProblem(p, "cuda:0")
+    with DecodeAttn(p, **T5) as op:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            op.run(dp, stream=side.cuda_stream)       # first call encodes the tensor maps (host work, not captured)
+        torch.cuda.synchronize()
+        want = dp.out.clone()
+        dp.out.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(3):
+                op.run(dp, stream=torch.cuda.current_stream().cuda_stream)
+        for _ in range(4):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dp.out, want)
+        assert op.check() == 0
+    assert_parity(want.float().cpu().numpy().astype(np.float64), oracle.decode_attn(p), "bf16", "graph")
+
+
+def test_decode_step_with_pre_step_on_this_path():
+    """plt_decode_attn_step (cache append with quantisation, window ring update, gate linear) ahead of this kernel: the
+    main kernel's loads may start while the query pack kernel runs, but never before the pre-step has finished."""
+    import test_gpu_prestep as TP
+    for spec in (custom(B=3, L=3, Hq=24, Hkv=4, w=50, lens=("list", [1700, 65, 3])),
+                 custom(B=4, L=4, Hq=16, Hkv=4, w=16, lens=("list", [16, 17, 33, 500]))):
+        p = make_problem(spec)
+        rows = TP.new_rows(p, 9)
+        dp = DeviceProblem(p, "cuda:0")
+        with DecodeAttn(p, **T5) as op:
+            got = TP.run_step(p, op, dp, *rows)
+        TP.check_against_oracle(p, dp, got, *rows, what="step on the tcgen05 path")
