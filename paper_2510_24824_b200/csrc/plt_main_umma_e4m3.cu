@@ -283,7 +283,7 @@ struct ECtx {
 // threads of a team call it together. `scale`: raw score -> log2 units; `done_bar` / `done_parity`: completion of
 // the last product into this O^T.
 template <int RP>
-__device__ __noinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, float scale, bool rescale,
+__device__ __forceinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, float scale, bool rescale,
                                          uint32_t tOb, uint64_t* done_bar, uint32_t done_parity, bool failed) {
     {
         float v[RP];
@@ -850,15 +850,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     }
                     // Copies, so that the arrays of the per-step path stay in registers (the out-of-line call takes
                     // the addresses of its arguments). The product before into this head's O^T was that of step g - HPC.
-                    float s_c[RP], ls_c[RP];
-#pragma unroll
-                    for (int r = 0; r < RP; ++r) {
-                        s_c[r] = s[r];
-                        ls_c[r] = lsum[r];
-                    }
-                    failed = e_slow_path<RP>(s_c, ls_c, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
-#pragma unroll
-                    for (int r = 0; r < RP; ++r) lsum[r] = ls_c[r];
+                    failed = e_slow_path<RP>(s, lsum, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
                 const uint32_t pb = g % kPBufs;   // last used by step g - kPBufs
