@@ -329,7 +329,7 @@ __device__ __forceinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[
 // scaled back), times the V scale of the head, and the denominators, out of tensor memory into the split partial.
 // tOb: O^T of the head in the piece; ob: piece parity; prow: first row of the head's partial.
 template <int RP>
-__device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
+__device__ __forceinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_t tOb, int ob, uint32_t parity, int64_t prow,
                                         float vscale, bool failed) {
     failed = sm_wait(&cx.bars[E_OFULL + ob], parity, cx.abort_flag, failed);
     float* dst = p.part_acc + prow * UD + cx.ltid;
@@ -361,7 +361,7 @@ __device__ __noinline__ bool e_epilogue(const Params& p, const ECtx& cx, uint32_
 
 // V rows of a boundary tile that hold no data may contain anything (NaN codes too): zero them so that 0 * garbage
 // stays 0. `vtile`: the V half of the slot. Called by the team that owns the step.
-__device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t* full_bar, uint32_t parity, const ECtx& cx,
+__device__ __forceinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t* full_bar, uint32_t parity, const ECtx& cx,
                                            bool failed) {
     failed = sm_wait(full_bar, parity, cx.abort_flag, failed);
     if (!failed && cx.ltid >= nvalid) {
@@ -374,7 +374,7 @@ __device__ __noinline__ bool e_zero_v_rows(uint8_t* vtile, int nvalid, uint64_t*
 
 // Start of a piece (shared cache) or of a window inside a windows piece: the visibility limit of each row; at the
 // start of a piece also the reference maxima. n: clamped length of the sequence.
-__device__ __noinline__ void e_set_limits(const Params& p, const ECtx& cx, int RP, int kind, int n, int win_loop, int wl,
+__device__ __forceinline__ void e_set_limits(const Params& p, const ECtx& cx, int RP, int kind, int n, int win_loop, int wl,
                                           bool new_piece) {
     // Threads still forming the probabilities of the tile before read lim: nobody rewrites it earlier.
     named_barrier_sync(cx.bar_id, kSmThreads);
