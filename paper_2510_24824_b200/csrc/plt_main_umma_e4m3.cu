@@ -192,7 +192,7 @@ struct EWalk {
     __device__ __forceinline__ EWalk(const Params& p, const int32_t* sp, int lo_, int hi_) : pos(lo_), hi(hi_), b(0) {
         if (pos < hi) b = find_seq(sp, p.B, pos);
     }
-    __device__ __noinline__ bool next(const Params& p, const int32_t* sp, const int32_t* lens, EPiece& pc, uint32_t& flags) {
+    __device__ __forceinline__ bool next(const Params& p, const int32_t* sp, const int32_t* lens, EPiece& pc, uint32_t& flags) {
         for (;;) {
             if (pos >= hi) return false;
             while (sp[b + 1] <= pos) ++b;
@@ -232,7 +232,7 @@ struct EWalk {
 // window's length.
 struct EWin {
     int l, key0, wl;
-    __device__ __noinline__ void seek(const Params& p, int b, int n, int t, uint32_t& flags) {
+    __device__ __forceinline__ void seek(const Params& p, int b, int n, int t, uint32_t& flags) {
         l = 1;
         wl = e_wl(p, b, n, 1, flags);
         while (l < p.L - 1) {
@@ -244,7 +244,7 @@ struct EWin {
         }
         key0 = t * UK;
     }
-    __device__ __noinline__ void advance(const Params& p, int b, int n, uint32_t& flags) {
+    __device__ __forceinline__ void advance(const Params& p, int b, int n, uint32_t& flags) {
         key0 += UK;
         while (key0 >= wl && l < p.L - 1) {
             ++l;
