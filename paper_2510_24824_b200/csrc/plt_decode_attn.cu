@@ -262,13 +262,14 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //    (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches of short sequences at any row
 //    count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one;
 //  - E4M3 caches, contiguous or in pages of a multiple of 128 tokens, at 25 to 32 packed rows when sequences can
-//    reach 16384 keys: the tcgen05 kernel for E4M3
-//    streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s) but pays more per launch
-//    for its pieces' starts and ends (measured at 32 rows: 237 vs 292 us at B = 16, N = 32768; 216 vs 279 us at
-//    B = 4, N = 131072; 157 vs 169 us at B = 16, N = 16384; 331 vs 347 us at B = 64, N = 8192; but 113 vs 107 us at
-//    B = 16, N = 8192; at 24 rows 224 vs 226 us at N = 32768 and 142 vs 129 us at N = 16384; with pages of 128 or 256
-//    tokens 232-236 vs 293 us, the page id of a tile being fetched one tile ahead; with pages of 64 tokens, two loads
-//    per tile through the producers' out-of-line path, 424 vs 293 us).
+//    reach 2048 keys and at 17 to 24 rows when they can reach 8192: the tcgen05 kernel for E4M3 streams at 6.5 TB/s
+//    where the warp-level one is bound by its conversions (4.4 TB/s). Measured steps, tcgen05 vs warp-level, B = 16:
+//    32 rows 208 vs 292 us at N = 32768, 124 vs 169 us at 16384, 83 vs 106 us at 8192, 62 vs 74 us at 4096, 52 vs
+//    56 us at 2048, 48 vs 47 us at 1024, 47 vs 42 us at 512 (B = 4, N = 131072: 200 vs 279 us; B = 64, N = 8192: 257
+//    vs 347 us; B = 128, N = 1024: 213 vs 241 us); 24 rows 202 vs 225 us at 32768, 119 vs 129 us at 16384, 77 vs
+//    79 us at 8192 (B = 64: 236 vs 259 us), 56 vs 53 us at 4096; 16 rows 177 vs 175 us at 32768 and slower below;
+//    pages of 128 or 256 tokens cost nothing (32 rows, N = 32768: 206 us; N = 4096: 62 us). With pages of 64 tokens
+//    (two loads per tile through the producers' out-of-line path) the warp-level kernel stays the faster one.
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
@@ -278,7 +279,8 @@ bool want_umma(const plt_decode_attn_config* c) {
         return false;
     const int rows = c->L * (c->Hq / c->Hkv);
     if (c->kv_dtype == PLT_KV_E4M3)
-        return umma_eligible(c) && rows > 24 && rows <= 32 && c->page_size % 128 == 0 && c->max_seq_len >= 16384 && c->stages == 0;
+        return umma_eligible(c) && rows > 16 && rows <= 32 && c->page_size % 128 == 0 && c->stages == 0 &&
+               c->max_seq_len >= (rows > 24 ? 2048 : 8192);
     return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
@@ -321,14 +323,14 @@ plt_status setup_kernels(plt_decode_attn* h, const plt_decode_attn_config* confi
         if (blocks < 1) return fail(nullptr, PLT_ERR_UNSUPPORTED, "tcgen05 main kernel does not fit an SM");
         h->umma = true;
         h->umma_e4m3 = true;
-        // Starting and finishing a piece costs this kernel as long as 4-5 tiles take it (7.6 us measured: plan step,
-        // limits, first-tile maxima, end-of-piece reduction, epilogue), and the tiles of a windows item (all masked, a
-        // limits update per window) cost more than shared-cache tiles. The plan charges every item a lead-in, so that
-        // blocks with more item starts get fewer tiles; with equal tile counts the blocks of workload 4 finished
-        // between 176 and 244 us. Measured per-step times for a lead-in of 0 / 8 / 14 / 20 tiles: 260.8 / 241.3 / 237 /
-        // 240 us at B = 16, N = 32768; 174.5 / 160.4 / 156.6 / 159.5 us at N = 16384; 244.3 / 230.7 / 216.0 / 219.0 us at
-        // B = 4, N = 131072; 337.4 / 332.6 / 331.3 / 337.7 us at B = 64, N = 8192.
-        h->piece_cost = 14;
+        // Starting and finishing a piece costs this kernel more than a tile (plan step, limits, first-tile maxima,
+        // end-of-piece reduction, epilogue), and the tiles of a windows item (all masked, a limits update per window)
+        // cost more than shared-cache tiles. The plan charges every item a lead-in, so that blocks with more item
+        // starts get fewer tiles. Measured per-step times for a lead-in of 0 / 4 / 8 / 14 / 20 tiles: 214.9 / 208.8 /
+        // 211.5 / 219.3 / 226.5 us at B = 16, N = 32768; 87.6 / 82.9 / 85.0 / 93.1 / 99.9 us at N = 8192; 208.5 /
+        // 200.1 / 199.9 / 201.7 / 203.4 us at B = 4, N = 131072; 260.0 / 257.0 / 259.3 / 262.8 / 267.1 us at B = 64,
+        // N = 8192 (3 to 6 tiles within 1 us of one another).
+        h->piece_cost = 4;
         h->var = MainVariant{config->d, 0, 0, hpc, 4, 1, 128, nslot, 0, smem, true};
         h->ctas_per_sm = 1;
         h->kbox = config->page_size > 0 ? (config->page_size < 128 ? config->page_size : 128)
