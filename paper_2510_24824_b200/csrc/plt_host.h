@@ -70,7 +70,7 @@ int main_umma_e4m3_max_slots();     // ring slots of 16 KB: 4 for K tiles, the r
 int main_umma_e4m3_min_slots();
 size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch);
 size_t main_umma_e4m3_image_bytes(int R);
-cudaError_t main_umma_e4m3_prepare(int R, int hpc, size_t smem, int* blocks_per_sm);
+cudaError_t main_umma_e4m3_prepare(int R, int hpc, bool half_pages, size_t smem, int* blocks_per_sm);
 cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream);
 cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                                   int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream);

@@ -405,14 +405,15 @@ struct ProdState {
     __device__ ProdState(const Params& p, const int32_t* sp, int lo, int hi) : walk(p, sp, lo, hi), t(0) { pc.t0 = pc.t1 = 0; }
 };
 
-// Next piece of a producer. Returns the steps it has (tiles x heads); `plain`: shared-cache tiles that are one TMA box
-// each (a contiguous cache, or pages that hold whole 128-key tiles).
+// Next piece of a producer. Returns the steps it has (tiles x heads); `plain`: shared-cache tiles that the per-step
+// loop loads itself (a contiguous cache or pages that hold whole 128-key tiles: one TMA box each; pages of 64 keys:
+// two boxes).
 __device__ __noinline__ int prod_next_piece(const Params& p, const int32_t* sp, const int32_t* lens, ProdState& st, int hpc, bool& plain,
                                             uint32_t& flags) {
     st.walk.next(p, sp, lens, st.pc, flags);
     st.t = st.pc.t0;
     if (st.pc.kind == 1) st.win.seek(p, st.pc.b, st.pc.n, st.t, flags);
-    plain = st.pc.kind == 0 && (p.page_size == 0 || p.page_size % UK == 0);
+    plain = st.pc.kind == 0 && (p.page_size == 0 || p.page_size % UK == 0 || 2 * p.page_size == UK);
     return (st.pc.t1 - st.pc.t0) * hpc;
 }
 
@@ -463,7 +464,7 @@ __device__ __noinline__ int issuer_next_piece(const Params& p, const int32_t* sp
     return (pc.t1 - pc.t0) * hpc;
 }
 
-template <int RP, int HPC>
+template <int RP, int HPC, bool HALVES>
 __global__ void __launch_bounds__(threads8(HPC), 1)
 plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                           const __grid_constant__ CUtensorMap tmKw, const __grid_constant__ CUtensorMap tmVw,
@@ -572,8 +573,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             int left = 0, hh = 0, key0 = 0, head0 = 0, outer = 0;   // of a plain piece: next tile's first key, first head, sequence
             // ... and with pages: the tile's offset in its page, the page's index in the sequence's table, its id, and
             // the id of the next tile's page, fetched one tile ahead so that the load is never waited for
+            // With pages of half a tile a tile is two boxes, the second only if it holds data; pidx then counts pages
+            // of the tile's first half and page_cur2 / page_next2 are the ids of the second half.
+            // (HALVES: a kernel of its own, so that the other page sizes' loop stays as short as it was.)
             const bool paged = p.page_size > 0;
-            int poff = 0, pidx = 0, page_cur = 0, page_next = 0;
+            int poff = 0, pidx = 0, page_cur = 0, page_next = 0, page_cur2 = 0, page_next2 = 0, cmax = 0;
             const int32_t* table = p.page_table;
             uint32_t n = 0;
             for (; n < U && ok; ++n) {
@@ -587,6 +591,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                         poff = key0 - pidx * p.page_size;
                         table = p.page_table + (int64_t)outer * p.max_pages;
                         page_cur = table[pidx];
+                        cmax = st.pc.cmax;
+                        if (HALVES && key0 + UK / 2 < cmax) page_cur2 = table[pidx + 1];
                     }
                 }
                 if (n >= (uint32_t)cap) {
@@ -598,20 +604,37 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                 uint8_t* dst = slots + (size_t)cur.slot * kTile8;
                 uint64_t* full = &fullb[cur.slot];
                 if (plain) {
-                    int c1 = key0, c3 = outer;
-                    if (paged) {
-                        if (hh == 0 && left > HPC)   // the piece has a next tile: its page id, if it starts a new page
-                            page_next = poff + UK == p.page_size ? table[pidx + 1] : page_cur;
-                        int page = page_cur;
-                        if (page < 0 || page >= p.num_pool_pages) {
-                            flags |= kDevPageIdClamped;
-                            page = page < 0 ? 0 : p.num_pool_pages - 1;
+                    if constexpr (HALVES) {
+                        if (hh == 0 && left > HPC) {   // the piece has a next tile: the ids of its one or two pages
+                            page_next = table[pidx + 2];
+                            if (key0 + UK + UK / 2 < cmax) page_next2 = table[pidx + 3];
                         }
-                        c1 = poff;
-                        c3 = page;
+                        const bool two = key0 + UK / 2 < cmax;
+                        int page = page_cur, page2 = page_cur2;
+                        if (page < 0 || page >= p.num_pool_pages || (two && (page2 < 0 || page2 >= p.num_pool_pages))) {
+                            flags |= kDevPageIdClamped;
+                            page = page < 0 ? 0 : (page >= p.num_pool_pages ? p.num_pool_pages - 1 : page);
+                            page2 = page2 < 0 ? 0 : (page2 >= p.num_pool_pages ? p.num_pool_pages - 1 : page2);
+                        }
+                        mbar_expect_tx(full, two ? (uint32_t)kTile8 : (uint32_t)(kTile8 / 2));
+                        tma_load_4d(dst, map, full, 0, 0, head0 + hh, page, pol);
+                        if (two) tma_load_4d(dst + kTile8 / 2, map, full, 0, 0, head0 + hh, page2, pol);
+                    } else {
+                        int c1 = key0, c3 = outer;
+                        if (paged) {
+                            if (hh == 0 && left > HPC)   // the piece has a next tile: its page id, if it starts a new page
+                                page_next = poff + UK == p.page_size ? table[pidx + 1] : page_cur;
+                            int page = page_cur;
+                            if (page < 0 || page >= p.num_pool_pages) {
+                                flags |= kDevPageIdClamped;
+                                page = page < 0 ? 0 : p.num_pool_pages - 1;
+                            }
+                            c1 = poff;
+                            c3 = page;
+                        }
+                        mbar_expect_tx(full, (uint32_t)(geo.kbox * 128));
+                        tma_load_4d(dst, map, full, 0, c1, head0 + hh, c3, pol);
                     }
-                    mbar_expect_tx(full, (uint32_t)(geo.kbox * 128));
-                    tma_load_4d(dst, map, full, 0, c1, head0 + hh, c3, pol);
                 } else {
                     prod_issue_special(p, geo, st, hh, HPC, dst, full, map, wmap, pol, flags);
                 }
@@ -621,7 +644,11 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     hh = 0;
                     key0 += UK;
                     ++st.t;
-                    if (paged) {
+                    if constexpr (HALVES) {
+                        pidx += 2;
+                        page_cur = page_next;
+                        page_cur2 = page_next2;
+                    } else if (paged) {
                         poff += UK;
                         if (poff == p.page_size) {
                             poff = 0;
@@ -962,15 +989,15 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
     }
 }
 
-template <int RP, int HPC>
+template <int RP, int HPC, bool HALVES>
 cudaError_t e4m3_prepare(size_t smem, int* blocks_per_sm) {
-    auto fn = plt_decode_main_umma_e4m3<RP, HPC>;
+    auto fn = plt_decode_main_umma_e4m3<RP, HPC, HALVES>;
     cudaError_t e = allow_max_dynamic_smem((const void*)fn);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, fn, threads8(HPC), smem);
 }
 
-template <int RP, int HPC>
+template <int RP, int HPC, bool HALVES>
 cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, const UmmaGeom& geo,
                         const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
     // Programmatic stream serialisation: the blocks set up and the producers start streaming the caches (which the
@@ -987,7 +1014,7 @@ cudaError_t e4m3_launch(const CUtensorMap maps[4], const Params& p, int grid, si
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, plt_decode_main_umma_e4m3<RP, HPC>, maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
+    return cudaLaunchKernelEx(&cfg, plt_decode_main_umma_e4m3<RP, HPC, HALVES>, maps[0], maps[1], maps[2], maps[3], p, geo, qimg, qinv);
 }
 
 }  // namespace
@@ -1005,10 +1032,19 @@ size_t main_umma_e4m3_smem(int R, int hpc, int nslot, int max_batch) {
 // Bytes of the query image of one (sequence, KV head).
 size_t main_umma_e4m3_image_bytes(int R) { return main_umma_e4m3_rows(R) == 16 ? ECfg<16>::QBUF : ECfg<32>::QBUF; }
 
-cudaError_t main_umma_e4m3_prepare(int R, int hpc, size_t smem, int* blocks_per_sm) {
-    if (main_umma_e4m3_rows(R) == 16)
-        return hpc == 2 ? e4m3_prepare<16, 2>(smem, blocks_per_sm) : e4m3_prepare<16, 1>(smem, blocks_per_sm);
-    return hpc == 2 ? e4m3_prepare<32, 2>(smem, blocks_per_sm) : e4m3_prepare<32, 1>(smem, blocks_per_sm);
+// `half_pages`: the cache is in pages of 64 tokens (half a tile), which have a kernel of their own.
+cudaError_t main_umma_e4m3_prepare(int R, int hpc, bool half_pages, size_t smem, int* blocks_per_sm) {
+    const int which = (main_umma_e4m3_rows(R) == 16 ? 0 : 4) + (hpc == 2 ? 2 : 0) + (half_pages ? 1 : 0);
+    switch (which) {
+        case 0: return e4m3_prepare<16, 1, false>(smem, blocks_per_sm);
+        case 1: return e4m3_prepare<16, 1, true>(smem, blocks_per_sm);
+        case 2: return e4m3_prepare<16, 2, false>(smem, blocks_per_sm);
+        case 3: return e4m3_prepare<16, 2, true>(smem, blocks_per_sm);
+        case 4: return e4m3_prepare<32, 1, false>(smem, blocks_per_sm);
+        case 5: return e4m3_prepare<32, 1, true>(smem, blocks_per_sm);
+        case 6: return e4m3_prepare<32, 2, false>(smem, blocks_per_sm);
+        default: return e4m3_prepare<32, 2, true>(smem, blocks_per_sm);
+    }
 }
 
 cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cudaStream_t stream) {
@@ -1020,11 +1056,17 @@ cudaError_t launch_pack_q_e4m3(const Params& p, uint8_t* qimg, float* qinv, cuda
 cudaError_t launch_main_umma_e4m3(const CUtensorMap maps[4], const Params& p, int grid, size_t smem, int nslot, int kbox,
                                   int wbox, int cap, const uint8_t* qimg, const float* qinv, cudaStream_t stream) {
     const UmmaGeom geo{nslot, kbox, wbox, cap < 1 ? 1 : (cap > nslot ? nslot : cap)};
-    if (main_umma_e4m3_rows(p.R) == 16)
-        return p.hpc == 2 ? e4m3_launch<16, 2>(maps, p, grid, smem, geo, qimg, qinv, stream)
-                          : e4m3_launch<16, 1>(maps, p, grid, smem, geo, qimg, qinv, stream);
-    return p.hpc == 2 ? e4m3_launch<32, 2>(maps, p, grid, smem, geo, qimg, qinv, stream)
-                      : e4m3_launch<32, 1>(maps, p, grid, smem, geo, qimg, qinv, stream);
+    const int which = (main_umma_e4m3_rows(p.R) == 16 ? 0 : 4) + (p.hpc == 2 ? 2 : 0) + (2 * p.page_size == UK ? 1 : 0);
+    switch (which) {
+        case 0: return e4m3_launch<16, 1, false>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 1: return e4m3_launch<16, 1, true>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 2: return e4m3_launch<16, 2, false>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 3: return e4m3_launch<16, 2, true>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 4: return e4m3_launch<32, 1, false>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 5: return e4m3_launch<32, 1, true>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        case 6: return e4m3_launch<32, 2, false>(maps, p, grid, smem, geo, qimg, qinv, stream);
+        default: return e4m3_launch<32, 2, true>(maps, p, grid, smem, geo, qimg, qinv, stream);
+    }
 }
 
 }  // namespace plt

@@ -32,17 +32,19 @@ def test_path_is_reported():
 
 
 def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
-    """E4M3 caches (contiguous or in pages that hold whole tiles) at 25 to 32 packed rows that can reach 2048 keys, or at
-    17 to 24 rows that can reach 8192: the library picks this kernel by itself."""
+    """E4M3 caches at 25 to 32 packed rows that can reach 2048 keys (contiguous, in pages that hold whole tiles or in
+    pages of 64 tokens), or at 17 to 24 rows that can reach 8192 (pages of 64 left out): the library picks this kernel
+    by itself."""
     spec = custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768)
     p = make_problem(spec)
     with DecodeAttn(p) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05 and op.info["heads_per_cta"] == 2
     assert_parity(run_gpu(p), oracle.decode_attn(p), "bf16", "automatic")
-    paged = make_problem(dict(spec, page_size=256))
-    with DecodeAttn(paged) as op:
-        assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
-    assert_parity(run_gpu(paged), oracle.decode_attn(paged), "bf16", "automatic, paged")
+    for page_size in (256, 64):
+        paged = make_problem(dict(spec, page_size=page_size))
+        with DecodeAttn(paged) as op:
+            assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
+        assert_parity(run_gpu(paged), oracle.decode_attn(paged), "bf16", f"automatic, pages of {page_size}")
     rows24 = make_problem(custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=8192))
     with DecodeAttn(rows24) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
@@ -50,7 +52,8 @@ def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
     for other in (custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=4096),      # 24 rows, shorter caches
                   custom(B=2, L=2, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768),     # 16 rows
                   custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=1024),      # 32 rows, short caches
-                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=64)):
+                  custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=64),   # 24 rows
+                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=32)):
         with DecodeAttn(make_problem(other)) as op:
             assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
 
@@ -136,6 +139,15 @@ def test_rows_of_very_different_magnitude_share_one_scale():
     q[:, :, 0::2] *= np.float32(2.0 ** -7)   # every other head 128 times smaller: its low term reaches the subnormal codes
     small = p.with_(q=f32_to_bf16_bits(q))
     assert_parity(run_gpu(small, **T5), oracle.decode_attn(small), "bf16", "mixed magnitudes")
+
+
+def test_pages_of_half_a_tile_with_every_kind_of_last_tile():
+    """Pages of 64 tokens are two loads per tile, the second only when that page holds data: lengths that end in the
+    first half of a tile, exactly at its middle, in the second half and at its end, on one and on several tiles."""
+    lens = [1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 1000, 1024, 1087, 1088, 1089]
+    for L, Hq in ((4, 16), (3, 6), (1, 4)):
+        p = make_problem(custom(B=len(lens), L=L, Hq=Hq, Hkv=2, w=70, lens=("list", lens), page_size=64, max_seq_len=1152))
+        assert_parity(run_gpu(p, **T5), oracle.decode_attn(p), "bf16", f"pages of 64, L={L}")
 
 
 @pytest.mark.parametrize("page_size", [64, 128, 256])
@@ -260,7 +272,9 @@ def test_out_of_range_device_values_are_clamped_and_flagged():
             op.run(dq)
             bits = op.check()
             assert bits & B.PLT_DEV_PAGE_ID_CLAMPED and not bits & B.PLT_DEV_WAIT_TIMEOUT
-        assert np.isfinite(dq.out.float().cpu().numpy()).all()
+        as_clamped = pp.with_(page_table=np.clip(table, 0, pp.num_pool_pages - 1).astype(np.int32))
+        assert_parity(dq.out.float().cpu().numpy().astype(np.float64), oracle.decode_attn(as_clamped), "bf16",
+                      f"clamped page ids, pages of {page_size}")
 
 
 def test_runs_can_be_captured_in_a_cuda_graph():
