@@ -875,8 +875,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                         aborted = true;
                         break;
                     }
-                    // Copies, so that the arrays of the per-step path stay in registers (the out-of-line call takes
-                    // the addresses of its arguments). The product before into this head's O^T was that of step g - HPC.
+                    // Inlined: an out-of-line call would take the addresses of the score and denominator arrays and put
+                    // them in local memory. The product before into this head's O^T was that of step g - HPC.
                     failed = e_slow_path<RP>(s, lsum, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
