@@ -267,10 +267,18 @@ __device__ __forceinline__ void note_piece(const Params& p, const Piece& pc, int
 struct WinCursor {
     int l;      // loop index (0-based), 1..L-1
     int key0;   // first key of the tile inside the window of loop l
+    // s.wl[l] picked by compares: an index that is not a constant would put the whole plan into local memory.
+    static __device__ __forceinline__ int32_t wl_of(const SeqPlan& s, int l) {
+        int32_t v = 0;
+#pragma unroll
+        for (int k = 1; k < kMaxLoops; ++k)
+            if (k == l) v = s.wl[k];
+        return v;
+    }
     __device__ void seek(const Params& p, const SeqPlan& s, int t) {
         l = 1;
         while (l < p.L - 1) {
-            int nt = ceil_div(s.wl[l], p.tile_keys);
+            int nt = ceil_div(wl_of(s, l), p.tile_keys);
             if (t < nt) break;
             t -= nt;
             ++l;
@@ -279,7 +287,7 @@ struct WinCursor {
     }
     __device__ void advance(const Params& p, const SeqPlan& s) {
         key0 += p.tile_keys;
-        while (key0 >= s.wl[l] && l < p.L - 1) {
+        while (key0 >= wl_of(s, l) && l < p.L - 1) {
             ++l;
             key0 = 0;
         }
