@@ -28,6 +28,11 @@
 // The query image (codes in the core-matrix order the instruction reads, and the power of two they were scaled
 // by) is written per (sequence, KV head) by plt_decode_pack_q_e4m3, launched before this kernel.
 // Online softmax with a lazily updated reference maximum, as in the bf16 tcgen05 kernel. Every wait is bounded.
+// Paged caches: a tile is one TMA box when a page holds whole tiles and two boxes with pages of 64 tokens (template
+// parameter HALVES), the page ids fetched one tile ahead by the producers' per-step loop; smaller pages go through
+// an out-of-line path with a page-table read per box.
+// Whatever the softmax teams call is inlined and takes no array or structure by reference: arguments in local
+// memory cost an L2 round trip each beside 213 KB of shared memory (measured: 240 -> 218 us on B = 16, N = 32768).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
