@@ -5,6 +5,7 @@ import pytest
 import torch
 
 import oracle
+from paper_2510_24824_b200 import binding as B
 from paper_2510_24824_b200.inputs import make_problem, workload
 from paper_2510_24824_b200.runner import DecodeAttn, DeviceProblem
 
@@ -20,12 +21,20 @@ def sample_rows(p, n, rng, forced=()):
     return np.array(sorted(rows), dtype=np.int32)
 
 
-@pytest.mark.parametrize("index,kv", [(1, ""), (2, ""), (3, ""), (4, ""), (1, "e4m3"), (4, "e4m3")])
-def test_full_size_sampled_rows(index, kv):
-    p = make_problem(dict(workload(index), kv_dtype=kv))
+# (workload index, cache type, page size or None for the workload's own): the E4M3 form of the long-context workload
+# runs on the tcgen05 kernel for E4M3, contiguous and in pages of 64 tokens (its two-boxes-per-tile variant)
+@pytest.mark.parametrize("index,kv,page_size", [(1, "", None), (2, "", None), (3, "", None), (4, "", None), (1, "e4m3", None),
+                                                (4, "e4m3", None), (3, "e4m3", None), (3, "e4m3", 64)])
+def test_full_size_sampled_rows(index, kv, page_size):
+    spec = dict(workload(index), kv_dtype=kv)
+    if page_size is not None:
+        spec["page_size"] = page_size
+    p = make_problem(spec)
     dp = DeviceProblem(p, "cuda:0")
     dp.out.fill_(float("nan"))
     with DecodeAttn(p) as op:
+        if index == 3 and kv:
+            assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
         op.run(dp)
         assert op.check() == 0
         first = dp.out.clone()
