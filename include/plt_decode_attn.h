@@ -69,10 +69,11 @@ typedef enum {
 /* Which main kernel streams the caches (plt_decode_attn_config.kernel_path). */
 typedef enum {
     PLT_PATH_AUTO = 0,      /* the library chooses: tcgen05 above 48 packed rows (L * Hq / Hkv) when max_seq_len >= 16384
-                               (bf16 caches), or on E4M3 caches at 25 to 32 packed rows when max_seq_len >= 2048 (contiguous,
-                               or in pages of 64 tokens or of a multiple of 128) and at 17 to 24 rows when max_seq_len >= 8192
+                               (bf16 caches), or on E4M3 caches at 25 to 32 packed rows when max_seq_len >= 8192 (contiguous,
+                               or in pages of 64 tokens or of a multiple of 128) and at 17 to 24 rows when max_seq_len >= 32768
                                (contiguous, or in pages of a multiple of 128 tokens), and it applies; else the warp-level
-                               kernel */
+                               kernel. With E4M3 caches at 17 to 32 rows, batches whose sequences are all longer than about
+                               2048 (25-32 rows) or 8192 (17-24 rows) tokens gain from PLT_PATH_TCGEN05 below these limits too */
     PLT_PATH_WARP_MMA = 1,  /* warp-level tensor-core products (mma.sync); fp32 inputs always use SIMT fp32 */
     PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16 queries, d = 128, pages that divide
                                or are a multiple of 128 tokens, q_len <= 1, with E4M3 caches at most 32 packed rows;

@@ -262,18 +262,22 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //    (64 rows, N = 16384: 337 vs 368 us); at 48 rows (226 vs 313 us) and on batches of short sequences at any row
 //    count (64 rows, N 512-4096: 252 vs 631 us) the warp-level kernel is the faster one;
 //  - E4M3 caches, contiguous or in pages of 64 tokens or of a multiple of 128, at 25 to 32 packed rows when sequences
-//    can reach 2048 keys, and (pages of 64 left out) at 17 to 24 rows when they can reach 8192: the tcgen05 kernel
-//    for E4M3 streams at 6.5 TB/s where the warp-level one is bound by its conversions (4.4 TB/s). Measured steps,
-//    tcgen05 vs warp-level, B = 16:
-//    32 rows 208 vs 292 us at N = 32768, 124 vs 169 us at 16384, 83 vs 106 us at 8192, 62 vs 74 us at 4096, 52 vs
-//    56 us at 2048, 48 vs 47 us at 1024, 47 vs 42 us at 512 (B = 4, N = 131072: 200 vs 279 us; B = 64, N = 8192: 257
-//    vs 347 us; B = 128, N = 1024: 213 vs 241 us); 24 rows 202 vs 225 us at 32768, 119 vs 129 us at 16384, 77 vs
-//    79 us at 8192 (B = 64: 236 vs 259 us), 56 vs 53 us at 4096; 16 rows 177 vs 175 us at 32768 and slower below;
-//    pages of 128 or 256 tokens cost nothing (32 rows, N = 32768: 206 us; N = 4096: 62 us), pages of 64 tokens (two
-//    boxes per tile, in a kernel of their own) 3 us (212 and 65 us). On a serving mix of 256 sequences of 128 to
-//    16384 tokens at 24 rows in pages of 64 the warp-level kernel is the faster one (228 vs 255 us: more than half of the
-//    sequences are shorter than 2048 tokens), hence no pages of 64 at 17 to 24 rows. Smaller pages go through the
-//    producers' out-of-line path, a dependent page-table read per box, and are left to the warp-level kernel.
+//    can reach 8192 keys, and (pages of 64 left out) at 17 to 24 rows when they can reach 32768: the tcgen05 kernel
+//    for E4M3 streams at 6.4 TB/s where the warp-level one is bound by its conversions (4.4 TB/s), but it pays more
+//    per work item, and the lengths a batch will really have are not known here. Measured steps, tcgen05 vs
+//    warp-level, equal lengths, B = 16: 32 rows 208 vs 292 us at N = 32768, 124 vs 169 us at 16384, 83 vs 106 us at
+//    8192, 62 vs 74 us at 4096, 52 vs 56 us at 2048, 48 vs 47 us at 1024, 47 vs 42 us at 512 (B = 4, N = 131072: 200
+//    vs 279 us; B = 64, N = 8192: 257 vs 347 us; B = 128, N = 1024: 213 vs 241 us); 24 rows 202 vs 225 us at 32768,
+//    119 vs 129 us at 16384, 77 vs 79 us at 8192 (B = 64: 236 vs 259 us), 56 vs 53 us at 4096; 16 rows 177 vs 175 us
+//    at 32768 and slower below; pages of 128 or 256 tokens cost nothing (32 rows, N = 32768: 206 us; N = 4096:
+//    62 us), pages of 64 tokens (two boxes per tile, in a kernel of their own) 3 us (212 and 65 us). Batches of 256
+//    sequences with log-uniform lengths (a serving mix: more than half of them under an eighth of the longest), 32
+//    rows: 313 vs 352 us with lengths up to 16384, 232 vs 248 us up to 8192 (B = 64: 75 vs 70 us), 193 vs 183 us up
+//    to 4096, 173 vs 143 us up to 2048; 24 rows: 369 vs 389 us up to 32768 (B = 64: 115 vs 115 us), 238 vs 229 us up
+//    to 16384 (pages of 64: 255 vs 228 us), 192 vs 162 us up to 8192. The thresholds are where the mixes stop
+//    losing; equal-length batches below them gain up to 15 % by asking for the path explicitly. Smaller pages go
+//    through the producers' out-of-line path, a dependent page-table read per box, and are left to the warp-level
+//    kernel.
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
 // kernel's variants.
 bool want_umma(const plt_decode_attn_config* c) {
@@ -284,8 +288,8 @@ bool want_umma(const plt_decode_attn_config* c) {
     const int rows = c->L * (c->Hq / c->Hkv);
     if (c->kv_dtype == PLT_KV_E4M3)
         return umma_eligible(c) && c->stages == 0 &&
-               ((rows > 24 && rows <= 32 && c->max_seq_len >= 2048 && (c->page_size % 128 == 0 || c->page_size == 64)) ||
-                (rows > 16 && rows <= 24 && c->max_seq_len >= 8192 && c->page_size % 128 == 0));
+               ((rows > 24 && rows <= 32 && c->max_seq_len >= 8192 && (c->page_size % 128 == 0 || c->page_size == 64)) ||
+                (rows > 16 && rows <= 24 && c->max_seq_len >= 32768 && c->page_size % 128 == 0));
     return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 

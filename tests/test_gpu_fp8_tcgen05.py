@@ -32,8 +32,8 @@ def test_path_is_reported():
 
 
 def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
-    """E4M3 caches at 25 to 32 packed rows that can reach 2048 keys (contiguous, in pages that hold whole tiles or in
-    pages of 64 tokens), or at 17 to 24 rows that can reach 8192 (pages of 64 left out): the library picks this kernel
+    """E4M3 caches at 25 to 32 packed rows that can reach 8192 keys (contiguous, in pages that hold whole tiles or in
+    pages of 64 tokens), or at 17 to 24 rows that can reach 32768 (pages of 64 left out): the library picks this kernel
     by itself."""
     spec = custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768)
     p = make_problem(spec)
@@ -45,13 +45,13 @@ def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
         with DecodeAttn(paged) as op:
             assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
         assert_parity(run_gpu(paged), oracle.decode_attn(paged), "bf16", f"automatic, pages of {page_size}")
-    rows24 = make_problem(custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=8192))
+    rows24 = make_problem(custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768))
     with DecodeAttn(rows24) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
     assert_parity(run_gpu(rows24), oracle.decode_attn(rows24), "bf16", "automatic, 24 rows")
-    for other in (custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=4096),      # 24 rows, shorter caches
+    for other in (custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=16384),     # 24 rows, shorter caches
                   custom(B=2, L=2, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768),     # 16 rows
-                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=1024),      # 32 rows, short caches
+                  custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=4096),      # 32 rows, short caches
                   custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=64),   # 24 rows
                   custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768, page_size=32)):
         with DecodeAttn(make_problem(other)) as op:

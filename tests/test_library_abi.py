@@ -87,8 +87,8 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert B.plt_decode_attn_workspace_bytes(B.make_config(**ok)) > 0
     # E4M3 caches on the tcgen05 path: at most 32 packed rows; its workspace (one block per SM, two heads per item, a
     # query image and a scale factor per (sequence, KV head)) differs from the warp-level path's, and the automatic
-    # choice is that path at 25-32 rows on caches (contiguous, pages of whole tiles or of 64 tokens) that can reach 2048
-    # keys and at 17-24 rows on caches (contiguous or pages of whole tiles) that can reach 8192
+    # choice is that path at 25-32 rows on caches (contiguous, pages of whole tiles or of 64 tokens) that can reach 8192
+    # keys and at 17-24 rows on caches (contiguous or pages of whole tiles) that can reach 32768
     fp8 = dict(ok, L=4, Hq=16, kv_dtype="e4m3")                                  # 32 packed rows
     size = lambda **kw: B.plt_decode_attn_workspace_bytes(B.make_config(**dict(fp8, **kw)))
     assert size(kernel_path=B.PLT_PATH_TCGEN05) > 4 * 2 * 8192
@@ -98,9 +98,9 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert size(max_seq_len=32768, page_size=64) == size(max_seq_len=32768, page_size=64, kernel_path=B.PLT_PATH_TCGEN05)
     assert size(max_seq_len=32768, page_size=32) == size(max_seq_len=32768, page_size=32, kernel_path=B.PLT_PATH_WARP_MMA)
     assert size(max_seq_len=32768, page_size=64, L=3) == size(max_seq_len=32768, page_size=64, L=3, kernel_path=B.PLT_PATH_WARP_MMA)
-    assert size(max_seq_len=2048) == size(max_seq_len=2048, kernel_path=B.PLT_PATH_TCGEN05)
-    assert size(max_seq_len=2047) == size(max_seq_len=2047, kernel_path=B.PLT_PATH_WARP_MMA)
-    for rows_24_or_16, longest, path in ((3, 8192, B.PLT_PATH_TCGEN05), (3, 8191, B.PLT_PATH_WARP_MMA), (2, 32768, B.PLT_PATH_WARP_MMA)):
+    assert size(max_seq_len=8192) == size(max_seq_len=8192, kernel_path=B.PLT_PATH_TCGEN05)
+    assert size(max_seq_len=8191) == size(max_seq_len=8191, kernel_path=B.PLT_PATH_WARP_MMA)
+    for rows_24_or_16, longest, path in ((3, 32768, B.PLT_PATH_TCGEN05), (3, 32767, B.PLT_PATH_WARP_MMA), (2, 65536, B.PLT_PATH_WARP_MMA)):
         assert size(max_seq_len=longest, L=rows_24_or_16) == size(max_seq_len=longest, L=rows_24_or_16, kernel_path=path)
         assert size(max_seq_len=longest, L=rows_24_or_16) != size(max_seq_len=longest, L=rows_24_or_16, kernel_path=3 - path)
     with pytest.raises(B.PltError) as e:
