@@ -285,15 +285,15 @@ struct ECtx {
 
 // Slow path of the online softmax: true maxima of the tile over its 128 keys, new reference maxima, and (unless this
 // is the head's first tile of the piece) the rescale of the three O^T column groups and of the denominators. The 128
-// threads of a team call it together. `scale`: raw score -> log2 units; `done_bar` / `done_parity`: completion of
-// the last product into this O^T.
+// threads of a team call it together. `s`: the scores in log2 units; `done_bar` / `done_parity`: completion of the
+// last product into this O^T.
 template <int RP>
-__device__ __forceinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, float scale, bool rescale,
+__device__ __forceinline__ bool e_slow_path(const float (&s)[RP], float (&lsum)[RP], const ECtx& cx, bool rescale,
                                          uint32_t tOb, uint64_t* done_bar, uint32_t done_parity, bool failed) {
     {
         float v[RP];
 #pragma unroll
-        for (int r = 0; r < RP; ++r) v[r] = s[r] * scale;
+        for (int r = 0; r < RP; ++r) v[r] = s[r];
         warp_reduce_rows<RP, true>(v, cx.lane, cx.red + cx.wq * RP);
     }
     named_barrier_sync(cx.bar_id, kSmThreads);
@@ -829,6 +829,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
             for (int t = t0; t < t1; ++t, g += HPC) {
                 int kbase, nvalid;
                 bool masked;
+                // fresh: a row may see its first key in this tile (first tile of the piece, first tile of a window)
+                bool fresh = t == t0;
                 if (kind == 0) {
                     kbase = t * UK;
                     nvalid = cmax - kbase;
@@ -837,6 +839,7 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     if (win.l != seg_l) {   // a new window: only the rows of its loop see it
                         seg_l = win.l;
                         e_set_limits(p, cx, RP, kind, pn, seg_l, win.wl, false);
+                        fresh = true;
                     }
                     kbase = win.key0;
                     nvalid = win.wl - kbase;
@@ -870,19 +873,36 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
                     for (int r = 0; r < RP; ++r)
                         if (key >= s_lim[r]) s[r] = -INFINITY;   // also replaces whatever a stale K row gave
                 }
-                // exponents against the reference maxima (rows beyond R: -1e30, never the largest), in place
+                // Exponents against the reference maxima (rows beyond R: -1e30, never the largest), in place. A fresh
+                // tile takes the slow path in any case (its rows have no reference yet), on the scaled scores.
                 float over = -INFINITY;
+                if (fresh) {
 #pragma unroll
-                for (int r = 0; r < RP; ++r) over = fmaxf(over, fmaf(s[r], scale, s_negm[r]));
+                    for (int r = 0; r < RP; ++r) s[r] *= scale;
+                } else {
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) {
+                        s[r] = fmaf(s[r], scale, s_negm[r]);
+                        over = fmaxf(over, s[r]);
+                    }
+                }
                 const bool trouble = failed || (*abort_flag != 0);
-                if (named_barrier_or(cx.bar_id, kSmThreads, over > kSlack8 || trouble)) {
+                if (named_barrier_or(cx.bar_id, kSmThreads, fresh || over > kSlack8 || trouble)) {
                     if (named_barrier_or(cx.bar_id, kSmThreads, trouble)) {
                         aborted = true;
                         break;
                     }
                     // Inlined: an out-of-line call would take the addresses of the score and denominator arrays and put
                     // them in local memory. The product before into this head's O^T was that of step g - HPC.
-                    failed = e_slow_path<RP>(s, lsum, cx, scale, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
+                    // Back to scaled scores first: outside a fresh tile a row either has a finite reference or has seen
+                    // no key at all (its scores are -inf and stay so).
+                    if (!fresh) {
+#pragma unroll
+                        for (int r = 0; r < RP; ++r) s[r] -= s_negm[r];
+                    }
+                    failed = e_slow_path<RP>(s, lsum, cx, t != t0, tOb, &bars[E_PFREE + ((g - HPC) % kPBufs)], ((g - HPC) / kPBufs) & 1, failed);
+#pragma unroll
+                    for (int r = 0; r < RP; ++r) s[r] += s_negm[r];   // against the new references
                 }
                 // ---- probabilities as three E4M3 terms into shared memory ----
                 const uint32_t pb = g % kPBufs;   // last used by step g - kPBufs
@@ -894,8 +914,8 @@ plt_decode_main_umma_e4m3(const __grid_constant__ CUtensorMap tmK, const __grid_
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         const int r0 = j * 16 + 2 * q;
-                        const float p0 = fast_exp2(fmaf(s[r0], scale, s_negm[r0]));
-                        const float p1 = fast_exp2(fmaf(s[r0 + 1], scale, s_negm[r0 + 1]));
+                        const float p0 = fast_exp2(s[r0]);
+                        const float p1 = fast_exp2(s[r0 + 1]);
                         lsum[r0] += p0;
                         lsum[r0 + 1] += p1;
                         const uint32_t h2 = pack_f16x2(p0, p1);
