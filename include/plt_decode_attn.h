@@ -73,7 +73,8 @@ typedef enum {
                                or in pages of 64 tokens or of a multiple of 128) and at 17 to 24 rows when max_seq_len >= 32768
                                (contiguous, or in pages of a multiple of 128 tokens), and it applies; else the warp-level
                                kernel. With E4M3 caches at 17 to 32 rows, batches whose sequences are all longer than about
-                               2048 (25-32 rows) or 8192 (17-24 rows) tokens gain from PLT_PATH_TCGEN05 below these limits too */
+                               2048 (25-32 rows) or 8192 (17-24 rows) tokens gain from the tcgen05 kernel below these limits
+                               too: say so with config.typical_seq_len, or ask for PLT_PATH_TCGEN05 */
     PLT_PATH_WARP_MMA = 1,  /* warp-level tensor-core products (mma.sync); fp32 inputs always use SIMT fp32 */
     PLT_PATH_TCGEN05 = 2    /* tcgen05.mma with accumulators in tensor memory: bf16 queries, d = 128, pages that divide
                                or are a multiple of 128 tokens, q_len <= 1, with E4M3 caches at most 32 packed rows;
@@ -129,6 +130,12 @@ typedef struct {
                               shared cache and the first wl - (Qn-1-j) slots of its loop's window (the loops are
                               displaced by whole tokens, Sec. 2.2.1, so the causal cutoff moves by one per token).
                               plt_decode_attn_step and plt_decode_attn_run_host take q_len <= 1 only. */
+    int32_t typical_seq_len; /* a length most sequences of a run will reach, if the caller knows one; 0: unknown. Only the
+                              automatic choice of the kernel path reads it (results do not depend on it): the lengths
+                              of a batch live on the device, so without it PLT_PATH_AUTO judges by max_seq_len and is
+                              cautious. With E4M3 caches the tcgen05 kernel is then taken at 25 to 32 packed rows from
+                              typical_seq_len >= 2048 and at 17 to 24 rows from >= 8192. < 0 is an error; values above
+                              max_seq_len count as max_seq_len. */
 } plt_decode_attn_config;
 
 /*

@@ -46,7 +46,7 @@ class Config(ctypes.Structure):
         ("heads_per_cta", ctypes.c_int32), ("key_slices", ctypes.c_int32), ("stages", ctypes.c_int32),
         ("ctas_per_sm", ctypes.c_int32), ("kernel_path", ctypes.c_int32),
         ("loads_in_flight", ctypes.c_int32), ("slices_per_warp", ctypes.c_int32), ("row_warps", ctypes.c_int32),
-        ("kv_dtype", ctypes.c_int32), ("q_len", ctypes.c_int32),
+        ("kv_dtype", ctypes.c_int32), ("q_len", ctypes.c_int32), ("typical_seq_len", ctypes.c_int32),
     ]
 
 
@@ -133,7 +133,8 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
                 page_size: int = 0, sm_scale: float = 0.0, device: int = 0,
                 loop_offset: Optional[Sequence[int]] = None, heads_per_cta: int = 0, key_slices: int = 0,
                 stages: int = 0, ctas_per_sm: int = 0, kernel_path: int = 0, loads_in_flight: int = 0,
-                row_warps: int = 0, slices_per_warp: int = 0, kv_dtype: int = 0, q_len: int = 0) -> Config:
+                row_warps: int = 0, slices_per_warp: int = 0, kv_dtype: int = 0, q_len: int = 0,
+                typical_seq_len: int = 0) -> Config:
     c = Config()
     c.struct_size = ctypes.sizeof(Config)
     c.dtype = {"f32": PLT_F32, "bf16": PLT_BF16}.get(dtype, dtype)
@@ -151,6 +152,7 @@ def make_config(dtype, max_batch: int, L: int, Hq: int, Hkv: int, d: int, max_se
     c.slices_per_warp = slices_per_warp
     c.kv_dtype = {"": PLT_KV_SAME, "e4m3": PLT_KV_E4M3}.get(kv_dtype, kv_dtype)
     c.q_len = q_len
+    c.typical_seq_len = typical_seq_len
     return c
 
 

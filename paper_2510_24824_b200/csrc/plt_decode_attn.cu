@@ -113,6 +113,7 @@ plt_status check_config(const plt_decode_attn_config* c, Geometry* g) {
             return fail(nullptr, PLT_ERR_UNSUPPORTED, "E4M3 caches need bf16 queries and head dim 128");
     }
     if (c->q_len < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "q_len %d < 0", c->q_len);
+    if (c->typical_seq_len < 0) return fail(nullptr, PLT_ERR_INVALID_ARG, "typical_seq_len %d < 0", c->typical_seq_len);
     g->Qn = c->q_len > 1 ? c->q_len : 1;
     if (g->Qn > 1 && (c->dtype != PLT_BF16 || c->kernel_path == PLT_PATH_TCGEN05))
         return fail(nullptr, PLT_ERR_UNSUPPORTED, "q_len > 1 is served by the warp-level bf16 kernel only");
@@ -275,7 +276,8 @@ bool umma_eligible(const plt_decode_attn_config* c) {
 //    rows: 313 vs 352 us with lengths up to 16384, 232 vs 248 us up to 8192 (B = 64: 75 vs 70 us), 193 vs 183 us up
 //    to 4096, 173 vs 143 us up to 2048; 24 rows: 369 vs 389 us up to 32768 (B = 64: 115 vs 115 us), 238 vs 229 us up
 //    to 16384 (pages of 64: 255 vs 228 us), 192 vs 162 us up to 8192. The thresholds are where the mixes stop
-//    losing; equal-length batches below them gain up to 15 % by asking for the path explicitly. Smaller pages go
+//    losing; a caller who knows that most sequences reach some length says so (typical_seq_len) and gets the kernel
+//    from 2048 tokens at 25 to 32 rows and from 8192 at 17 to 24, where equal-length batches gain up to 15 %. Smaller pages go
 //    through the producers' out-of-line path, a dependent page-table read per box, and are left to the warp-level
 //    kernel.
 // An explicit heads_per_cta / key_slices / ctas_per_sm / row_warps / slices_per_warp asks for the warp-level
@@ -286,10 +288,15 @@ bool want_umma(const plt_decode_attn_config* c) {
     if (c->heads_per_cta != 0 || c->key_slices != 0 || c->ctas_per_sm != 0 || c->row_warps != 0 || c->slices_per_warp != 0)
         return false;
     const int rows = c->L * (c->Hq / c->Hkv);
-    if (c->kv_dtype == PLT_KV_E4M3)
+    if (c->kv_dtype == PLT_KV_E4M3) {
+        // With a length the caller expects most sequences to reach, the equal-length figures above decide.
+        const int len = c->typical_seq_len < c->max_seq_len ? c->typical_seq_len : c->max_seq_len;
+        const bool long32 = len > 0 ? len >= 2048 : c->max_seq_len >= 8192;
+        const bool long24 = len > 0 ? len >= 8192 : c->max_seq_len >= 32768;
         return umma_eligible(c) && c->stages == 0 &&
-               ((rows > 24 && rows <= 32 && c->max_seq_len >= 8192 && (c->page_size % 128 == 0 || c->page_size == 64)) ||
-                (rows > 16 && rows <= 24 && c->max_seq_len >= 32768 && c->page_size % 128 == 0));
+               ((rows > 24 && rows <= 32 && long32 && (c->page_size % 128 == 0 || c->page_size == 64)) ||
+                (rows > 16 && rows <= 24 && long24 && c->page_size % 128 == 0));
+    }
     return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
@@ -851,7 +858,7 @@ bool same_config(const NoAllocDevice& dv, const plt_decode_attn_config* c) {
         a.heads_per_cta != c->heads_per_cta || a.key_slices != c->key_slices || a.stages != c->stages ||
         a.ctas_per_sm != c->ctas_per_sm || a.kernel_path != c->kernel_path || a.loads_in_flight != c->loads_in_flight ||
         a.slices_per_warp != c->slices_per_warp || a.row_warps != c->row_warps || a.kv_dtype != c->kv_dtype ||
-        a.q_len != c->q_len)
+        a.q_len != c->q_len || a.typical_seq_len != c->typical_seq_len)
         return false;
     for (int l = 0; l < c->L; ++l)
         if ((c->loop_offset ? c->loop_offset[l] : l) != dv.offsets[l]) return false;

@@ -49,6 +49,15 @@ def test_automatic_choice_for_long_unpaged_caches_at_32_rows():
     with DecodeAttn(rows24) as op:
         assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
     assert_parity(run_gpu(rows24), oracle.decode_attn(rows24), "bf16", "automatic, 24 rows")
+    # a length the caller expects most sequences to reach decides instead of the capacity
+    hinted = make_problem(custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [2100, 2050]), max_seq_len=4096))
+    with DecodeAttn(hinted, typical_seq_len=2048) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_TCGEN05
+    with DecodeAttn(hinted) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
+    assert_parity(run_gpu(hinted, typical_seq_len=2048), oracle.decode_attn(hinted), "bf16", "automatic with a typical length")
+    with DecodeAttn(make_problem(spec), typical_seq_len=512) as op:
+        assert op.info["kernel_path"] == B.PLT_PATH_WARP_MMA
     for other in (custom(B=2, L=3, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=16384),     # 24 rows, shorter caches
                   custom(B=2, L=2, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=32768),     # 16 rows
                   custom(B=2, L=4, Hq=16, Hkv=2, w=90, lens=("list", [900, 130]), max_seq_len=4096),      # 32 rows, short caches

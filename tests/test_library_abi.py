@@ -100,6 +100,14 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert size(max_seq_len=32768, page_size=64, L=3) == size(max_seq_len=32768, page_size=64, L=3, kernel_path=B.PLT_PATH_WARP_MMA)
     assert size(max_seq_len=8192) == size(max_seq_len=8192, kernel_path=B.PLT_PATH_TCGEN05)
     assert size(max_seq_len=8191) == size(max_seq_len=8191, kernel_path=B.PLT_PATH_WARP_MMA)
+    # a length the caller expects most sequences to reach replaces the cautious judgement by max_seq_len
+    assert size(max_seq_len=4096, typical_seq_len=2048) == size(max_seq_len=4096, kernel_path=B.PLT_PATH_TCGEN05, typical_seq_len=2048)
+    assert size(max_seq_len=32768, typical_seq_len=1024) == size(max_seq_len=32768, kernel_path=B.PLT_PATH_WARP_MMA, typical_seq_len=1024)
+    assert size(max_seq_len=16384, L=3, typical_seq_len=8192) == size(max_seq_len=16384, L=3, kernel_path=B.PLT_PATH_TCGEN05, typical_seq_len=8192)
+    assert size(max_seq_len=4096, typical_seq_len=10 ** 6) == size(max_seq_len=4096, kernel_path=B.PLT_PATH_TCGEN05, typical_seq_len=10 ** 6)
+    with pytest.raises(B.PltError) as e:
+        size(typical_seq_len=-1)
+    assert e.value.status == B.PLT_ERR_INVALID_ARG
     for rows_24_or_16, longest, path in ((3, 32768, B.PLT_PATH_TCGEN05), (3, 32767, B.PLT_PATH_WARP_MMA), (2, 65536, B.PLT_PATH_WARP_MMA)):
         assert size(max_seq_len=longest, L=rows_24_or_16) == size(max_seq_len=longest, L=rows_24_or_16, kernel_path=path)
         assert size(max_seq_len=longest, L=rows_24_or_16) != size(max_seq_len=longest, L=rows_24_or_16, kernel_path=3 - path)
