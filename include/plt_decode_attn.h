@@ -134,8 +134,9 @@ typedef struct {
                               automatic choice of the kernel path reads it (results do not depend on it): the lengths
                               of a batch live on the device, so without it PLT_PATH_AUTO judges by max_seq_len and is
                               cautious. With E4M3 caches the tcgen05 kernel is then taken at 25 to 32 packed rows from
-                              typical_seq_len >= 2048 and at 17 to 24 rows from >= 8192. < 0 is an error; values above
-                              max_seq_len count as max_seq_len. */
+                              typical_seq_len >= 2048 and at 17 to 24 rows from >= 8192; with bf16 caches above 48 rows
+                              it stands in for max_seq_len in the rule. < 0 is an error; values above max_seq_len count
+                              as max_seq_len. */
 } plt_decode_attn_config;
 
 /*

@@ -297,7 +297,8 @@ bool want_umma(const plt_decode_attn_config* c) {
                ((rows > 24 && rows <= 32 && long32 && (c->page_size % 128 == 0 || c->page_size == 64)) ||
                 (rows > 16 && rows <= 24 && long24 && c->page_size % 128 == 0));
     }
-    return umma_eligible(c) && rows > 48 && c->max_seq_len >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
+    const int reach = c->typical_seq_len > 0 && c->typical_seq_len < c->max_seq_len ? c->typical_seq_len : c->max_seq_len;
+    return umma_eligible(c) && rows > 48 && reach >= 16384 && (c->stages == 0 || c->stages == 4 || c->stages == 6);
 }
 
 // Chooses the kernel path and variant, prepares the kernels (shared-memory attribute, occupancy) and fills
